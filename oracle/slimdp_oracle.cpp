@@ -1,0 +1,224 @@
+// Slim-DP communication round: the plain CPU oracle.
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, single-threaded, obviously
+// correct statement of what one Slim-DP communication round computes.  It is
+// used by the test-suite, by the smoke check and by the benchmark's CPU
+// baseline leg, and by nothing else: the CUDA library neither includes, links
+// nor calls it, and it shares no code, table or constant generator with the
+// CUDA sources.  Build: g++ -O2 -std=c++17 -ffp-contract=off -shared -fPIC.
+//
+// Where the paper gives a plain definition the function below is that
+// definition written out:
+//   score   Eq. 1 (Section 3.2):  S_i = |w_i| + c |g_i|
+//   select  Section 3.2: rank all parameters by S_i, keep the top beta*n (full sort)
+//   pack    Section 3.1 / 3.5: T_C(delta_k) = the updates on core U explorer
+//   merge   Section 3.3 step 3: w <- w - eta' * T_C(delta_k), every worker, k ascending
+//   pull    Section 3.3 step 4: T_C(w) = the merged values on core U explorer
+//   dense   Section 2.1: Plump-DP pushes and merges every parameter
+// Readings the paper leaves open (all also listed in the design notes):
+//   * g_i is the fp32 sum of the K workers' dense updates, k ascending
+//     (Section 3.3 step 6 scores with the updates pushed densely before reselection);
+//   * score arithmetic is fp32: left-to-right sum, then one fused multiply-add;
+//     a NaN score is stored as 0x7FC00000 and ranks above +inf;
+//   * ties in the ranking are broken by ascending parameter index;
+//   * the explorer (Section 3.1 item 2, Section 3.3 step 2: a random subset of
+//     the parameters outside the core, drawn anew per worker and per
+//     communication) is an exact-size uniform subset: the first k_exp images
+//     of a keyed pseudo-random permutation of the M = n - k_core non-core
+//     ranks.  The paper fixes only "random, outside the core"; the generator
+//     (Philox-4x32-10 round keys feeding a cycle-walking Feistel network) is
+//     this library's own definition.  It is pinned by the generator's
+//     published known answers, by exhaustive bijection checks, by an
+//     independent big-integer restatement in the tests, and by a chi-square
+//     test of uniform inclusion; the paper prints no sequence to compare with.
+//
+// Indices are 0-based here (the paper's i in {1..n} is i-1).
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+namespace {
+
+inline uint32_t f32_bits(float x) {
+    uint32_t u;
+    std::memcpy(&u, &x, 4);
+    return u;
+}
+inline float bits_f32(uint32_t u) {
+    float x;
+    std::memcpy(&x, &u, 4);
+    return x;
+}
+
+// Philox-4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as
+// easy as 1, 2, 3", SC'11): ten rounds of two 32x32->64 multiplies, with the
+// key bumped by the Weyl constants between rounds.
+void philox4x32_10(const uint32_t key_in[2], const uint32_t ctr_in[4], uint32_t out[4]) {
+    const uint64_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+    const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t k0 = key_in[0], k1 = key_in[1];
+    uint32_t c0 = ctr_in[0], c1 = ctr_in[1], c2 = ctr_in[2], c3 = ctr_in[3];
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = M0 * c0;
+        uint64_t p1 = M1 * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        if (r < 9) { k0 += W0; k1 += W1; }
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+const int FEISTEL_ROUNDS = 10;
+const uint32_t STREAM_TAG = 0x534C494Du;
+
+// Twelve round-key words for (seed, worker, round): three Philox blocks with
+// key = (seed low word, seed high word), counter = (block, worker, round, tag).
+void round_keys(uint64_t seed, uint32_t worker, uint32_t round, uint32_t rk[12]) {
+    uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    for (uint32_t b = 0; b < 3; ++b) {
+        uint32_t ctr[4] = {b, worker, round, STREAM_TAG};
+        philox4x32_10(key, ctr, rk + 4 * b);
+    }
+}
+
+// Half-width h of the Feistel domain for M ranks: b = least integer >= 1 with
+// 2^b >= M, h = ceil(b / 2); the network permutes [0, 2^(2h)).
+int half_bits(uint64_t M) {
+    int b = 1;
+    while (((uint64_t)1 << b) < M) ++b;
+    return (b + 1) / 2;
+}
+
+// pi(j) on [0, M): apply the balanced Feistel network to j, and while the
+// image falls outside [0, M) apply it again (cycle walking).
+uint64_t feistel_perm(uint64_t j, uint64_t M, const uint32_t rk[12]) {
+    const int h = half_bits(M);
+    const uint32_t mask = (uint32_t)(((uint64_t)1 << h) - 1);
+    uint64_t x = j;
+    do {
+        uint32_t L = (uint32_t)(x >> h);
+        uint32_t R = (uint32_t)(x & mask);
+        for (int r = 0; r < FEISTEL_ROUNDS; ++r) {
+            const uint64_t mult = (r % 2 == 0) ? 0xD2511F53u : 0xCD9E8D57u;
+            uint64_t p = (uint64_t)(uint32_t)(R ^ rk[r]) * mult;
+            uint32_t F = (uint32_t)(p >> 32) ^ (uint32_t)p;
+            uint32_t newR = (L ^ F) & mask;
+            L = R;
+            R = newR;
+        }
+        x = ((uint64_t)L << h) | R;
+    } while (x >= M);
+    return x;
+}
+
+struct Ranked {
+    uint32_t key;   // bit pattern of the score
+    uint32_t idx;   // parameter index
+};
+
+}  // namespace
+
+extern "C" {
+
+void oracle_philox4x32_10(const uint32_t* key, const uint32_t* ctr, uint32_t* out) {
+    philox4x32_10(key, ctr, out);
+}
+
+void oracle_round_keys(uint64_t seed, uint32_t worker, uint32_t round, uint32_t* rk) {
+    round_keys(seed, worker, round, rk);
+}
+
+uint64_t oracle_feistel_perm(uint64_t j, uint64_t M, const uint32_t* rk) {
+    return feistel_perm(j, M, rk);
+}
+
+// Eq. 1.  grads: K pointers to float[n].
+void oracle_score(const float* w, const float* const* grads, uint32_t K, float c, uint64_t n, float* scores) {
+    for (uint64_t i = 0; i < n; ++i) {
+        float g = grads[0][i];
+        for (uint32_t k = 1; k < K; ++k) g = g + grads[k][i];
+        float s = std::fmaf(c, std::fabs(g), std::fabs(w[i]));
+        if (std::isnan(s)) s = bits_f32(0x7FC00000u);
+        scores[i] = s;
+    }
+}
+
+// Section 3.2: sort every parameter by (score descending, index ascending),
+// keep the first k_core, report them in ascending index order.  Scores are
+// >= +0 or the canonical NaN, so the unsigned bit pattern orders them.
+void oracle_select_core(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx) {
+    std::vector<Ranked> v(n);
+    for (uint64_t i = 0; i < n; ++i) {
+        v[i].key = f32_bits(scores[i]);
+        v[i].idx = (uint32_t)i;
+    }
+    std::sort(v.begin(), v.end(), [](const Ranked& a, const Ranked& b) {
+        if (a.key != b.key) return a.key > b.key;
+        return a.idx < b.idx;
+    });
+    for (uint64_t j = 0; j < k_core; ++j) core_idx[j] = v[j].idx;
+    std::sort(core_idx, core_idx + k_core);
+}
+
+// Section 3.3 step 2: worker `worker`'s explorer for communication `round`.
+// core_idx ascending.  noncore = ascending complement; explorer =
+// { noncore[pi(j)] : j < k_exp }, ascending.
+void oracle_sample_explore(const uint32_t* core_idx, uint64_t n, uint64_t k_core, uint64_t k_exp,
+                           uint64_t seed, uint32_t worker, uint32_t round, uint32_t* exp_idx) {
+    if (k_exp == 0) return;
+    const uint64_t M = n - k_core;
+    std::vector<uint32_t> noncore;
+    noncore.reserve(M);
+    uint64_t c = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        if (c < k_core && core_idx[c] == i) { ++c; continue; }
+        noncore.push_back((uint32_t)i);
+    }
+    uint32_t rk[12];
+    round_keys(seed, worker, round, rk);
+    for (uint64_t j = 0; j < k_exp; ++j) exp_idx[j] = noncore[feistel_perm(j, M, rk)];
+    std::sort(exp_idx, exp_idx + k_exp);
+}
+
+// T_C(delta_k): core values first, explorer values second.
+void oracle_pack(const float* delta, const uint32_t* core_idx, uint64_t k_core,
+                 const uint32_t* exp_idx, uint64_t k_exp, float* val) {
+    for (uint64_t j = 0; j < k_core; ++j) val[j] = delta[core_idx[j]];
+    for (uint64_t j = 0; j < k_exp; ++j) val[k_core + j] = delta[exp_idx[j]];
+}
+
+// Section 3.3 step 3: every worker's push applied to the global model, k ascending.
+void oracle_merge(float* w, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+                  const uint32_t* const* exp_idx, uint64_t k_exp, const float* const* val, float eta) {
+    for (uint32_t k = 0; k < K; ++k) {
+        for (uint64_t j = 0; j < k_core; ++j) {
+            uint32_t i = core_idx[j];
+            w[i] = std::fmaf(-eta, val[k][j], w[i]);
+        }
+        for (uint64_t j = 0; j < k_exp; ++j) {
+            uint32_t i = exp_idx[k][j];
+            w[i] = std::fmaf(-eta, val[k][k_core + j], w[i]);
+        }
+    }
+}
+
+// T_C(w) after the merge.
+void oracle_pull(const float* w, const uint32_t* core_idx, uint64_t k_core,
+                 const uint32_t* exp_idx, uint64_t k_exp, float* out) {
+    for (uint64_t j = 0; j < k_core; ++j) out[j] = w[core_idx[j]];
+    for (uint64_t j = 0; j < k_exp; ++j) out[k_core + j] = w[exp_idx[j]];
+}
+
+// Plump-DP (Section 2.1): every worker pushes its whole update.
+void oracle_dense_merge(float* w, uint64_t n, uint32_t K, const float* const* grads, float eta) {
+    for (uint32_t k = 0; k < K; ++k)
+        for (uint64_t i = 0; i < n; ++i) w[i] = std::fmaf(-eta, grads[k][i], w[i]);
+}
+
+}  // extern "C"

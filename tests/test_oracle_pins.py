@@ -1,0 +1,390 @@
+"""CPU-only pins of the oracle against what the paper and the mathematics fix.
+
+Each test names the passage it pins.  None of the expected values comes from
+the oracle itself or from the CUDA path: they are hand-computed exact binary
+values, exact rational arithmetic, brute force over all subsets, published
+known answers of the counter-based generator, or invariants stated in the
+paper.
+"""
+import itertools
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+from _exact import (explore_py, fma_f32, frac, perm_py, philox_py, round_f32,
+                    round_keys_py)
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bits(a):
+    return np.asarray(a, dtype=np.float32).view(np.uint32)
+
+
+# ----------------------------------------------------------------- generator
+
+def _kat_rows():
+    rows = []
+    with open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            v = [int(x, 16) for x in line.split()]
+            rows.append((v[0:4], v[4:6], v[6:10]))
+    assert len(rows) == 3
+    return rows
+
+
+@pytest.mark.parametrize("ctr,key,out", _kat_rows())
+def test_philox_known_answers(ctr, key, out):
+    # published known answers of Philox-4x32-10 (Salmon et al., SC'11)
+    assert oracle.philox4x32_10(key, ctr) == out
+    assert philox_py(key, ctr) == out
+
+
+def test_round_keys_and_permutation_match_bigint_restatement():
+    rng = np.random.default_rng(7)
+    for _ in range(40):
+        seed = int(rng.integers(0, 2 ** 63)) * 2 + int(rng.integers(0, 2))
+        worker, rnd = int(rng.integers(0, 64)), int(rng.integers(0, 2 ** 32))
+        rk = oracle.round_keys(seed, worker, rnd)
+        assert [int(x) for x in rk] == round_keys_py(seed, worker, rnd)
+        M = int(rng.integers(1, 2 ** 32))
+        for j in rng.integers(0, M, size=8):
+            assert oracle.feistel_perm(int(j), M, rk) == perm_py(int(j), M, list(map(int, rk)))
+
+
+def test_permutation_is_a_bijection_for_every_small_M():
+    # cycle-walking a bijection of [0, 2^(2h)) restricted to [0, M) is a bijection of [0, M)
+    for M in range(1, 301):
+        rk = oracle.round_keys(12345 + M, M % 7, M % 5)
+        img = sorted(oracle.feistel_perm(j, M, rk) for j in range(M))
+        assert img == list(range(M)), M
+
+
+def test_permutation_bijection_at_power_of_two_edges():
+    for M in (255, 256, 257, 4095, 4096, 4097, 65536, 65537):
+        rk = oracle.round_keys(99, 1, M)
+        img = np.array([oracle.feistel_perm(j, M, rk) for j in range(M)])
+        assert np.array_equal(np.sort(img), np.arange(M)), M
+
+
+# --------------------------------------------------------------------- score
+
+def test_score_hand_example_eq1():
+    # Eq. 1 with values exact in binary: S = |w| + c|g|
+    w = np.array([0.5, -0.25, 0.0, 1.0], np.float32)
+    g = np.array([0.0, 1.0, -2.0, 0.125], np.float32)
+    S = oracle.score(w, [g], 0.5)
+    assert S.tolist() == [0.5, 0.75, 1.0, 1.0625]
+
+
+def test_score_reduces_to_magnitude_and_to_gradient():
+    rng = np.random.default_rng(0)
+    w = rng.standard_normal(1000).astype(np.float32)
+    g = rng.standard_normal(1000).astype(np.float32)
+    z = np.zeros(1000, np.float32)
+    # g = 0: pure magnitude ranking (the weight-pruning measure of Section 3.2)
+    assert np.array_equal(bits(oracle.score(w, [z], 3.0)), bits(np.abs(w)))
+    # w = 0, c = 1: |g|
+    assert np.array_equal(bits(oracle.score(z, [g], 1.0)), bits(np.abs(g)))
+    # sign symmetry of both terms
+    assert np.array_equal(bits(oracle.score(-w, [-g], 0.7)), bits(oracle.score(w, [g], 0.7)))
+
+
+def test_score_is_one_rounding_of_the_exact_value():
+    rng = np.random.default_rng(1)
+    n = 400
+    w = (rng.standard_normal(n) * 10.0 ** rng.integers(-42, 3, n)).astype(np.float32)
+    g = (rng.standard_normal(n) * 10.0 ** rng.integers(-42, 3, n)).astype(np.float32)
+    c = np.float32(0.3)
+    S = oracle.score(w, [g], float(c))
+    for i in range(n):
+        exact = abs(frac(w[i])) + frac(c) * abs(frac(g[i]))
+        assert bits(S[i]) == bits(round_f32(exact)), i
+
+
+def test_score_sums_workers_left_to_right_in_fp32():
+    # (a + b) + c differs from a + (b + c) in binary32 for these values
+    a, b, c_ = np.float32(1.0), np.float32(2.0 ** -24), np.float32(2.0 ** -24)
+    left = np.float32(np.float32(a + b) + c_)
+    right = np.float32(a + np.float32(b + c_))
+    assert left != right
+    z = np.zeros(1, np.float32)
+    S = oracle.score(z, [np.array([a]), np.array([b]), np.array([c_])], 1.0)
+    assert S[0] == left
+    rng = np.random.default_rng(2)
+    gs = [rng.standard_normal(500).astype(np.float32) for _ in range(5)]
+    acc = gs[0].copy()
+    for g in gs[1:]:
+        acc = (acc + g).astype(np.float32)
+    assert np.array_equal(bits(oracle.score(np.zeros(500, np.float32), gs, 1.0)), bits(np.abs(acc)))
+
+
+def test_score_nonfinite():
+    w = np.array([np.inf, 1.0, np.nan, 0.0, -0.0], np.float32)
+    g = np.array([0.0, np.inf, 0.0, np.nan, -0.0], np.float32)
+    S = oracle.score(w, [g], 1.0)
+    assert bits(S).tolist() == [0x7F800000, 0x7F800000, 0x7FC00000, 0x7FC00000, 0]
+
+
+# -------------------------------------------------------------------- select
+
+def _valid_core(S, C):
+    """C is the top set under (score descending, index ascending): every member beats every non-member."""
+    key = bits(S)
+    inside = set(C)
+    for a in C:
+        for b in range(len(S)):
+            if b in inside:
+                continue
+            if not (key[a] > key[b] or (key[a] == key[b] and a < b)):
+                return False
+    return True
+
+
+def test_select_brute_force_over_all_subsets():
+    rng = np.random.default_rng(3)
+    for trial in range(30):
+        n = int(rng.integers(1, 11))
+        S = rng.integers(0, 4, n).astype(np.float32) * np.float32(0.25)   # many ties
+        for k in range(n + 1):
+            valid = [C for C in itertools.combinations(range(n), k) if _valid_core(S, C)]
+            assert len(valid) == 1
+            assert oracle.select_core(S, k).tolist() == list(valid[0])
+
+
+def test_select_closed_cases():
+    n, k = 1000, 137
+    assert oracle.select_core(np.full(n, 0.5, np.float32), k).tolist() == list(range(k))
+    inc = np.arange(n, dtype=np.float32)
+    assert oracle.select_core(inc, k).tolist() == list(range(n - k, n))
+    assert oracle.select_core(inc[::-1].copy(), k).tolist() == list(range(k))
+    assert oracle.select_core(inc, 0).size == 0
+    assert oracle.select_core(inc, n).tolist() == list(range(n))
+    # NaN (canonical) ranks above +inf, +inf above everything finite
+    S = np.array([1.0, np.inf, 3.0, 2.0], np.float32)
+    S[3] = np.uint32(0x7FC00000).view(np.float32)
+    assert oracle.select_core(S, 2).tolist() == [1, 3]
+
+
+def test_select_against_partition_on_random_scores():
+    rng = np.random.default_rng(4)
+    n, k = 200_000, 20_000
+    S = np.abs(rng.standard_normal(n)).astype(np.float32)
+    S[rng.integers(0, n, 5000)] = S[17]          # a tie group
+    core = oracle.select_core(S, k)
+    assert core.size == k and np.all(np.diff(core.astype(np.int64)) > 0)
+    kth = np.partition(S, n - k)[n - k]           # library routine: k-th largest value
+    inside = np.zeros(n, bool)
+    inside[core] = True
+    assert S[inside].min() == kth
+    assert np.all(S[~inside] <= kth) and np.all(S[inside] >= kth)
+    tied = np.flatnonzero(S == kth)
+    sel_tied, unsel_tied = tied[inside[tied]], tied[~inside[tied]]
+    if sel_tied.size and unsel_tied.size:
+        assert sel_tied.max() < unsel_tied.min()  # ties go to the smaller indices
+
+
+# ------------------------------------------------------------------- explore
+
+def _random_core(rng, n, k):
+    return np.sort(rng.choice(n, size=k, replace=False)).astype(np.uint32)
+
+
+def test_explore_invariants():
+    # Section 3.1 item 2 / Section 3.3 step 2: exact size, outside the core, distinct
+    rng = np.random.default_rng(5)
+    for n, k_core, k_exp in [(1000, 100, 45), (1000, 0, 300), (1000, 1000, 0), (1000, 999, 1),
+                             (4097, 1234, 2863), (50_000, 5000, 2250), (1, 0, 1), (2, 1, 1)]:
+        core = _random_core(rng, n, k_core)
+        e = oracle.sample_explore(core, n, k_exp, seed=11, worker=2, rnd=3)
+        assert e.size == k_exp
+        assert np.all(np.diff(e.astype(np.int64)) > 0)
+        assert e.size == 0 or int(e.max()) < n
+        assert np.intersect1d(core, e).size == 0
+        if k_exp == n - k_core:           # everything outside the core
+            assert np.array_equal(e, np.setdiff1d(np.arange(n, dtype=np.uint32), core))
+
+
+def test_explore_resampled_per_worker_and_per_round_but_reproducible():
+    rng = np.random.default_rng(6)
+    n = 20_000
+    core = _random_core(rng, n, 2000)
+    a = oracle.sample_explore(core, n, 900, 5, 0, 0)
+    assert np.array_equal(a, oracle.sample_explore(core, n, 900, 5, 0, 0))
+    for seed, worker, rnd in [(5, 1, 0), (5, 0, 1), (6, 0, 0), (5 + 2 ** 32, 0, 0)]:
+        b = oracle.sample_explore(core, n, 900, seed, worker, rnd)
+        assert not np.array_equal(a, b)
+        # two independent 5 % samples overlap in about 5 % of their members, not in most
+        assert np.intersect1d(a, b).size < 200
+
+
+def test_explore_matches_bigint_restatement():
+    rng = np.random.default_rng(8)
+    for n, k_core, k_exp in [(300, 30, 40), (1025, 100, 925), (5000, 4000, 100)]:
+        core = _random_core(rng, n, k_core)
+        got = oracle.sample_explore(core, n, k_exp, seed=2 ** 40 + 17, worker=3, rnd=9)
+        assert got.tolist() == explore_py(core, n, k_exp, 2 ** 40 + 17, 3, 9)
+
+
+def test_explore_inclusion_is_uniform_over_the_noncore():
+    # "randomly picking ... from those other than the core": every non-core
+    # parameter is included equally often (chi-square over many rounds)
+    n, k_core, k_exp, rounds = 1100, 100, 50, 4000
+    core = np.arange(0, n, 11, dtype=np.uint32)         # every 11th parameter is core
+    assert core.size == k_core
+    counts = np.zeros(n, np.int64)
+    for t in range(rounds):
+        counts[oracle.sample_explore(core, n, k_exp, seed=0, worker=0, rnd=t)] += 1
+    assert counts[core].sum() == 0
+    M = n - k_core
+    noncore = np.setdiff1d(np.arange(n), core)
+    expect = rounds * k_exp / M
+    chi2 = float(((counts[noncore] - expect) ** 2 / expect).sum())
+    dof = M - 1
+    assert abs(chi2 - dof) < 5 * np.sqrt(2 * dof), chi2
+    # per-worker streams are independent as well
+    counts_w = np.zeros(n, np.int64)
+    for k in range(64):
+        for t in range(60):
+            counts_w[oracle.sample_explore(core, n, k_exp, seed=1, worker=k, rnd=t)] += 1
+    expect = 64 * 60 * k_exp / M
+    chi2 = float(((counts_w[noncore] - expect) ** 2 / expect).sum())
+    assert abs(chi2 - dof) < 5 * np.sqrt(2 * dof), chi2
+
+
+# --------------------------------------------------------- pack / merge / pull
+
+def test_pack_and_pull_identity_and_layout():
+    rng = np.random.default_rng(9)
+    n = 1000
+    d = rng.standard_normal(n).astype(np.float32)
+    allidx = np.arange(n, dtype=np.uint32)
+    none = np.zeros(0, np.uint32)
+    assert np.array_equal(oracle.pack(d, allidx, none), d)
+    assert np.array_equal(oracle.pack(d, none, allidx), d)
+    core, exp = np.array([3, 10, 999], np.uint32), np.array([0, 7], np.uint32)
+    assert oracle.pack(d, core, exp).tolist() == [d[3], d[10], d[999], d[0], d[7]]
+    assert oracle.pull(d, core, exp).tolist() == [d[3], d[10], d[999], d[0], d[7]]
+
+
+def test_merge_single_worker_closed_form_and_sign():
+    # Section 3.3 step 3: w <- w - eta' * delta on the communication set
+    w = np.array([1.0, 2.0, 3.0, 4.0], np.float32)
+    core, exp = np.array([1], np.uint32), [np.array([3], np.uint32)]
+    val = [np.array([0.5, -2.0], np.float32)]
+    out = oracle.merge(w, core, exp, val, 0.5)
+    assert out.tolist() == [1.0, 1.75, 3.0, 5.0]
+    rng = np.random.default_rng(10)
+    n = 300
+    w = rng.standard_normal(n).astype(np.float32)
+    d = rng.standard_normal(n).astype(np.float32)
+    eta = np.float32(0.37)
+    idx = np.arange(n, dtype=np.uint32)
+    out = oracle.merge(w, idx, [np.zeros(0, np.uint32)], [d], float(eta))
+    for i in range(n):      # one rounding of the exact w - eta*d
+        assert bits(out[i]) == bits(fma_f32(-eta, d[i], w[i])), i
+
+
+def test_merge_applies_workers_in_ascending_order():
+    # two workers whose explorers collide on one parameter; values chosen so
+    # the two application orders round differently in binary32
+    w0 = np.float32(1.0)
+    a, b = np.float32(2.0 ** -24), np.float32(-1.5 * 2.0 ** -23)
+    first_a = fma_f32(-1.0, b, fma_f32(-1.0, a, w0))
+    first_b = fma_f32(-1.0, a, fma_f32(-1.0, b, w0))
+    assert bits(first_a) != bits(first_b)
+    w = np.array([w0, 5.0], np.float32)
+    none = np.zeros(0, np.uint32)
+    e = [np.array([0], np.uint32), np.array([0], np.uint32)]
+    out = oracle.merge(w, none, e, [np.array([a]), np.array([b])], 1.0)
+    assert bits(out[0]) == bits(first_a) and out[1] == 5.0
+    out = oracle.merge(w, none, e, [np.array([b]), np.array([a])], 1.0)
+    assert bits(out[0]) == bits(first_b)
+
+
+def test_dense_merge_is_sequential_rounding_of_exact_updates():
+    rng = np.random.default_rng(11)
+    n, K = 200, 3
+    w = rng.standard_normal(n).astype(np.float32)
+    gs = [rng.standard_normal(n).astype(np.float32) for _ in range(K)]
+    eta = np.float32(1.0 / 3.0)
+    out = oracle.dense_merge(w, gs, float(eta))
+    for i in range(n):
+        x = w[i]
+        for k in range(K):
+            x = fma_f32(-eta, gs[k][i], x)
+        assert bits(out[i]) == bits(x), i
+
+
+@pytest.mark.parametrize("form", ["all_core", "all_explore", "core_plus_rest"])
+def test_full_communication_ratio_reproduces_plump_dp(form):
+    # alpha = 100 %: Slim-DP transfers everything, i.e. Plump-DP (Sections 2.1, 3.5)
+    rng = np.random.default_rng(12)
+    n, K = 5000, 4
+    w = rng.standard_normal(n).astype(np.float32)
+    gs = [(rng.standard_normal(n) * 1e-2).astype(np.float32) for _ in range(K)]
+    k_core = {"all_core": n, "all_explore": 0, "core_plus_rest": 1234}[form]
+    r = oracle.run_round(w, gs, 1.0, k_core, n - k_core, seed=3, rnd=0, eta=1.0 / K)
+    assert np.array_equal(bits(r["w"]), bits(oracle.dense_merge(w, gs, 1.0 / K)))
+    for k in range(K):      # and every worker pulls the whole merged model
+        both = np.concatenate([r["core_idx"], r["exp_idx"][k]])
+        full = np.empty(n, np.float32)
+        full[both] = r["pulled"][k]
+        assert np.array_equal(bits(full), bits(r["w"]))
+
+
+def test_round_invariants_on_tiny_shape():
+    rng = np.random.default_rng(13)
+    n, K, k_core, k_exp = 20_000, 4, 2000, 900
+    w = (rng.standard_normal(n) * 0.05).astype(np.float32)
+    gs = [(rng.standard_normal(n) * 1e-3).astype(np.float32) for _ in range(K)]
+    r = oracle.run_round(w, gs, 1.0, k_core, k_exp, seed=0, rnd=0, eta=0.25)
+    core = r["core_idx"]
+    assert core.size == k_core
+    touched = np.zeros(n, bool)
+    touched[core] = True
+    for k in range(K):
+        e = r["exp_idx"][k]
+        assert e.size == k_exp and np.intersect1d(e, core).size == 0     # core and explorer disjoint
+        touched[e] = True
+        # pushed values are the worker's updates on its communication set
+        assert np.array_equal(r["val"][k], gs[k][np.concatenate([core, e])])
+        assert np.array_equal(r["pulled"][k], r["w"][np.concatenate([core, e])])
+    # parameters outside every communication set are untouched, bit for bit
+    assert np.array_equal(bits(r["w"][~touched]), bits(w[~touched]))
+    # eta' = 0: nothing moves, pull returns the old values
+    r0 = oracle.run_round(w, gs, 1.0, k_core, k_exp, seed=0, rnd=0, eta=0.0)
+    assert np.array_equal(bits(r0["w"]), bits(w))
+
+
+def test_degenerate_ratios():
+    # beta = 0 (pure exploration) and beta = alpha (no exploration) are legal (Section 3.4)
+    rng = np.random.default_rng(14)
+    n, K = 3000, 2
+    w = rng.standard_normal(n).astype(np.float32)
+    gs = [rng.standard_normal(n).astype(np.float32) for _ in range(K)]
+    r = oracle.run_round(w, gs, 1.0, 0, 300, seed=1, rnd=0, eta=0.5)
+    assert r["core_idx"].size == 0 and all(v.size == 300 for v in r["val"])
+    r = oracle.run_round(w, gs, 1.0, 300, 0, seed=1, rnd=0, eta=0.5)
+    assert all(e.size == 0 for e in r["exp_idx"]) and all(v.size == 300 for v in r["val"])
+
+
+# ----------------------------------------------------------------- wire size
+
+def test_wire_words_match_table1_ratios():
+    # Section 3.5: core costs beta*n words (keys cached), explorer 2(alpha-beta)n;
+    # Table 1's measured T_comm ratios agree with (2 alpha - beta) to a few percent.
+    with open(os.path.join(GOLDEN, "table1_comm_time.txt")) as f:
+        rows = [l.split() for l in f if l.strip() and not l.startswith("#")]
+    n = 10 ** 6
+    for model, K, alpha, beta, t_plump, t_slim in rows:
+        alpha, beta = float(alpha), float(beta)
+        k_core, k_exp = round(beta * n), round((alpha - beta) * n)
+        words = k_core + 2 * k_exp           # values for the core, (index, value) for the explorer
+        assert words == round((2 * alpha - beta) * n)
+        assert abs(words / n - float(t_slim) / float(t_plump)) < 0.03, model
