@@ -41,23 +41,24 @@ def _chunk(cfg: Config, tensor: int, worker: int, ci: int) -> np.ndarray:
     a = ci * CHUNK
     b = min(a + CHUNK, cfg.N)
     rng = np.random.default_rng([cfg.seed, tensor, worker, ci])
-    n = b - a
+    n = CHUNK      # always a whole chunk, so a prefix of a config sees the same draws
     if tensor == _TENSOR_W:
-        x = rng.standard_normal(n, dtype=np.float32)
+        x = rng.standard_normal(n, dtype=np.float32)[:b - a]
         _scale_by_segment(cfg, x, a, b, 1.0, True)
         if cfg.quantise:
             x = (np.clip(np.rint(x * np.float32(512.0)), -128, 127) * np.float32(2.0 ** -9)).astype(np.float32)
         return x
     if cfg.grad_dist == "normal":
-        x = rng.standard_normal(n, dtype=np.float32)
+        x = rng.standard_normal(n, dtype=np.float32)[:b - a]
         x *= np.float32(cfg.grad_scale)
     elif cfg.grad_dist == "normal_layer":
-        x = rng.standard_normal(n, dtype=np.float32)
+        x = rng.standard_normal(n, dtype=np.float32)[:b - a]
         _scale_by_segment(cfg, x, a, b, cfg.grad_scale, False)
     elif cfg.grad_dist == "laplace":
         # Laplace(0, b) as b * (E1 - E2), E1 and E2 independent Exp(1)
         x = rng.standard_exponential(n, dtype=np.float32)
         x -= rng.standard_exponential(n, dtype=np.float32)
+        x = x[:b - a]
         x *= np.float32(cfg.grad_scale)
     else:
         raise ValueError(cfg.grad_dist)
