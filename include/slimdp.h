@@ -1,0 +1,227 @@
+/* slimdp.h - C ABI of the Slim-DP communication round for NVIDIA B200 (sm_100a).
+ *
+ * One Slim-DP communication round (Sun et al., "Slim-DP: A Light Communication
+ * Data Parallelism for DNN", Algorithm 1 and Section 3.3) touches a flat fp32
+ * parameter vector w-bar of n entries and K workers' accumulated updates
+ * delta_k of n entries each:
+ *
+ *   score    S_i = |w_i| + c |g_i|                         (Eq. 1, Section 3.2)
+ *   select   core = the k_core parameters of largest S     (Section 3.2; T_S of Section 3.1)
+ *   explore  per worker, per round: k_exp random parameters outside the core
+ *                                                          (T_R^k, Section 3.1 item 2, Section 3.3 step 2)
+ *   pack     T_C(delta_k): the worker's updates on core U explorer
+ *                                                          (Section 3.1; extraction, Section 3.5)
+ *   merge    w-bar <- w-bar - eta' T_C(delta_k), all k     (Section 3.3 step 3)
+ *   pull     T_C(w-bar): merged values on core U explorer  (Section 3.3 step 4)
+ *
+ * General rules, valid for every entry point unless it says otherwise:
+ *   - Every pointer is a DEVICE pointer (memory of the current CUDA device)
+ *     unless its comment says HOST.  "HOST array of K device pointers" means a
+ *     host-side array whose K entries are device pointers; it is read during
+ *     the call and may be freed as soon as the call returns.
+ *   - The caller owns every buffer.  The library allocates no device memory,
+ *     creates no stream, and never synchronises except in slimdp_read_status
+ *     and slimdp_round_host.  All work is enqueued on `stream` (a cudaStream_t
+ *     passed as void*; NULL is the legacy default stream) and is ordered with
+ *     other work on that stream.
+ *   - Arguments are validated on the host before anything is enqueued.  A
+ *     negative return value means nothing (more) was enqueued by that call.
+ *   - Indices are 0-based uint32_t, so 1 <= n < 2^32.  fp32 buffers must be
+ *     4-byte aligned; 16-byte alignment of all of them selects the vectorised
+ *     kernels (any alignment is still computed correctly).  Index buffers and
+ *     core_aux / workspaces must be 16-byte aligned.
+ *   - Input and output buffers of one call must not overlap, except where a
+ *     buffer is documented as updated in place.
+ *   - Results are deterministic: the same inputs give the same bytes on every
+ *     call, whatever the launch shape.
+ */
+#ifndef SLIMDP_H_
+#define SLIMDP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t slimdp_status;
+
+enum {
+    SLIMDP_OK = 0,
+    SLIMDP_ERR_INVALID_ARG = -1, /* null pointer, count out of range, non-finite coefficient, misaligned buffer */
+    SLIMDP_ERR_WORKSPACE = -2,   /* workspace / arena smaller than the matching *_bytes query              */
+    SLIMDP_ERR_CUDA = -3,        /* a CUDA runtime call or kernel launch failed                             */
+    SLIMDP_ERR_INTERNAL = -4,    /* a device-side consistency check failed (reported by slimdp_read_status) */
+    SLIMDP_ERR_UNSUPPORTED = -5
+};
+
+/* Largest K: the K per-worker device pointers travel by value as kernel arguments. */
+#define SLIMDP_MAX_WORKERS 64
+
+/* Parameters per bitmap block: core_aux keeps one directory entry per block. */
+#define SLIMDP_BLOCK 1024
+
+const char* slimdp_status_string(slimdp_status s);
+
+/* ---------------------------------------------------------------- sizes ---
+ * core_aux is the device-side description of the core that the explorer
+ * sampler reads.  Layout (all uint32_t, little-endian bit order):
+ *   bitmap    [nb * 32] words, nb = ceil(n / 1024): bit (i & 31) of word (i >> 5)
+ *             is 1 iff parameter i is in the core; bits at i >= n are 0;
+ *   directory [nb + 1] words starting at byte offset slimdp_core_aux_dir_offset(n):
+ *             directory[b] = number of NON-core parameters with index < 1024 b,
+ *             directory[nb] = n - k_core.
+ */
+size_t slimdp_core_aux_bytes(uint64_t n);
+size_t slimdp_core_aux_dir_offset(uint64_t n);
+
+/* Bytes of scratch that slimdp_select_core needs for n parameters. */
+size_t slimdp_select_workspace_bytes(uint64_t n);
+
+/* Bytes of scratch that slimdp_sample_explore (num_workers = 1) or
+ * slimdp_sample_explore_batched (num_workers workers in one call) needs. */
+size_t slimdp_explore_workspace_bytes(uint64_t n, uint32_t num_workers);
+
+/* max(select, explore for K workers): one workspace that serves every call of a round. */
+size_t slimdp_workspace_bytes(uint64_t n, uint32_t K);
+
+/* ---------------------------------------------------------------- score ---
+ * Eq. 1 (Section 3.2).  For every i < n, in fp32:
+ *     g      = ((grads[0][i] + grads[1][i]) + ...) + grads[K-1][i]   (left to right)
+ *     S[i]   = fma(c, |g|, |w[i]|)                                   (one rounding)
+ * and a NaN result is stored as the bit pattern 0x7FC00000.  g is the sum of
+ * the updates all K workers pushed densely before a reselection (Section 3.3
+ * steps 3 and 6); a caller that already holds an aggregated gradient passes
+ * K = 1.  Scores are >= +0, +inf or that NaN, so their bit patterns order them.
+ *   w       [n] global model                       (read)
+ *   grads   HOST array of K device pointers, each [n] (read), 1 <= K <= SLIMDP_MAX_WORKERS
+ *   c       finite, the coefficient of Eq. 1
+ *   scores  [n] (written)
+ */
+slimdp_status slimdp_score(const float* w, const float* const* grads, uint32_t K, float c, uint64_t n,
+                           float* scores, void* stream);
+
+/* --------------------------------------------------------------- select ---
+ * Core selection T_S (Section 3.1 item 1, Section 3.2: "rank the parameters by
+ * their significance, and select the top"): the k_core parameters that come
+ * first when all n are ordered by (score bit pattern descending as unsigned
+ * 32-bit, index ascending).  For scores from slimdp_score this is score
+ * descending with ties going to the smaller index and NaN ranking highest.
+ *   scores    [n] (read)
+ *   k_core    0 <= k_core <= n
+ *   core_idx  [k_core] (written): the core, ascending
+ *   core_aux  [slimdp_core_aux_bytes(n)] (written): bitmap + directory, see above
+ *   ws        [ws_bytes >= slimdp_select_workspace_bytes(n)] scratch, contents undefined after
+ * Device-side consistency failures are recorded in the first word of ws; read
+ * them with slimdp_read_status(ws, stream).
+ */
+slimdp_status slimdp_select_core(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx,
+                                 void* core_aux, void* ws, size_t ws_bytes, void* stream);
+
+/* -------------------------------------------------------------- explore ---
+ * Exploration operator T_R^k (Section 3.1 item 2, Section 3.3 step 2): worker
+ * `worker` draws, for communication `round`, k_exp distinct parameters
+ * uniformly from the M = n - k_core parameters outside the core.  The paper
+ * fixes "random"; this library fixes the generator so that results can be
+ * reproduced bit for bit:
+ *   round keys rk[0..11] = three Philox-4x32-10 blocks with key
+ *       (seed low word, seed high word) and counters (b, worker, round, 0x534C494D), b = 0, 1, 2;
+ *   pi = a 10-round balanced Feistel network on 2h bits, h = ceil(b/2) with b the least
+ *       integer >= 1 such that 2^b >= M; round r maps (L, R) to (R, (L ^ F) & (2^h - 1)),
+ *       F = hi32(p) ^ lo32(p), p = (uint64)(R ^ rk[r]) * (r even ? 0xD2511F53 : 0xCD9E8D57);
+ *       images >= M are fed through the network again (cycle walking);
+ *   explorer = { the pi(j)-th non-core parameter (0-based, ascending) : j < k_exp }.
+ *   core_aux  as written by slimdp_select_core for the same n and k_core (read)
+ *   k_exp     0 <= k_exp <= n - k_core
+ *   exp_idx   [k_exp] (written): the explorer, ascending
+ *   ws        [ws_bytes >= slimdp_explore_workspace_bytes(n, 1)] scratch
+ */
+slimdp_status slimdp_sample_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp,
+                                    uint64_t seed, uint32_t worker, uint32_t round, uint32_t* exp_idx,
+                                    void* ws, size_t ws_bytes, void* stream);
+
+/* The same for workers first_worker .. first_worker + num_workers - 1 in one
+ * call; exp_idx is a HOST array of num_workers device pointers, each [k_exp].
+ * ws_bytes >= slimdp_explore_workspace_bytes(n, num_workers).  Results are
+ * identical to num_workers single calls. */
+slimdp_status slimdp_sample_explore_batched(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp,
+                                            uint64_t seed, uint32_t first_worker, uint32_t num_workers,
+                                            uint32_t round, uint32_t* const* exp_idx, void* ws,
+                                            size_t ws_bytes, void* stream);
+
+/* ----------------------------------------------------------------- pack ---
+ * Extraction of T_C(delta_k) = T_S(delta_k) U T_R^k(delta_k) (Section 3.1; the
+ * "extract ... by scanning" cost of Section 3.5):
+ *     val[j]          = delta[core_idx[j]]   j < k_core
+ *     val[k_core + j] = delta[exp_idx[j]]    j < k_exp
+ * The worker's <key, value> buffer (Section 3.5) is the pair
+ * (core_idx || exp_idx, val); the core keys are stored once and shared by all
+ * workers, which is the key-caching of Section 3.5, so a push carries
+ * 4 (k_core + 2 k_exp) bytes.
+ *   delta [n] (read), core_idx [k_core], exp_idx [k_exp] (read; entries < n), val [k_core + k_exp] (written)
+ */
+slimdp_status slimdp_pack(const float* delta, uint64_t n, const uint32_t* core_idx, uint64_t k_core,
+                          const uint32_t* exp_idx, uint64_t k_exp, float* val, void* stream);
+
+/* K workers in one call: deltas, exp_idx and val are HOST arrays of K device pointers. */
+slimdp_status slimdp_pack_batched(const float* const* deltas, uint32_t K, uint64_t n, const uint32_t* core_idx,
+                                  uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
+                                  float* const* val, void* stream);
+
+/* ---------------------------------------------------------------- merge ---
+ * Server update (Algorithm 1, Section 3.3 step 3): every worker's push is
+ * applied to the global model, workers in ascending order:
+ *     for k = 0 .. K-1:  for every pushed (i, v) of worker k:  w[i] = fma(-eta, v, w[i])
+ * Explorers of different workers may contain the same parameter; it then
+ * receives its updates in ascending k, so the fp32 result is unique.
+ * Parameters outside every worker's communication set are not written.
+ *   w_global  [n] (updated in place)
+ *   exp_idx   HOST array of K device pointers, each [k_exp], ascending, disjoint from core_idx
+ *   val       HOST array of K device pointers, each [k_core + k_exp], as written by slimdp_pack
+ *   eta       finite, the server step eta'
+ */
+slimdp_status slimdp_merge(float* w_global, uint64_t n, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+                           const uint32_t* const* exp_idx, uint64_t k_exp, const float* const* val, float eta,
+                           void* stream);
+
+/* ----------------------------------------------------------------- pull ---
+ * Pull of T_C(w-bar) (Algorithm 1, Section 3.3 step 4):
+ *     out[j] = w_global[core_idx[j]],  out[k_core + j] = w_global[exp_idx[j]].
+ */
+slimdp_status slimdp_pull(const float* w_global, uint64_t n, const uint32_t* core_idx, uint64_t k_core,
+                          const uint32_t* exp_idx, uint64_t k_exp, float* out, void* stream);
+
+/* K workers in one call: exp_idx and out are HOST arrays of K device pointers. */
+slimdp_status slimdp_pull_batched(const float* w_global, uint32_t K, uint64_t n, const uint32_t* core_idx,
+                                  uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
+                                  float* const* out, void* stream);
+
+/* --------------------------------------------------------------- status ---
+ * Synchronises `stream`, then returns the sticky status word kept in the first
+ * 4 bytes of a workspace used by slimdp_select_core / slimdp_sample_explore*:
+ * SLIMDP_OK, or SLIMDP_ERR_INTERNAL if a device-side consistency check failed
+ * (the outputs of that call are then undefined), or SLIMDP_ERR_CUDA. */
+slimdp_status slimdp_read_status(const void* ws, void* stream);
+
+/* ----------------------------------------------------- whole round, host ---
+ * One whole round (score, select, K x explore, K x pack, merge, K x pull) on
+ * HOST buffers: copies w and the K updates to the device, runs the round
+ * above, copies the results back, and synchronises before returning.
+ *   w_host       HOST [n]: global model, replaced by the merged model
+ *   grads_host   HOST array of K HOST pointers, each [n]
+ *   core_idx_host HOST [k_core] (written)
+ *   exp_idx_host  HOST array of K HOST pointers, each [k_exp] (written)
+ *   pulled_host   HOST array of K HOST pointers, each [k_core + k_exp] (written)
+ *   arena         DEVICE scratch of at least slimdp_round_arena_bytes(n, K, k_core, k_exp) bytes, 256-byte aligned
+ * Host buffers should be page-locked for full copy bandwidth. */
+size_t slimdp_round_arena_bytes(uint64_t n, uint32_t K, uint64_t k_core, uint64_t k_exp);
+slimdp_status slimdp_round_host(float* w_host, const float* const* grads_host, uint32_t K, uint64_t n, float c,
+                                uint64_t k_core, uint64_t k_exp, uint64_t seed, uint32_t round, float eta,
+                                uint32_t* core_idx_host, uint32_t* const* exp_idx_host,
+                                float* const* pulled_host, void* arena, size_t arena_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLIMDP_H_ */

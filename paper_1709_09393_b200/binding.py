@@ -1,0 +1,261 @@
+"""ctypes binding of libslimdp.so.  Argument marshalling only.
+
+The shared library must have been built in-tree (python -m
+paper_1709_09393_b200.build); importing this module without it raises.
+There is no fallback path of any kind.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libslimdp.so")
+
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build the CUDA library first (python -m paper_1709_09393_b200.build)")
+
+lib = ctypes.CDLL(_LIB_PATH)
+
+_vp = ctypes.c_void_p
+_u64 = ctypes.c_uint64
+_u32 = ctypes.c_uint32
+_f32 = ctypes.c_float
+_sz = ctypes.c_size_t
+_pp = ctypes.POINTER(ctypes.c_void_p)
+
+EXPORTS = {
+    "slimdp_status_string": (ctypes.c_char_p, [ctypes.c_int32]),
+    "slimdp_core_aux_bytes": (_sz, [_u64]),
+    "slimdp_core_aux_dir_offset": (_sz, [_u64]),
+    "slimdp_select_workspace_bytes": (_sz, [_u64]),
+    "slimdp_explore_workspace_bytes": (_sz, [_u64, _u32]),
+    "slimdp_workspace_bytes": (_sz, [_u64, _u32]),
+    "slimdp_score": (ctypes.c_int32, [_vp, _pp, _u32, _f32, _u64, _vp, _vp]),
+    "slimdp_select_core": (ctypes.c_int32, [_vp, _u64, _u64, _vp, _vp, _vp, _sz, _vp]),
+    "slimdp_sample_explore": (ctypes.c_int32, [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _vp, _vp, _sz, _vp]),
+    "slimdp_sample_explore_batched": (ctypes.c_int32,
+                                      [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _u32, _pp, _vp, _sz, _vp]),
+    "slimdp_pack": (ctypes.c_int32, [_vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp]),
+    "slimdp_pack_batched": (ctypes.c_int32, [_pp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _vp]),
+    "slimdp_merge": (ctypes.c_int32, [_vp, _u64, _u32, _vp, _u64, _pp, _u64, _pp, _f32, _vp]),
+    "slimdp_pull": (ctypes.c_int32, [_vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp]),
+    "slimdp_pull_batched": (ctypes.c_int32, [_vp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _vp]),
+    "slimdp_read_status": (ctypes.c_int32, [_vp, _vp]),
+    "slimdp_round_arena_bytes": (_sz, [_u64, _u32, _u64, _u64]),
+    "slimdp_round_host": (ctypes.c_int32, [_vp, _pp, _u32, _u64, _f32, _u64, _u64, _u64, _u32, _f32, _vp, _pp, _pp,
+                                           _vp, _sz, _vp]),
+}
+
+for _name, (_res, _args) in EXPORTS.items():
+    _fn = getattr(lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class SlimDPError(RuntimeError):
+    def __init__(self, call: str, status: int):
+        self.status = status
+        msg = lib.slimdp_status_string(status).decode()
+        super().__init__(f"{call} failed: {msg} ({status})")
+
+
+def _check(call: str, status: int) -> None:
+    if status != 0:
+        raise SlimDPError(call, status)
+
+
+def _stream(stream: Optional[torch.cuda.Stream] = None) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    """Device/host address, or NULL for a missing or empty tensor."""
+    if t is None:
+        return None
+    return t.data_ptr() or None
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+def _ptr_array(ts: Sequence[torch.Tensor]):
+    return (ctypes.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+
+
+# int32 carries uint32 indices (torch has no full uint32 support); values are reinterpreted, not converted
+IDX = torch.int32
+
+
+def core_aux_bytes(n: int) -> int:
+    return lib.slimdp_core_aux_bytes(n)
+
+
+def core_aux_dir_offset(n: int) -> int:
+    return lib.slimdp_core_aux_dir_offset(n)
+
+
+def select_workspace_bytes(n: int) -> int:
+    return lib.slimdp_select_workspace_bytes(n)
+
+
+def explore_workspace_bytes(n: int, num_workers: int) -> int:
+    return lib.slimdp_explore_workspace_bytes(n, num_workers)
+
+
+def workspace_bytes(n: int, K: int) -> int:
+    return lib.slimdp_workspace_bytes(n, K)
+
+
+def round_arena_bytes(n: int, K: int, k_core: int, k_exp: int) -> int:
+    return lib.slimdp_round_arena_bytes(n, K, k_core, k_exp)
+
+
+def read_status(ws: torch.Tensor, stream=None) -> None:
+    _check("slimdp_read_status", lib.slimdp_read_status(ws.data_ptr(), _stream(stream)))
+
+
+def slimdp_score(w: torch.Tensor, grads: Sequence[torch.Tensor], c: float, scores: torch.Tensor, stream=None):
+    n = w.numel()
+    _dev(w, torch.float32, "w")
+    _dev(scores, torch.float32, "scores")
+    for g in grads:
+        if _dev(g, torch.float32, "grads").numel() != n:
+            raise ValueError("grads: length differs from w")
+    if scores.numel() != n:
+        raise ValueError("scores: length differs from w")
+    _check("slimdp_score", lib.slimdp_score(w.data_ptr(), _ptr_array(grads), len(grads), c, n, scores.data_ptr(),
+                                            _stream(stream)))
+
+
+def slimdp_select_core(scores: torch.Tensor, k_core: int, core_idx: torch.Tensor, core_aux: torch.Tensor,
+                       ws: torch.Tensor, stream=None):
+    _dev(scores, torch.float32, "scores")
+    _dev(core_idx, IDX, "core_idx")
+    if core_idx.numel() != k_core:
+        raise ValueError("core_idx: length differs from k_core")
+    _check("slimdp_select_core",
+           lib.slimdp_select_core(scores.data_ptr(), scores.numel(), k_core, _ptr(core_idx), core_aux.data_ptr(),
+                                  ws.data_ptr(), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def slimdp_sample_explore(core_aux: torch.Tensor, n: int, k_core: int, k_exp: int, seed: int, worker: int,
+                          rnd: int, exp_idx: torch.Tensor, ws: torch.Tensor, stream=None):
+    _dev(exp_idx, IDX, "exp_idx")
+    if exp_idx.numel() != k_exp:
+        raise ValueError("exp_idx: length differs from k_exp")
+    _check("slimdp_sample_explore",
+           lib.slimdp_sample_explore(core_aux.data_ptr(), n, k_core, k_exp, seed, worker, rnd, _ptr(exp_idx),
+                                     ws.data_ptr(), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def slimdp_sample_explore_batched(core_aux: torch.Tensor, n: int, k_core: int, k_exp: int, seed: int,
+                                  first_worker: int, rnd: int, exp_idx: Sequence[torch.Tensor], ws: torch.Tensor,
+                                  stream=None):
+    for e in exp_idx:
+        if _dev(e, IDX, "exp_idx").numel() != k_exp:
+            raise ValueError("exp_idx: length differs from k_exp")
+    _check("slimdp_sample_explore_batched",
+           lib.slimdp_sample_explore_batched(core_aux.data_ptr(), n, k_core, k_exp, seed, first_worker,
+                                             len(exp_idx), rnd, _ptr_array(exp_idx), ws.data_ptr(),
+                                             ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def _check_sets(core_idx, exp_idx, out, what):
+    _dev(core_idx, IDX, "core_idx")
+    _dev(exp_idx, IDX, "exp_idx")
+    _dev(out, torch.float32, what)
+    if out.numel() != core_idx.numel() + exp_idx.numel():
+        raise ValueError(f"{what}: length differs from k_core + k_exp")
+
+
+def slimdp_pack(delta: torch.Tensor, core_idx: torch.Tensor, exp_idx: torch.Tensor, val: torch.Tensor, stream=None):
+    _dev(delta, torch.float32, "delta")
+    _check_sets(core_idx, exp_idx, val, "val")
+    _check("slimdp_pack", lib.slimdp_pack(delta.data_ptr(), delta.numel(), _ptr(core_idx), core_idx.numel(),
+                                          _ptr(exp_idx), exp_idx.numel(), _ptr(val), _stream(stream)))
+
+
+def slimdp_pack_batched(deltas: Sequence[torch.Tensor], core_idx: torch.Tensor, exp_idx: Sequence[torch.Tensor],
+                        val: Sequence[torch.Tensor], stream=None):
+    K = len(deltas)
+    if len(exp_idx) != K or len(val) != K:
+        raise ValueError("deltas, exp_idx and val must have K entries each")
+    for d, e, v in zip(deltas, exp_idx, val):
+        _dev(d, torch.float32, "deltas")
+        _check_sets(core_idx, e, v, "val")
+    _check("slimdp_pack_batched",
+           lib.slimdp_pack_batched(_ptr_array(deltas), K, deltas[0].numel(), _ptr(core_idx), core_idx.numel(),
+                                   _ptr_array(exp_idx), exp_idx[0].numel(), _ptr_array(val), _stream(stream)))
+
+
+def slimdp_merge(w_global: torch.Tensor, core_idx: torch.Tensor, exp_idx: Sequence[torch.Tensor],
+                 val: Sequence[torch.Tensor], eta: float, stream=None):
+    _dev(w_global, torch.float32, "w_global")
+    K = len(val)
+    if len(exp_idx) != K:
+        raise ValueError("exp_idx and val must have K entries each")
+    for e, v in zip(exp_idx, val):
+        _check_sets(core_idx, e, v, "val")
+    _check("slimdp_merge",
+           lib.slimdp_merge(w_global.data_ptr(), w_global.numel(), K, _ptr(core_idx), core_idx.numel(),
+                            _ptr_array(exp_idx), exp_idx[0].numel(), _ptr_array(val), eta, _stream(stream)))
+
+
+def slimdp_pull(w_global: torch.Tensor, core_idx: torch.Tensor, exp_idx: torch.Tensor, out: torch.Tensor,
+                stream=None):
+    _dev(w_global, torch.float32, "w_global")
+    _check_sets(core_idx, exp_idx, out, "out")
+    _check("slimdp_pull", lib.slimdp_pull(w_global.data_ptr(), w_global.numel(), _ptr(core_idx), core_idx.numel(),
+                                          _ptr(exp_idx), exp_idx.numel(), _ptr(out), _stream(stream)))
+
+
+def slimdp_pull_batched(w_global: torch.Tensor, core_idx: torch.Tensor, exp_idx: Sequence[torch.Tensor],
+                        out: Sequence[torch.Tensor], stream=None):
+    _dev(w_global, torch.float32, "w_global")
+    K = len(out)
+    if len(exp_idx) != K:
+        raise ValueError("exp_idx and out must have K entries each")
+    for e, o in zip(exp_idx, out):
+        _check_sets(core_idx, e, o, "out")
+    _check("slimdp_pull_batched",
+           lib.slimdp_pull_batched(w_global.data_ptr(), K, w_global.numel(), _ptr(core_idx), core_idx.numel(),
+                                   _ptr_array(exp_idx), exp_idx[0].numel(), _ptr_array(out), _stream(stream)))
+
+
+def _host(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name}: expected a contiguous host tensor of {dtype}")
+    return t
+
+
+def slimdp_round_host(w_host: torch.Tensor, grads_host: Sequence[torch.Tensor], c: float, k_core: int, k_exp: int,
+                      seed: int, rnd: int, eta: float, core_idx_host: torch.Tensor,
+                      exp_idx_host: Sequence[torch.Tensor], pulled_host: Sequence[torch.Tensor],
+                      arena: torch.Tensor, stream=None):
+    """One whole round on host tensors (pinned for speed); w_host is replaced by the merged model."""
+    n, K = w_host.numel(), len(grads_host)
+    _host(w_host, torch.float32, "w_host")
+    _host(core_idx_host, IDX, "core_idx_host")
+    for g, e, p in zip(grads_host, exp_idx_host, pulled_host):
+        if _host(g, torch.float32, "grads_host").numel() != n:
+            raise ValueError("grads_host: length differs from w_host")
+        if _host(e, IDX, "exp_idx_host").numel() != k_exp:
+            raise ValueError("exp_idx_host: length differs from k_exp")
+        if _host(p, torch.float32, "pulled_host").numel() != k_core + k_exp:
+            raise ValueError("pulled_host: length differs from k_core + k_exp")
+    if core_idx_host.numel() != k_core or len(exp_idx_host) != K or len(pulled_host) != K:
+        raise ValueError("output buffers do not match k_core / K")
+    if not arena.is_cuda:
+        raise TypeError("arena: expected a CUDA tensor")
+    _check("slimdp_round_host",
+           lib.slimdp_round_host(w_host.data_ptr(), _ptr_array(grads_host), K, n, c, k_core, k_exp, seed, rnd, eta,
+                                 _ptr(core_idx_host), _ptr_array(exp_idx_host), _ptr_array(pulled_host),
+                                 arena.data_ptr(), arena.numel() * arena.element_size(), _stream(stream)))

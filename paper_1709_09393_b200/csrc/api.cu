@@ -1,0 +1,318 @@
+// The exported C ABI: argument validation, workspace sizing, and the order
+// of kernel launches for each call.  No step of the round runs on the host.
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "layout.cuh"
+
+namespace slimdp {
+
+slimdp_status launch_score(const float* w, const PtrArray<const float>& g, uint32_t K, float c, uint64_t n,
+                           float* S, bool vec, cudaStream_t st);
+slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx, void* core_aux,
+                            void* ws, cudaStream_t st);
+slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
+                             uint32_t first_worker, uint32_t workers, uint32_t round,
+                             const PtrArray<uint32_t>& out, void* ws, cudaStream_t st);
+slimdp_status launch_gather(const PtrArray<const float>& src, uint32_t workers, const uint32_t* core_idx,
+                            uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp,
+                            const PtrArray<float>& out, cudaStream_t st);
+slimdp_status launch_merge(float* w, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+                           const PtrArray<const uint32_t>& exp, uint64_t k_exp, const PtrArray<const float>& val,
+                           float eta, cudaStream_t st);
+
+int sm_count() {
+    static int cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+    if (cached[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return -1;
+        cached[dev] = v;
+    }
+    return cached[dev];
+}
+
+namespace {
+
+constexpr uint64_t kMaxN = 0xFFFFFFFFull;   // indices are uint32_t
+
+bool n_ok(uint64_t n) { return n >= 1 && n <= kMaxN; }
+bool k_ok(uint32_t K) { return K >= 1 && K <= SLIMDP_MAX_WORKERS; }
+
+template <typename T>
+bool fill(PtrArray<T>& dst, T* const* src, uint32_t count, bool need, size_t align) {
+    memset(&dst, 0, sizeof(dst));
+    if (src == nullptr) return !need;
+    for (uint32_t k = 0; k < count; ++k) {
+        if (need && (src[k] == nullptr || (reinterpret_cast<uintptr_t>(src[k]) & (align - 1)) != 0)) return false;
+        dst.p[k] = src[k];
+    }
+    return true;
+}
+
+bool sets_ok(uint64_t n, uint64_t k_core, uint64_t k_exp) {
+    return n_ok(n) && k_core <= n && k_exp <= n - k_core;
+}
+
+}  // namespace
+}  // namespace slimdp
+
+using namespace slimdp;
+
+extern "C" {
+
+const char* slimdp_status_string(slimdp_status s) {
+    switch (s) {
+        case SLIMDP_OK: return "ok";
+        case SLIMDP_ERR_INVALID_ARG: return "invalid argument";
+        case SLIMDP_ERR_WORKSPACE: return "workspace too small";
+        case SLIMDP_ERR_CUDA: return "CUDA error";
+        case SLIMDP_ERR_INTERNAL: return "device-side consistency check failed";
+        case SLIMDP_ERR_UNSUPPORTED: return "unsupported";
+        default: return "unknown status";
+    }
+}
+
+size_t slimdp_core_aux_dir_offset(uint64_t n) {
+    if (!n_ok(n)) return 0;
+    return align_up(num_blocks(n) * kWordsPerBlock * 4, 256);
+}
+
+size_t slimdp_core_aux_bytes(uint64_t n) {
+    if (!n_ok(n)) return 0;
+    return slimdp_core_aux_dir_offset(n) + align_up((num_blocks(n) + 1) * 4, 256);
+}
+
+size_t slimdp_select_workspace_bytes(uint64_t n) {
+    if (!n_ok(n)) return 0;
+    return select_ws_layout(nullptr, n).bytes;
+}
+
+size_t slimdp_explore_workspace_bytes(uint64_t n, uint32_t num_workers) {
+    if (!n_ok(n) || !k_ok(num_workers)) return 0;
+    return explore_ws_layout(nullptr, n, num_workers).bytes;
+}
+
+size_t slimdp_workspace_bytes(uint64_t n, uint32_t K) {
+    const size_t a = slimdp_select_workspace_bytes(n), b = slimdp_explore_workspace_bytes(n, K);
+    if (a == 0 || b == 0) return 0;
+    return a > b ? a : b;
+}
+
+slimdp_status slimdp_score(const float* w, const float* const* grads, uint32_t K, float c, uint64_t n,
+                           float* scores, void* stream) {
+    if (!n_ok(n) || !k_ok(K) || !w || !grads || !scores || !isfinite(c)) return SLIMDP_ERR_INVALID_ARG;
+    if (!aligned4(w) || !aligned4(scores)) return SLIMDP_ERR_INVALID_ARG;
+    PtrArray<const float> g;
+    if (!fill<const float>(g, grads, K, true, 4)) return SLIMDP_ERR_INVALID_ARG;
+    bool vec = aligned16(w) && aligned16(scores);
+    for (uint32_t k = 0; k < K; ++k) vec = vec && aligned16(g.p[k]);
+    return launch_score(w, g, K, c, n, scores, vec, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_select_core(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx,
+                                 void* core_aux, void* ws, size_t ws_bytes, void* stream) {
+    if (!n_ok(n) || k_core > n || !scores || !core_aux || !ws) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && !core_idx) return SLIMDP_ERR_INVALID_ARG;
+    if (!aligned4(scores) || !aligned16(core_aux) || !aligned16(ws) || (core_idx && !aligned16(core_idx)))
+        return SLIMDP_ERR_INVALID_ARG;
+    if (ws_bytes < slimdp_select_workspace_bytes(n)) return SLIMDP_ERR_WORKSPACE;
+    return launch_select(scores, n, k_core, core_idx, core_aux, ws, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_sample_explore_batched(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp,
+                                            uint64_t seed, uint32_t first_worker, uint32_t num_workers,
+                                            uint32_t round, uint32_t* const* exp_idx, void* ws, size_t ws_bytes,
+                                            void* stream) {
+    if (!sets_ok(n, k_core, k_exp) || !k_ok(num_workers) || !core_aux || !ws) return SLIMDP_ERR_INVALID_ARG;
+    if ((uint64_t)first_worker + num_workers > 0x100000000ull) return SLIMDP_ERR_INVALID_ARG;
+    if (!aligned16(core_aux) || !aligned16(ws)) return SLIMDP_ERR_INVALID_ARG;
+    PtrArray<uint32_t> out;
+    if (!fill<uint32_t>(out, exp_idx, num_workers, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (ws_bytes < slimdp_explore_workspace_bytes(n, num_workers)) return SLIMDP_ERR_WORKSPACE;
+    return launch_explore(core_aux, n, k_core, k_exp, seed, first_worker, num_workers, round, out, ws,
+                          (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_sample_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp,
+                                    uint64_t seed, uint32_t worker, uint32_t round, uint32_t* exp_idx, void* ws,
+                                    size_t ws_bytes, void* stream) {
+    uint32_t* one[1] = {exp_idx};
+    return slimdp_sample_explore_batched(core_aux, n, k_core, k_exp, seed, worker, 1, round, one, ws, ws_bytes,
+                                         stream);
+}
+
+static slimdp_status gather_common(const float* const* srcs, bool same_src, const float* src0, uint32_t K,
+                                   uint64_t n, const uint32_t* core_idx, uint64_t k_core,
+                                   const uint32_t* const* exp_idx, uint64_t k_exp, float* const* out, void* stream) {
+    if (!sets_ok(n, k_core, k_exp) || !k_ok(K)) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    PtrArray<const float> src;
+    PtrArray<const uint32_t> exp;
+    PtrArray<float> dst;
+    if (same_src) {
+        if (!src0 || !aligned4(src0)) return SLIMDP_ERR_INVALID_ARG;
+        memset(&src, 0, sizeof(src));
+        for (uint32_t k = 0; k < K; ++k) src.p[k] = src0;
+    } else if (!fill<const float>(src, srcs, K, true, 4)) {
+        return SLIMDP_ERR_INVALID_ARG;
+    }
+    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<float>(dst, out, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
+    return launch_gather(src, K, core_idx, k_core, exp, k_exp, dst, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_pack_batched(const float* const* deltas, uint32_t K, uint64_t n, const uint32_t* core_idx,
+                                  uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
+                                  float* const* val, void* stream) {
+    if (!deltas) return SLIMDP_ERR_INVALID_ARG;
+    return gather_common(deltas, false, nullptr, K, n, core_idx, k_core, exp_idx, k_exp, val, stream);
+}
+
+slimdp_status slimdp_pack(const float* delta, uint64_t n, const uint32_t* core_idx, uint64_t k_core,
+                          const uint32_t* exp_idx, uint64_t k_exp, float* val, void* stream) {
+    const uint32_t* e[1] = {exp_idx};
+    float* o[1] = {val};
+    return gather_common(nullptr, true, delta, 1, n, core_idx, k_core, e, k_exp, o, stream);
+}
+
+slimdp_status slimdp_pull_batched(const float* w_global, uint32_t K, uint64_t n, const uint32_t* core_idx,
+                                  uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
+                                  float* const* out, void* stream) {
+    return gather_common(nullptr, true, w_global, K, n, core_idx, k_core, exp_idx, k_exp, out, stream);
+}
+
+slimdp_status slimdp_pull(const float* w_global, uint64_t n, const uint32_t* core_idx, uint64_t k_core,
+                          const uint32_t* exp_idx, uint64_t k_exp, float* out, void* stream) {
+    const uint32_t* e[1] = {exp_idx};
+    float* o[1] = {out};
+    return gather_common(nullptr, true, w_global, 1, n, core_idx, k_core, e, k_exp, o, stream);
+}
+
+slimdp_status slimdp_merge(float* w_global, uint64_t n, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+                           const uint32_t* const* exp_idx, uint64_t k_exp, const float* const* val, float eta,
+                           void* stream) {
+    if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !w_global || !aligned4(w_global) || !isfinite(eta))
+        return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    PtrArray<const uint32_t> exp;
+    PtrArray<const float> v;
+    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const float>(v, val, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core + k_exp == 0) return SLIMDP_OK;
+    return launch_merge(w_global, K, core_idx, k_core, exp, k_exp, v, eta, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_read_status(const void* ws, void* stream) {
+    if (!ws) return SLIMDP_ERR_INVALID_ARG;
+    int32_t s = 0;
+    if (cudaMemcpyAsync(&s, ws, sizeof(s), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+        return SLIMDP_ERR_CUDA;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return SLIMDP_ERR_CUDA;
+    return (s == SLIMDP_OK) ? SLIMDP_OK : SLIMDP_ERR_INTERNAL;
+}
+
+// ---- whole round on host buffers ------------------------------------------
+
+namespace {
+struct Arena {
+    float* w;
+    float* delta[SLIMDP_MAX_WORKERS];
+    float* scores;
+    uint32_t* core_idx;
+    void* core_aux;
+    void* select_ws;
+    size_t select_ws_bytes;
+    void* explore_ws;
+    size_t explore_ws_bytes;
+    uint32_t* exp_idx[SLIMDP_MAX_WORKERS];
+    float* val[SLIMDP_MAX_WORKERS];
+    float* pulled[SLIMDP_MAX_WORKERS];
+    size_t bytes;
+};
+
+Arena arena_layout(void* base, uint64_t n, uint32_t K, uint64_t k_core, uint64_t k_exp) {
+    char* p = reinterpret_cast<char*>(base);
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        char* r = p + off;
+        off += align_up(bytes ? bytes : 1, 256);
+        return r;
+    };
+    Arena A;
+    memset(&A, 0, sizeof(A));
+    const uint64_t m = k_core + k_exp;
+    A.w = reinterpret_cast<float*>(take(n * 4));
+    for (uint32_t k = 0; k < K; ++k) A.delta[k] = reinterpret_cast<float*>(take(n * 4));
+    A.scores = reinterpret_cast<float*>(take(n * 4));
+    A.core_idx = reinterpret_cast<uint32_t*>(take(k_core * 4));
+    A.core_aux = take(slimdp_core_aux_bytes(n));
+    A.select_ws_bytes = slimdp_select_workspace_bytes(n);
+    A.select_ws = take(A.select_ws_bytes);
+    A.explore_ws_bytes = slimdp_explore_workspace_bytes(n, K);
+    A.explore_ws = take(A.explore_ws_bytes);
+    for (uint32_t k = 0; k < K; ++k) A.exp_idx[k] = reinterpret_cast<uint32_t*>(take(k_exp * 4));
+    for (uint32_t k = 0; k < K; ++k) A.val[k] = reinterpret_cast<float*>(take(m * 4));
+    for (uint32_t k = 0; k < K; ++k) A.pulled[k] = reinterpret_cast<float*>(take(m * 4));
+    A.bytes = off;
+    return A;
+}
+}  // namespace
+
+size_t slimdp_round_arena_bytes(uint64_t n, uint32_t K, uint64_t k_core, uint64_t k_exp) {
+    if (!sets_ok(n, k_core, k_exp) || !k_ok(K)) return 0;
+    return arena_layout(nullptr, n, K, k_core, k_exp).bytes;
+}
+
+slimdp_status slimdp_round_host(float* w_host, const float* const* grads_host, uint32_t K, uint64_t n, float c,
+                                uint64_t k_core, uint64_t k_exp, uint64_t seed, uint32_t round, float eta,
+                                uint32_t* core_idx_host, uint32_t* const* exp_idx_host, float* const* pulled_host,
+                                void* arena, size_t arena_bytes, void* stream) {
+    if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !w_host || !grads_host || !arena || !isfinite(c) || !isfinite(eta))
+        return SLIMDP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && !core_idx_host) return SLIMDP_ERR_INVALID_ARG;
+    if (k_exp > 0 && !exp_idx_host) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core + k_exp > 0 && !pulled_host) return SLIMDP_ERR_INVALID_ARG;
+    for (uint32_t k = 0; k < K; ++k) {
+        if (!grads_host[k]) return SLIMDP_ERR_INVALID_ARG;
+        if (k_exp > 0 && !exp_idx_host[k]) return SLIMDP_ERR_INVALID_ARG;
+        if (k_core + k_exp > 0 && !pulled_host[k]) return SLIMDP_ERR_INVALID_ARG;
+    }
+    if (arena_bytes < slimdp_round_arena_bytes(n, K, k_core, k_exp)) return SLIMDP_ERR_WORKSPACE;
+    const Arena A = arena_layout(arena, n, K, k_core, k_exp);
+    cudaStream_t st = (cudaStream_t)stream;
+    const uint64_t m = k_core + k_exp;
+#define SLIMDP_CUDA(x) \
+    if ((x) != cudaSuccess) return SLIMDP_ERR_CUDA
+#define SLIMDP_TRY(x)                   \
+    do {                                \
+        slimdp_status s_ = (x);         \
+        if (s_ != SLIMDP_OK) return s_; \
+    } while (0)
+    SLIMDP_CUDA(cudaMemcpyAsync(A.w, w_host, n * 4, cudaMemcpyHostToDevice, st));
+    for (uint32_t k = 0; k < K; ++k)
+        SLIMDP_CUDA(cudaMemcpyAsync(A.delta[k], grads_host[k], n * 4, cudaMemcpyHostToDevice, st));
+    SLIMDP_TRY(slimdp_score(A.w, A.delta, K, c, n, A.scores, stream));
+    SLIMDP_TRY(slimdp_select_core(A.scores, n, k_core, A.core_idx, A.core_aux, A.select_ws, A.select_ws_bytes,
+                                  stream));
+    SLIMDP_TRY(slimdp_sample_explore_batched(A.core_aux, n, k_core, k_exp, seed, 0, K, round, A.exp_idx,
+                                             A.explore_ws, A.explore_ws_bytes, stream));
+    SLIMDP_TRY(slimdp_pack_batched(A.delta, K, n, A.core_idx, k_core, A.exp_idx, k_exp, A.val, stream));
+    SLIMDP_TRY(slimdp_merge(A.w, n, K, A.core_idx, k_core, A.exp_idx, k_exp, A.val, eta, stream));
+    SLIMDP_TRY(slimdp_pull_batched(A.w, K, n, A.core_idx, k_core, A.exp_idx, k_exp, A.pulled, stream));
+    SLIMDP_CUDA(cudaMemcpyAsync(w_host, A.w, n * 4, cudaMemcpyDeviceToHost, st));
+    if (k_core) SLIMDP_CUDA(cudaMemcpyAsync(core_idx_host, A.core_idx, k_core * 4, cudaMemcpyDeviceToHost, st));
+    for (uint32_t k = 0; k < K; ++k) {
+        if (k_exp) SLIMDP_CUDA(cudaMemcpyAsync(exp_idx_host[k], A.exp_idx[k], k_exp * 4, cudaMemcpyDeviceToHost, st));
+        if (m) SLIMDP_CUDA(cudaMemcpyAsync(pulled_host[k], A.pulled[k], m * 4, cudaMemcpyDeviceToHost, st));
+    }
+    SLIMDP_TRY(slimdp_read_status(A.select_ws, stream));
+    return slimdp_read_status(A.explore_ws, stream);
+#undef SLIMDP_CUDA
+#undef SLIMDP_TRY
+}
+
+}  // extern "C"

@@ -1,0 +1,116 @@
+// Shared declarations of the Slim-DP CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "slimdp.h"
+
+namespace slimdp {
+
+constexpr uint32_t kBlock = SLIMDP_BLOCK;        // parameters per bitmap block
+constexpr uint32_t kWordsPerBlock = kBlock / 32; // 32 bitmap words per block
+constexpr uint32_t kScanTile = 1024;             // bitmap blocks per scan tile
+
+// K device pointers passed by value as a kernel argument (512 bytes).
+template <typename T>
+struct PtrArray {
+    T* p[SLIMDP_MAX_WORKERS];
+};
+
+// First 256 bytes of every workspace.
+struct WsHeader {
+    int32_t status;      // sticky: SLIMDP_OK or SLIMDP_ERR_INTERNAL
+    uint32_t prefix;     // radix prefix found so far; after the last pass the threshold key T
+    uint32_t k_rem;      // rank still to resolve inside the prefix; after the last pass the tie quota r
+    uint32_t ties;       // r: how many keys equal to T are admitted (smallest indices first)
+    uint32_t reserved[60];
+};
+static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline uint64_t num_blocks(uint64_t n) { return (n + kBlock - 1) / kBlock; }
+inline uint64_t num_scan_tiles(uint64_t n) { return (num_blocks(n) + kScanTile - 1) / kScanTile; }
+
+// Number of SMs of the current device (cached per device id).
+int sm_count();
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+#define SLIMDP_CHECK_LAUNCH()                                   \
+    do {                                                        \
+        if (cudaGetLastError() != cudaSuccess) return SLIMDP_ERR_CUDA; \
+    } while (0)
+
+// ---- device helpers -------------------------------------------------------
+
+// Position of the n-th (0-based) set bit of word; word must have more than n set bits.
+__device__ __forceinline__ uint32_t nth_set_bit(uint32_t word, uint32_t n) {
+    uint32_t pos = 0;
+#pragma unroll
+    for (int width = 16; width >= 1; width >>= 1) {
+        uint32_t low = (word >> pos) & ((1u << width) - 1u);
+        uint32_t c = __popc(low);
+        if (n >= c) {
+            n -= c;
+            pos += width;
+        }
+    }
+    return pos;
+}
+
+__device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31u; }
+
+// Inclusive warp scan (all 32 lanes active).
+__device__ __forceinline__ uint32_t warp_inclusive_scan(uint32_t v) {
+    const uint32_t lane = lane_id();
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t t = __shfl_up_sync(0xFFFFFFFFu, v, d);
+        if (lane >= (uint32_t)d) v += t;
+    }
+    return v;
+}
+
+__device__ __forceinline__ unsigned long long warp_inclusive_scan64(unsigned long long v) {
+    const uint32_t lane = lane_id();
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, v, d);
+        if (lane >= (uint32_t)d) v += t;
+    }
+    return v;
+}
+
+// Exclusive scan of one value per thread over a block of 1024 threads.
+// Returns the exclusive prefix; *total receives the block sum.  smem: 33 words.
+__device__ __forceinline__ unsigned long long block_exclusive_scan64_1024(unsigned long long v,
+                                                                          unsigned long long* smem,
+                                                                          unsigned long long* total) {
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    unsigned long long inc = warp_inclusive_scan64(v);
+    if (lane == 31) smem[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned long long s = smem[lane];
+        unsigned long long sinc = warp_inclusive_scan64(s);
+        smem[lane] = sinc - s;
+        if (lane == 31) smem[32] = sinc;
+    }
+    __syncthreads();
+    unsigned long long out = smem[warp] + inc - v;
+    *total = smem[32];
+    __syncthreads();
+    return out;
+}
+
+// ---- internal launchers (each enqueues on `st`, returns a slimdp_status) ---
+
+// Exclusive scan over bitmap blocks of 64-bit counters: cnt[y][nb] -> pref[y][nb],
+// totals[y] = sum.  y = 0 .. batch-1; rows are `stride` entries apart.
+slimdp_status launch_block_scan(const unsigned long long* cnt, unsigned long long* pref,
+                                unsigned long long* tile_sums, unsigned long long* totals, uint64_t nb,
+                                uint32_t batch, uint64_t stride, uint64_t tile_stride, cudaStream_t st);
+
+}  // namespace slimdp

@@ -1,0 +1,114 @@
+// slimdp_score: significance S_i = |w_i| + c |g_i| (Eq. 1, Section 3.2) as one
+// streaming pass: 128-bit loads of w and of the K updates, fp32 left-to-right
+// sum over workers, one fused multiply-add, 128-bit store.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace slimdp {
+
+namespace {
+
+__device__ __forceinline__ float score_one(float c, float g, float w) {
+    float s = __fmaf_rn(c, fabsf(g), fabsf(w));
+    return (s != s) ? __uint_as_float(0x7FC00000u) : s;
+}
+
+// KT > 0: K known at compile time (all loads of one element group are issued
+// before the first add).  KT == 0: K from the argument.
+template <int KT>
+__global__ void __launch_bounds__(256) score_vec4_kernel(const float4* __restrict__ w, PtrArray<const float> g,
+                                                         int K, float c, uint64_t n4, uint64_t n,
+                                                         float4* __restrict__ S) {
+    const int kk = (KT > 0) ? KT : K;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        float4 a = __ldcs(reinterpret_cast<const float4*>(g.p[0]) + i);
+        if (KT > 0) {
+            float4 b[KT > 1 ? KT - 1 : 1];
+#pragma unroll
+            for (int k = 1; k < KT; ++k) b[k - 1] = __ldcs(reinterpret_cast<const float4*>(g.p[k]) + i);
+#pragma unroll
+            for (int k = 1; k < KT; ++k) {
+                a.x = __fadd_rn(a.x, b[k - 1].x);
+                a.y = __fadd_rn(a.y, b[k - 1].y);
+                a.z = __fadd_rn(a.z, b[k - 1].z);
+                a.w = __fadd_rn(a.w, b[k - 1].w);
+            }
+        } else {
+#pragma unroll 4
+            for (int k = 1; k < kk; ++k) {
+                float4 b = __ldcs(reinterpret_cast<const float4*>(g.p[k]) + i);
+                a.x = __fadd_rn(a.x, b.x);
+                a.y = __fadd_rn(a.y, b.y);
+                a.z = __fadd_rn(a.z, b.z);
+                a.w = __fadd_rn(a.w, b.w);
+            }
+        }
+        float4 ww = __ldcs(w + i);
+        float4 s;
+        s.x = score_one(c, a.x, ww.x);
+        s.y = score_one(c, a.y, ww.y);
+        s.z = score_one(c, a.z, ww.z);
+        s.w = score_one(c, a.w, ww.w);
+        S[i] = s;
+    }
+    // ragged tail (n % 4 elements)
+    if (blockIdx.x == 0 && threadIdx.x < (uint32_t)(n - 4 * n4)) {
+        const uint64_t i = 4 * n4 + threadIdx.x;
+        const float* ws = reinterpret_cast<const float*>(w);
+        float a = g.p[0][i];
+        for (int k = 1; k < kk; ++k) a = __fadd_rn(a, g.p[k][i]);
+        reinterpret_cast<float*>(S)[i] = score_one(c, a, ws[i]);
+    }
+}
+
+// Any 4-byte alignment.
+__global__ void __launch_bounds__(256) score_scalar_kernel(const float* __restrict__ w, PtrArray<const float> g,
+                                                           int K, float c, uint64_t n, float* __restrict__ S) {
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        float a = g.p[0][i];
+        for (int k = 1; k < K; ++k) a = __fadd_rn(a, g.p[k][i]);
+        S[i] = score_one(c, a, w[i]);
+    }
+}
+
+}  // namespace
+
+slimdp_status launch_score(const float* w, const PtrArray<const float>& g, uint32_t K, float c, uint64_t n,
+                           float* S, bool vec, cudaStream_t st) {
+    const int sms = sm_count();
+    if (sms <= 0) return SLIMDP_ERR_CUDA;
+    if (!vec) {
+        uint64_t blocks = (n + 255) / 256;
+        if (blocks > (uint64_t)sms * 32) blocks = (uint64_t)sms * 32;
+        score_scalar_kernel<<<(unsigned)blocks, 256, 0, st>>>(w, g, (int)K, c, n, S);
+        SLIMDP_CHECK_LAUNCH();
+        return SLIMDP_OK;
+    }
+    const uint64_t n4 = n / 4;
+    uint64_t blocks = (n4 + 255) / 256;
+    if (blocks > (uint64_t)sms * 32) blocks = (uint64_t)sms * 32;
+    if (blocks == 0) blocks = 1;
+    const float4* w4 = reinterpret_cast<const float4*>(w);
+    float4* S4 = reinterpret_cast<float4*>(S);
+#define SLIMDP_SCORE_CASE(KK)                                                                        \
+    case KK:                                                                                         \
+        score_vec4_kernel<KK><<<(unsigned)blocks, 256, 0, st>>>(w4, g, (int)K, c, n4, n, S4);        \
+        break;
+    switch (K) {
+        SLIMDP_SCORE_CASE(1)
+        SLIMDP_SCORE_CASE(2)
+        SLIMDP_SCORE_CASE(4)
+        SLIMDP_SCORE_CASE(8)
+        SLIMDP_SCORE_CASE(16)
+        default:
+            score_vec4_kernel<0><<<(unsigned)blocks, 256, 0, st>>>(w4, g, (int)K, c, n4, n, S4);
+    }
+#undef SLIMDP_SCORE_CASE
+    SLIMDP_CHECK_LAUNCH();
+    return SLIMDP_OK;
+}
+
+}  // namespace slimdp

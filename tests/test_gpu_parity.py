@@ -1,0 +1,353 @@
+"""GPU parity: every C-ABI call against the CPU oracle, element by element,
+on the same seeded inputs.  Integer results (indices, bitmaps) and all fp32
+results (scores, packed values, merged model, pulled values) must match bit
+for bit: both sides use the same operation order (fp32 left-to-right worker
+sum, one fused multiply-add), so the tolerance is 0 ULP.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from workloads import CONFIGS, all_inputs, scaled_config
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def P():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    import paper_1709_09393_b200 as pkg
+    return pkg
+
+
+def dev(a: np.ndarray) -> torch.Tensor:
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint32:
+        a = a.view(np.int32)
+    return torch.from_numpy(a).cuda()
+
+
+def host_u32(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy().view(np.uint32)
+
+
+def host_bits(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy().view(np.uint32)
+
+
+def bits(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+def expected_aux(P, core: np.ndarray, n: int):
+    """core_aux by its definition: bitmap of the core, non-core counts before each 1024-block."""
+    nb = (n + 1023) // 1024
+    member = np.zeros(nb * 1024, np.uint8)
+    member[core] = 1
+    words = np.packbits(member.reshape(-1, 8), axis=1, bitorder="little").reshape(-1).view(np.uint32)
+    per_block = member.reshape(nb, 1024).sum(axis=1, dtype=np.int64)
+    sizes = np.full(nb, 1024, np.int64)
+    directory = np.zeros(nb + 1, np.int64)
+    directory[1:] = np.cumsum(sizes - per_block)
+    directory[nb] = n - core.size
+    return words, directory.astype(np.uint32)
+
+
+def gpu_select(P, S: np.ndarray, k: int):
+    n = S.size
+    scores = dev(S.astype(np.float32, copy=False))
+    core_idx = torch.empty(k, dtype=torch.int32, device="cuda")
+    aux = torch.empty(P.core_aux_bytes(n), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(P.select_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    P.slimdp_select_core(scores, k, core_idx, aux, ws)
+    P.read_status(ws)
+    return core_idx, aux
+
+
+def check_aux(P, aux: torch.Tensor, core: np.ndarray, n: int):
+    nb = (n + 1023) // 1024
+    raw = aux.cpu().numpy()
+    words, directory = expected_aux(P, core, n)
+    assert np.array_equal(raw[:nb * 128].view(np.uint32), words)
+    off = P.core_aux_dir_offset(n)
+    assert np.array_equal(raw[off:off + 4 * (nb + 1)].view(np.uint32), directory)
+
+
+# --------------------------------------------------------------------- score
+
+@pytest.mark.parametrize("n", [1, 3, 4, 5, 31, 1023, 1025, 100_007])
+@pytest.mark.parametrize("K", [1, 2, 3, 4, 8, 16, 17, 64])
+def test_score_parity(P, n, K):
+    rng = np.random.default_rng(n * 131 + K)
+    w = (rng.standard_normal(n) * 0.05).astype(np.float32)
+    gs = [(rng.standard_normal(n) * 1e-3).astype(np.float32) for _ in range(K)]
+    if n >= 31:
+        w[:8] = [np.inf, -np.inf, np.nan, 0.0, -0.0, 1e-42, -1e-45, 3e38]
+        gs[0][:8] = [0.0, 1.0, 0.0, np.nan, -0.0, 1e-44, 1e-45, 3e38]
+    c = 0.73
+    out = torch.empty(n, dtype=torch.float32, device="cuda")
+    P.slimdp_score(dev(w), [dev(g) for g in gs], c, out)
+    assert np.array_equal(host_bits(out), bits(oracle.score(w, gs, c)))
+
+
+def test_score_unaligned_views(P):
+    n, K = 10_001, 3
+    rng = np.random.default_rng(5)
+    w = rng.standard_normal(n + 3).astype(np.float32)
+    gs = [rng.standard_normal(n + 3).astype(np.float32) for _ in range(K)]
+    dw, dg = dev(w), [dev(g) for g in gs]
+    out = torch.zeros(n + 3, dtype=torch.float32, device="cuda")
+    # every buffer starts 4, 8 or 12 bytes past a 16-byte boundary
+    P.slimdp_score(dw[1:n + 1], [dg[0][2:n + 2], dg[1][3:n + 3], dg[2][1:n + 1]], 1.0, out[3:n + 3])
+    exp = oracle.score(w[1:n + 1], [gs[0][2:n + 2], gs[1][3:n + 3], gs[2][1:n + 1]], 1.0)
+    got = out.cpu().numpy()
+    assert np.array_equal(got[3:].view(np.uint32), bits(exp)) and np.all(got[:3] == 0)
+
+
+# -------------------------------------------------------------------- select
+
+def _score_patterns(n, rng):
+    yield "random", np.abs(rng.standard_normal(n)).astype(np.float32)
+    yield "all_equal", np.full(n, 0.25, np.float32)
+    yield "increasing", np.arange(n, dtype=np.float32)
+    yield "decreasing", np.arange(n, dtype=np.float32)[::-1].copy()
+    yield "two_values", rng.integers(0, 2, n).astype(np.float32)
+    yield "coarse_grid", (rng.integers(0, 37, n) * 2.0 ** -7).astype(np.float32)
+    s = np.abs(rng.standard_normal(n)).astype(np.float32)
+    s[rng.integers(0, n, max(1, n // 50))] = np.inf
+    s[rng.integers(0, n, max(1, n // 70))] = np.uint32(0x7FC00000).view(np.float32)
+    s[rng.integers(0, n, max(1, n // 30))] = 0.0
+    s[rng.integers(0, n, max(1, n // 40))] = 1e-42
+    yield "nonfinite_zero_denormal", s
+    yield "arbitrary_bit_patterns", rng.integers(0, 2 ** 32, n, dtype=np.uint64).astype(np.uint32).view(np.float32)
+
+
+@pytest.mark.parametrize("n", [1, 31, 32, 33, 1023, 1024, 1025, 4097, 100_007])
+def test_select_parity_small_and_adversarial(P, n):
+    rng = np.random.default_rng(n)
+    for name, S in _score_patterns(n, rng):
+        for k in sorted({0, 1, n // 10, n // 2, n - 1, n} - {-1}):
+            if k < 0 or k > n:
+                continue
+            core_idx, aux = gpu_select(P, S, k)
+            exp = oracle.select_core(S, k)
+            assert np.array_equal(host_u32(core_idx), exp), (name, n, k)
+            check_aux(P, aux, exp, n)
+
+
+def test_select_large_tie_group_spanning_many_blocks(P):
+    n, k = 3_000_000, 1_234_567
+    rng = np.random.default_rng(77)
+    S = (rng.integers(0, 5, n) * 0.125).astype(np.float32)     # 5 distinct scores, ~600k each
+    core_idx, aux = gpu_select(P, S, k)
+    exp = oracle.select_core(S, k)
+    assert np.array_equal(host_u32(core_idx), exp)
+    check_aux(P, aux, exp, n)
+
+
+# ------------------------------------------------------------------- explore
+
+def _gpu_core_aux(P, n, core: np.ndarray):
+    """Build core_aux on the device from a chosen core: scores 1 on the core, 0 elsewhere."""
+    S = np.zeros(n, np.float32)
+    S[core] = 1.0
+    core_idx, aux = gpu_select(P, S, core.size)
+    assert np.array_equal(host_u32(core_idx), core)
+    return aux
+
+
+@pytest.mark.parametrize("n,k_core,k_exp", [
+    (1, 0, 1), (2, 1, 1), (1000, 100, 45), (1000, 0, 1000), (1000, 1000, 0), (1000, 999, 1), (1024, 24, 1000),
+    (4097, 1234, 2863), (50_000, 5000, 2250), (100_007, 20_000, 4000), (1_000_003, 300_000, 7000),
+])
+def test_explore_parity(P, n, k_core, k_exp):
+    rng = np.random.default_rng(n + k_core)
+    core = np.sort(rng.choice(n, size=k_core, replace=False)).astype(np.uint32)
+    aux = _gpu_core_aux(P, n, core)
+    ws = torch.empty(P.explore_workspace_bytes(n, 1), dtype=torch.uint8, device="cuda")
+    for seed, worker, rnd in [(0, 0, 0), (2 ** 40 + 17, 3, 9), (2 ** 64 - 1, 63, 2 ** 32 - 1)]:
+        out = torch.empty(k_exp, dtype=torch.int32, device="cuda")
+        P.slimdp_sample_explore(aux, n, k_core, k_exp, seed, worker, rnd, out, ws)
+        P.read_status(ws)
+        assert np.array_equal(host_u32(out), oracle.sample_explore(core, n, k_exp, seed, worker, rnd))
+
+
+def test_explore_batched_equals_single_calls(P):
+    n, k_core, k_exp, K = 300_000, 30_000, 13_500, 16
+    rng = np.random.default_rng(3)
+    core = np.sort(rng.choice(n, size=k_core, replace=False)).astype(np.uint32)
+    aux = _gpu_core_aux(P, n, core)
+    ws = torch.empty(P.explore_workspace_bytes(n, K), dtype=torch.uint8, device="cuda")
+    outs = [torch.empty(k_exp, dtype=torch.int32, device="cuda") for _ in range(K)]
+    P.slimdp_sample_explore_batched(aux, n, k_core, k_exp, 9, 5, 2, outs, ws)
+    P.read_status(ws)
+    for k in range(K):
+        assert np.array_equal(host_u32(outs[k]), oracle.sample_explore(core, n, k_exp, 9, 5 + k, 2))
+
+
+# --------------------------------------------------------- pack / merge / pull
+
+@pytest.mark.parametrize("n,k_core,k_exp,K", [(1, 1, 0, 1), (1, 0, 1, 2), (1000, 0, 0, 2), (1000, 100, 45, 4),
+                                               (100_007, 20_000, 4000, 3), (100_007, 0, 100_007, 2),
+                                               (100_007, 100_007, 0, 64), (300_001, 100_000, 200_001, 5)])
+def test_pack_merge_pull_parity(P, n, k_core, k_exp, K):
+    rng = np.random.default_rng(n + K)
+    w = rng.standard_normal(n).astype(np.float32)
+    ds = [(rng.standard_normal(n) * 0.1).astype(np.float32) for _ in range(K)]
+    core = np.sort(rng.choice(n, size=k_core, replace=False)).astype(np.uint32)
+    rest = np.setdiff1d(np.arange(n, dtype=np.uint32), core)
+    exps = [np.sort(rng.choice(rest, size=k_exp, replace=False)).astype(np.uint32) for _ in range(K)]
+    eta = 0.3
+    d_core, d_exps, d_ds = dev(core), [dev(e) for e in exps], [dev(d) for d in ds]
+    m = k_core + k_exp
+    vals = [torch.empty(m, dtype=torch.float32, device="cuda") for _ in range(K)]
+    # single-worker calls and the batched call must agree with the oracle
+    for k in range(K):
+        P.slimdp_pack(d_ds[k], d_core, d_exps[k], vals[k])
+    exp_vals = [oracle.pack(ds[k], core, exps[k]) for k in range(K)]
+    for k in range(K):
+        assert np.array_equal(host_bits(vals[k]), bits(exp_vals[k]))
+    vals_b = [torch.zeros(m, dtype=torch.float32, device="cuda") for _ in range(K)]
+    P.slimdp_pack_batched(d_ds, d_core, d_exps, vals_b)
+    for k in range(K):
+        assert np.array_equal(host_bits(vals_b[k]), bits(exp_vals[k]))
+    d_w = dev(w)
+    P.slimdp_merge(d_w, d_core, d_exps, vals, eta)
+    exp_w = oracle.merge(w, core, exps, exp_vals, eta)
+    assert np.array_equal(host_bits(d_w), bits(exp_w))
+    outs = [torch.empty(m, dtype=torch.float32, device="cuda") for _ in range(K)]
+    P.slimdp_pull_batched(d_w, d_core, d_exps, outs)
+    one = torch.empty(m, dtype=torch.float32, device="cuda")
+    for k in range(K):
+        exp_out = oracle.pull(exp_w, core, exps[k])
+        assert np.array_equal(host_bits(outs[k]), bits(exp_out))
+        P.slimdp_pull(d_w, d_core, d_exps[k], one)
+        assert np.array_equal(host_bits(one), bits(exp_out))
+
+
+def test_merge_collisions_follow_worker_order(P):
+    # every worker's explorer is the same set: each parameter receives K updates in ascending k
+    n, K = 50_000, 7
+    rng = np.random.default_rng(21)
+    w = rng.standard_normal(n).astype(np.float32)
+    exp = np.sort(rng.choice(n, size=20_000, replace=False)).astype(np.uint32)
+    vals = [rng.standard_normal(exp.size).astype(np.float32) for _ in range(K)]
+    none = np.zeros(0, np.uint32)
+    d_w = dev(w)
+    P.slimdp_merge(d_w, dev(none), [dev(exp)] * K, [dev(v) for v in vals], 1.0 / 3.0)
+    fwd = oracle.merge(w, none, [exp] * K, vals, 1.0 / 3.0)
+    rev = oracle.merge(w, none, [exp] * K, vals[::-1], 1.0 / 3.0)
+    assert not np.array_equal(bits(fwd), bits(rev))        # the order matters for these values
+    assert np.array_equal(host_bits(d_w), bits(fwd))
+
+
+# --------------------------------------------------------------- whole round
+
+def gpu_round(P, w, gs, cfg_c, k_core, k_exp, seed, rnd, eta):
+    n, K = w.size, len(gs)
+    buf = P.RoundBuffers(n, K, k_core, k_exp)
+    d_w, d_gs = dev(w), [dev(g) for g in gs]
+    P.run_round(d_w, d_gs, cfg_c, seed, rnd, eta, buf)
+    P.read_status(buf.select_ws)
+    P.read_status(buf.explore_ws)
+    return d_w, buf
+
+
+def assert_round_equal(P, d_w, buf, ref, n):
+    assert np.array_equal(host_bits(buf.scores), bits(ref["scores"])), "scores"
+    assert np.array_equal(host_u32(buf.core_idx), ref["core_idx"]), "core_idx"
+    check_aux(P, buf.core_aux, ref["core_idx"], n)
+    for k in range(buf.K):
+        assert np.array_equal(host_u32(buf.exp_idx[k]), ref["exp_idx"][k]), f"exp_idx[{k}]"
+        assert np.array_equal(host_bits(buf.val[k]), bits(ref["val"][k])), f"val[{k}]"
+        assert np.array_equal(host_bits(buf.pulled[k]), bits(ref["pulled"][k])), f"pulled[{k}]"
+    assert np.array_equal(host_bits(d_w), bits(ref["w"])), "merged model"
+
+
+def _round_case(P, cfg, rnd=0):
+    w, gs = all_inputs(cfg)
+    ref = oracle.run_round(w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta)
+    d_w, buf = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta)
+    assert_round_equal(P, d_w, buf, ref, cfg.N)
+    return w, gs, ref
+
+
+@pytest.mark.parametrize("rnd", [0, 1, 2])
+def test_round_tiny(P, rnd):
+    _round_case(P, CONFIGS["tiny"], rnd)
+
+
+def test_round_googlenet_shaped(P):
+    _round_case(P, CONFIGS["googlenet"])
+
+
+def test_round_resnet50_tie_stress(P):
+    cfg = CONFIGS["resnet50_ties"]
+    w, gs, ref = _round_case(P, cfg)
+    # the recipe really does produce a large tie group at the threshold
+    S = ref["scores"]
+    thr = S[ref["core_idx"]].min()
+    assert np.count_nonzero(S == thr) > 1000
+
+
+def test_round_vgg16_shaped_full_size(P):
+    _round_case(P, CONFIGS["vgg16"])
+
+
+@pytest.mark.parametrize("case", ["beta_zero", "beta_equals_alpha", "everything_core", "everything_explored",
+                                  "core_plus_rest"])
+def test_round_degenerate_ratios(P, case):
+    cfg = scaled_config(CONFIGS["googlenet"], 200_003)
+    w, gs = all_inputs(cfg)
+    n = cfg.N
+    k_core, k_exp = {"beta_zero": (0, 30_000), "beta_equals_alpha": (30_000, 0), "everything_core": (n, 0),
+                     "everything_explored": (0, n), "core_plus_rest": (12_345, n - 12_345)}[case]
+    ref = oracle.run_round(w, gs, 1.0, k_core, k_exp, 5, 1, cfg.eta)
+    d_w, buf = gpu_round(P, w, gs, 1.0, k_core, k_exp, 5, 1, cfg.eta)
+    assert_round_equal(P, d_w, buf, ref, n)
+    if k_core + k_exp == n:       # 100 % communication ratio: the dense Plump-DP merge
+        assert np.array_equal(host_bits(d_w), bits(oracle.dense_merge(w, gs, cfg.eta)))
+
+
+def test_round_is_deterministic(P):
+    cfg = CONFIGS["tiny"]
+    w, gs = all_inputs(cfg)
+    a_w, a = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 0, cfg.eta)
+    b_w, b = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 0, cfg.eta)
+    assert torch.equal(a_w, b_w) and torch.equal(a.core_idx, b.core_idx) and torch.equal(a.core_aux, b.core_aux)
+    for k in range(cfg.K):
+        assert torch.equal(a.exp_idx[k], b.exp_idx[k]) and torch.equal(a.pulled[k], b.pulled[k])
+
+
+def test_round_on_host_buffers(P):
+    cfg = scaled_config(CONFIGS["vgg16"], 3_000_017)
+    w, gs = all_inputs(cfg)
+    ref = oracle.run_round(w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 0, cfg.eta)
+    pin = lambda a: torch.from_numpy(a.view(np.int32) if a.dtype == np.uint32 else a).pin_memory()
+    w_h = pin(w.copy())
+    g_h = [pin(g) for g in gs]
+    core_h = torch.empty(cfg.k_core, dtype=torch.int32).pin_memory()
+    exp_h = [torch.empty(cfg.k_exp, dtype=torch.int32).pin_memory() for _ in range(cfg.K)]
+    pulled_h = [torch.empty(cfg.m, dtype=torch.float32).pin_memory() for _ in range(cfg.K)]
+    arena = torch.empty(P.round_arena_bytes(cfg.N, cfg.K, cfg.k_core, cfg.k_exp), dtype=torch.uint8, device="cuda")
+    P.slimdp_round_host(w_h, g_h, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 0, cfg.eta, core_h, exp_h, pulled_h, arena)
+    assert np.array_equal(w_h.numpy().view(np.uint32), bits(ref["w"]))
+    assert np.array_equal(core_h.numpy().view(np.uint32), ref["core_idx"])
+    for k in range(cfg.K):
+        assert np.array_equal(exp_h[k].numpy().view(np.uint32), ref["exp_idx"][k])
+        assert np.array_equal(pulled_h[k].numpy().view(np.uint32), bits(ref["pulled"][k]))
+
+
+def test_untouched_parameters_keep_their_bits(P):
+    cfg = CONFIGS["tiny"]
+    w, gs = all_inputs(cfg)
+    d_w, buf = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 0, cfg.eta)
+    touched = np.zeros(cfg.N, bool)
+    touched[host_u32(buf.core_idx)] = True
+    for k in range(cfg.K):
+        e = host_u32(buf.exp_idx[k])
+        assert np.intersect1d(e, host_u32(buf.core_idx)).size == 0
+        touched[e] = True
+    got = d_w.cpu().numpy()
+    assert np.array_equal(got[~touched].view(np.uint32), w[~touched].view(np.uint32))
