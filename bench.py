@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of one Slim-DP communication round on B200.
+
+A step is one whole round (score, select, K x explore, K x pack, merge,
+K x pull) over the VGG-16-shaped synthetic workload, every step a C-ABI call
+sequence of the CUDA library.  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+N > 1 (under torchrun): the round does not shard (K workers are buffers on one
+GPU, there is no exchange step), so every rank runs an independent replica of
+the same workload; value = N * params / max-over-ranks time ("weak").
+--impl reference times the CPU oracle on a bounded sample of the workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "Gparams/s per Slim-DP round (score+select+pack+merge) and % of HBM roofline"
+UNIT = "Gparams/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+CPU_BASELINE_SAMPLE = 1 << 25      # leading parameters of the workload for the cpu_baseline leg
+REFERENCE_BUDGET_S = 120.0         # wall-clock target of a whole --impl reference run
+
+
+# ------------------------------------------------------------ byte model ---
+
+def model_bytes(N: int, K: int, k_core: int, k_exp: int) -> dict:
+    """Algorithmic bytes per step: every input element the method must examine
+    read once, every output written once, gathers / scatters at 4 B per element."""
+    m = k_core + k_exp
+    b = {
+        "score": 4 * N * (K + 1) + 4 * N,
+        "select": 4 * N + 4 * k_core + N // 8,
+        "explore": K * (N // 8 + 4 * k_exp),
+        "pack": K * 12 * m,
+        "merge": 4 * k_core + 8 * k_core + 4 * K * k_core + K * 16 * k_exp,
+        "pull": K * 12 * m,
+    }
+    b["round"] = sum(b.values())
+    b["round_without_score"] = b["round"] - b["score"]
+    return b
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "MEASURED_PEAKS.json hbm_gbs (of measured)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "profiling-recipe fallback 6.65 TB/s (of fallback)"
+
+
+# --------------------------------------------------------- clock sampling ---
+
+_REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+            0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, torch_device_index: int, period_s: float = 0.01):
+        self.period = period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self.handle = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(torch_device_index).uuid)
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+                idx = int(vis.split(",")[torch_device_index]) if vis else torch_device_index
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.handle = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
+                for bit, name in _REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.handle is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self) -> dict:
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------- multi-rank glue ---
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(value_ms: float, world: int, device=None) -> float:
+    """Max of a per-rank duration over all ranks (the job is as slow as its slowest replica)."""
+    if world == 1:
+        return value_ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(params_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job Gparams/s: all ranks' parameters over the slowest rank's step time."""
+    return params_per_rank * world / (ms_per_step * 1e-3) / 1e9
+
+
+# ------------------------------------------------------------ CPU oracle ---
+
+def time_oracle(cfg, n_sample: int, steps: int, warmup: int):
+    import oracle
+    from workloads import all_inputs, scaled_config
+    sample = scaled_config(cfg, n_sample)
+    w, gs = all_inputs(sample)
+    times = []
+    for s in range(warmup + steps):
+        t0 = time.perf_counter()
+        r = oracle.run_round(w, gs, sample.c, sample.k_core, sample.k_exp, sample.seed, s, sample.eta)
+        dt = time.perf_counter() - t0
+        w = r["w"]
+        if s >= warmup:
+            times.append(dt)
+    return sample, times
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    from workloads import CONFIGS
+    cfg = CONFIGS[args.config]
+    # size the per-step sample from a short probe so that warmup + steps rounds fit the budget
+    probe, probe_t = time_oracle(cfg, 1 << 20, 1, 0)
+    per_step = REFERENCE_BUDGET_S / (args.steps + args.warmup)
+    n_sample = 1 << 16
+    while n_sample * 2 <= min(cfg.N, 1 << 25) and (n_sample * 2) * 1.3 * probe_t[0] / probe.N <= per_step:
+        n_sample *= 2
+    sample, times = time_oracle(cfg, n_sample, args.steps, args.warmup)
+    ms = 1e3 * sum(times) / len(times)
+    value = sample.N / (ms * 1e-3) / 1e9
+    desc = (f"leading {sample.N} parameters of the {cfg.name}-shaped workload (K={sample.K}, "
+            f"k_core={sample.k_core}, k_exp={sample.k_exp}), one oracle round per step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ ours ---
+
+def run_ours(args):
+    import numpy as np
+    import torch
+
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl")
+    torch.cuda.set_device(local_rank if world > 1 else 0)
+    device = torch.device("cuda", torch.cuda.current_device())
+
+    import paper_1709_09393_b200 as P
+    from workloads import CONFIGS, all_inputs
+
+    cfg = CONFIGS[args.config]
+    N, K, k_core, k_exp, m = cfg.N, cfg.K, cfg.k_core, cfg.k_exp, cfg.m
+    w_host, g_host = all_inputs(cfg)
+    w = torch.from_numpy(w_host).to(device)
+    grads = [torch.from_numpy(g).to(device) for g in g_host]
+    buf = P.RoundBuffers(N, K, k_core, k_exp, device)
+    bytes_model = model_bytes(N, K, k_core, k_exp)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+
+    def round_after_score(t):
+        P.slimdp_select_core(buf.scores, k_core, buf.core_idx, buf.core_aux, buf.select_ws)
+        P.slimdp_sample_explore_batched(buf.core_aux, N, k_core, k_exp, cfg.seed, 0, t, buf.exp_idx, buf.explore_ws)
+        P.slimdp_pack_batched(grads, buf.core_idx, buf.exp_idx, buf.val)
+        P.slimdp_merge(w, buf.core_idx, buf.exp_idx, buf.val, cfg.eta)
+        P.slimdp_pull_batched(w, buf.core_idx, buf.exp_idx, buf.pulled)
+
+    # warm-up: successive rounds t = 0, 1, ... on the evolving model, as in training
+    t = 0
+    for _ in range(args.warmup):
+        P.slimdp_score(w, grads, cfg.c, buf.scores)
+        round_after_score(t)
+        t += 1
+    torch.cuda.synchronize()
+    P.read_status(buf.select_ws)
+    P.read_status(buf.explore_ws)
+
+    # ---- timed region: exactly `steps` rounds, device-timed -----------------
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    ev_start, ev_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(torch.cuda.current_device())
+    launches0 = P.launch_count()
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev_start.record()
+    for s in range(args.steps):
+        ev[s][0].record()
+        P.slimdp_score(w, grads, cfg.c, buf.scores)
+        ev[s][1].record()
+        round_after_score(t)
+        t += 1
+    ev_end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    barrier()
+    launches = P.launch_count() - launches0
+    P.read_status(buf.select_ws)
+    P.read_status(buf.explore_ws)
+    total_ms = max_over_ranks(ev_start.elapsed_time(ev_end), world, device)
+    ms_per_step = total_ms / args.steps
+    score_ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
+    value = aggregate_value(N, world, ms_per_step)
+
+    # ---- per-call breakdown (untimed for the headline; 5 more rounds) -------
+    names = ["score", "select", "explore", "pack", "merge", "pull"]
+    acc = {nm: [] for nm in names}
+    for _ in range(5):
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(7)]
+        marks[0].record()
+        P.slimdp_score(w, grads, cfg.c, buf.scores); marks[1].record()
+        P.slimdp_select_core(buf.scores, k_core, buf.core_idx, buf.core_aux, buf.select_ws); marks[2].record()
+        P.slimdp_sample_explore_batched(buf.core_aux, N, k_core, k_exp, cfg.seed, 0, t, buf.exp_idx, buf.explore_ws)
+        marks[3].record()
+        P.slimdp_pack_batched(grads, buf.core_idx, buf.exp_idx, buf.val); marks[4].record()
+        P.slimdp_merge(w, buf.core_idx, buf.exp_idx, buf.val, cfg.eta); marks[5].record()
+        P.slimdp_pull_batched(w, buf.core_idx, buf.exp_idx, buf.pulled); marks[6].record()
+        torch.cuda.synchronize()
+        t += 1
+        for i, nm in enumerate(names):
+            acc[nm].append(marks[i].elapsed_time(marks[i + 1]) * 1e3)
+    breakdown_us = {nm: round(statistics.median(v), 1) for nm, v in acc.items()}
+
+    peak, peak_src = measured_peak()
+    achieved = bytes_model["score"] / (score_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": f"score_vec4_kernel<{K}>", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "traffic": TRAFFIC_SCORE_BYTES.get(cfg.name),
+                "algorithmic_bytes_per_launch": bytes_model["score"], "avg_launch_ms": score_ms,
+                "peak_source": peak_src}
+    round_gbs = bytes_model["round"] / (ms_per_step * 1e-3) / 1e9
+    rest_ms = ms_per_step - score_ms
+    rest_gbs = bytes_model["round_without_score"] / (rest_ms * 1e-3) / 1e9
+    round_roofline = {
+        "model_bytes": bytes_model["round"], "achieved_gbs": round_gbs,
+        "frac_of_8TBs": round_gbs / NOMINAL_HBM_GBS, "frac_of_measured": round_gbs / peak,
+        "without_score": {"model_bytes": bytes_model["round_without_score"], "ms": rest_ms, "achieved_gbs": rest_gbs,
+                          "frac_of_8TBs": rest_gbs / NOMINAL_HBM_GBS, "frac_of_measured": rest_gbs / peak},
+    }
+
+    # ---- end to end: host buffers through the C ABI, copies inside the timed region
+    e2e = None
+    if rank == 0 or world > 1:
+        pin = lambda a: torch.from_numpy(a).pin_memory()
+        w_pin = pin(w_host.copy())
+        g_pin = [pin(g) for g in g_host]
+        core_pin = torch.empty(k_core, dtype=torch.int32).pin_memory()
+        exp_pin = [torch.empty(k_exp, dtype=torch.int32).pin_memory() for _ in range(K)]
+        pulled_pin = [torch.empty(m, dtype=torch.float32).pin_memory() for _ in range(K)]
+        del buf
+        torch.cuda.empty_cache()
+        arena = torch.empty(P.round_arena_bytes(N, K, k_core, k_exp), dtype=torch.uint8, device=device)
+        e2e_steps = max(1, min(args.steps, 5))
+        P.slimdp_round_host(w_pin, g_pin, cfg.c, k_core, k_exp, cfg.seed, 0, cfg.eta, core_pin, exp_pin, pulled_pin,
+                            arena)      # warm-up
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        torch.cuda.synchronize()
+        e0.record()
+        for s in range(e2e_steps):
+            P.slimdp_round_host(w_pin, g_pin, cfg.c, k_core, k_exp, cfg.seed, 1 + s, cfg.eta, core_pin, exp_pin,
+                                pulled_pin, arena)
+        e1.record()
+        torch.cuda.synchronize()
+        barrier()
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, device) / e2e_steps
+        e2e = {"value": aggregate_value(N, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms, "steps": e2e_steps,
+               "h2d_bytes_per_step": 4 * N * (K + 1),
+               "d2h_bytes_per_step": 4 * N + 4 * k_core + K * (4 * k_exp + 4 * m)}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample, times = time_oracle(cfg, CPU_BASELINE_SAMPLE, 1, 0)
+        cpu_baseline = {"value": sample.N / times[0] / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "seconds": times[0],
+                        "sample": f"one oracle round on the leading {sample.N} parameters of the {cfg.name}-shaped "
+                                  f"workload (K={sample.K}, k_core={sample.k_core}, k_exp={sample.k_exp})"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}-shaped: N={N} fp32 parameters, K={K} workers, k_core={k_core} "
+                                   f"({cfg.core_pct}%), k_exp={k_exp} ({cfg.explore_pct}% of the non-core)",
+                       "N": N, "K": K, "k_core": k_core, "k_exp": k_exp, "seed": cfg.seed,
+                       "l2": "inputs larger than L2 (no flush needed)" if 4 * N * (K + 1) > 4 * 126e6
+                       else "inputs fit L2 (warm)",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+            "round_roofline": round_roofline, "breakdown_us": breakdown_us, "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+# DRAM bytes (read + write) of one score launch from an ncu capture, per workload;
+# absent until a capture of the current kernel exists.
+TRAFFIC_SCORE_BYTES: dict = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="vgg16")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

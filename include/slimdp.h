@@ -204,6 +204,11 @@ slimdp_status slimdp_pull_batched(const float* w_global, uint32_t K, uint64_t n,
  * (the outputs of that call are then undefined), or SLIMDP_ERR_CUDA. */
 slimdp_status slimdp_read_status(const void* ws, void* stream);
 
+/* Number of kernels this library has launched in this process so far (all
+ * devices, all streams).  An accounting aid for benchmarks: read it before and
+ * after a timed region.  The paper has no counterpart. */
+uint64_t slimdp_launch_count(void);
+
 /* ----------------------------------------------------- whole round, host ---
  * One whole round (score, select, K x explore, K x pack, merge, K x pull) on
  * HOST buffers: copies w and the K updates to the device, runs the round

@@ -46,6 +46,7 @@ EXPORTS = {
     "slimdp_pull": (ctypes.c_int32, [_vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp]),
     "slimdp_pull_batched": (ctypes.c_int32, [_vp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _vp]),
     "slimdp_read_status": (ctypes.c_int32, [_vp, _vp]),
+    "slimdp_launch_count": (_u64, []),
     "slimdp_round_arena_bytes": (_sz, [_u64, _u32, _u64, _u64]),
     "slimdp_round_host": (ctypes.c_int32, [_vp, _pp, _u32, _u64, _f32, _u64, _u64, _u64, _u32, _f32, _vp, _pp, _pp,
                                            _vp, _sz, _vp]),
@@ -116,6 +117,11 @@ def workspace_bytes(n: int, K: int) -> int:
 
 def round_arena_bytes(n: int, K: int, k_core: int, k_exp: int) -> int:
     return lib.slimdp_round_arena_bytes(n, K, k_core, k_exp)
+
+
+def launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return lib.slimdp_launch_count()
 
 
 def read_status(ws: torch.Tensor, stream=None) -> None:

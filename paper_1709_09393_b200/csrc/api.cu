@@ -3,6 +3,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "layout.cuh"
 
@@ -21,6 +23,10 @@ slimdp_status launch_gather(const PtrArray<const float>& src, uint32_t workers, 
 slimdp_status launch_merge(float* w, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
                            const PtrArray<const uint32_t>& exp, uint64_t k_exp, const PtrArray<const float>& val,
                            float eta, cudaStream_t st);
+
+static std::atomic<unsigned long long> g_launches{0};
+
+void count_launches(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 int sm_count() {
     static int cached[64];
@@ -204,6 +210,8 @@ slimdp_status slimdp_merge(float* w_global, uint64_t n, uint32_t K, const uint32
     if (k_core + k_exp == 0) return SLIMDP_OK;
     return launch_merge(w_global, K, core_idx, k_core, exp, k_exp, v, eta, (cudaStream_t)stream);
 }
+
+uint64_t slimdp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 slimdp_status slimdp_read_status(const void* ws, void* stream) {
     if (!ws) return SLIMDP_ERR_INVALID_ARG;

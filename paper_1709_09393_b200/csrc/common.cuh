@@ -35,12 +35,17 @@ inline uint64_t num_scan_tiles(uint64_t n) { return (num_blocks(n) + kScanTile -
 // Number of SMs of the current device (cached per device id).
 int sm_count();
 
+// Adds n to the process-wide count of launched kernels.
+void count_launches(unsigned n);
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
-#define SLIMDP_CHECK_LAUNCH()                                   \
-    do {                                                        \
-        if (cudaGetLastError() != cudaSuccess) return SLIMDP_ERR_CUDA; \
+// After a group of `count` kernel launches: fail on a launch error, else count them.
+#define SLIMDP_LAUNCHED(count)                                          \
+    do {                                                                \
+        if (cudaGetLastError() != cudaSuccess) return SLIMDP_ERR_CUDA;  \
+        count_launches(count);                                          \
     } while (0)
 
 // ---- device helpers -------------------------------------------------------

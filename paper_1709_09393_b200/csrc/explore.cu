@@ -176,7 +176,7 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
 
     explore_setup_kernel<<<1, 256, 0, st>>>(L.hdr, L.round_keys, (uint32_t)seed, (uint32_t)(seed >> 32),
                                             first_worker, workers, round);
-    SLIMDP_CHECK_LAUNCH();
+    SLIMDP_LAUNCHED(1);
     if (k_exp == 0) return SLIMDP_OK;
     if (cudaMemsetAsync(L.marks, 0, (size_t)workers * L.mark_stride * 4, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
 
@@ -189,20 +189,20 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
     mark_kernel<<<dim3((unsigned)mgrid, workers), 256, 0, st>>>(bitmap, dir, (uint32_t)nb, (uint32_t)M,
                                                                 (uint32_t)k_exp, h, L.round_keys, L.marks,
                                                                 L.mark_stride, L.hdr);
-    SLIMDP_CHECK_LAUNCH();
+    SLIMDP_LAUNCHED(1);
     uint64_t cgrid = (nb + 7) / 8;
     const uint64_t cap = ((uint64_t)sms * 8 + workers - 1) / workers;
     if (cgrid > cap) cgrid = cap;
     if (cgrid == 0) cgrid = 1;
     count_marks_kernel<<<dim3((unsigned)cgrid, workers), 256, 0, st>>>(L.marks, L.mark_stride, nb, L.cnt,
                                                                        L.cnt_stride);
-    SLIMDP_CHECK_LAUNCH();
+    SLIMDP_LAUNCHED(1);
     slimdp_status s =
         launch_block_scan(L.cnt, L.pref, L.tile_sums, L.totals, nb, workers, L.cnt_stride, L.tile_stride, st);
     if (s != SLIMDP_OK) return s;
     expand_marks_kernel<<<dim3((unsigned)cgrid, workers), 256, 0, st>>>(L.marks, L.mark_stride, nb, L.pref, L.totals,
                                                                         L.cnt_stride, (uint32_t)k_exp, out, L.hdr);
-    SLIMDP_CHECK_LAUNCH();
+    SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }
 

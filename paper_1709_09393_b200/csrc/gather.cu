@@ -52,7 +52,7 @@ slimdp_status launch_gather(const PtrArray<const float>& src, uint32_t workers, 
     const uint64_t cap = ((uint64_t)sms * 32 + workers - 1) / workers;
     if (grid > cap) grid = cap;
     gather_kernel<<<dim3((unsigned)grid, workers), 256, 0, st>>>(src, core_idx, k_core, exp, k_exp, out);
-    SLIMDP_CHECK_LAUNCH();
+    SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }
 

@@ -48,14 +48,14 @@ slimdp_status launch_merge(float* w, uint32_t K, const uint32_t* core_idx, uint6
         uint64_t grid = (k_core + 255) / 256;
         if (grid > (uint64_t)sms * 32) grid = (uint64_t)sms * 32;
         merge_core_kernel<<<(unsigned)grid, 256, 0, st>>>(w, core_idx, k_core, val, (int)K, neg_eta);
-        SLIMDP_CHECK_LAUNCH();
+        SLIMDP_LAUNCHED(1);
     }
     if (k_exp > 0) {
         uint64_t grid = (k_exp + 255) / 256;
         if (grid > (uint64_t)sms * 32) grid = (uint64_t)sms * 32;
         for (uint32_t k = 0; k < K; ++k) {
             merge_explore_kernel<<<(unsigned)grid, 256, 0, st>>>(w, exp.p[k], k_exp, val.p[k] + k_core, neg_eta);
-            SLIMDP_CHECK_LAUNCH();
+            SLIMDP_LAUNCHED(1);
         }
     }
     return SLIMDP_OK;

@@ -46,9 +46,8 @@ slimdp_status launch_block_scan(const unsigned long long* cnt, unsigned long lon
     const uint32_t tiles = (uint32_t)((nb + kScanTile - 1) / kScanTile);
     dim3 grid(tiles, batch);
     tile_sum_kernel<<<grid, 1024, 0, st>>>(cnt, tile_sums, nb, stride, tile_stride);
-    SLIMDP_CHECK_LAUNCH();
     tile_scan_kernel<<<grid, 1024, 0, st>>>(cnt, tile_sums, pref, totals, nb, stride, tile_stride);
-    SLIMDP_CHECK_LAUNCH();
+    SLIMDP_LAUNCHED(2);
     return SLIMDP_OK;
 }
 

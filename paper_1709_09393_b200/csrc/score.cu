@@ -84,7 +84,7 @@ slimdp_status launch_score(const float* w, const PtrArray<const float>& g, uint3
         uint64_t blocks = (n + 255) / 256;
         if (blocks > (uint64_t)sms * 32) blocks = (uint64_t)sms * 32;
         score_scalar_kernel<<<(unsigned)blocks, 256, 0, st>>>(w, g, (int)K, c, n, S);
-        SLIMDP_CHECK_LAUNCH();
+        SLIMDP_LAUNCHED(1);
         return SLIMDP_OK;
     }
     const uint64_t n4 = n / 4;
@@ -107,7 +107,7 @@ slimdp_status launch_score(const float* w, const PtrArray<const float>& g, uint3
             score_vec4_kernel<0><<<(unsigned)blocks, 256, 0, st>>>(w4, g, (int)K, c, n4, n, S4);
     }
 #undef SLIMDP_SCORE_CASE
-    SLIMDP_CHECK_LAUNCH();
+    SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }
 

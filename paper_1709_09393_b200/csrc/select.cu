@@ -227,7 +227,7 @@ slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, ui
     uint32_t* dir = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(core_aux) + slimdp_core_aux_dir_offset(n));
 
     select_init_kernel<<<1, 1, 0, st>>>(L.hdr, (uint32_t)k_core);
-    SLIMDP_CHECK_LAUNCH();
+    SLIMDP_LAUNCHED(1);
     if (k_core > 0) {
         if (cudaMemsetAsync(L.hist, 0, 3 * kBins0 * sizeof(uint32_t), st) != cudaSuccess) return SLIMDP_ERR_CUDA;
         const unsigned hgrid = (unsigned)sms * 4;
@@ -237,17 +237,17 @@ slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, ui
         find_bin_kernel<1><<<1, 1024, 0, st>>>(L.hdr, L.hist + kBins0);
         hist_kernel<2><<<hgrid, kHistThreads, 0, st>>>(keys, n, L.hdr, L.hist + 2 * kBins0);
         find_bin_kernel<2><<<1, 1024, 0, st>>>(L.hdr, L.hist + 2 * kBins0);
-        SLIMDP_CHECK_LAUNCH();
+        SLIMDP_LAUNCHED(6);
     }
     uint64_t cgrid = (nb + 7) / 8;
     if (cgrid > (uint64_t)sms * 8) cgrid = (uint64_t)sms * 8;
     classify_kernel<<<(unsigned)cgrid, 256, 0, st>>>(keys, n, nb, L.hdr, L.G, L.E, L.cnt);
-    SLIMDP_CHECK_LAUNCH();
+    SLIMDP_LAUNCHED(1);
     slimdp_status s = launch_block_scan(L.cnt, L.pref, L.tile_sums, L.totals, nb, 1, nb, num_scan_tiles(n), st);
     if (s != SLIMDP_OK) return s;
     emit_kernel<<<(unsigned)cgrid, 256, 0, st>>>(L.G, L.E, L.pref, L.totals, n, nb, (uint32_t)k_core, L.hdr,
                                                  core_idx, bitmap, dir);
-    SLIMDP_CHECK_LAUNCH();
+    SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }
 
