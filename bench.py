@@ -207,6 +207,9 @@ def run_ours(args):
     from workloads import CONFIGS, all_inputs
 
     cfg = CONFIGS[args.config]
+    if args.scale:
+        from workloads import scaled_config
+        cfg = scaled_config(cfg, args.scale)     # leading parameters only: a small case for profiling
     N, K, k_core, k_exp, m = cfg.N, cfg.K, cfg.k_core, cfg.k_exp, cfg.m
     w_host, g_host = all_inputs(cfg)
     w = torch.from_numpy(w_host).to(device)
@@ -299,7 +302,7 @@ def run_ours(args):
 
     # ---- end to end: host buffers through the C ABI, copies inside the timed region
     e2e = None
-    if rank == 0 or world > 1:
+    if (rank == 0 or world > 1) and not args.no_e2e:
         pin = lambda a: torch.from_numpy(a).pin_memory()
         w_pin = pin(w_host.copy())
         g_pin = [pin(g) for g in g_host]
@@ -367,6 +370,9 @@ def main():
     ap.add_argument("--config", default="vgg16")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--scale", type=int, default=0,
+                    help="run on the leading SCALE parameters of the config (small case for profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

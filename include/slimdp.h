@@ -80,11 +80,12 @@ size_t slimdp_core_aux_dir_offset(uint64_t n);
 size_t slimdp_select_workspace_bytes(uint64_t n);
 
 /* Bytes of scratch that slimdp_sample_explore (num_workers = 1) or
- * slimdp_sample_explore_batched (num_workers workers in one call) needs. */
-size_t slimdp_explore_workspace_bytes(uint64_t n, uint32_t num_workers);
+ * slimdp_sample_explore_batched (num_workers workers in one call) needs to
+ * draw k_exp parameters per worker (any k_core). */
+size_t slimdp_explore_workspace_bytes(uint64_t n, uint64_t k_exp, uint32_t num_workers);
 
 /* max(select, explore for K workers): one workspace that serves every call of a round. */
-size_t slimdp_workspace_bytes(uint64_t n, uint32_t K);
+size_t slimdp_workspace_bytes(uint64_t n, uint64_t k_exp, uint32_t K);
 
 /* ---------------------------------------------------------------- score ---
  * Eq. 1 (Section 3.2).  For every i < n, in fp32:
@@ -135,7 +136,7 @@ slimdp_status slimdp_select_core(const float* scores, uint64_t n, uint64_t k_cor
  *   core_aux  as written by slimdp_select_core for the same n and k_core (read)
  *   k_exp     0 <= k_exp <= n - k_core
  *   exp_idx   [k_exp] (written): the explorer, ascending
- *   ws        [ws_bytes >= slimdp_explore_workspace_bytes(n, 1)] scratch
+ *   ws        [ws_bytes >= slimdp_explore_workspace_bytes(n, k_exp, 1)] scratch
  */
 slimdp_status slimdp_sample_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp,
                                     uint64_t seed, uint32_t worker, uint32_t round, uint32_t* exp_idx,
@@ -143,7 +144,7 @@ slimdp_status slimdp_sample_explore(const void* core_aux, uint64_t n, uint64_t k
 
 /* The same for workers first_worker .. first_worker + num_workers - 1 in one
  * call; exp_idx is a HOST array of num_workers device pointers, each [k_exp].
- * ws_bytes >= slimdp_explore_workspace_bytes(n, num_workers).  Results are
+ * ws_bytes >= slimdp_explore_workspace_bytes(n, k_exp, num_workers).  Results are
  * identical to num_workers single calls. */
 slimdp_status slimdp_sample_explore_batched(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp,
                                             uint64_t seed, uint32_t first_worker, uint32_t num_workers,

@@ -33,8 +33,8 @@ EXPORTS = {
     "slimdp_core_aux_bytes": (_sz, [_u64]),
     "slimdp_core_aux_dir_offset": (_sz, [_u64]),
     "slimdp_select_workspace_bytes": (_sz, [_u64]),
-    "slimdp_explore_workspace_bytes": (_sz, [_u64, _u32]),
-    "slimdp_workspace_bytes": (_sz, [_u64, _u32]),
+    "slimdp_explore_workspace_bytes": (_sz, [_u64, _u64, _u32]),
+    "slimdp_workspace_bytes": (_sz, [_u64, _u64, _u32]),
     "slimdp_score": (ctypes.c_int32, [_vp, _pp, _u32, _f32, _u64, _vp, _vp]),
     "slimdp_select_core": (ctypes.c_int32, [_vp, _u64, _u64, _vp, _vp, _vp, _sz, _vp]),
     "slimdp_sample_explore": (ctypes.c_int32, [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _vp, _vp, _sz, _vp]),
@@ -107,12 +107,12 @@ def select_workspace_bytes(n: int) -> int:
     return lib.slimdp_select_workspace_bytes(n)
 
 
-def explore_workspace_bytes(n: int, num_workers: int) -> int:
-    return lib.slimdp_explore_workspace_bytes(n, num_workers)
+def explore_workspace_bytes(n: int, k_exp: int, num_workers: int) -> int:
+    return lib.slimdp_explore_workspace_bytes(n, k_exp, num_workers)
 
 
-def workspace_bytes(n: int, K: int) -> int:
-    return lib.slimdp_workspace_bytes(n, K)
+def workspace_bytes(n: int, k_exp: int, K: int) -> int:
+    return lib.slimdp_workspace_bytes(n, k_exp, K)
 
 
 def round_arena_bytes(n: int, K: int, k_core: int, k_exp: int) -> int:

@@ -17,10 +17,10 @@ slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, ui
 slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                              uint32_t first_worker, uint32_t workers, uint32_t round,
                              const PtrArray<uint32_t>& out, void* ws, cudaStream_t st);
-slimdp_status launch_gather(const PtrArray<const float>& src, uint32_t workers, const uint32_t* core_idx,
-                            uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp,
-                            const PtrArray<float>& out, cudaStream_t st);
-slimdp_status launch_merge(float* w, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+slimdp_status launch_gather(const PtrArray<const float>& src, bool same_src, uint32_t workers,
+                            const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,
+                            uint64_t k_exp, const PtrArray<float>& out, cudaStream_t st);
+slimdp_status launch_merge(float* w, uint64_t n, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
                            const PtrArray<const uint32_t>& exp, uint64_t k_exp, const PtrArray<const float>& val,
                            float eta, cudaStream_t st);
 
@@ -96,13 +96,13 @@ size_t slimdp_select_workspace_bytes(uint64_t n) {
     return select_ws_layout(nullptr, n).bytes;
 }
 
-size_t slimdp_explore_workspace_bytes(uint64_t n, uint32_t num_workers) {
-    if (!n_ok(n) || !k_ok(num_workers)) return 0;
-    return explore_ws_layout(nullptr, n, num_workers).bytes;
+size_t slimdp_explore_workspace_bytes(uint64_t n, uint64_t k_exp, uint32_t num_workers) {
+    if (!n_ok(n) || k_exp > n || !k_ok(num_workers)) return 0;
+    return explore_ws_layout(nullptr, n, k_exp, num_workers).bytes;
 }
 
-size_t slimdp_workspace_bytes(uint64_t n, uint32_t K) {
-    const size_t a = slimdp_select_workspace_bytes(n), b = slimdp_explore_workspace_bytes(n, K);
+size_t slimdp_workspace_bytes(uint64_t n, uint64_t k_exp, uint32_t K) {
+    const size_t a = slimdp_select_workspace_bytes(n), b = slimdp_explore_workspace_bytes(n, k_exp, K);
     if (a == 0 || b == 0) return 0;
     return a > b ? a : b;
 }
@@ -137,7 +137,7 @@ slimdp_status slimdp_sample_explore_batched(const void* core_aux, uint64_t n, ui
     if (!aligned16(core_aux) || !aligned16(ws)) return SLIMDP_ERR_INVALID_ARG;
     PtrArray<uint32_t> out;
     if (!fill<uint32_t>(out, exp_idx, num_workers, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
-    if (ws_bytes < slimdp_explore_workspace_bytes(n, num_workers)) return SLIMDP_ERR_WORKSPACE;
+    if (ws_bytes < slimdp_explore_workspace_bytes(n, k_exp, num_workers)) return SLIMDP_ERR_WORKSPACE;
     return launch_explore(core_aux, n, k_core, k_exp, seed, first_worker, num_workers, round, out, ws,
                           (cudaStream_t)stream);
 }
@@ -167,7 +167,8 @@ static slimdp_status gather_common(const float* const* srcs, bool same_src, cons
     }
     if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
     if (!fill<float>(dst, out, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
-    return launch_gather(src, K, core_idx, k_core, exp, k_exp, dst, (cudaStream_t)stream);
+    if (k_core + k_exp == 0) return SLIMDP_OK;
+    return launch_gather(src, same_src, K, core_idx, k_core, exp, k_exp, dst, (cudaStream_t)stream);
 }
 
 slimdp_status slimdp_pack_batched(const float* const* deltas, uint32_t K, uint64_t n, const uint32_t* core_idx,
@@ -208,7 +209,7 @@ slimdp_status slimdp_merge(float* w_global, uint64_t n, uint32_t K, const uint32
     if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
     if (!fill<const float>(v, val, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (k_core + k_exp == 0) return SLIMDP_OK;
-    return launch_merge(w_global, K, core_idx, k_core, exp, k_exp, v, eta, (cudaStream_t)stream);
+    return launch_merge(w_global, n, K, core_idx, k_core, exp, k_exp, v, eta, (cudaStream_t)stream);
 }
 
 uint64_t slimdp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
@@ -259,7 +260,7 @@ Arena arena_layout(void* base, uint64_t n, uint32_t K, uint64_t k_core, uint64_t
     A.core_aux = take(slimdp_core_aux_bytes(n));
     A.select_ws_bytes = slimdp_select_workspace_bytes(n);
     A.select_ws = take(A.select_ws_bytes);
-    A.explore_ws_bytes = slimdp_explore_workspace_bytes(n, K);
+    A.explore_ws_bytes = slimdp_explore_workspace_bytes(n, k_exp, K);
     A.explore_ws = take(A.explore_ws_bytes);
     for (uint32_t k = 0; k < K; ++k) A.exp_idx[k] = reinterpret_cast<uint32_t*>(take(k_exp * 4));
     for (uint32_t k = 0; k < K; ++k) A.val[k] = reinterpret_cast<float*>(take(m * 4));

@@ -2,20 +2,34 @@
 // Section 3.3 step 2): k_exp distinct parameters drawn uniformly from outside
 // the core, anew for every worker and every communication round.
 //
-//   1. round keys: three Philox-4x32-10 blocks per worker;
-//   2. thread j evaluates the keyed permutation pi(j) of the non-core ranks
-//      (10-round Feistel network with cycle walking), turns the rank into a
-//      parameter index with a select-zero query on the core bitmap (binary
-//      search of the per-1024 rank directory, then a popcount walk over the 32
-//      words of the block) and sets that bit in the worker's mark bitmap;
-//   3. the mark bitmap is compacted into the ascending index list (per-block
-//      popcounts, two-kernel scan, warp-ordered expansion).
+// The explorer is { select0(pi(j)) : j < k_exp }, ascending, where pi is the
+// keyed permutation of the M non-core ranks and select0(r) the r-th non-core
+// parameter.  select0 is monotone, so sorting the ranks sorts the indices, and
+// the ranks are uniform on [0, M), so a bucket sort by the ranks' high bits
+// is balanced:
+//   1. setup: round keys (three Philox-4x32-10 blocks per worker);
+//   2. rank: thread j evaluates pi(j) (10-round Feistel network with cycle
+//      walking), stores it and counts it into its bucket (rank >> s);
+//   3. two-kernel exclusive scan of the bucket counts;
+//   4. scatter: every rank goes to its bucket's slice (order inside a bucket
+//      is arbitrary here and is fixed by the next step);
+//   5. bucket: one CTA per (bucket, worker) marks its ranks in a 2^s-bit
+//      shared-memory bitmap, which sorts them; a block scan of the popcounts
+//      gives each rank its output position, and a select0 query (binary
+//      search of the per-1024 non-core directory inside the bucket's block
+//      range, then a popcount walk over the block's 32 bitmap words) turns
+//      it into the parameter index.
+// No global bitmap, no inter-CTA waiting; the result does not depend on the
+// order in which atomics land.
 #include "common.cuh"
 #include "layout.cuh"
 
 namespace slimdp {
 
 namespace {
+
+constexpr int kBucketThreads = 256;
+constexpr uint64_t kMaxSmemBuckets = 5120;   // 20 KB / 40 KB of static-limit shared memory per CTA
 
 __device__ __forceinline__ void philox4x32_10(uint32_t k0, uint32_t k1, uint32_t c0, uint32_t c1, uint32_t c2,
                                               uint32_t c3, uint32_t out[4]) {
@@ -40,34 +54,84 @@ __device__ __forceinline__ void philox4x32_10(uint32_t k0, uint32_t k1, uint32_t
     out[3] = c3;
 }
 
-__global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, uint32_t seed_lo, uint32_t seed_hi,
-                                     uint32_t first_worker, uint32_t workers, uint32_t round) {
-    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
-    if (t == 0) hdr->status = SLIMDP_OK;
-    if (t >= workers * 3) return;
-    const uint32_t w = t / 3, b = t % 3;
-    uint32_t out[4];
-    philox4x32_10(seed_lo, seed_hi, b, first_worker + w, round, 0x534C494Du, out);
-#pragma unroll
-    for (int q = 0; q < 4; ++q) rk[w * 12 + b * 4 + q] = out[q];
+// Largest block b in [lo, hi] with dir[b] <= x (dir[lo] <= x is given).
+__device__ __forceinline__ uint32_t find_block(const uint32_t* __restrict__ dir, uint32_t lo, uint32_t hi,
+                                               uint32_t x) {
+    while (lo < hi) {
+        const uint32_t mid = lo + ((hi - lo + 1) >> 1);
+        if (__ldg(dir + mid) <= x)
+            lo = mid;
+        else
+            hi = mid - 1;
+    }
+    return lo;
 }
 
-__global__ void __launch_bounds__(256) mark_kernel(const uint32_t* __restrict__ bitmap,
-                                                   const uint32_t* __restrict__ dir, uint32_t nb, uint32_t M,
-                                                   uint32_t k_exp, uint32_t h, const uint32_t* __restrict__ rk_all,
-                                                   uint32_t* __restrict__ marks, uint64_t mark_stride,
-                                                   WsHeader* hdr) {
-    const uint32_t worker = blockIdx.y;
+// Round keys per worker, and per rank bucket the bitmap block that holds the bucket's first rank
+// (bounds[buckets] = the block of the last rank M - 1).  The bounds depend on the core only.
+__global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, uint32_t seed_lo, uint32_t seed_hi,
+                                     uint32_t first_worker, uint32_t workers, uint32_t round,
+                                     const uint32_t* __restrict__ dir, uint32_t nb, uint32_t M, uint32_t s,
+                                     uint32_t buckets, uint32_t* __restrict__ bounds) {
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t == 0) hdr->status = SLIMDP_OK;
+    if (t < workers * 3) {
+        const uint32_t w = t / 3, b = t % 3;
+        uint32_t out[4];
+        philox4x32_10(seed_lo, seed_hi, b, first_worker + w, round, 0x534C494Du, out);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) rk[w * 12 + b * 4 + q] = out[q];
+    }
+    if (M > 0 && t <= buckets) {
+        const uint64_t first = (uint64_t)t << s;
+        const uint32_t rank = (first < M) ? (uint32_t)first : M - 1;
+        bounds[t] = find_block(dir, 0, nb - 1, rank);
+    }
+}
+
+// grid = (chunks, workers).  rho[w][j] = pi(j) for the CTA's chunk of j; cnt[w][rho >> s] += 1.
+// Lanes whose walk has ended take the next j of their warp's range at once, so a
+// long cycle walk in one lane does not idle the other 31.
+template <bool SMEM_HIST>
+__global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, uint32_t chunk, uint32_t h,
+                                                    uint32_t s, uint32_t buckets,
+                                                    const uint32_t* __restrict__ rk_all, uint32_t* __restrict__ rho,
+                                                    uint64_t rho_stride, unsigned long long* __restrict__ cnt,
+                                                    uint64_t cnt_stride) {
+    extern __shared__ uint32_t sh_hist[];
+    const uint32_t worker = blockIdx.y, lane = lane_id();
+    if (SMEM_HIST) {
+        for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) sh_hist[b] = 0;
+        __syncthreads();
+    }
     uint32_t rk[10];
 #pragma unroll
     for (int r = 0; r < 10; ++r) rk[r] = rk_all[worker * 12 + r];
-    const uint32_t mask = (h >= 32) ? 0xFFFFFFFFu : ((1u << h) - 1u);
-    uint32_t* my_marks = marks + (uint64_t)worker * mark_stride;
-    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k_exp; j += stride) {
-        // pi(j): Feistel network, re-applied while the image is outside [0, M)
-        uint32_t x = (uint32_t)j;
-        do {
+    const uint32_t mask = (1u << h) - 1u;
+    uint32_t* my_rho = rho + (uint64_t)worker * rho_stride;
+    unsigned long long* my_cnt = cnt + (uint64_t)worker * cnt_stride;
+    // this warp's contiguous range of j
+    const uint64_t c0 = (uint64_t)blockIdx.x * chunk;
+    const uint64_t c1 = (c0 + chunk < k_exp) ? c0 + chunk : k_exp;
+    const uint32_t warps = blockDim.x >> 5, wid = threadIdx.x >> 5;
+    const uint64_t span = (c1 > c0) ? (c1 - c0 + warps - 1) / warps : 0;
+    uint64_t next = c0 + (uint64_t)wid * span;
+    const uint64_t stop = (next + span < c1) ? next + span : c1;
+    bool have = false;
+    uint32_t x = 0, j = 0;
+    while (true) {
+        const uint32_t want = __ballot_sync(0xFFFFFFFFu, !have);
+        if (!have) {
+            const uint64_t cand = next + __popc(want & ((1u << lane) - 1u));
+            if (cand < stop) {
+                j = (uint32_t)cand;
+                x = j;
+                have = true;
+            }
+        }
+        next += __popc(want);
+        if (__ballot_sync(0xFFFFFFFFu, have) == 0) break;
+        if (have) {
             uint32_t L = x >> h, R = x & mask;
 #pragma unroll
             for (int r = 0; r < 10; ++r) {
@@ -79,129 +143,246 @@ __global__ void __launch_bounds__(256) mark_kernel(const uint32_t* __restrict__ 
                 R = nr;
             }
             x = (L << h) | R;
-        } while (x >= M);
-        // select0(x): the x-th (0-based) non-core parameter
-        uint32_t lo = 0, hi = nb - 1;
-        while (lo < hi) {
-            const uint32_t mid = lo + ((hi - lo + 1) >> 1);
-            if (__ldg(dir + mid) <= x)
-                lo = mid;
-            else
-                hi = mid - 1;
+            if (x < M) {          // the walk ends at the first image inside [0, M)
+                my_rho[j] = x;
+                if (SMEM_HIST)
+                    atomicAdd(&sh_hist[x >> s], 1u);
+                else
+                    atomicAdd(&my_cnt[x >> s], 1ull);
+                have = false;
+            }
         }
-        uint32_t rem = x - __ldg(dir + lo);
-        const uint4* words = reinterpret_cast<const uint4*>(bitmap + (uint64_t)lo * kWordsPerBlock);
-        uint32_t found = 0xFFFFFFFFu;
-#pragma unroll 1
-        for (int q = 0; q < 8 && found == 0xFFFFFFFFu; ++q) {
-            const uint4 v = __ldg(words + q);
-            const uint32_t z[4] = {~v.x, ~v.y, ~v.z, ~v.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const uint32_t c = __popc(z[e]);
-                if (found == 0xFFFFFFFFu) {
-                    if (rem < c)
-                        found = (uint32_t)(q * 4 + e) * 32u + nth_set_bit(z[e], rem);
-                    else
-                        rem -= c;
+    }
+    if (SMEM_HIST) {
+        __syncthreads();
+        for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) {
+            const uint32_t c = sh_hist[b];
+            if (c) atomicAdd(&my_cnt[b], (unsigned long long)c);
+        }
+    }
+}
+
+// grid = (chunks, workers).  Move every rank of the chunk into its bucket's slice of `sorted`.
+// SMEM: the CTA counts its chunk per bucket, reserves one contiguous piece of every bucket's
+// slice with a single global atomic per bucket, and hands out places inside it from shared memory.
+template <bool SMEM>
+__global__ void __launch_bounds__(1024) scatter_kernel(uint32_t k_exp, uint32_t chunk, uint32_t s, uint32_t buckets,
+                                                       const uint32_t* __restrict__ rho, uint64_t rho_stride,
+                                                       const unsigned long long* __restrict__ pref,
+                                                       uint64_t cnt_stride, uint32_t* __restrict__ cursor,
+                                                       uint32_t* __restrict__ sorted) {
+    extern __shared__ uint32_t sh[];
+    uint32_t* sh_count = sh;              // per bucket: entries of this chunk
+    uint32_t* sh_base = sh + buckets;     // per bucket: first place of this CTA's piece, then the running place
+    const uint32_t worker = blockIdx.y;
+    const uint32_t* my_rho = rho + (uint64_t)worker * rho_stride;
+    uint32_t* my_sorted = sorted + (uint64_t)worker * rho_stride;
+    const unsigned long long* my_pref = pref + (uint64_t)worker * cnt_stride;
+    uint32_t* my_cur = cursor + (uint64_t)worker * cnt_stride;
+    const uint64_t c0 = (uint64_t)blockIdx.x * chunk;
+    const uint64_t c1 = (c0 + chunk < k_exp) ? c0 + chunk : k_exp;
+    if (SMEM) {
+        for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) sh_count[b] = 0;
+        __syncthreads();
+        for (uint64_t j = c0 + threadIdx.x; j < c1; j += blockDim.x) atomicAdd(&sh_count[my_rho[j] >> s], 1u);
+        __syncthreads();
+        for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) {
+            const uint32_t c = sh_count[b];
+            sh_base[b] = c ? (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], c) : 0u;
+        }
+        __syncthreads();
+    }
+    for (uint64_t j = c0 + threadIdx.x; j < c1; j += blockDim.x) {
+        const uint32_t x = my_rho[j];
+        const uint32_t b = x >> s;
+        const uint32_t pos = SMEM ? atomicAdd(&sh_base[b], 1u) : (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], 1u);
+        if (pos < k_exp) my_sorted[pos] = x;
+    }
+}
+
+constexpr uint32_t kDirCache = 1024;
+constexpr uint32_t kListCap = 4096;
+
+// grid = (buckets, workers).  Sort the bucket's ranks through a shared bitmap and emit parameter indices.
+__global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
+    const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ dir, const uint32_t* __restrict__ bounds,
+    uint32_t k_exp, uint32_t s, const uint32_t* __restrict__ sorted, uint64_t rho_stride,
+    const unsigned long long* __restrict__ cnt, const unsigned long long* __restrict__ pref,
+    const unsigned long long* __restrict__ totals, uint64_t cnt_stride, PtrArray<uint32_t> out, WsHeader* hdr) {
+    __shared__ uint32_t bm[2048];            // up to 2^16 rank bits
+    __shared__ uint32_t dir_sh[kDirCache];   // the directory entries of the bucket's blocks
+    __shared__ uint16_t list[kListCap];      // sorted ranks (low s bits) of the current round
+    __shared__ uint32_t warp_sums[kBucketThreads / 32];
+    const uint32_t worker = blockIdx.y, bucket = blockIdx.x, t = threadIdx.x;
+    const uint32_t words = 1u << (s - 5);
+    const uint32_t per = words / kBucketThreads;   // 1, 2, 4 or 8 words per thread
+    const uint32_t count = (uint32_t)cnt[(uint64_t)worker * cnt_stride + bucket];
+    const uint32_t offset = (uint32_t)pref[(uint64_t)worker * cnt_stride + bucket];
+    if (bucket == 0 && t == 0 && totals[worker] != k_exp) hdr->status = SLIMDP_ERR_INTERNAL;
+    if (count == 0) return;
+    for (uint32_t i = t; i < words; i += kBucketThreads) bm[i] = 0;
+    // the bucket's ranks live in bitmap blocks [blk_lo, blk_hi]
+    const uint32_t blk_lo = __ldg(bounds + bucket), blk_hi = __ldg(bounds + bucket + 1);
+    const uint32_t nblk = blk_hi - blk_lo + 1;
+    const bool cached = nblk <= kDirCache;
+    if (cached)
+        for (uint32_t i = t; i < nblk; i += kBucketThreads) dir_sh[i] = __ldg(dir + blk_lo + i);
+    __syncthreads();
+    const uint32_t* my_sorted = sorted + (uint64_t)worker * rho_stride + offset;
+    const uint32_t low_mask = (1u << s) - 1u;
+    for (uint32_t e = t; e < count; e += kBucketThreads) {
+        const uint32_t r = my_sorted[e] & low_mask;
+        atomicOr(&bm[r >> 5], 1u << (r & 31u));
+    }
+    __syncthreads();
+    // place of this thread's first rank in the sorted order: exclusive scan of the popcounts
+    uint32_t mine = 0;
+    for (uint32_t q = 0; q < per; ++q) mine += __popc(bm[t * per + q]);
+    const uint32_t inc = warp_inclusive_scan(mine);
+    if ((t & 31u) == 31u) warp_sums[t >> 5] = inc;
+    __syncthreads();
+    uint32_t base = inc - mine;
+    for (uint32_t wdx = 0; wdx < (t >> 5); ++wdx) base += warp_sums[wdx];
+    uint32_t total = 0;
+    for (uint32_t wdx = 0; wdx < kBucketThreads / 32; ++wdx) total += warp_sums[wdx];
+    if (t == 0 && total != count) hdr->status = SLIMDP_ERR_INTERNAL;   // two ranks collided: pi is not injective
+    uint32_t* dst = out.p[worker] + offset;
+    const uint32_t first_rank = bucket << s;
+    // rounds of up to kListCap ranks: write them to `list` in sorted order, then share them out evenly
+    for (uint32_t r0 = 0; r0 < count; r0 += kListCap) {
+        if (base < r0 + kListCap && base + mine > r0) {
+            uint32_t p = base;
+            for (uint32_t q = 0; q < per; ++q) {
+                uint32_t word = bm[t * per + q];
+                while (word) {
+                    const uint32_t bit = __ffs(word) - 1;
+                    word &= word - 1;
+                    if (p >= r0 && p < r0 + kListCap) list[p - r0] = (uint16_t)((t * per + q) * 32u + bit);
+                    ++p;
                 }
             }
         }
-        if (found == 0xFFFFFFFFu) {
-            hdr->status = SLIMDP_ERR_INTERNAL;   // directory and bitmap disagree
-            continue;
-        }
-        const uint32_t idx = lo * kBlock + found;
-        atomicOr(&my_marks[idx >> 5], 1u << (idx & 31u));
-    }
-}
-
-__global__ void __launch_bounds__(256) count_marks_kernel(const uint32_t* __restrict__ marks, uint64_t mark_stride,
-                                                          uint64_t nb, unsigned long long* __restrict__ cnt,
-                                                          uint64_t cnt_stride) {
-    const uint32_t worker = blockIdx.y, lane = lane_id();
-    const uint32_t* my = marks + (uint64_t)worker * mark_stride;
-    const uint64_t warps = (uint64_t)gridDim.x * (blockDim.x >> 5);
-    for (uint64_t blk = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); blk < nb; blk += warps) {
-        const uint32_t c = __reduce_add_sync(0xFFFFFFFFu, __popc(my[blk * kWordsPerBlock + lane]));
-        if (lane == 0) cnt[(uint64_t)worker * cnt_stride + blk] = c;
-    }
-}
-
-__global__ void __launch_bounds__(256) expand_marks_kernel(const uint32_t* __restrict__ marks, uint64_t mark_stride,
-                                                           uint64_t nb, const unsigned long long* __restrict__ pref,
-                                                           const unsigned long long* __restrict__ totals,
-                                                           uint64_t cnt_stride, uint32_t k_exp,
-                                                           PtrArray<uint32_t> out, WsHeader* hdr) {
-    const uint32_t worker = blockIdx.y, lane = lane_id();
-    const uint32_t* my = marks + (uint64_t)worker * mark_stride;
-    uint32_t* dst = out.p[worker];
-    const uint64_t warps = (uint64_t)gridDim.x * (blockDim.x >> 5);
-    const uint64_t warp0 = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (warp0 == 0 && lane == 0 && totals[worker] != k_exp) hdr->status = SLIMDP_ERR_INTERNAL;
-    for (uint64_t blk = warp0; blk < nb; blk += warps) {
-        const uint32_t sel = my[blk * kWordsPerBlock + lane];
-        const uint32_t ps = __popc(sel);
-        const uint32_t any = __ballot_sync(0xFFFFFFFFu, sel != 0);
-        if (any == 0) continue;
-        const uint32_t out_base = (uint32_t)pref[(uint64_t)worker * cnt_stride + blk] + warp_inclusive_scan(ps) - ps;
-        for (uint32_t m = any; m; m &= m - 1) {
-            const int wd = __ffs(m) - 1;
-            const uint32_t word = __shfl_sync(0xFFFFFFFFu, sel, wd);
-            const uint32_t base = __shfl_sync(0xFFFFFFFFu, out_base, wd);
-            if ((word >> lane) & 1u) {
-                const uint32_t pos = base + __popc(word & ((1u << lane) - 1u));
-                if (pos < k_exp)
-                    dst[pos] = (uint32_t)(blk * kBlock + wd * 32 + lane);
-                else
-                    hdr->status = SLIMDP_ERR_INTERNAL;
+        __syncthreads();
+        const uint32_t m = (count - r0 < kListCap) ? count - r0 : kListCap;
+        uint32_t rel = 0;     // block relative to blk_lo; ranks ascend inside a thread, so it only moves up
+        for (uint32_t e = t; e < m; e += kBucketThreads) {
+            const uint32_t rank = first_rank + list[e];
+            // select0(rank): block by binary search of the directory ...
+            uint32_t rem;
+            if (cached) {
+                uint32_t lo = rel, hi = nblk - 1;
+                while (lo < hi) {
+                    const uint32_t mid = lo + ((hi - lo + 1) >> 1);
+                    if (dir_sh[mid] <= rank)
+                        lo = mid;
+                    else
+                        hi = mid - 1;
+                }
+                rel = lo;
+                rem = rank - dir_sh[rel];
+            } else {
+                rel = find_block(dir, blk_lo + rel, blk_hi, rank) - blk_lo;
+                rem = rank - __ldg(dir + blk_lo + rel);
+            }
+            // ... then the word holding the rem-th zero bit of the block, then the bit
+            const uint32_t blk = blk_lo + rel;
+            const uint32_t* blk_words = bitmap + (uint64_t)blk * kWordsPerBlock;
+            const uint4* wordsp = reinterpret_cast<const uint4*>(blk_words);
+            uint4 v[8];
+#pragma unroll
+            for (int g = 0; g < 8; ++g) v[g] = __ldg(wordsp + g);
+            uint32_t zeros = 0, wsel = 0, before = 0;
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+                const uint32_t c[4] = {32u - __popc(v[g].x), 32u - __popc(v[g].y), 32u - __popc(v[g].z),
+                                       32u - __popc(v[g].w)};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    zeros += c[q];
+                    const bool passed = zeros <= rem;   // the whole word lies before the wanted zero
+                    wsel += passed ? 1u : 0u;
+                    before = passed ? zeros : before;
+                }
+            }
+            if (wsel >= kWordsPerBlock || offset + r0 + e >= k_exp) {
+                hdr->status = SLIMDP_ERR_INTERNAL;   // directory and bitmap disagree
+            } else {
+                const uint32_t z = ~__ldg(blk_words + wsel);
+                dst[r0 + e] = blk * kBlock + wsel * 32u + nth_set_bit(z, rem - before);
             }
         }
+        __syncthreads();
     }
 }
 
 }  // namespace
+
+uint32_t explore_bucket_shift(uint64_t M) {
+    int lg = 0;
+    while (lg < 63 && (2ull << lg) <= M) ++lg;   // floor(log2(M)) for M >= 1
+    int extra = lg - 22;
+    if (extra < 0) extra = 0;
+    if (extra > 3) extra = 3;
+    return (uint32_t)(13 + extra);
+}
 
 slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                              uint32_t first_worker, uint32_t workers, uint32_t round,
                              const PtrArray<uint32_t>& out, void* ws, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
-    const ExploreWs L = explore_ws_layout(ws, n, workers);
+    const ExploreWs L = explore_ws_layout(ws, n, k_exp, workers);
     const uint64_t nb = num_blocks(n);
     const uint64_t M = n - k_core;
     const uint32_t* bitmap = reinterpret_cast<const uint32_t*>(core_aux);
     const uint32_t* dir =
         reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(core_aux) + slimdp_core_aux_dir_offset(n));
+    const uint32_t s = explore_bucket_shift(M);
+    const uint64_t buckets = (M + (1ull << s) - 1) >> s;
 
-    explore_setup_kernel<<<1, 256, 0, st>>>(L.hdr, L.round_keys, (uint32_t)seed, (uint32_t)(seed >> 32),
-                                            first_worker, workers, round);
+    const unsigned setup_threads = (unsigned)((buckets + 1 > 3ull * workers) ? buckets + 1 : 3ull * workers);
+    explore_setup_kernel<<<(setup_threads + 255) / 256, 256, 0, st>>>(L.hdr, L.round_keys, (uint32_t)seed,
+                                                                      (uint32_t)(seed >> 32), first_worker, workers,
+                                                                      round, dir, (uint32_t)nb, (uint32_t)M, s,
+                                                                      (uint32_t)buckets, L.bounds);
     SLIMDP_LAUNCHED(1);
     if (k_exp == 0) return SLIMDP_OK;
-    if (cudaMemsetAsync(L.marks, 0, (size_t)workers * L.mark_stride * 4, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
+    if (cudaMemsetAsync(L.cnt, 0, L.zero_bytes, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
 
     int b = 1;
     while (((uint64_t)1 << b) < M) ++b;
     const uint32_t h = (uint32_t)((b + 1) / 2);
 
-    uint64_t mgrid = (k_exp + 255) / 256;
-    if (mgrid > (uint64_t)sms * 16) mgrid = (uint64_t)sms * 16;
-    mark_kernel<<<dim3((unsigned)mgrid, workers), 256, 0, st>>>(bitmap, dir, (uint32_t)nb, (uint32_t)M,
-                                                                (uint32_t)k_exp, h, L.round_keys, L.marks,
-                                                                L.mark_stride, L.hdr);
+    // about two 1024-thread CTAs per SM over all workers; every CTA owns one contiguous chunk of j
+    uint64_t chunks = ((uint64_t)sms * 2 + workers - 1) / workers;
+    if (chunks > (k_exp + 1023) / 1024) chunks = (k_exp + 1023) / 1024;
+    if (chunks == 0) chunks = 1;
+    const uint32_t chunk = (uint32_t)((k_exp + chunks - 1) / chunks);
+    const dim3 grid((unsigned)chunks, workers);
+    const bool smem = buckets <= kMaxSmemBuckets;
+    if (smem) {
+        rank_kernel<true><<<grid, 1024, buckets * 4, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, h, s,
+                                                           (uint32_t)buckets, L.round_keys, L.rho, L.rho_stride,
+                                                           L.cnt, L.cnt_stride);
+    } else {
+        rank_kernel<false><<<grid, 1024, 0, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, h, s, (uint32_t)buckets,
+                                                  L.round_keys, L.rho, L.rho_stride, L.cnt, L.cnt_stride);
+    }
     SLIMDP_LAUNCHED(1);
-    uint64_t cgrid = (nb + 7) / 8;
-    const uint64_t cap = ((uint64_t)sms * 8 + workers - 1) / workers;
-    if (cgrid > cap) cgrid = cap;
-    if (cgrid == 0) cgrid = 1;
-    count_marks_kernel<<<dim3((unsigned)cgrid, workers), 256, 0, st>>>(L.marks, L.mark_stride, nb, L.cnt,
-                                                                       L.cnt_stride);
+    slimdp_status rc =
+        launch_block_scan(L.cnt, L.pref, L.tile_sums, L.totals, buckets, workers, L.cnt_stride, L.tile_stride, st);
+    if (rc != SLIMDP_OK) return rc;
+    if (smem) {
+        scatter_kernel<true><<<grid, 1024, buckets * 8, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets, L.rho,
+                                                              L.rho_stride, L.pref, L.cnt_stride, L.cursor, L.sorted);
+    } else {
+        scatter_kernel<false><<<grid, 1024, 0, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets, L.rho,
+                                                     L.rho_stride, L.pref, L.cnt_stride, L.cursor, L.sorted);
+    }
     SLIMDP_LAUNCHED(1);
-    slimdp_status s =
-        launch_block_scan(L.cnt, L.pref, L.tile_sums, L.totals, nb, workers, L.cnt_stride, L.tile_stride, st);
-    if (s != SLIMDP_OK) return s;
-    expand_marks_kernel<<<dim3((unsigned)cgrid, workers), 256, 0, st>>>(L.marks, L.mark_stride, nb, L.pref, L.totals,
-                                                                        L.cnt_stride, (uint32_t)k_exp, out, L.hdr);
+    bucket_kernel<<<dim3((unsigned)buckets, workers), kBucketThreads, 0, st>>>(
+        bitmap, dir, L.bounds, (uint32_t)k_exp, s, L.sorted, L.rho_stride, L.cnt, L.pref, L.totals, L.cnt_stride,
+        out, L.hdr);
     SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }

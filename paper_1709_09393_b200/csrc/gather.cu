@@ -2,57 +2,95 @@
 // T_C = core U explorer (Section 3.1) out of a full-length vector: the
 // worker's updates for the push (the extraction step of Section 3.5), the
 // merged global parameters for the pull (Section 3.3 step 4).
+//
+// Core segment: the core keys are shared by all workers (Section 3.5, key
+// caching), so one thread reads core_idx[j] once and serves all K workers:
+// K independent gathers in flight for the push, a single gather written K
+// times for the pull.  Explorer segments: one grid row per worker.
 #include "common.cuh"
 
 namespace slimdp {
 
 namespace {
 
-// grid.y = worker.  out[w][j] = src[w][core_idx[j]] (j < k_core), out[w][k_core + j] = src[w][exp[w][j]].
-__global__ void __launch_bounds__(256) gather_kernel(PtrArray<const float> src, const uint32_t* __restrict__ core_idx,
-                                                     uint64_t k_core, PtrArray<const uint32_t> exp, uint64_t k_exp,
-                                                     PtrArray<float> out) {
+// out[k][j] = src[k][core_idx[j]] for every worker k.  SAME: all workers read the same source.
+template <bool SAME>
+__global__ void __launch_bounds__(256) gather_core_kernel(PtrArray<const float> src,
+                                                          const uint32_t* __restrict__ core_idx, uint64_t k_core,
+                                                          PtrArray<float> out, int K) {
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k_core; j += stride) {
+        const uint32_t i = __ldg(core_idx + j);
+        if (SAME) {
+            const float v = __ldg(src.p[0] + i);
+#pragma unroll 8
+            for (int k = 0; k < K; ++k) __stcs(out.p[k] + j, v);
+        } else {
+            int k = 0;
+            for (; k + 8 <= K; k += 8) {
+                float v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = __ldg(src.p[k + q] + i);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) __stcs(out.p[k + q] + j, v[q]);
+            }
+            for (; k < K; ++k) __stcs(out.p[k] + j, __ldg(src.p[k] + i));
+        }
+    }
+}
+
+// grid.y = worker.  out[w][k_core + j] = src[w][exp[w][j]].
+__global__ void __launch_bounds__(256) gather_explore_kernel(PtrArray<const float> src, PtrArray<const uint32_t> exp,
+                                                             uint64_t k_exp, PtrArray<float> out, uint64_t k_core) {
     const uint32_t worker = blockIdx.y;
     const float* __restrict__ s = src.p[worker];
     const uint32_t* __restrict__ e = exp.p[worker];
-    float* __restrict__ o = out.p[worker];
-    const uint64_t m = k_core + k_exp;
+    float* __restrict__ o = out.p[worker] + k_core;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x * 4;
-    for (uint64_t j0 = ((uint64_t)blockIdx.x * blockDim.x) * 4 + threadIdx.x; j0 < m; j0 += stride) {
+    for (uint64_t j0 = ((uint64_t)blockIdx.x * blockDim.x) * 4 + threadIdx.x; j0 < k_exp; j0 += stride) {
         uint32_t idx[4];
         float v[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const uint64_t j = j0 + (uint64_t)q * blockDim.x;
-            if (j < m) idx[q] = (j < k_core) ? __ldg(core_idx + j) : __ldg(e + (j - k_core));
+            if (j < k_exp) idx[q] = __ldg(e + j);
         }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const uint64_t j = j0 + (uint64_t)q * blockDim.x;
-            if (j < m) v[q] = __ldg(s + idx[q]);
+            if (j < k_exp) v[q] = __ldg(s + idx[q]);
         }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const uint64_t j = j0 + (uint64_t)q * blockDim.x;
-            if (j < m) o[j] = v[q];
+            if (j < k_exp) __stcs(o + j, v[q]);
         }
     }
 }
 
 }  // namespace
 
-slimdp_status launch_gather(const PtrArray<const float>& src, uint32_t workers, const uint32_t* core_idx,
-                            uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp,
-                            const PtrArray<float>& out, cudaStream_t st) {
-    const uint64_t m = k_core + k_exp;
-    if (m == 0) return SLIMDP_OK;
+slimdp_status launch_gather(const PtrArray<const float>& src, bool same_src, uint32_t workers,
+                            const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,
+                            uint64_t k_exp, const PtrArray<float>& out, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
-    uint64_t grid = (m + 1023) / 1024;
-    const uint64_t cap = ((uint64_t)sms * 32 + workers - 1) / workers;
-    if (grid > cap) grid = cap;
-    gather_kernel<<<dim3((unsigned)grid, workers), 256, 0, st>>>(src, core_idx, k_core, exp, k_exp, out);
-    SLIMDP_LAUNCHED(1);
+    if (k_core > 0) {
+        uint64_t grid = (k_core + 255) / 256;
+        if (grid > (uint64_t)sms * 32) grid = (uint64_t)sms * 32;
+        if (same_src)
+            gather_core_kernel<true><<<(unsigned)grid, 256, 0, st>>>(src, core_idx, k_core, out, (int)workers);
+        else
+            gather_core_kernel<false><<<(unsigned)grid, 256, 0, st>>>(src, core_idx, k_core, out, (int)workers);
+        SLIMDP_LAUNCHED(1);
+    }
+    if (k_exp > 0) {
+        uint64_t grid = (k_exp + 1023) / 1024;
+        const uint64_t cap = ((uint64_t)sms * 32 + workers - 1) / workers;
+        if (grid > cap) grid = cap;
+        gather_explore_kernel<<<dim3((unsigned)grid, workers), 256, 0, st>>>(src, exp, k_exp, out, k_core);
+        SLIMDP_LAUNCHED(1);
+    }
     return SLIMDP_OK;
 }
 

@@ -42,34 +42,49 @@ inline SelectWs select_ws_layout(void* ws, uint64_t n) {
 struct ExploreWs {
     WsHeader* hdr;
     uint32_t* round_keys;           // 12 words per worker
-    uint32_t* marks;                // per worker: nb * 32 words
-    unsigned long long* cnt;        // per worker: nb
-    unsigned long long* pref;       // per worker: nb
-    unsigned long long* tile_sums;  // per worker: nt
+    uint32_t* bounds;               // per bucket: bitmap block of its first rank (+1 entry)
+    uint32_t* rho;                  // per worker: pi(j), j < k_exp
+    uint32_t* sorted;               // per worker: the same ranks grouped by bucket
+    unsigned long long* cnt;        // per worker: ranks per bucket
+    uint32_t* cursor;               // per worker: scatter cursors per bucket
+    unsigned long long* pref;       // per worker: exclusive scan of cnt
+    unsigned long long* tile_sums;  // per worker: per scan tile
     unsigned long long* totals;     // per worker: 1
-    uint64_t mark_stride;           // words between workers' bitmaps
-    uint64_t cnt_stride;            // entries between workers' counter rows
+    uint64_t rho_stride;            // entries between workers' rank rows
+    uint64_t cnt_stride;            // entries between workers' bucket rows
     uint64_t tile_stride;
+    size_t zero_bytes;              // cnt and cursor, contiguous, cleared before every call
     size_t bytes;
 };
 
-inline ExploreWs explore_ws_layout(void* ws, uint64_t n, uint32_t workers) {
-    const uint64_t nb = num_blocks(n), nt = num_scan_tiles(n);
+// Upper bound on the number of rank buckets for any core size: buckets hold
+// 2^13 .. 2^16 ranks, 2^16 once there are at least 2^25 non-core parameters.
+inline uint64_t explore_max_buckets(uint64_t n) {
+    const uint64_t big = (n + 65535) / 65536;
+    return big > 1024 ? big : 1024;
+}
+
+inline ExploreWs explore_ws_layout(void* ws, uint64_t n, uint64_t k_exp, uint32_t workers) {
     char* p = reinterpret_cast<char*>(ws);
     size_t off = 0;
     ExploreWs L;
     auto take = [&](size_t bytes) {
         char* r = p + off;
-        off += align_up(bytes, 256);
+        off += align_up(bytes ? bytes : 1, 256);
         return r;
     };
-    L.mark_stride = align_up(nb * kWordsPerBlock, 64);
-    L.cnt_stride = align_up(nb, 32);
-    L.tile_stride = align_up(nt, 32);
+    L.rho_stride = align_up(k_exp, 64);
+    L.cnt_stride = align_up(explore_max_buckets(n), 64);
+    L.tile_stride = align_up((L.cnt_stride + kScanTile - 1) / kScanTile, 32);
     L.hdr = reinterpret_cast<WsHeader*>(take(sizeof(WsHeader)));
     L.round_keys = reinterpret_cast<uint32_t*>(take((size_t)workers * 12 * 4));
-    L.marks = reinterpret_cast<uint32_t*>(take((size_t)workers * L.mark_stride * 4));
+    L.bounds = reinterpret_cast<uint32_t*>(take((L.cnt_stride + 1) * 4));
+    L.rho = reinterpret_cast<uint32_t*>(take((size_t)workers * L.rho_stride * 4));
+    L.sorted = reinterpret_cast<uint32_t*>(take((size_t)workers * L.rho_stride * 4));
+    const size_t zero_begin = off;
     L.cnt = reinterpret_cast<unsigned long long*>(take((size_t)workers * L.cnt_stride * 8));
+    L.cursor = reinterpret_cast<uint32_t*>(take((size_t)workers * L.cnt_stride * 4));
+    L.zero_bytes = off - zero_begin;
     L.pref = reinterpret_cast<unsigned long long*>(take((size_t)workers * L.cnt_stride * 8));
     L.tile_sums = reinterpret_cast<unsigned long long*>(take((size_t)workers * L.tile_stride * 8));
     L.totals = reinterpret_cast<unsigned long long*>(take((size_t)workers * 8));

@@ -22,7 +22,7 @@ class RoundBuffers:
         self.core_idx = torch.empty(k_core, dtype=B.IDX, device=dev)
         self.core_aux = torch.empty(B.core_aux_bytes(n), dtype=torch.uint8, device=dev)
         self.select_ws = torch.empty(B.select_workspace_bytes(n), dtype=torch.uint8, device=dev)
-        self.explore_ws = torch.empty(B.explore_workspace_bytes(n, K), dtype=torch.uint8, device=dev)
+        self.explore_ws = torch.empty(B.explore_workspace_bytes(n, k_exp, K), dtype=torch.uint8, device=dev)
         self.exp_idx: List[torch.Tensor] = [torch.empty(k_exp, dtype=B.IDX, device=dev) for _ in range(K)]
         self.val: List[torch.Tensor] = [torch.empty(m, dtype=torch.float32, device=dev) for _ in range(K)]
         self.pulled: List[torch.Tensor] = [torch.empty(m, dtype=torch.float32, device=dev) for _ in range(K)]

@@ -49,11 +49,15 @@ def test_size_queries(P):
         assert off >= nb * 128 and off % 256 == 0
         assert P.core_aux_bytes(n) >= off + 4 * (nb + 1)
         assert P.select_workspace_bytes(n) >= 256 + 3 * 4096 * 4 + 2 * nb * 128 + 2 * nb * 8
-        assert P.explore_workspace_bytes(n, 8) > P.explore_workspace_bytes(n, 1) >= 256 + nb * 128 + 2 * nb * 8
-        assert P.workspace_bytes(n, 8) == max(P.select_workspace_bytes(n), P.explore_workspace_bytes(n, 8))
+        k_exp = n // 100
+        assert P.explore_workspace_bytes(n, k_exp, 8) > P.explore_workspace_bytes(n, k_exp, 1) >= 256 + 8 * k_exp
+        assert P.explore_workspace_bytes(n, n, 1) >= 8 * n
+        assert P.workspace_bytes(n, k_exp, 8) == max(P.select_workspace_bytes(n),
+                                                     P.explore_workspace_bytes(n, k_exp, 8))
     # out-of-range arguments size to zero
     assert P.core_aux_bytes(0) == 0 and P.core_aux_bytes(2 ** 32) == 0
-    assert P.explore_workspace_bytes(1000, 0) == 0 and P.explore_workspace_bytes(1000, 65) == 0
+    assert P.explore_workspace_bytes(1000, 10, 0) == 0 and P.explore_workspace_bytes(1000, 10, 65) == 0
+    assert P.explore_workspace_bytes(1000, 1001, 1) == 0
     assert P.round_arena_bytes(1000, 4, 1001, 0) == 0 and P.round_arena_bytes(1000, 4, 600, 401) == 0
     a = P.round_arena_bytes(10 ** 6, 4, 10 ** 5, 45_000)
     assert a >= 4 * 10 ** 6 * 6 + 4 * 145_000 * 8

@@ -165,7 +165,7 @@ def test_explore_parity(P, n, k_core, k_exp):
     rng = np.random.default_rng(n + k_core)
     core = np.sort(rng.choice(n, size=k_core, replace=False)).astype(np.uint32)
     aux = _gpu_core_aux(P, n, core)
-    ws = torch.empty(P.explore_workspace_bytes(n, 1), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(P.explore_workspace_bytes(n, k_exp, 1), dtype=torch.uint8, device="cuda")
     for seed, worker, rnd in [(0, 0, 0), (2 ** 40 + 17, 3, 9), (2 ** 64 - 1, 63, 2 ** 32 - 1)]:
         out = torch.empty(k_exp, dtype=torch.int32, device="cuda")
         P.slimdp_sample_explore(aux, n, k_core, k_exp, seed, worker, rnd, out, ws)
@@ -178,7 +178,7 @@ def test_explore_batched_equals_single_calls(P):
     rng = np.random.default_rng(3)
     core = np.sort(rng.choice(n, size=k_core, replace=False)).astype(np.uint32)
     aux = _gpu_core_aux(P, n, core)
-    ws = torch.empty(P.explore_workspace_bytes(n, K), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(P.explore_workspace_bytes(n, k_exp, K), dtype=torch.uint8, device="cuda")
     outs = [torch.empty(k_exp, dtype=torch.int32, device="cuda") for _ in range(K)]
     P.slimdp_sample_explore_batched(aux, n, k_core, k_exp, 9, 5, 2, outs, ws)
     P.read_status(ws)
