@@ -59,8 +59,9 @@ enum {
 /* Largest K: the K per-worker device pointers travel by value as kernel arguments. */
 #define SLIMDP_MAX_WORKERS 64
 
-/* Parameters per bitmap block: core_aux keeps one directory entry per block. */
+/* Parameters per bitmap block (32 words), and per directory entry of core_aux. */
 #define SLIMDP_BLOCK 1024
+#define SLIMDP_DIR_STRIDE 256
 
 const char* slimdp_status_string(slimdp_status s);
 
@@ -69,9 +70,10 @@ const char* slimdp_status_string(slimdp_status s);
  * sampler reads.  Layout (all uint32_t, little-endian bit order):
  *   bitmap    [nb * 32] words, nb = ceil(n / 1024): bit (i & 31) of word (i >> 5)
  *             is 1 iff parameter i is in the core; bits at i >= n are 0;
- *   directory [nb + 1] words starting at byte offset slimdp_core_aux_dir_offset(n):
- *             directory[b] = number of NON-core parameters with index < 1024 b,
- *             directory[nb] = n - k_core.
+ *   directory [nd + 1] words, nd = 4 nb, starting at byte offset slimdp_core_aux_dir_offset(n):
+ *             directory[d] = 256 d - (number of core parameters with index < 256 d) for d < nd,
+ *             i.e. the number of NON-core parameters below 256 d wherever 256 d <= n;
+ *             directory[nd] = n - k_core.
  */
 size_t slimdp_core_aux_bytes(uint64_t n);
 size_t slimdp_core_aux_dir_offset(uint64_t n);

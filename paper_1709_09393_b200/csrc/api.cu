@@ -88,7 +88,7 @@ size_t slimdp_core_aux_dir_offset(uint64_t n) {
 
 size_t slimdp_core_aux_bytes(uint64_t n) {
     if (!n_ok(n)) return 0;
-    return slimdp_core_aux_dir_offset(n) + align_up((num_blocks(n) + 1) * 4, 256);
+    return slimdp_core_aux_dir_offset(n) + align_up((num_blocks(n) * kDirPerBlock + 1) * 4, 256);
 }
 
 size_t slimdp_select_workspace_bytes(uint64_t n) {

@@ -10,7 +10,12 @@ namespace slimdp {
 
 constexpr uint32_t kBlock = SLIMDP_BLOCK;        // parameters per bitmap block
 constexpr uint32_t kWordsPerBlock = kBlock / 32; // 32 bitmap words per block
+constexpr uint32_t kDirStride = SLIMDP_DIR_STRIDE;      // parameters per directory entry
+constexpr uint32_t kDirPerBlock = kBlock / kDirStride;  // 4 directory entries per bitmap block
+constexpr uint32_t kWordsPerDir = kDirStride / 32;      // 8 bitmap words per directory entry
 constexpr uint32_t kScanTile = 1024;             // bitmap blocks per scan tile
+constexpr uint32_t kSampleBits = 18;             // the selection's bracket is estimated from 2^18 sampled keys
+constexpr uint64_t kBracketMinN = 1ull << 21;    // below this the selection reads the keys three more times instead
 
 // K device pointers passed by value as a kernel argument (512 bytes).
 template <typename T>
@@ -24,7 +29,12 @@ struct WsHeader {
     uint32_t prefix;     // radix prefix found so far; after the last pass the threshold key T
     uint32_t k_rem;      // rank still to resolve inside the prefix; after the last pass the tie quota r
     uint32_t ties;       // r: how many keys equal to T are admitted (smallest indices first)
-    uint32_t reserved[60];
+    uint32_t n_def;      // bracket pass: keys in bins >= b_top (certainly in the core)
+    uint32_t n_cand;     // bracket pass: keys inside the bracket (candidates)
+    uint32_t b_top;      // first 16-bit bin certainly above T (65536: none)
+    uint32_t b_bot;      // lowest 16-bit bin that may hold T
+    uint32_t ticket[8];  // "last CTA done" counters, one per kernel that needs one
+    uint32_t reserved[48];
 };
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 
@@ -88,17 +98,18 @@ __device__ __forceinline__ unsigned long long warp_inclusive_scan64(unsigned lon
     return v;
 }
 
-// Exclusive scan of one value per thread over a block of 1024 threads.
+// Exclusive scan of one value per thread over a block of NWARPS * 32 threads.
 // Returns the exclusive prefix; *total receives the block sum.  smem: 33 words.
-__device__ __forceinline__ unsigned long long block_exclusive_scan64_1024(unsigned long long v,
-                                                                          unsigned long long* smem,
-                                                                          unsigned long long* total) {
+template <int NWARPS>
+__device__ __forceinline__ unsigned long long block_exclusive_scan64(unsigned long long v,
+                                                                     unsigned long long* smem,
+                                                                     unsigned long long* total) {
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
     unsigned long long inc = warp_inclusive_scan64(v);
     if (lane == 31) smem[warp] = inc;
     __syncthreads();
     if (warp == 0) {
-        unsigned long long s = smem[lane];
+        unsigned long long s = (lane < (uint32_t)NWARPS) ? smem[lane] : 0ull;
         unsigned long long sinc = warp_inclusive_scan64(s);
         smem[lane] = sinc - s;
         if (lane == 31) smem[32] = sinc;
@@ -108,6 +119,12 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan64_1024(unsign
     *total = smem[32];
     __syncthreads();
     return out;
+}
+
+__device__ __forceinline__ unsigned long long block_exclusive_scan64_1024(unsigned long long v,
+                                                                          unsigned long long* smem,
+                                                                          unsigned long long* total) {
+    return block_exclusive_scan64<32>(v, smem, total);
 }
 
 // ---- internal launchers (each enqueues on `st`, returns a slimdp_status) ---

@@ -16,9 +16,9 @@
 //   5. bucket: one CTA per (bucket, worker) marks its ranks in a 2^s-bit
 //      shared-memory bitmap, which sorts them; a block scan of the popcounts
 //      gives each rank its output position, and a select0 query (binary
-//      search of the per-1024 non-core directory inside the bucket's block
-//      range, then a popcount walk over the block's 32 bitmap words) turns
-//      it into the parameter index.
+//      search of the per-256 non-core directory inside the bucket's range,
+//      then a popcount walk over the group's 8 bitmap words, skipped when
+//      the group holds no core parameter) turns it into the parameter index.
 // No global bitmap, no inter-CTA waiting; the result does not depend on the
 // order in which atomics land.
 #include "common.cuh"
@@ -29,7 +29,7 @@ namespace slimdp {
 namespace {
 
 constexpr int kBucketThreads = 256;
-constexpr uint64_t kMaxSmemBuckets = 5120;   // 20 KB / 40 KB of static-limit shared memory per CTA
+
 
 __device__ __forceinline__ void philox4x32_10(uint32_t k0, uint32_t k1, uint32_t c0, uint32_t c1, uint32_t c2,
                                               uint32_t c3, uint32_t out[4]) {
@@ -67,11 +67,12 @@ __device__ __forceinline__ uint32_t find_block(const uint32_t* __restrict__ dir,
     return lo;
 }
 
-// Round keys per worker, and per rank bucket the bitmap block that holds the bucket's first rank
-// (bounds[buckets] = the block of the last rank M - 1).  The bounds depend on the core only.
+// Round keys per worker, and per rank bucket the directory entry (256-parameter group) that holds
+// the bucket's first rank (bounds[buckets] = the group of the last rank M - 1).  The bounds
+// depend on the core only.
 __global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, uint32_t seed_lo, uint32_t seed_hi,
                                      uint32_t first_worker, uint32_t workers, uint32_t round,
-                                     const uint32_t* __restrict__ dir, uint32_t nb, uint32_t M, uint32_t s,
+                                     const uint32_t* __restrict__ dir, uint32_t nd, uint32_t M, uint32_t s,
                                      uint32_t buckets, uint32_t* __restrict__ bounds) {
     const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t == 0) hdr->status = SLIMDP_OK;
@@ -85,7 +86,7 @@ __global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, u
     if (M > 0 && t <= buckets) {
         const uint64_t first = (uint64_t)t << s;
         const uint32_t rank = (first < M) ? (uint32_t)first : M - 1;
-        bounds[t] = find_block(dir, 0, nb - 1, rank);
+        bounds[t] = find_block(dir, 0, nd - 1, rank);
     }
 }
 
@@ -97,7 +98,7 @@ __global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, 
                                                     uint32_t s, uint32_t buckets,
                                                     const uint32_t* __restrict__ rk_all, uint32_t* __restrict__ rho,
                                                     uint64_t rho_stride, unsigned long long* __restrict__ cnt,
-                                                    uint64_t cnt_stride) {
+                                                    uint64_t cnt_stride, uint32_t* __restrict__ cta_hist) {
     extern __shared__ uint32_t sh_hist[];
     const uint32_t worker = blockIdx.y, lane = lane_id();
     if (SMEM_HIST) {
@@ -135,9 +136,9 @@ __global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, 
             uint32_t L = x >> h, R = x & mask;
 #pragma unroll
             for (int r = 0; r < 10; ++r) {
-                const uint32_t mult = (r & 1) ? 0xCD9E8D57u : 0xD2511F53u;
-                const uint32_t v = R ^ rk[r];
-                const uint32_t F = __umulhi(v, mult) ^ (v * mult);
+                const unsigned long long mult = (r & 1) ? 0xCD9E8D57ull : 0xD2511F53ull;
+                const unsigned long long prod = (unsigned long long)(R ^ rk[r]) * mult;   // one 32x32->64 multiply
+                const uint32_t F = (uint32_t)(prod >> 32) ^ (uint32_t)prod;
                 const uint32_t nr = (L ^ F) & mask;
                 L = R;
                 R = nr;
@@ -155,25 +156,28 @@ __global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, 
     }
     if (SMEM_HIST) {
         __syncthreads();
+        // the chunk's own histogram is kept for the scatter step, which reserves bucket space with it
+        uint32_t* mine = cta_hist + ((uint64_t)worker * gridDim.x + blockIdx.x) * buckets;
         for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) {
             const uint32_t c = sh_hist[b];
+            mine[b] = c;
             if (c) atomicAdd(&my_cnt[b], (unsigned long long)c);
         }
     }
 }
 
 // grid = (chunks, workers).  Move every rank of the chunk into its bucket's slice of `sorted`.
-// SMEM: the CTA counts its chunk per bucket, reserves one contiguous piece of every bucket's
-// slice with a single global atomic per bucket, and hands out places inside it from shared memory.
+// SMEM: with the chunk's histogram from the rank step the CTA reserves one contiguous piece of
+// every bucket's slice (a single global atomic per bucket) and hands out places inside it from
+// shared memory.
 template <bool SMEM>
 __global__ void __launch_bounds__(1024) scatter_kernel(uint32_t k_exp, uint32_t chunk, uint32_t s, uint32_t buckets,
                                                        const uint32_t* __restrict__ rho, uint64_t rho_stride,
                                                        const unsigned long long* __restrict__ pref,
                                                        uint64_t cnt_stride, uint32_t* __restrict__ cursor,
+                                                       const uint32_t* __restrict__ cta_hist,
                                                        uint32_t* __restrict__ sorted) {
-    extern __shared__ uint32_t sh[];
-    uint32_t* sh_count = sh;              // per bucket: entries of this chunk
-    uint32_t* sh_base = sh + buckets;     // per bucket: first place of this CTA's piece, then the running place
+    extern __shared__ uint32_t sh_place[];   // per bucket: next free place of this CTA's piece
     const uint32_t worker = blockIdx.y;
     const uint32_t* my_rho = rho + (uint64_t)worker * rho_stride;
     uint32_t* my_sorted = sorted + (uint64_t)worker * rho_stride;
@@ -182,25 +186,34 @@ __global__ void __launch_bounds__(1024) scatter_kernel(uint32_t k_exp, uint32_t 
     const uint64_t c0 = (uint64_t)blockIdx.x * chunk;
     const uint64_t c1 = (c0 + chunk < k_exp) ? c0 + chunk : k_exp;
     if (SMEM) {
-        for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) sh_count[b] = 0;
-        __syncthreads();
-        for (uint64_t j = c0 + threadIdx.x; j < c1; j += blockDim.x) atomicAdd(&sh_count[my_rho[j] >> s], 1u);
-        __syncthreads();
+        const uint32_t* mine = cta_hist + ((uint64_t)worker * gridDim.x + blockIdx.x) * buckets;
         for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) {
-            const uint32_t c = sh_count[b];
-            sh_base[b] = c ? (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], c) : 0u;
+            const uint32_t c = mine[b];
+            sh_place[b] = c ? (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], c) : 0u;
         }
         __syncthreads();
     }
-    for (uint64_t j = c0 + threadIdx.x; j < c1; j += blockDim.x) {
-        const uint32_t x = my_rho[j];
-        const uint32_t b = x >> s;
-        const uint32_t pos = SMEM ? atomicAdd(&sh_base[b], 1u) : (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], 1u);
-        if (pos < k_exp) my_sorted[pos] = x;
+    for (uint64_t j0 = c0 + threadIdx.x; j0 < c1; j0 += 4ull * blockDim.x) {
+        uint32_t x[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint64_t j = j0 + (uint64_t)q * blockDim.x;
+            x[q] = (j < c1) ? my_rho[j] : 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint64_t j = j0 + (uint64_t)q * blockDim.x;
+            if (j < c1) {
+                const uint32_t b = x[q] >> s;
+                const uint32_t pos =
+                    SMEM ? atomicAdd(&sh_place[b], 1u) : (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], 1u);
+                if (pos < k_exp) my_sorted[pos] = x[q];
+            }
+        }
     }
 }
 
-constexpr uint32_t kDirCache = 1024;
+constexpr uint32_t kDirCache = 2048;
 constexpr uint32_t kListCap = 4096;
 
 // grid = (buckets, workers).  Sort the bucket's ranks through a shared bitmap and emit parameter indices.
@@ -209,9 +222,9 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
     uint32_t k_exp, uint32_t s, const uint32_t* __restrict__ sorted, uint64_t rho_stride,
     const unsigned long long* __restrict__ cnt, const unsigned long long* __restrict__ pref,
     const unsigned long long* __restrict__ totals, uint64_t cnt_stride, PtrArray<uint32_t> out, WsHeader* hdr) {
-    __shared__ uint32_t bm[2048];            // up to 2^16 rank bits
-    __shared__ uint32_t dir_sh[kDirCache];   // the directory entries of the bucket's blocks
-    __shared__ uint16_t list[kListCap];      // sorted ranks (low s bits) of the current round
+    __shared__ uint32_t bm[2048];                // up to 2^16 rank bits
+    __shared__ uint32_t dir_sh[kDirCache + 1];   // directory entries of the bucket's 256-parameter groups (+1)
+    __shared__ uint16_t list[kListCap];          // sorted ranks (low s bits) of the current round
     __shared__ uint32_t warp_sums[kBucketThreads / 32];
     const uint32_t worker = blockIdx.y, bucket = blockIdx.x, t = threadIdx.x;
     const uint32_t words = 1u << (s - 5);
@@ -221,12 +234,12 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
     if (bucket == 0 && t == 0 && totals[worker] != k_exp) hdr->status = SLIMDP_ERR_INTERNAL;
     if (count == 0) return;
     for (uint32_t i = t; i < words; i += kBucketThreads) bm[i] = 0;
-    // the bucket's ranks live in bitmap blocks [blk_lo, blk_hi]
-    const uint32_t blk_lo = __ldg(bounds + bucket), blk_hi = __ldg(bounds + bucket + 1);
-    const uint32_t nblk = blk_hi - blk_lo + 1;
-    const bool cached = nblk <= kDirCache;
+    // the bucket's ranks live in directory groups [grp_lo, grp_hi]
+    const uint32_t grp_lo = __ldg(bounds + bucket), grp_hi = __ldg(bounds + bucket + 1);
+    const uint32_t ngrp = grp_hi - grp_lo + 1;
+    const bool cached = ngrp <= kDirCache;
     if (cached)
-        for (uint32_t i = t; i < nblk; i += kBucketThreads) dir_sh[i] = __ldg(dir + blk_lo + i);
+        for (uint32_t i = t; i <= ngrp; i += kBucketThreads) dir_sh[i] = __ldg(dir + grp_lo + i);
     __syncthreads();
     const uint32_t* my_sorted = sorted + (uint64_t)worker * rho_stride + offset;
     const uint32_t low_mask = (1u << s) - 1u;
@@ -264,13 +277,13 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
         }
         __syncthreads();
         const uint32_t m = (count - r0 < kListCap) ? count - r0 : kListCap;
-        uint32_t rel = 0;     // block relative to blk_lo; ranks ascend inside a thread, so it only moves up
+        uint32_t rel = 0;     // group relative to grp_lo; ranks ascend inside a thread, so it only moves up
         for (uint32_t e = t; e < m; e += kBucketThreads) {
             const uint32_t rank = first_rank + list[e];
-            // select0(rank): block by binary search of the directory ...
-            uint32_t rem;
+            // select0(rank): the 256-parameter group by binary search of the directory ...
+            uint32_t d0, d1;
             if (cached) {
-                uint32_t lo = rel, hi = nblk - 1;
+                uint32_t lo = rel, hi = ngrp - 1;
                 while (lo < hi) {
                     const uint32_t mid = lo + ((hi - lo + 1) >> 1);
                     if (dir_sh[mid] <= rank)
@@ -279,36 +292,43 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
                         hi = mid - 1;
                 }
                 rel = lo;
-                rem = rank - dir_sh[rel];
+                d0 = dir_sh[rel];
+                d1 = dir_sh[rel + 1];
             } else {
-                rel = find_block(dir, blk_lo + rel, blk_hi, rank) - blk_lo;
-                rem = rank - __ldg(dir + blk_lo + rel);
+                rel = find_block(dir, grp_lo + rel, grp_hi, rank) - grp_lo;
+                d0 = __ldg(dir + grp_lo + rel);
+                d1 = __ldg(dir + grp_lo + rel + 1);
             }
-            // ... then the word holding the rem-th zero bit of the block, then the bit
-            const uint32_t blk = blk_lo + rel;
-            const uint32_t* blk_words = bitmap + (uint64_t)blk * kWordsPerBlock;
-            const uint4* wordsp = reinterpret_cast<const uint4*>(blk_words);
-            uint4 v[8];
+            const uint32_t grp = grp_lo + rel;
+            const uint32_t rem = rank - d0;
+            uint32_t idx;
+            if (d1 - d0 == kDirStride) {
+                idx = grp * kDirStride + rem;   // no core parameter in this group
+            } else {
+                // ... then the word holding the rem-th zero bit of the group, then the bit
+                const uint32_t* grp_words = bitmap + (uint64_t)grp * kWordsPerDir;
+                const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(grp_words));
+                const uint4 v1 = __ldg(reinterpret_cast<const uint4*>(grp_words) + 1);
+                const uint32_t w8[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                uint32_t zeros = 0, wsel = 0, before = 0, zword = 0;
 #pragma unroll
-            for (int g = 0; g < 8; ++g) v[g] = __ldg(wordsp + g);
-            uint32_t zeros = 0, wsel = 0, before = 0;
-#pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                const uint32_t c[4] = {32u - __popc(v[g].x), 32u - __popc(v[g].y), 32u - __popc(v[g].z),
-                                       32u - __popc(v[g].w)};
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    zeros += c[q];
-                    const bool passed = zeros <= rem;   // the whole word lies before the wanted zero
+                for (int q = 0; q < 8; ++q) {
+                    const uint32_t z = ~w8[q];
+                    const uint32_t after = zeros + __popc(z);
+                    const bool passed = after <= rem;          // the whole word lies before the wanted zero
+                    const bool here = !passed && zeros <= rem;  // the wanted zero is in this word
                     wsel += passed ? 1u : 0u;
-                    before = passed ? zeros : before;
+                    before = passed ? after : before;
+                    zword = here ? z : zword;
+                    zeros = after;
                 }
+                idx = (wsel < kWordsPerDir) ? grp * kDirStride + wsel * 32u + nth_set_bit(zword, rem - before)
+                                            : 0xFFFFFFFFu;
             }
-            if (wsel >= kWordsPerBlock || offset + r0 + e >= k_exp) {
+            if (idx == 0xFFFFFFFFu || offset + r0 + e >= k_exp) {
                 hdr->status = SLIMDP_ERR_INTERNAL;   // directory and bitmap disagree
             } else {
-                const uint32_t z = ~__ldg(blk_words + wsel);
-                dst[r0 + e] = blk * kBlock + wsel * 32u + nth_set_bit(z, rem - before);
+                dst[r0 + e] = idx;
             }
         }
         __syncthreads();
@@ -332,7 +352,7 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
     const ExploreWs L = explore_ws_layout(ws, n, k_exp, workers);
-    const uint64_t nb = num_blocks(n);
+    const uint64_t nd = num_blocks(n) * kDirPerBlock;
     const uint64_t M = n - k_core;
     const uint32_t* bitmap = reinterpret_cast<const uint32_t*>(core_aux);
     const uint32_t* dir =
@@ -343,7 +363,7 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
     const unsigned setup_threads = (unsigned)((buckets + 1 > 3ull * workers) ? buckets + 1 : 3ull * workers);
     explore_setup_kernel<<<(setup_threads + 255) / 256, 256, 0, st>>>(L.hdr, L.round_keys, (uint32_t)seed,
                                                                       (uint32_t)(seed >> 32), first_worker, workers,
-                                                                      round, dir, (uint32_t)nb, (uint32_t)M, s,
+                                                                      round, dir, (uint32_t)nd, (uint32_t)M, s,
                                                                       (uint32_t)buckets, L.bounds);
     SLIMDP_LAUNCHED(1);
     if (k_exp == 0) return SLIMDP_OK;
@@ -355,6 +375,7 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
 
     // about two 1024-thread CTAs per SM over all workers; every CTA owns one contiguous chunk of j
     uint64_t chunks = ((uint64_t)sms * 2 + workers - 1) / workers;
+    if (chunks * workers > kMaxExploreCtas) chunks = kMaxExploreCtas / workers;
     if (chunks > (k_exp + 1023) / 1024) chunks = (k_exp + 1023) / 1024;
     if (chunks == 0) chunks = 1;
     const uint32_t chunk = (uint32_t)((k_exp + chunks - 1) / chunks);
@@ -363,21 +384,24 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
     if (smem) {
         rank_kernel<true><<<grid, 1024, buckets * 4, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, h, s,
                                                            (uint32_t)buckets, L.round_keys, L.rho, L.rho_stride,
-                                                           L.cnt, L.cnt_stride);
+                                                           L.cnt, L.cnt_stride, L.cta_hist);
     } else {
         rank_kernel<false><<<grid, 1024, 0, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, h, s, (uint32_t)buckets,
-                                                  L.round_keys, L.rho, L.rho_stride, L.cnt, L.cnt_stride);
+                                                  L.round_keys, L.rho, L.rho_stride, L.cnt, L.cnt_stride,
+                                                  L.cta_hist);
     }
     SLIMDP_LAUNCHED(1);
     slimdp_status rc =
         launch_block_scan(L.cnt, L.pref, L.tile_sums, L.totals, buckets, workers, L.cnt_stride, L.tile_stride, st);
     if (rc != SLIMDP_OK) return rc;
     if (smem) {
-        scatter_kernel<true><<<grid, 1024, buckets * 8, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets, L.rho,
-                                                              L.rho_stride, L.pref, L.cnt_stride, L.cursor, L.sorted);
+        scatter_kernel<true><<<grid, 1024, buckets * 4, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets, L.rho,
+                                                              L.rho_stride, L.pref, L.cnt_stride, L.cursor,
+                                                              L.cta_hist, L.sorted);
     } else {
         scatter_kernel<false><<<grid, 1024, 0, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets, L.rho,
-                                                     L.rho_stride, L.pref, L.cnt_stride, L.cursor, L.sorted);
+                                                     L.rho_stride, L.pref, L.cnt_stride, L.cursor, L.cta_hist,
+                                                     L.sorted);
     }
     SLIMDP_LAUNCHED(1);
     bucket_kernel<<<dim3((unsigned)buckets, workers), kBucketThreads, 0, st>>>(

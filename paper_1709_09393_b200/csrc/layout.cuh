@@ -7,13 +7,19 @@ namespace slimdp {
 
 struct SelectWs {
     WsHeader* hdr;
-    uint32_t* hist;                 // 3 x 4096 bins
+    uint32_t* hist;                 // 6 x 4096 bins: three passes over all keys, three over the candidates
+    uint32_t* sample_hist;          // 65536 bins (top 16 key bits of the sampled keys)
+    uint32_t* coarse_hist;          // 256 bins (top 8 key bits of the sampled keys)
     uint32_t* G;                    // greater-than-threshold bitmap, nb * 32 words
     uint32_t* E;                    // equal-to-threshold bitmap, nb * 32 words
     unsigned long long* cnt;        // per block: #greater | #equal << 32
     unsigned long long* pref;       // exclusive scan of cnt
     unsigned long long* tile_sums;  // per scan tile
     unsigned long long* totals;     // [1]
+    uint32_t* cand_key;             // keys inside the bracket
+    uint32_t* cand_idx;             // and their parameter indices
+    uint64_t cand_cap;              // entries in each candidate array
+    size_t zero_bytes;              // header + histograms, contiguous, cleared at the start of every call
     size_t bytes;
 };
 
@@ -28,13 +34,19 @@ inline SelectWs select_ws_layout(void* ws, uint64_t n) {
         return r;
     };
     L.hdr = reinterpret_cast<WsHeader*>(take(sizeof(WsHeader)));
-    L.hist = reinterpret_cast<uint32_t*>(take(3 * 4096 * sizeof(uint32_t)));
+    L.hist = reinterpret_cast<uint32_t*>(take(6 * 4096 * sizeof(uint32_t)));
+    L.sample_hist = reinterpret_cast<uint32_t*>(take(65536 * sizeof(uint32_t)));
+    L.coarse_hist = reinterpret_cast<uint32_t*>(take(256 * sizeof(uint32_t)));
+    L.zero_bytes = off;
     L.G = reinterpret_cast<uint32_t*>(take(nb * kWordsPerBlock * 4));
     L.E = reinterpret_cast<uint32_t*>(take(nb * kWordsPerBlock * 4));
     L.cnt = reinterpret_cast<unsigned long long*>(take(nb * 8));
     L.pref = reinterpret_cast<unsigned long long*>(take(nb * 8));
     L.tile_sums = reinterpret_cast<unsigned long long*>(take(nt * 8));
     L.totals = reinterpret_cast<unsigned long long*>(take(8));
+    L.cand_cap = (n >= kBracketMinN) ? (n / 16 > 65536 ? n / 16 : 65536) : 0;
+    L.cand_key = reinterpret_cast<uint32_t*>(take(L.cand_cap * 4 + 16));
+    L.cand_idx = reinterpret_cast<uint32_t*>(take(L.cand_cap * 4 + 16));
     L.bytes = off;
     return L;
 }
@@ -47,6 +59,7 @@ struct ExploreWs {
     uint32_t* sorted;               // per worker: the same ranks grouped by bucket
     unsigned long long* cnt;        // per worker: ranks per bucket
     uint32_t* cursor;               // per worker: scatter cursors per bucket
+    uint32_t* cta_hist;             // per rank-step CTA: its chunk's ranks per bucket
     unsigned long long* pref;       // per worker: exclusive scan of cnt
     unsigned long long* tile_sums;  // per worker: per scan tile
     unsigned long long* totals;     // per worker: 1
@@ -56,6 +69,9 @@ struct ExploreWs {
     size_t zero_bytes;              // cnt and cursor, contiguous, cleared before every call
     size_t bytes;
 };
+
+constexpr uint64_t kMaxSmemBuckets = 5120;   // bucket histograms up to this size live in shared memory (20 KB)
+constexpr uint64_t kMaxExploreCtas = 1024;   // rank / scatter CTAs over all workers of one call
 
 // Upper bound on the number of rank buckets for any core size: buckets hold
 // 2^13 .. 2^16 ranks, 2^16 once there are at least 2^25 non-core parameters.
@@ -88,6 +104,8 @@ inline ExploreWs explore_ws_layout(void* ws, uint64_t n, uint64_t k_exp, uint32_
     L.pref = reinterpret_cast<unsigned long long*>(take((size_t)workers * L.cnt_stride * 8));
     L.tile_sums = reinterpret_cast<unsigned long long*>(take((size_t)workers * L.tile_stride * 8));
     L.totals = reinterpret_cast<unsigned long long*>(take((size_t)workers * 8));
+    const uint64_t hist_buckets = explore_max_buckets(n) < kMaxSmemBuckets ? explore_max_buckets(n) : kMaxSmemBuckets;
+    L.cta_hist = reinterpret_cast<uint32_t*>(take((size_t)kMaxExploreCtas * hist_buckets * 4));
     L.bytes = off;
     return L;
 }

@@ -1,17 +1,33 @@
 // slimdp_select_core: exact top-k_core of the scores (Section 3.2: rank by
 // significance, keep the top), ties to the smaller index.
 //
-// Keys are the scores' 32-bit patterns compared as unsigned integers.
-//   1. three most-significant-digit-first histogram passes (12 + 10 + 10 bits,
-//      shared-memory histograms flushed to global) find the exact k-th largest
-//      key T and the number r of keys equal to T that belong to the core;
-//   2. one pass classifies every key against T into two bitmaps (greater,
-//      equal) and counts both per 1024-parameter block;
-//   3. a two-kernel exclusive scan over the block counts;
-//   4. one pass over the bitmaps admits the first r equal keys in index order,
-//      writes the final core bitmap, the non-core rank directory and the
-//      ascending index list (ordered compaction: ballot/popc inside a warp,
-//      scanned block offsets across warps; no atomic cursors, no spinning).
+// Keys are the scores' 32-bit patterns compared as unsigned integers.  The
+// result is defined by the k-th largest key T and the number r of keys equal
+// to T that belong to the core (those with the smallest indices).
+//
+// Large inputs (n >= 2^21) take the bracketed path, which reads the scores once:
+//   1. sample: 2^18 evenly spaced keys are histogrammed by their top 16 bits
+//      (and by their top 8 bits); the last CTA to finish turns the histograms
+//      into a bracket of 16-bit bins [b_bot, b_top) that holds T with
+//      overwhelming probability;
+//   2. bracket pass (one read of all keys): keys in bins >= b_top are
+//      certainly in the core and go straight into the "greater" bitmap; keys
+//      inside the bracket are copied, with their indices, to a candidate list;
+//   3. if the counts prove the bracket right (n_def < k <= n_def + n_cand and
+//      the list did not overflow), three radix histogram passes over the
+//      candidates alone find T and r exactly, and one pass over the
+//      candidates adds them to the "greater" / "equal" bitmaps;
+//   4. otherwise the full path below runs (its kernels are always enqueued and
+//      return at once when the bracket held), so the result is exact for every input.
+// Full path (small inputs, or a failed bracket, e.g. one score value repeated
+// millions of times): three most-significant-digit-first histogram passes over
+// all keys (12 + 10 + 10 bits), then one classifying pass that writes both bitmaps.
+// Both paths end the same way: a two-kernel exclusive scan over per-1024-block
+// counts and one pass over the bitmaps that admits the first r equal keys in
+// index order and writes the core bitmap, the non-core rank directory and the
+// ascending index list (ordered compaction, no atomic cursors, no spinning).
+// Each histogram kernel's last CTA (found with an atomic ticket) also locates
+// the bin of the wanted rank, so no separate single-CTA launches are needed.
 #include "common.cuh"
 #include "layout.cuh"
 
@@ -23,12 +39,206 @@ constexpr int kHistThreads = 512;
 constexpr uint32_t kBins0 = 4096;   // pass 0: bits 31..20
 constexpr uint32_t kBins12 = 1024;  // pass 1: bits 19..10, pass 2: bits 9..0
 
+enum Mode : int { kFullAlways = 0, kFullIfBracketFailed = 1, kCandidates = 2 };
+
 __global__ void select_init_kernel(WsHeader* hdr, uint32_t k) {
     hdr->status = SLIMDP_OK;
     hdr->prefix = (k == 0) ? 0xFFFFFFFFu : 0u;   // k = 0: no key is greater than or (with r = 0) admitted at T
     hdr->k_rem = k;
     hdr->ties = 0;
 }
+
+// True when the bracket pass proved that T lies inside the bracket and every candidate was stored.
+__device__ __forceinline__ bool bracket_ok(const WsHeader* hdr, uint32_t k, uint32_t cap) {
+    const uint32_t n_def = hdr->n_def, n_cand = hdr->n_cand;
+    return n_def < k && k - n_def <= n_cand && n_cand <= cap;
+}
+
+__device__ __forceinline__ bool mode_runs(int mode, const WsHeader* hdr, uint32_t k, uint32_t cap) {
+    if (mode == kFullAlways) return true;
+    const bool ok = bracket_ok(hdr, k, cap);
+    return (mode == kCandidates) ? ok : !ok;
+}
+
+// ---- step 1: sample histogram and bracket ------------------------------------------------
+
+// 2^18 evenly spaced keys are counted by their top 16 bits (fine, 65536 bins) and by their top
+// 8 bits (coarse, 256 bins).  The last CTA to finish locates, in the coarse histogram, the two
+// coarse bins where the count from the top crosses the two target ranks, and resolves each
+// crossing inside the 256 fine bins of that coarse bin.
+__global__ void __launch_bounds__(1024) sample_bracket_kernel(const uint32_t* __restrict__ keys, uint64_t n,
+                                                              uint32_t k, WsHeader* hdr,
+                                                              uint32_t* __restrict__ sample_hist,
+                                                              uint32_t* __restrict__ coarse_hist) {
+    __shared__ bool last;
+    __shared__ unsigned long long smem[33];
+    __shared__ uint32_t sh_coarse[256];
+    __shared__ long long s_incl[256];
+    __shared__ uint32_t s_val[2];
+    const uint32_t t = threadIdx.x;
+    if (t < 256) sh_coarse[t] = 0;
+    __syncthreads();
+    const uint32_t j = blockIdx.x * 1024 + t;   // sample number, < 2^18
+    const uint64_t pos = ((uint64_t)j * n) >> kSampleBits;
+    const uint32_t key = __ldg(keys + pos);
+    atomicAdd(&sample_hist[key >> 16], 1u);
+    atomicAdd(&sh_coarse[key >> 24], 1u);
+    __syncthreads();
+    if (t < 256 && sh_coarse[t]) atomicAdd(&coarse_hist[t], sh_coarse[t]);
+    __threadfence();
+    __syncthreads();
+    if (t == 0) last = atomicAdd(&hdr->ticket[6], 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    // the sample rank of T is about r = k * samples / n; keep 6 standard deviations (+16) on each side
+    const double samples = (double)(1u << kSampleBits);
+    const double p = (double)k / (double)n;
+    const double r = p * samples;
+    const double margin = 6.0 * sqrt(samples * p * (1.0 - p)) + 16.0;
+    const long long lo_target = (long long)floor(r - margin);
+    const long long hi_target = (long long)ceil(r + margin);
+    const volatile uint32_t* fine = sample_hist;
+    const volatile uint32_t* coarse = coarse_hist;
+    // coarse bins from the top down: thread t < 256 owns coarse bin 255 - t
+    unsigned long long total;
+    const unsigned long long c = (t < 256) ? coarse[255 - t] : 0ull;
+    const long long c_above = (long long)block_exclusive_scan64<32>(c, smem, &total);
+    if (t < 256) s_incl[255 - t] = c_above + (long long)c;   // samples in coarse bins >= 255 - t
+    if (t < 2) s_val[t] = 0xFFFFFFFFu;
+    __syncthreads();
+    // b_top: lowest fine bin b with (samples in bins >= b) <= lo_target; 65536 if there is none.
+    // b_bot: highest fine bin b with (samples in bins >= b) >= hi_target; 0 if there is none.
+    // which = 0 resolves b_top, which = 1 resolves b_bot; both walk one coarse bin's 256 fine bins.
+    for (int which = 0; which < 2; ++which) {
+        const long long target = which ? hi_target : lo_target;
+        // crossing coarse bin: the highest one whose inclusive count exceeds (which = 0) / reaches (which = 1) the target
+        if (t < 256) {
+            const long long incl = s_incl[t], above = (t == 255) ? 0 : s_incl[t + 1];
+            const bool here = which ? (incl >= target && above < target) : (incl > target && above <= target);
+            if (here) s_val[which] = t;
+        }
+        __syncthreads();
+        const uint32_t cx = s_val[which];
+        __syncthreads();
+        uint32_t result;
+        if (cx == 0xFFFFFFFFu) {
+            // no crossing: which = 0: target < 0 (nothing certain, 65536) or every bin qualifies (0);
+            //              which = 1: target above the sample size, or target <= 0: every bin may hold T
+            result = which ? 0u : ((target < 0) ? 65536u : 0u);
+            if (t == 0) s_val[which] = result;
+            __syncthreads();
+            continue;
+        }
+        const long long above_cx = (cx == 255) ? 0 : s_incl[cx + 1];
+        // fine bins of coarse bin cx from the top down: thread t < 256 owns fine bin cx * 256 + 255 - t
+        const unsigned long long f = (t < 256) ? fine[cx * 256 + 255 - t] : 0ull;
+        const long long f_above = (long long)block_exclusive_scan64<32>(f, smem, &total);
+        if (t == 0) s_val[which] = which ? 0u : (cx + 1) * 256u;   // default when no fine bin of cx qualifies
+        __syncthreads();
+        if (t < 256) {
+            const uint32_t b = cx * 256 + 255 - t;
+            const long long incl = above_cx + f_above + (long long)f;
+            if (which == 0) {
+                if (incl <= target) atomicMin(&s_val[0], b);
+            } else {
+                if (incl >= target) atomicMax(&s_val[1], b);
+            }
+        }
+        __syncthreads();
+    }
+    if (t == 0) {
+        hdr->b_top = s_val[0];
+        hdr->b_bot = s_val[1];
+    }
+}
+
+// ---- step 2: one pass over all keys ------------------------------------------------------
+
+constexpr uint32_t kFlushAt = 128;             // a warp appends its staged candidates once it holds this many
+constexpr uint32_t kStage = kFlushAt + 256;    // staging capacity: below kFlushAt before a quarter block, +256 in it
+
+// Warp per 1024-parameter block, a quarter block (8 words) at a time.  Candidates are staged per
+// warp in shared memory and appended to the global list at least kFlushAt at a time, so the
+// list cursor sees one atomic per kFlushAt candidates or more.
+__global__ void __launch_bounds__(256) bracket_pass_kernel(const uint32_t* __restrict__ keys, uint64_t n, uint64_t nb,
+                                                           WsHeader* hdr, uint32_t cap, uint32_t* __restrict__ G,
+                                                           uint32_t* __restrict__ E,
+                                                           unsigned long long* __restrict__ cnt,
+                                                           uint32_t* __restrict__ cand_key,
+                                                           uint32_t* __restrict__ cand_idx) {
+    __shared__ uint32_t st_key[8][kStage], st_idx[8][kStage];
+    __shared__ uint32_t cta_def;
+    const uint32_t b_top = hdr->b_top, b_bot = hdr->b_bot;
+    const uint32_t lane = lane_id(), wid = threadIdx.x >> 5;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    uint32_t* my_key = st_key[wid];
+    uint32_t* my_idx = st_idx[wid];
+    if (threadIdx.x == 0) cta_def = 0;
+    __syncthreads();
+    uint32_t staged = 0, def_acc = 0;
+    auto flush = [&](uint32_t m) {
+        uint32_t base = 0;
+        if (lane == 0) base = atomicAdd(&hdr->n_cand, m);
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        if ((uint64_t)base + m <= cap) {   // else: overflow, n_cand > cap sends the call down the full path
+            for (uint32_t e = lane; e < m; e += 32) {
+                cand_key[base + e] = my_key[e];
+                cand_idx[base + e] = my_idx[e];
+            }
+        }
+        __syncwarp();
+    };
+    const uint64_t warps = (uint64_t)gridDim.x * (blockDim.x >> 5);
+    for (uint64_t blk = (uint64_t)blockIdx.x * (blockDim.x >> 5) + wid; blk < nb; blk += warps) {
+        const uint64_t base = blk * kBlock;
+        const bool full = base + kBlock <= n;
+        uint32_t myG = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint32_t key[8];
+#pragma unroll
+            for (int wd = 0; wd < 8; ++wd) {
+                const uint64_t i = base + (q * 8 + wd) * 32 + lane;
+                key[wd] = (full || i < n) ? __ldcs(keys + i) : 0u;
+            }
+            uint32_t place = staged;
+#pragma unroll
+            for (int wd = 0; wd < 8; ++wd) {
+                const uint32_t off = (q * 8 + wd) * 32 + lane;
+                const bool in = full || (base + off < n);
+                const uint32_t bin = key[wd] >> 16;
+                const bool cand = in && bin >= b_bot && bin < b_top;
+                const uint32_t bg = __ballot_sync(0xFFFFFFFFu, in && bin >= b_top);
+                const uint32_t bc = __ballot_sync(0xFFFFFFFFu, cand);
+                if (lane == (uint32_t)(q * 8 + wd)) myG = bg;
+                if (cand) {
+                    const uint32_t slot = place + __popc(bc & lt_mask);
+                    my_key[slot] = key[wd];
+                    my_idx[slot] = (uint32_t)(base + off);
+                }
+                place += __popc(bc);
+            }
+            staged = place;
+            __syncwarp();
+            if (staged >= kFlushAt) {
+                flush(staged);
+                staged = 0;
+            }
+        }
+        G[blk * kWordsPerBlock + lane] = myG;
+        E[blk * kWordsPerBlock + lane] = 0u;
+        const uint32_t cg = __reduce_add_sync(0xFFFFFFFFu, __popc(myG));
+        if (lane == 0) cnt[blk] = cg;
+        def_acc += cg;
+    }
+    if (staged) flush(staged);
+    if (lane == 0 && def_acc) atomicAdd(&cta_def, def_acc);
+    __syncthreads();
+    if (threadIdx.x == 0 && cta_def) atomicAdd(&hdr->n_def, cta_def);
+}
+
+// ---- radix histogram passes (over all keys, or over the candidates) -----------------------
 
 template <int PASS>
 __device__ __forceinline__ void hist_key(uint32_t key, uint32_t prefix, uint32_t* sh) {
@@ -41,12 +251,22 @@ __device__ __forceinline__ void hist_key(uint32_t key, uint32_t prefix, uint32_t
     }
 }
 
+// Histogram of one radix digit; the last CTA to finish then walks the histogram
+// from the top bin down and records the bin that holds the wanted rank.
 template <int PASS>
-__global__ void __launch_bounds__(kHistThreads) hist_kernel(const uint32_t* __restrict__ keys, uint64_t n,
-                                                            const WsHeader* __restrict__ hdr,
-                                                            uint32_t* __restrict__ hist) {
+__global__ void __launch_bounds__(kHistThreads) hist_kernel(const uint32_t* __restrict__ all_keys, uint64_t n_all,
+                                                            const uint32_t* __restrict__ cand_key, WsHeader* hdr,
+                                                            uint32_t* __restrict__ hist, uint32_t k, uint32_t cap,
+                                                            int mode) {
     constexpr uint32_t NB = (PASS == 0) ? kBins0 : kBins12;
+    constexpr uint32_t PER = NB / kHistThreads;
+    constexpr uint32_t SHIFT = (PASS == 0) ? 20 : (PASS == 1 ? 10 : 0);
     __shared__ uint32_t sh[NB];
+    __shared__ unsigned long long smem[33];
+    __shared__ bool last;
+    if (!mode_runs(mode, hdr, k, cap)) return;
+    const uint32_t* keys = (mode == kCandidates) ? cand_key : all_keys;
+    const uint64_t n = (mode == kCandidates) ? hdr->n_cand : n_all;
     for (uint32_t b = threadIdx.x; b < NB; b += kHistThreads) sh[b] = 0;
     __syncthreads();
     const uint32_t prefix = (PASS == 0) ? 0u : hdr->prefix;
@@ -74,36 +294,38 @@ __global__ void __launch_bounds__(kHistThreads) hist_kernel(const uint32_t* __re
         uint32_t c = sh[b];
         if (c) atomicAdd(&hist[b], c);
     }
-}
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(&hdr->ticket[PASS + (mode == kCandidates ? 0 : 3)], 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
 
-// One block of 1024 threads: walk the histogram from the top bin down and
-// find the bin holding the k_rem-th largest key.
-template <int PASS>
-__global__ void __launch_bounds__(1024) find_bin_kernel(WsHeader* hdr, const uint32_t* __restrict__ hist) {
-    constexpr uint32_t NB = (PASS == 0) ? kBins0 : kBins12;
-    constexpr uint32_t PER = NB / 1024;
-    constexpr uint32_t SHIFT = (PASS == 0) ? 20 : (PASS == 1 ? 10 : 0);
-    __shared__ unsigned long long smem[33];
-    const uint32_t k = hdr->k_rem;
-    const uint32_t prefix = hdr->prefix;
+    // rank wanted inside the current prefix
+    uint32_t want;
+    if (PASS == 0)
+        want = (mode == kCandidates) ? k - hdr->n_def : k;
+    else
+        want = hdr->k_rem;
+    const volatile uint32_t* gh = hist;
     const uint32_t top = NB - 1 - threadIdx.x * PER;   // this thread's highest bin
     uint32_t h[PER];
     unsigned long long sum = 0;
 #pragma unroll
     for (uint32_t q = 0; q < PER; ++q) {
-        h[q] = hist[top - q];
+        h[q] = gh[top - q];
         sum += h[q];
     }
     unsigned long long total;
-    unsigned long long above = block_exclusive_scan64_1024(sum, smem, &total);
-    if (total < k) {
+    unsigned long long above = block_exclusive_scan64<kHistThreads / 32>(sum, smem, &total);
+    if (total < want) {
         if (threadIdx.x == 0) hdr->status = SLIMDP_ERR_INTERNAL;
         return;
     }
 #pragma unroll
     for (uint32_t q = 0; q < PER; ++q) {
-        if (above < k && (unsigned long long)k <= above + h[q]) {
-            const uint32_t rem = k - (uint32_t)above;
+        if (above < want && (unsigned long long)want <= above + h[q]) {
+            const uint32_t rem = want - (uint32_t)above;
             hdr->prefix = prefix | ((top - q) << SHIFT);
             hdr->k_rem = rem;
             if (PASS == 2) hdr->ties = rem;
@@ -112,11 +334,39 @@ __global__ void __launch_bounds__(1024) find_bin_kernel(WsHeader* hdr, const uin
     }
 }
 
+// ---- step 3: candidates into the bitmaps --------------------------------------------------
+
+__global__ void __launch_bounds__(256) mark_candidates_kernel(const uint32_t* __restrict__ cand_key,
+                                                              const uint32_t* __restrict__ cand_idx,
+                                                              const WsHeader* __restrict__ hdr, uint32_t k,
+                                                              uint32_t cap, uint32_t* __restrict__ G,
+                                                              uint32_t* __restrict__ E,
+                                                              unsigned long long* __restrict__ cnt) {
+    if (!bracket_ok(hdr, k, cap)) return;
+    const uint32_t T = hdr->prefix, n_cand = hdr->n_cand;
+    const uint32_t stride = gridDim.x * blockDim.x;
+    for (uint32_t c = blockIdx.x * blockDim.x + threadIdx.x; c < n_cand; c += stride) {
+        const uint32_t key = __ldg(cand_key + c);
+        if (key < T) continue;
+        const uint32_t i = __ldg(cand_idx + c);
+        if (key > T) {
+            atomicOr(&G[i >> 5], 1u << (i & 31u));
+            atomicAdd(&cnt[i / kBlock], 1ull);
+        } else {
+            atomicOr(&E[i >> 5], 1u << (i & 31u));
+            atomicAdd(&cnt[i / kBlock], 1ull << 32);
+        }
+    }
+}
+
+// ---- full path: classify every key against T ----------------------------------------------
+
 // Warp per 1024-parameter block: two bitmap words per lane and the block's counts.
 __global__ void __launch_bounds__(256) classify_kernel(const uint32_t* __restrict__ keys, uint64_t n, uint64_t nb,
-                                                       const WsHeader* __restrict__ hdr, uint32_t* __restrict__ G,
-                                                       uint32_t* __restrict__ E,
+                                                       const WsHeader* __restrict__ hdr, uint32_t k, uint32_t cap,
+                                                       int mode, uint32_t* __restrict__ G, uint32_t* __restrict__ E,
                                                        unsigned long long* __restrict__ cnt) {
+    if (!mode_runs(mode, hdr, k, cap)) return;
     const uint32_t T = hdr->prefix;
     const uint32_t lane = lane_id();
     const uint64_t warps = (uint64_t)gridDim.x * (blockDim.x >> 5);
@@ -157,6 +407,8 @@ __global__ void __launch_bounds__(256) classify_kernel(const uint32_t* __restric
     }
 }
 
+// ---- last step: bitmaps to core bitmap, directory and ascending index list ----------------
+
 // Warp per 1024-parameter block, bitmaps only.
 __global__ void __launch_bounds__(256) emit_kernel(const uint32_t* __restrict__ G, const uint32_t* __restrict__ E,
                                                    const unsigned long long* __restrict__ pref,
@@ -173,7 +425,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const uint32_t* __restrict__ 
         const unsigned long long t = totals[0];
         const uint32_t ng = (uint32_t)t, ne = (uint32_t)(t >> 32);
         if (ng + min(ne, ties) != k_core) hdr->status = SLIMDP_ERR_INTERNAL;
-        dir[nb] = (uint32_t)(n - k_core);
+        dir[nb * kDirPerBlock] = (uint32_t)(n - k_core);
     }
     for (uint64_t blk = warp0; blk < nb; blk += warps) {
         const uint32_t Gw = G[blk * kWordsPerBlock + lane];
@@ -195,20 +447,40 @@ __global__ void __launch_bounds__(256) emit_kernel(const uint32_t* __restrict__ 
         const uint32_t sel = Gw | Ea;
         const uint32_t ps = __popc(sel);
         const uint32_t sel_before = g_before + min(e_before, ties);
-        const uint32_t out_base = sel_before + warp_inclusive_scan(ps) - ps;
+        const uint32_t ps_incl = warp_inclusive_scan(ps);
+        const uint32_t out_base = sel_before + ps_incl - ps;
         bitmap[blk * kWordsPerBlock + lane] = sel;
-        if (lane == 0) dir[blk] = (uint32_t)(blk * kBlock - sel_before);
-        const uint32_t any = __ballot_sync(0xFFFFFFFFu, sel != 0);
-        for (uint32_t m = any; m; m &= m - 1) {
-            const int wd = __ffs(m) - 1;
-            const uint32_t word = __shfl_sync(0xFFFFFFFFu, sel, wd);
-            const uint32_t base = __shfl_sync(0xFFFFFFFFu, out_base, wd);
-            if ((word >> lane) & 1u) {
-                const uint32_t pos = base + __popc(word & ((1u << lane) - 1u));
+        if ((lane & (kWordsPerDir - 1)) == 0)   // one directory entry per 256 parameters (8 words)
+            dir[blk * kDirPerBlock + lane / kWordsPerDir] = (uint32_t)(blk * kBlock + lane * 32 - out_base);
+        const uint32_t in_block = __shfl_sync(0xFFFFFFFFu, ps_incl, 31);
+        if (in_block == 0) continue;
+        const uint32_t first = (uint32_t)(blk * kBlock);
+        if (in_block <= 256) {
+            // sparse block: every lane writes out its own word's members
+            uint32_t word = sel, pos = out_base;
+            while (word) {
+                const uint32_t bit = __ffs(word) - 1;
+                word &= word - 1;
                 if (pos < k_core)
-                    core_idx[pos] = (uint32_t)(blk * kBlock + wd * 32 + lane);
+                    core_idx[pos] = first + lane * 32 + bit;
                 else
                     hdr->status = SLIMDP_ERR_INTERNAL;
+                ++pos;
+            }
+        } else {
+            // dense block: the warp writes one word's members at a time (coalesced)
+            const uint32_t any = __ballot_sync(0xFFFFFFFFu, sel != 0);
+            for (uint32_t m = any; m; m &= m - 1) {
+                const int wd = __ffs(m) - 1;
+                const uint32_t word = __shfl_sync(0xFFFFFFFFu, sel, wd);
+                const uint32_t base = __shfl_sync(0xFFFFFFFFu, out_base, wd);
+                if ((word >> lane) & 1u) {
+                    const uint32_t pos = base + __popc(word & ((1u << lane) - 1u));
+                    if (pos < k_core)
+                        core_idx[pos] = first + wd * 32 + lane;
+                    else
+                        hdr->status = SLIMDP_ERR_INTERNAL;
+                }
             }
         }
     }
@@ -225,28 +497,48 @@ slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, ui
     const uint32_t* keys = reinterpret_cast<const uint32_t*>(scores);
     uint32_t* bitmap = reinterpret_cast<uint32_t*>(core_aux);
     uint32_t* dir = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(core_aux) + slimdp_core_aux_dir_offset(n));
+    const uint32_t k = (uint32_t)k_core;
+    const uint32_t cap = (uint32_t)L.cand_cap;
 
-    select_init_kernel<<<1, 1, 0, st>>>(L.hdr, (uint32_t)k_core);
+    // header, radix histograms and sample histogram are contiguous: one clear
+    if (cudaMemsetAsync(L.hdr, 0, L.zero_bytes, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
+    select_init_kernel<<<1, 1, 0, st>>>(L.hdr, k);
     SLIMDP_LAUNCHED(1);
-    if (k_core > 0) {
-        if (cudaMemsetAsync(L.hist, 0, 3 * kBins0 * sizeof(uint32_t), st) != cudaSuccess) return SLIMDP_ERR_CUDA;
-        const unsigned hgrid = (unsigned)sms * 4;
-        hist_kernel<0><<<hgrid, kHistThreads, 0, st>>>(keys, n, L.hdr, L.hist);
-        find_bin_kernel<0><<<1, 1024, 0, st>>>(L.hdr, L.hist);
-        hist_kernel<1><<<hgrid, kHistThreads, 0, st>>>(keys, n, L.hdr, L.hist + kBins0);
-        find_bin_kernel<1><<<1, 1024, 0, st>>>(L.hdr, L.hist + kBins0);
-        hist_kernel<2><<<hgrid, kHistThreads, 0, st>>>(keys, n, L.hdr, L.hist + 2 * kBins0);
-        find_bin_kernel<2><<<1, 1024, 0, st>>>(L.hdr, L.hist + 2 * kBins0);
-        SLIMDP_LAUNCHED(6);
-    }
     uint64_t cgrid = (nb + 7) / 8;
     if (cgrid > (uint64_t)sms * 8) cgrid = (uint64_t)sms * 8;
-    classify_kernel<<<(unsigned)cgrid, 256, 0, st>>>(keys, n, nb, L.hdr, L.G, L.E, L.cnt);
+    const unsigned hgrid = (unsigned)sms * 4;
+    const bool bracketed = k_core > 0 && n >= kBracketMinN;
+    if (bracketed) {
+        sample_bracket_kernel<<<(1u << kSampleBits) / 1024, 1024, 0, st>>>(keys, n, k, L.hdr, L.sample_hist,
+                                                                              L.coarse_hist);
+        bracket_pass_kernel<<<(unsigned)cgrid, 256, 0, st>>>(keys, n, nb, L.hdr, cap, L.G, L.E, L.cnt, L.cand_key,
+                                                             L.cand_idx);
+        // T and r from the candidates (these return at once if the bracket failed) ...
+        const unsigned cand_grid = (unsigned)sms;
+        hist_kernel<0><<<cand_grid, kHistThreads, 0, st>>>(keys, n, L.cand_key, L.hdr, L.hist + 3 * kBins0, k, cap,
+                                                           kCandidates);
+        hist_kernel<1><<<cand_grid, kHistThreads, 0, st>>>(keys, n, L.cand_key, L.hdr, L.hist + 4 * kBins0, k, cap,
+                                                           kCandidates);
+        hist_kernel<2><<<cand_grid, kHistThreads, 0, st>>>(keys, n, L.cand_key, L.hdr, L.hist + 5 * kBins0, k, cap,
+                                                           kCandidates);
+        mark_candidates_kernel<<<(unsigned)sms * 4, 256, 0, st>>>(L.cand_key, L.cand_idx, L.hdr, k, cap, L.G, L.E,
+                                                                  L.cnt);
+        SLIMDP_LAUNCHED(6);
+    }
+    if (k_core > 0) {
+        // ... or from all keys (these return at once if the bracket held)
+        const int mode = bracketed ? kFullIfBracketFailed : kFullAlways;
+        hist_kernel<0><<<hgrid, kHistThreads, 0, st>>>(keys, n, L.cand_key, L.hdr, L.hist, k, cap, mode);
+        hist_kernel<1><<<hgrid, kHistThreads, 0, st>>>(keys, n, L.cand_key, L.hdr, L.hist + kBins0, k, cap, mode);
+        hist_kernel<2><<<hgrid, kHistThreads, 0, st>>>(keys, n, L.cand_key, L.hdr, L.hist + 2 * kBins0, k, cap, mode);
+        SLIMDP_LAUNCHED(3);
+    }
+    classify_kernel<<<(unsigned)cgrid, 256, 0, st>>>(keys, n, nb, L.hdr, k, cap,
+                                                     bracketed ? kFullIfBracketFailed : kFullAlways, L.G, L.E, L.cnt);
     SLIMDP_LAUNCHED(1);
     slimdp_status s = launch_block_scan(L.cnt, L.pref, L.tile_sums, L.totals, nb, 1, nb, num_scan_tiles(n), st);
     if (s != SLIMDP_OK) return s;
-    emit_kernel<<<(unsigned)cgrid, 256, 0, st>>>(L.G, L.E, L.pref, L.totals, n, nb, (uint32_t)k_core, L.hdr,
-                                                 core_idx, bitmap, dir);
+    emit_kernel<<<(unsigned)cgrid, 256, 0, st>>>(L.G, L.E, L.pref, L.totals, n, nb, k, L.hdr, core_idx, bitmap, dir);
     SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }

@@ -46,11 +46,11 @@ def expected_aux(P, core: np.ndarray, n: int):
     member = np.zeros(nb * 1024, np.uint8)
     member[core] = 1
     words = np.packbits(member.reshape(-1, 8), axis=1, bitorder="little").reshape(-1).view(np.uint32)
-    per_block = member.reshape(nb, 1024).sum(axis=1, dtype=np.int64)
-    sizes = np.full(nb, 1024, np.int64)
-    directory = np.zeros(nb + 1, np.int64)
-    directory[1:] = np.cumsum(sizes - per_block)
-    directory[nb] = n - core.size
+    nd = nb * 4
+    per_group = member.reshape(nd, 256).sum(axis=1, dtype=np.int64)
+    directory = np.zeros(nd + 1, np.int64)
+    directory[1:] = np.cumsum(256 - per_group)       # 256 d minus the core members below 256 d
+    directory[nd] = n - core.size
     return words, directory.astype(np.uint32)
 
 
@@ -71,7 +71,7 @@ def check_aux(P, aux: torch.Tensor, core: np.ndarray, n: int):
     words, directory = expected_aux(P, core, n)
     assert np.array_equal(raw[:nb * 128].view(np.uint32), words)
     off = P.core_aux_dir_offset(n)
-    assert np.array_equal(raw[off:off + 4 * (nb + 1)].view(np.uint32), directory)
+    assert np.array_equal(raw[off:off + 4 * (4 * nb + 1)].view(np.uint32), directory)
 
 
 # --------------------------------------------------------------------- score
@@ -144,6 +144,30 @@ def test_select_large_tie_group_spanning_many_blocks(P):
     exp = oracle.select_core(S, k)
     assert np.array_equal(host_u32(core_idx), exp)
     check_aux(P, aux, exp, n)
+
+
+@pytest.mark.parametrize("case", ["random", "all_equal", "sampler_fooled", "two_values", "narrow_band"])
+def test_select_bracketed_path_and_its_fallback(P, case):
+    # n >= 2^21 takes the sampled-bracket path; inputs that defeat the sample or
+    # overflow the candidate list must still give the exact core through the full path
+    n = (1 << 22) + 77
+    rng = np.random.default_rng(len(case))
+    if case == "random":
+        S = np.abs(rng.standard_normal(n)).astype(np.float32)
+    elif case == "all_equal":
+        S = np.full(n, 0.5, np.float32)
+    elif case == "sampler_fooled":
+        S = np.abs(rng.standard_normal(n)).astype(np.float32)
+        S[::16] = 100.0                      # the evenly spaced sample sees (almost) only these
+    elif case == "two_values":
+        S = rng.integers(0, 2, n).astype(np.float32)
+    else:
+        S = (1.0 + rng.integers(0, 4000, n) * 2.0 ** -23).astype(np.float32)   # 4000 adjacent bit patterns
+    for k in (1, 1000, n // 20, n // 3, n - 1, n):
+        core_idx, aux = gpu_select(P, S, k)
+        exp = oracle.select_core(S, k)
+        assert np.array_equal(host_u32(core_idx), exp), (case, k)
+        check_aux(P, aux, exp, n)
 
 
 # ------------------------------------------------------------------- explore
@@ -319,7 +343,7 @@ def test_round_is_deterministic(P):
     nb = (cfg.N + 1023) // 1024
     off = P.core_aux_dir_offset(cfg.N)
     assert torch.equal(a.core_aux[:nb * 128], b.core_aux[:nb * 128])                      # bitmap
-    assert torch.equal(a.core_aux[off:off + 4 * (nb + 1)], b.core_aux[off:off + 4 * (nb + 1)])   # directory
+    assert torch.equal(a.core_aux[off:off + 4 * (4 * nb + 1)], b.core_aux[off:off + 4 * (4 * nb + 1)])   # directory
     for k in range(cfg.K):
         assert torch.equal(a.exp_idx[k], b.exp_idx[k]) and torch.equal(a.pulled[k], b.pulled[k])
 
