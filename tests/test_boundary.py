@@ -12,8 +12,12 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 @pytest.fixture(scope="module")
 def P():
-    from paper_1709_09393_b200 import build
-    build.build()
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("_slimdp_cuda_build",
+                                                  os.path.join(ROOT, "paper_1709_09393_b200", "build.py"))
+    build = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(build)
+    build.build()          # the package refuses to import without its library, so build by file path first
     import paper_1709_09393_b200 as pkg
     return pkg
 
