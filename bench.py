@@ -224,9 +224,8 @@ def run_ours(args):
     def round_after_score(t):
         P.slimdp_select_core(buf.scores, k_core, buf.core_idx, buf.core_aux, buf.select_ws)
         P.slimdp_sample_explore_batched(buf.core_aux, N, k_core, k_exp, cfg.seed, 0, t, buf.exp_idx, buf.explore_ws)
-        P.slimdp_pack_batched(grads, buf.core_idx, buf.exp_idx, buf.val)
-        P.slimdp_merge(w, buf.core_idx, buf.exp_idx, buf.val, cfg.eta)
-        P.slimdp_pull_batched(w, buf.core_idx, buf.exp_idx, buf.pulled)
+        # push (pack), server update (merge) and pull of all K workers in one fused call
+        P.slimdp_exchange(w, grads, buf.core_idx, buf.exp_idx, cfg.eta, buf.val, buf.pulled)
 
     # warm-up: successive rounds t = 0, 1, ... on the evolving model, as in training
     t = 0
@@ -266,18 +265,21 @@ def run_ours(args):
     value = aggregate_value(N, world, ms_per_step)
 
     # ---- per-call breakdown (untimed for the headline; 5 more rounds) -------
-    names = ["score", "select", "explore", "pack", "merge", "pull"]
+    # "exchange" is the fused pack + merge + pull the timed rounds use; the three separate calls
+    # are timed after it for comparison (they repeat the exchange's work on the next model state)
+    names = ["score", "select", "explore", "exchange", "pack_alone", "merge_alone", "pull_alone"]
     acc = {nm: [] for nm in names}
     for _ in range(5):
-        marks = [torch.cuda.Event(enable_timing=True) for _ in range(7)]
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(8)]
         marks[0].record()
         P.slimdp_score(w, grads, cfg.c, buf.scores); marks[1].record()
         P.slimdp_select_core(buf.scores, k_core, buf.core_idx, buf.core_aux, buf.select_ws); marks[2].record()
         P.slimdp_sample_explore_batched(buf.core_aux, N, k_core, k_exp, cfg.seed, 0, t, buf.exp_idx, buf.explore_ws)
         marks[3].record()
-        P.slimdp_pack_batched(grads, buf.core_idx, buf.exp_idx, buf.val); marks[4].record()
-        P.slimdp_merge(w, buf.core_idx, buf.exp_idx, buf.val, cfg.eta); marks[5].record()
-        P.slimdp_pull_batched(w, buf.core_idx, buf.exp_idx, buf.pulled); marks[6].record()
+        P.slimdp_exchange(w, grads, buf.core_idx, buf.exp_idx, cfg.eta, buf.val, buf.pulled); marks[4].record()
+        P.slimdp_pack_batched(grads, buf.core_idx, buf.exp_idx, buf.val); marks[5].record()
+        P.slimdp_merge(w, buf.core_idx, buf.exp_idx, buf.val, cfg.eta); marks[6].record()
+        P.slimdp_pull_batched(w, buf.core_idx, buf.exp_idx, buf.pulled); marks[7].record()
         torch.cuda.synchronize()
         t += 1
         for i, nm in enumerate(names):

@@ -200,6 +200,19 @@ slimdp_status slimdp_pull_batched(const float* w_global, uint32_t K, uint64_t n,
                                   uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
                                   float* const* out, void* stream);
 
+/* ------------------------------------------------------------- exchange ---
+ * Push, server update and pull of one round for all K workers in one call
+ * (Section 3.3 steps 3 and 4; Algorithm 1's Push, Update, Pull).  The results
+ * are bit-identical to slimdp_pack_batched, then slimdp_merge, then
+ * slimdp_pull_batched on the same arguments; the three steps share one pass
+ * over the communication set, so every gathered line is fetched once.
+ *   w_global [n] (updated in place), deltas HOST array of K device pointers [n] (read)
+ *   val, pulled  HOST arrays of K device pointers, each [k_core + k_exp] (written)
+ */
+slimdp_status slimdp_exchange(float* w_global, uint64_t n, uint32_t K, const float* const* deltas,
+                              const uint32_t* core_idx, uint64_t k_core, const uint32_t* const* exp_idx,
+                              uint64_t k_exp, float eta, float* const* val, float* const* pulled, void* stream);
+
 /* --------------------------------------------------------------- status ---
  * Synchronises `stream`, then returns the sticky status word kept in the first
  * 4 bytes of a workspace used by slimdp_select_core / slimdp_sample_explore*:
@@ -213,8 +226,8 @@ slimdp_status slimdp_read_status(const void* ws, void* stream);
 uint64_t slimdp_launch_count(void);
 
 /* ----------------------------------------------------- whole round, host ---
- * One whole round (score, select, K x explore, K x pack, merge, K x pull) on
- * HOST buffers: copies w and the K updates to the device, runs the round
+ * One whole round (score, select, K x explore, then the exchange: K x pack,
+ * merge, K x pull) on HOST buffers: copies w and the K updates to the device, runs the round
  * above, copies the results back, and synchronises before returning.
  *   w_host       HOST [n]: global model, replaced by the merged model
  *   grads_host   HOST array of K HOST pointers, each [n]

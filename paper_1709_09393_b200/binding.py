@@ -45,6 +45,7 @@ EXPORTS = {
     "slimdp_merge": (ctypes.c_int32, [_vp, _u64, _u32, _vp, _u64, _pp, _u64, _pp, _f32, _vp]),
     "slimdp_pull": (ctypes.c_int32, [_vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp]),
     "slimdp_pull_batched": (ctypes.c_int32, [_vp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _vp]),
+    "slimdp_exchange": (ctypes.c_int32, [_vp, _u64, _u32, _pp, _vp, _u64, _pp, _u64, _f32, _pp, _pp, _vp]),
     "slimdp_read_status": (ctypes.c_int32, [_vp, _vp]),
     "slimdp_launch_count": (_u64, []),
     "slimdp_round_arena_bytes": (_sz, [_u64, _u32, _u64, _u64]),
@@ -234,6 +235,25 @@ def slimdp_pull_batched(w_global: torch.Tensor, core_idx: torch.Tensor, exp_idx:
     _check("slimdp_pull_batched",
            lib.slimdp_pull_batched(w_global.data_ptr(), K, w_global.numel(), _ptr(core_idx), core_idx.numel(),
                                    _ptr_array(exp_idx), exp_idx[0].numel(), _ptr_array(out), _stream(stream)))
+
+
+def slimdp_exchange(w_global: torch.Tensor, deltas: Sequence[torch.Tensor], core_idx: torch.Tensor,
+                    exp_idx: Sequence[torch.Tensor], eta: float, val: Sequence[torch.Tensor],
+                    pulled: Sequence[torch.Tensor], stream=None):
+    """Push + update + pull for all workers; same results as pack_batched, merge, pull_batched."""
+    _dev(w_global, torch.float32, "w_global")
+    K = len(deltas)
+    if len(exp_idx) != K or len(val) != K or len(pulled) != K:
+        raise ValueError("deltas, exp_idx, val and pulled must have K entries each")
+    for d, e, v, o in zip(deltas, exp_idx, val, pulled):
+        if _dev(d, torch.float32, "deltas").numel() != w_global.numel():
+            raise ValueError("deltas: length differs from w_global")
+        _check_sets(core_idx, e, v, "val")
+        _check_sets(core_idx, e, o, "pulled")
+    _check("slimdp_exchange",
+           lib.slimdp_exchange(w_global.data_ptr(), w_global.numel(), K, _ptr_array(deltas), _ptr(core_idx),
+                               core_idx.numel(), _ptr_array(exp_idx), exp_idx[0].numel(), eta, _ptr_array(val),
+                               _ptr_array(pulled), _stream(stream)))
 
 
 def _host(t: torch.Tensor, dtype, name: str) -> torch.Tensor:

@@ -28,6 +28,11 @@ static std::atomic<unsigned long long> g_launches{0};
 
 void count_launches(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<const float>& delta,
+                              const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,
+                              uint64_t k_exp, float eta, const PtrArray<float>& val, const PtrArray<float>& pulled,
+                              cudaStream_t st);
+
 int sm_count() {
     static int cached[64];
     int dev = 0;
@@ -212,6 +217,23 @@ slimdp_status slimdp_merge(float* w_global, uint64_t n, uint32_t K, const uint32
     return launch_merge(w_global, n, K, core_idx, k_core, exp, k_exp, v, eta, (cudaStream_t)stream);
 }
 
+slimdp_status slimdp_exchange(float* w_global, uint64_t n, uint32_t K, const float* const* deltas,
+                              const uint32_t* core_idx, uint64_t k_core, const uint32_t* const* exp_idx,
+                              uint64_t k_exp, float eta, float* const* val, float* const* pulled, void* stream) {
+    if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !w_global || !aligned4(w_global) || !isfinite(eta))
+        return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    PtrArray<const float> d;
+    PtrArray<const uint32_t> exp;
+    PtrArray<float> v, o;
+    if (!fill<const float>(d, deltas, K, true, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<float>(v, val, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<float>(o, pulled, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core + k_exp == 0) return SLIMDP_OK;
+    return launch_exchange(w_global, n, K, d, core_idx, k_core, exp, k_exp, eta, v, o, (cudaStream_t)stream);
+}
+
 uint64_t slimdp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 slimdp_status slimdp_read_status(const void* ws, void* stream) {
@@ -309,9 +331,8 @@ slimdp_status slimdp_round_host(float* w_host, const float* const* grads_host, u
                                   stream));
     SLIMDP_TRY(slimdp_sample_explore_batched(A.core_aux, n, k_core, k_exp, seed, 0, K, round, A.exp_idx,
                                              A.explore_ws, A.explore_ws_bytes, stream));
-    SLIMDP_TRY(slimdp_pack_batched(A.delta, K, n, A.core_idx, k_core, A.exp_idx, k_exp, A.val, stream));
-    SLIMDP_TRY(slimdp_merge(A.w, n, K, A.core_idx, k_core, A.exp_idx, k_exp, A.val, eta, stream));
-    SLIMDP_TRY(slimdp_pull_batched(A.w, K, n, A.core_idx, k_core, A.exp_idx, k_exp, A.pulled, stream));
+    SLIMDP_TRY(slimdp_exchange(A.w, n, K, A.delta, A.core_idx, k_core, A.exp_idx, k_exp, eta, A.val, A.pulled,
+                               stream));
     SLIMDP_CUDA(cudaMemcpyAsync(w_host, A.w, n * 4, cudaMemcpyDeviceToHost, st));
     if (k_core) SLIMDP_CUDA(cudaMemcpyAsync(core_idx_host, A.core_idx, k_core * 4, cudaMemcpyDeviceToHost, st));
     for (uint32_t k = 0; k < K; ++k) {

@@ -1,22 +1,25 @@
 // slimdp_merge: the server update of Section 3.3 step 3,
 // w <- w - eta' * T_C(delta_k) for every worker, applied in ascending worker
-// order so that the fp32 result is unique.
+// order so that the fp32 result is unique; and slimdp_exchange, which does the
+// push (extraction), that update and the pull (Section 3.3 step 4) in one pass.
 //
 // Core segment: one thread owns one core parameter and folds the K pushed
 // values into it in worker order (K coalesced value streams, one gather and
 // one scatter).
 // Explorer segments: different workers' explorers may contain the same
 // parameter (never a core one), so the order across workers matters.  The
-// parameter vector is cut into ranges; one CTA owns one range, finds each
+// parameter vector is cut into ranges; one warp owns one range, finds each
 // worker's entries inside it by binary search of the ascending index lists,
-// and applies worker 0's entries, a block barrier, worker 1's entries, ...
-// Inside one worker the indices are distinct, and no other CTA touches the
+// and applies worker 0's entries, a warp barrier, worker 1's entries, ...
+// Inside one worker the indices are distinct, and no other warp touches the
 // range, so a parameter receives its updates in ascending k without atomics.
 #include "common.cuh"
 
 namespace slimdp {
 
 namespace {
+
+constexpr int kMergeWarps = 8;
 
 __global__ void __launch_bounds__(256) merge_core_kernel(float* __restrict__ w, const uint32_t* __restrict__ core_idx,
                                                          uint64_t k_core, PtrArray<const float> val, int K,
@@ -51,32 +54,127 @@ __device__ __forceinline__ uint32_t lower_bound(const uint32_t* __restrict__ a, 
     return lo;
 }
 
-__global__ void __launch_bounds__(256) merge_explore_kernel(float* w, uint64_t n, PtrArray<const uint32_t> exp,
-                                                            uint32_t k_exp, PtrArray<const float> val,
-                                                            uint64_t k_core, int K, float neg_eta,
-                                                            uint32_t range_shift) {
-    __shared__ uint32_t begin[SLIMDP_MAX_WORKERS], end[SLIMDP_MAX_WORKERS];
-    const uint64_t first = (uint64_t)blockIdx.x << range_shift;
-    const uint64_t last = first + (1ull << range_shift);
-    for (int t = threadIdx.x; t < 2 * K; t += blockDim.x) {
-        const int k = (t < K) ? t : t - K;
-        const uint32_t pos = lower_bound(exp.p[k], k_exp, (t < K) ? first : last);
-        if (t < K)
-            begin[k] = pos;
-        else
-            end[k] = pos;
+// bound[k][r]: where the r-th of the CTA's 9 range boundaries falls in worker k's index list.
+__device__ __forceinline__ void find_bounds(uint32_t (*bound)[kMergeWarps + 1], const PtrArray<const uint32_t>& exp,
+                                            uint32_t k_exp, int K, uint32_t range_shift) {
+    const uint64_t first = ((uint64_t)blockIdx.x * kMergeWarps) << range_shift;
+    for (int t = threadIdx.x; t < K * (kMergeWarps + 1); t += blockDim.x) {
+        const int k = t / (kMergeWarps + 1), r = t % (kMergeWarps + 1);
+        bound[k][r] = lower_bound(exp.p[k], k_exp, first + ((uint64_t)r << range_shift));
     }
     __syncthreads();
+}
+
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// One CTA owns 8 consecutive ranges of 2^range_shift parameters, one per warp.  Every warp, on
+// its own, first requests all lines it is going to touch (L2 prefetch), then applies worker 0's
+// entries of its range, a warp barrier, worker 1's entries, ...
+__global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* w, PtrArray<const uint32_t> exp,
+                                                                         uint32_t k_exp, PtrArray<const float> val,
+                                                                         uint64_t k_core, int K, float neg_eta,
+                                                                         uint32_t range_shift) {
+    __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
+    find_bounds(bound, exp, k_exp, K, range_shift);
+    const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
+    for (int k = 0; k < K; ++k) {
+        const uint32_t* __restrict__ idx = exp.p[k];
+        const uint32_t b = bound[k][wid + 1];
+        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) prefetch_l2(w + __ldg(idx + e));
+    }
     for (int k = 0; k < K; ++k) {
         const uint32_t* __restrict__ idx = exp.p[k];
         const float* __restrict__ v = val.p[k] + k_core;
-        const uint32_t b = end[k];
-        for (uint32_t e = begin[k] + threadIdx.x; e < b; e += blockDim.x) {
+        const uint32_t b = bound[k][wid + 1];
+        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) {
             const uint32_t i = __ldg(idx + e);
             w[i] = __fmaf_rn(neg_eta, __ldcs(v + e), w[i]);
         }
-        __syncthreads();   // worker k's updates are visible to the whole CTA before worker k+1 starts
+        __syncwarp();   // worker k's updates are visible to the whole warp before worker k+1 starts
     }
+}
+
+// ---- push + server update + pull in one pass (slimdp_exchange) -----------------------------
+
+// Core segment: thread j gathers the K workers' updates of core parameter core_idx[j] (the
+// push), folds them into the parameter in worker order (the update) and hands the merged value
+// back to all K workers (the pull).  One read of the key, K gathers, one read-modify-write.
+__global__ void __launch_bounds__(256) exchange_core_kernel(float* __restrict__ w,
+                                                            const uint32_t* __restrict__ core_idx, uint64_t k_core,
+                                                            PtrArray<const float> delta, PtrArray<float> val,
+                                                            PtrArray<float> pulled, int K, float neg_eta) {
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k_core; j += stride) {
+        const uint32_t i = __ldg(core_idx + j);
+        float x = w[i];
+        int k = 0;
+        for (; k + 8 <= K; k += 8) {
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = __ldg(delta.p[k + q] + i);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                __stcs(val.p[k + q] + j, v[q]);
+                x = __fmaf_rn(neg_eta, v[q], x);
+            }
+        }
+        for (; k < K; ++k) {
+            const float v = __ldg(delta.p[k] + i);
+            __stcs(val.p[k] + j, v);
+            x = __fmaf_rn(neg_eta, v, x);
+        }
+        w[i] = x;
+#pragma unroll 8
+        for (int q = 0; q < K; ++q) __stcs(pulled.p[q] + j, x);
+    }
+}
+
+// Explorer segments: warp-owned ranges as in merge_explore_kernel.  Per worker, in ascending
+// order, the warp gathers the worker's updates inside its range, stores them as the pushed
+// values and applies them; after the last worker it reads the merged values back for every
+// worker's pull (they are still in cache).
+__global__ void __launch_bounds__(kMergeWarps * 32) exchange_explore_kernel(
+    float* w, PtrArray<const uint32_t> exp, uint32_t k_exp, PtrArray<const float> delta, PtrArray<float> val,
+    PtrArray<float> pulled, uint64_t k_core, int K, float neg_eta, uint32_t range_shift) {
+    __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
+    find_bounds(bound, exp, k_exp, K, range_shift);
+    const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
+    for (int k = 0; k < K; ++k) {
+        const uint32_t* __restrict__ idx = exp.p[k];
+        const float* __restrict__ d = delta.p[k];
+        const uint32_t b = bound[k][wid + 1];
+        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) {
+            const uint32_t i = __ldg(idx + e);
+            prefetch_l2(w + i);
+            prefetch_l2(d + i);
+        }
+    }
+    for (int k = 0; k < K; ++k) {
+        const uint32_t* __restrict__ idx = exp.p[k];
+        const float* __restrict__ d = delta.p[k];
+        float* __restrict__ v = val.p[k] + k_core;
+        const uint32_t b = bound[k][wid + 1];
+        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) {
+            const uint32_t i = __ldg(idx + e);
+            const float u = __ldg(d + i);
+            __stcs(v + e, u);
+            w[i] = __fmaf_rn(neg_eta, u, w[i]);
+        }
+        __syncwarp();   // worker k's updates are visible to the whole warp before worker k+1 starts
+    }
+    for (int k = 0; k < K; ++k) {
+        const uint32_t* __restrict__ idx = exp.p[k];
+        float* __restrict__ o = pulled.p[k] + k_core;
+        const uint32_t b = bound[k][wid + 1];
+        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) __stcs(o + e, w[__ldg(idx + e)]);
+    }
+}
+
+// Range per warp: a power of two with 16 to 32 entries per worker on average, at least 32 parameters.
+uint32_t explore_range_shift(uint64_t n, uint64_t k_exp) {
+    uint32_t shift = 5;
+    while (shift < 24 && ((k_exp << (shift + 1)) / n) <= 32) ++shift;
+    return shift;
 }
 
 }  // namespace
@@ -94,12 +192,35 @@ slimdp_status launch_merge(float* w, uint64_t n, uint32_t K, const uint32_t* cor
         SLIMDP_LAUNCHED(1);
     }
     if (k_exp > 0) {
-        // range length: a power of two with about 256 entries per worker per range, at least 1024 parameters
-        uint32_t shift = 10;
-        while (shift < 24 && ((k_exp << shift) / n) < 256) ++shift;
-        const uint64_t ranges = (n + (1ull << shift) - 1) >> shift;
-        merge_explore_kernel<<<(unsigned)ranges, 256, 0, st>>>(w, n, exp, (uint32_t)k_exp, val, k_core, (int)K,
-                                                               neg_eta, shift);
+        const uint32_t shift = explore_range_shift(n, k_exp);
+        const uint64_t per_cta = (uint64_t)kMergeWarps << shift;
+        const uint64_t ctas = (n + per_cta - 1) / per_cta;
+        merge_explore_kernel<<<(unsigned)ctas, kMergeWarps * 32, 0, st>>>(w, exp, (uint32_t)k_exp, val, k_core,
+                                                                          (int)K, neg_eta, shift);
+        SLIMDP_LAUNCHED(1);
+    }
+    return SLIMDP_OK;
+}
+
+slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<const float>& delta,
+                              const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,
+                              uint64_t k_exp, float eta, const PtrArray<float>& val, const PtrArray<float>& pulled,
+                              cudaStream_t st) {
+    const int sms = sm_count();
+    if (sms <= 0) return SLIMDP_ERR_CUDA;
+    const float neg_eta = -eta;
+    if (k_core > 0) {
+        uint64_t grid = (k_core + 255) / 256;
+        if (grid > (uint64_t)sms * 32) grid = (uint64_t)sms * 32;
+        exchange_core_kernel<<<(unsigned)grid, 256, 0, st>>>(w, core_idx, k_core, delta, val, pulled, (int)K, neg_eta);
+        SLIMDP_LAUNCHED(1);
+    }
+    if (k_exp > 0) {
+        const uint32_t shift = explore_range_shift(n, k_exp);
+        const uint64_t per_cta = (uint64_t)kMergeWarps << shift;
+        const uint64_t ctas = (n + per_cta - 1) / per_cta;
+        exchange_explore_kernel<<<(unsigned)ctas, kMergeWarps * 32, 0, st>>>(w, exp, (uint32_t)k_exp, delta, val, pulled,
+                                                                             k_core, (int)K, neg_eta, shift);
         SLIMDP_LAUNCHED(1);
     }
     return SLIMDP_OK;

@@ -29,13 +29,17 @@ class RoundBuffers:
 
 
 def run_round(w: torch.Tensor, grads: Sequence[torch.Tensor], c: float, seed: int, rnd: int, eta: float,
-              buf: RoundBuffers, with_score: bool = True) -> None:
-    """Enqueue one round on the current stream; w is merged in place."""
+              buf: RoundBuffers, with_score: bool = True, fused_exchange: bool = True) -> None:
+    """Enqueue one round on the current stream; w is merged in place.  fused_exchange selects
+    slimdp_exchange over the three separate calls (identical results)."""
     n, k_core, k_exp = buf.n, buf.k_core, buf.k_exp
     if with_score:
         B.slimdp_score(w, grads, c, buf.scores)
     B.slimdp_select_core(buf.scores, k_core, buf.core_idx, buf.core_aux, buf.select_ws)
     B.slimdp_sample_explore_batched(buf.core_aux, n, k_core, k_exp, seed, 0, rnd, buf.exp_idx, buf.explore_ws)
+    if fused_exchange:
+        B.slimdp_exchange(w, grads, buf.core_idx, buf.exp_idx, eta, buf.val, buf.pulled)
+        return
     B.slimdp_pack_batched(grads, buf.core_idx, buf.exp_idx, buf.val)
     B.slimdp_merge(w, buf.core_idx, buf.exp_idx, buf.val, eta)
     B.slimdp_pull_batched(w, buf.core_idx, buf.exp_idx, buf.pulled)

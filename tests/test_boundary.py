@@ -98,6 +98,9 @@ def test_invalid_arguments_are_rejected_on_the_host(P):
     assert lib.slimdp_merge(fake, 10, 2, fake, 5, arr, 5, arr, float("inf"), None) == INVALID
     assert lib.slimdp_merge(fake, 10, 2, fake, 5, null_in, 5, arr, 0.5, None) == INVALID
     assert lib.slimdp_merge(None, 10, 2, fake, 5, arr, 5, arr, 0.5, None) == INVALID
+    assert lib.slimdp_exchange(fake, 10, 2, arr, fake, 5, arr, 5, 0.5, arr, null_in, None) == INVALID
+    assert lib.slimdp_exchange(fake, 10, 2, null_in, fake, 5, arr, 5, 0.5, arr, arr, None) == INVALID
+    assert lib.slimdp_exchange(fake, 10, 2, arr, fake, 5, arr, 6, 0.5, arr, arr, None) == INVALID
     # whole round on host buffers
     assert lib.slimdp_round_host(fake, arr, 2, 10, 1.0, 5, 5, 0, 0, 0.5, fake, arr, arr, None, 0, None) == INVALID
     assert lib.slimdp_round_host(fake, arr, 2, 10, 1.0, 5, 5, 0, 0, 0.5, fake, arr, arr, fake, 16, None) == WORKSPACE

@@ -248,6 +248,15 @@ def test_pack_merge_pull_parity(P, n, k_core, k_exp, K):
         assert np.array_equal(host_bits(outs[k]), bits(exp_out))
         P.slimdp_pull(d_w, d_core, d_exps[k], one)
         assert np.array_equal(host_bits(one), bits(exp_out))
+    # the fused push + update + pull gives the same three results
+    f_w = dev(w)
+    f_vals = [torch.zeros(m, dtype=torch.float32, device="cuda") for _ in range(K)]
+    f_outs = [torch.zeros(m, dtype=torch.float32, device="cuda") for _ in range(K)]
+    P.slimdp_exchange(f_w, d_ds, d_core, d_exps, eta, f_vals, f_outs)
+    assert np.array_equal(host_bits(f_w), bits(exp_w))
+    for k in range(K):
+        assert np.array_equal(host_bits(f_vals[k]), bits(exp_vals[k]))
+        assert np.array_equal(host_bits(f_outs[k]), bits(oracle.pull(exp_w, core, exps[k])))
 
 
 def test_merge_collisions_follow_worker_order(P):
@@ -264,15 +273,28 @@ def test_merge_collisions_follow_worker_order(P):
     rev = oracle.merge(w, none, [exp] * K, vals[::-1], 1.0 / 3.0)
     assert not np.array_equal(bits(fwd), bits(rev))        # the order matters for these values
     assert np.array_equal(host_bits(d_w), bits(fwd))
+    # same through the fused call: worker k's update vector holds vals[k] on the shared explorer
+    ds = []
+    for k in range(K):
+        d = np.zeros(n, np.float32)
+        d[exp] = vals[k]
+        ds.append(dev(d))
+    f_w = dev(w)
+    f_vals = [torch.empty(exp.size, dtype=torch.float32, device="cuda") for _ in range(K)]
+    f_outs = [torch.empty(exp.size, dtype=torch.float32, device="cuda") for _ in range(K)]
+    P.slimdp_exchange(f_w, ds, dev(none), [dev(exp)] * K, 1.0 / 3.0, f_vals, f_outs)
+    assert np.array_equal(host_bits(f_w), bits(fwd))
+    for k in range(K):
+        assert np.array_equal(host_bits(f_outs[k]), bits(fwd[exp]))
 
 
 # --------------------------------------------------------------- whole round
 
-def gpu_round(P, w, gs, cfg_c, k_core, k_exp, seed, rnd, eta):
+def gpu_round(P, w, gs, cfg_c, k_core, k_exp, seed, rnd, eta, fused=True):
     n, K = w.size, len(gs)
     buf = P.RoundBuffers(n, K, k_core, k_exp)
     d_w, d_gs = dev(w), [dev(g) for g in gs]
-    P.run_round(d_w, d_gs, cfg_c, seed, rnd, eta, buf)
+    P.run_round(d_w, d_gs, cfg_c, seed, rnd, eta, buf, fused_exchange=fused)
     P.read_status(buf.select_ws)
     P.read_status(buf.explore_ws)
     return d_w, buf
@@ -292,8 +314,10 @@ def assert_round_equal(P, d_w, buf, ref, n):
 def _round_case(P, cfg, rnd=0):
     w, gs = all_inputs(cfg)
     ref = oracle.run_round(w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta)
-    d_w, buf = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta)
-    assert_round_equal(P, d_w, buf, ref, cfg.N)
+    for fused in (True, False):      # slimdp_exchange, and the three separate calls
+        d_w, buf = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta, fused)
+        assert_round_equal(P, d_w, buf, ref, cfg.N)
+        del d_w, buf
     return w, gs, ref
 
 
