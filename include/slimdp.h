@@ -153,6 +153,34 @@ slimdp_status slimdp_sample_explore_batched(const void* core_aux, uint64_t n, ui
                                             uint32_t round, uint32_t* const* exp_idx, void* ws,
                                             size_t ws_bytes, void* stream);
 
+/* The paper has no counterpart of this call; it exists for callers that cannot
+ * allocate.  slimdp_sample_explore needs a workspace, and some callers have no
+ * way to get one: code that runs after a host application has handed all device
+ * memory to its own pool, a plug-in whose host forbids cudaMalloc inside the
+ * training loop because it would stall every stream, or a process running
+ * under a memory cap that is already spent.  For them this variant draws one
+ * worker's explorer with the library's own scratch: a static device array of
+ * SLIMDP_STATIC_SCRATCH_MIB MiB that every GPU holding this library keeps from
+ * load until the process exits.  It calls no allocator of any kind.
+ *   Same arguments and same result (bit for bit) as slimdp_sample_explore,
+ *   without ws / ws_bytes.  Limits: n <= SLIMDP_STATIC_MAX_N and
+ *   k_exp <= SLIMDP_STATIC_MAX_K_EXP; anything larger returns
+ *   SLIMDP_ERR_UNSUPPORTED and enqueues nothing.
+ *   status   optional DEVICE int32 (may be NULL): receives, in stream order, the
+ *            call's device-side consistency status (SLIMDP_OK or SLIMDP_ERR_INTERNAL).
+ * The first call on each device looks up the scratch array's device address
+ * (cudaGetSymbolAddress, with that device current); make that first call
+ * outside any stream capture.  All calls on a device share the one array and
+ * each call overwrites what the last one left (it clears what it needs at zero
+ * itself), so two calls that may run at the same time on the GPU, e.g. on
+ * different streams, race; order them. */
+#define SLIMDP_STATIC_SCRATCH_MIB 8
+#define SLIMDP_STATIC_MAX_N (1ull << 25)
+#define SLIMDP_STATIC_MAX_K_EXP (1ull << 18)
+slimdp_status slimdp_sample_explore_static(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp,
+                                           uint64_t seed, uint32_t worker, uint32_t round, uint32_t* exp_idx,
+                                           int32_t* status, void* stream);
+
 /* ----------------------------------------------------------------- pack ---
  * Extraction of T_C(delta_k) = T_S(delta_k) U T_R^k(delta_k) (Section 3.1; the
  * "extract ... by scanning" cost of Section 3.5):

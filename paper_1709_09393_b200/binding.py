@@ -40,6 +40,7 @@ EXPORTS = {
     "slimdp_sample_explore": (ctypes.c_int32, [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _vp, _vp, _sz, _vp]),
     "slimdp_sample_explore_batched": (ctypes.c_int32,
                                       [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _u32, _pp, _vp, _sz, _vp]),
+    "slimdp_sample_explore_static": (ctypes.c_int32, [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _vp, _vp, _vp]),
     "slimdp_pack": (ctypes.c_int32, [_vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp]),
     "slimdp_pack_batched": (ctypes.c_int32, [_pp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _vp]),
     "slimdp_merge": (ctypes.c_int32, [_vp, _u64, _u32, _vp, _u64, _pp, _u64, _pp, _f32, _vp]),
@@ -173,6 +174,22 @@ def slimdp_sample_explore_batched(core_aux: torch.Tensor, n: int, k_core: int, k
            lib.slimdp_sample_explore_batched(core_aux.data_ptr(), n, k_core, k_exp, seed, first_worker,
                                              len(exp_idx), rnd, _ptr_array(exp_idx), ws.data_ptr(),
                                              ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def slimdp_sample_explore_static(core_aux: torch.Tensor, n: int, k_core: int, k_exp: int, seed: int, worker: int,
+                                 rnd: int, exp_idx: torch.Tensor, status: Optional[torch.Tensor] = None,
+                                 stream=None):
+    """slimdp_sample_explore for callers that cannot allocate a workspace: the library's own
+    static scratch is used (n <= 2^25, k_exp <= 2^18).  `status`, if given, is a one-element
+    int32 CUDA tensor that receives the device-side consistency status in stream order."""
+    _dev(exp_idx, IDX, "exp_idx")
+    if exp_idx.numel() != k_exp:
+        raise ValueError("exp_idx: length differs from k_exp")
+    if status is not None:
+        _dev(status, torch.int32, "status")
+    _check("slimdp_sample_explore_static",
+           lib.slimdp_sample_explore_static(core_aux.data_ptr(), n, k_core, k_exp, seed, worker, rnd, _ptr(exp_idx),
+                                            _ptr(status), _stream(stream)))
 
 
 def _check_sets(core_idx, exp_idx, out, what):

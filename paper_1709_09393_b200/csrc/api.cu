@@ -33,6 +33,10 @@ slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<c
                               uint64_t k_exp, float eta, const PtrArray<float>& val, const PtrArray<float>& pulled,
                               cudaStream_t st);
 
+slimdp_status launch_explore_static(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
+                                    uint32_t worker, uint32_t round, uint32_t* exp_idx, int32_t* status_out,
+                                    cudaStream_t st);
+
 int sm_count() {
     static int cached[64];
     int dev = 0;
@@ -153,6 +157,17 @@ slimdp_status slimdp_sample_explore(const void* core_aux, uint64_t n, uint64_t k
     uint32_t* one[1] = {exp_idx};
     return slimdp_sample_explore_batched(core_aux, n, k_core, k_exp, seed, worker, 1, round, one, ws, ws_bytes,
                                          stream);
+}
+
+slimdp_status slimdp_sample_explore_static(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp,
+                                           uint64_t seed, uint32_t worker, uint32_t round, uint32_t* exp_idx,
+                                           int32_t* status, void* stream) {
+    if (!sets_ok(n, k_core, k_exp) || !core_aux || !aligned16(core_aux)) return SLIMDP_ERR_INVALID_ARG;
+    if (k_exp > 0 && (!exp_idx || !aligned16(exp_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (status && !aligned4(status)) return SLIMDP_ERR_INVALID_ARG;
+    if (n > SLIMDP_STATIC_MAX_N || k_exp > SLIMDP_STATIC_MAX_K_EXP) return SLIMDP_ERR_UNSUPPORTED;
+    return launch_explore_static(core_aux, n, k_core, k_exp, seed, worker, round, exp_idx, status,
+                                 (cudaStream_t)stream);
 }
 
 static slimdp_status gather_common(const float* const* srcs, bool same_src, const float* src0, uint32_t K,

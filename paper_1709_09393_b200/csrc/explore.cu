@@ -411,4 +411,37 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
     return SLIMDP_OK;
 }
 
+// ---- explorer sampling without a caller-supplied workspace ---------------------------------
+
+// Scratch for slimdp_sample_explore_static.  The array lives in every device that loads this
+// library, from load to process exit.  Its name is only a handle in host code; the device
+// address comes from cudaGetSymbolAddress (once per device, cached below).
+constexpr size_t kStaticScratchBytes = (size_t)SLIMDP_STATIC_SCRATCH_MIB << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+slimdp_status launch_explore_static(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
+                                    uint32_t worker, uint32_t round, uint32_t* exp_idx, int32_t* status_out,
+                                    cudaStream_t st) {
+    static void* scratch_addr[64];   // per device; every thread that races here stores the same value
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SLIMDP_ERR_CUDA;
+    if (scratch_addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return SLIMDP_ERR_CUDA;
+        scratch_addr[dev] = p;
+    }
+    if (explore_ws_layout(nullptr, n, k_exp, 1).bytes > kStaticScratchBytes) return SLIMDP_ERR_UNSUPPORTED;
+    PtrArray<uint32_t> out;
+    for (auto& q : out.p) q = nullptr;
+    out.p[0] = exp_idx;
+    void* ws = scratch_addr[dev];
+    // launch_explore clears the counters it needs at zero and resets the status word on every call
+    slimdp_status rc = launch_explore(core_aux, n, k_core, k_exp, seed, worker, 1, round, out, ws, st);
+    if (rc != SLIMDP_OK) return rc;
+    if (status_out != nullptr &&
+        cudaMemcpyAsync(status_out, ws, sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return SLIMDP_ERR_CUDA;
+    return SLIMDP_OK;
+}
+
 }  // namespace slimdp
