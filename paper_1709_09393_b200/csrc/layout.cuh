@@ -8,8 +8,10 @@ namespace slimdp {
 struct SelectWs {
     WsHeader* hdr;
     uint32_t* hist;                 // 6 x 4096 bins: three passes over all keys, three over the candidates
-    uint32_t* sample_hist;          // 65536 bins (top 16 key bits of the sampled keys)
     uint32_t* coarse_hist;          // 256 bins (top 8 key bits of the sampled keys)
+    uint32_t* fine_hist;            // 2 x 256 bins (top 16 key bits inside the two crossing coarse bins)
+    uint32_t* coarse_incl;          // 256: samples in coarse bins >= c
+    uint32_t* sample;               // 2^18 sampled keys
     uint32_t* G;                    // greater-than-threshold bitmap, nb * 32 words
     uint32_t* E;                    // equal-to-threshold bitmap, nb * 32 words
     unsigned long long* cnt;        // per block: #greater | #equal << 32
@@ -35,9 +37,11 @@ inline SelectWs select_ws_layout(void* ws, uint64_t n) {
     };
     L.hdr = reinterpret_cast<WsHeader*>(take(sizeof(WsHeader)));
     L.hist = reinterpret_cast<uint32_t*>(take(6 * 4096 * sizeof(uint32_t)));
-    L.sample_hist = reinterpret_cast<uint32_t*>(take(65536 * sizeof(uint32_t)));
     L.coarse_hist = reinterpret_cast<uint32_t*>(take(256 * sizeof(uint32_t)));
+    L.fine_hist = reinterpret_cast<uint32_t*>(take(512 * sizeof(uint32_t)));
     L.zero_bytes = off;
+    L.coarse_incl = reinterpret_cast<uint32_t*>(take(256 * sizeof(uint32_t)));
+    L.sample = reinterpret_cast<uint32_t*>(take((size_t)(1u << kSampleBits) * sizeof(uint32_t)));
     L.G = reinterpret_cast<uint32_t*>(take(nb * kWordsPerBlock * 4));
     L.E = reinterpret_cast<uint32_t*>(take(nb * kWordsPerBlock * 4));
     L.cnt = reinterpret_cast<unsigned long long*>(take(nb * 8));

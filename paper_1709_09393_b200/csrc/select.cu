@@ -6,10 +6,11 @@
 // to T that belong to the core (those with the smallest indices).
 //
 // Large inputs (n >= 2^21) take the bracketed path, which reads the scores once:
-//   1. sample: 2^18 evenly spaced keys are histogrammed by their top 16 bits
-//      (and by their top 8 bits); the last CTA to finish turns the histograms
-//      into a bracket of 16-bit bins [b_bot, b_top) that holds T with
-//      overwhelming probability;
+//   1. sample (two small kernels): 2^18 evenly spaced keys are copied out and
+//      counted by their top 8 bits, then, around the two target ranks, by their
+//      top 16 bits; the last CTA of each kernel turns the counts into a
+//      bracket of 16-bit bins [b_bot, b_top) that holds T with overwhelming
+//      probability;
 //   2. bracket pass (one read of all keys): keys in bins >= b_top are
 //      certainly in the core and go straight into the "greater" bitmap; keys
 //      inside the bracket are copied, with their indices, to a candidate list;
@@ -62,77 +63,116 @@ __device__ __forceinline__ bool mode_runs(int mode, const WsHeader* hdr, uint32_
 
 // ---- step 1: sample histogram and bracket ------------------------------------------------
 
-// 2^18 evenly spaced keys are counted by their top 16 bits (fine, 65536 bins) and by their top
-// 8 bits (coarse, 256 bins).  The last CTA to finish locates, in the coarse histogram, the two
-// coarse bins where the count from the top crosses the two target ranks, and resolves each
-// crossing inside the 256 fine bins of that coarse bin.
-__global__ void __launch_bounds__(1024) sample_bracket_kernel(const uint32_t* __restrict__ keys, uint64_t n,
-                                                              uint32_t k, WsHeader* hdr,
-                                                              uint32_t* __restrict__ sample_hist,
-                                                              uint32_t* __restrict__ coarse_hist) {
+// "Last CTA done": every CTA ends with this; it returns true in exactly one CTA, the last to
+// arrive, and that CTA then sees all global writes and atomics the others made before arriving.
+// The block barrier orders the CTA's own accesses before thread 0's device-wide fence, the
+// fence orders them before the ticket.
+__device__ __forceinline__ bool last_cta_done(uint32_t* ticket) {
     __shared__ bool last;
-    __shared__ unsigned long long smem[33];
-    __shared__ uint32_t sh_coarse[256];
-    __shared__ long long s_incl[256];
-    __shared__ uint32_t s_val[2];
-    const uint32_t t = threadIdx.x;
-    if (t < 256) sh_coarse[t] = 0;
     __syncthreads();
-    const uint32_t j = blockIdx.x * 1024 + t;   // sample number, < 2^18
-    const uint64_t pos = ((uint64_t)j * n) >> kSampleBits;
-    const uint32_t key = __ldg(keys + pos);
-    atomicAdd(&sample_hist[key >> 16], 1u);
-    atomicAdd(&sh_coarse[key >> 24], 1u);
+    if (threadIdx.x == 0) {
+        __threadfence();
+        last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+        __threadfence();
+    }
     __syncthreads();
-    if (t < 256 && sh_coarse[t]) atomicAdd(&coarse_hist[t], sh_coarse[t]);
-    __threadfence();
-    __syncthreads();
-    if (t == 0) last = atomicAdd(&hdr->ticket[6], 1u) == gridDim.x - 1;
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
-    // the sample rank of T is about r = k * samples / n; keep 6 standard deviations (+16) on each side
+    return last;
+}
+
+// The sample rank of T is about r = k * samples / n; the bracket keeps 6 standard deviations
+// (+16) of the sample count on each side of it.
+__device__ __forceinline__ void bracket_targets(uint32_t k, uint64_t n, long long* lo_target, long long* hi_target) {
     const double samples = (double)(1u << kSampleBits);
     const double p = (double)k / (double)n;
     const double r = p * samples;
     const double margin = 6.0 * sqrt(samples * p * (1.0 - p)) + 16.0;
-    const long long lo_target = (long long)floor(r - margin);
-    const long long hi_target = (long long)ceil(r + margin);
-    const volatile uint32_t* fine = sample_hist;
-    const volatile uint32_t* coarse = coarse_hist;
+    *lo_target = (long long)floor(r - margin);
+    *hi_target = (long long)ceil(r + margin);
+}
+
+// Sample kernel A: 2^18 evenly spaced keys are copied to `sample` and counted by their top 8
+// bits (256 coarse bins: shared memory per CTA, then a few global atomics).  The last CTA finds
+// the two coarse bins in which the count from the top crosses the two target ranks:
+// coarse_x[0] for b_top (highest coarse bin whose inclusive count exceeds lo_target),
+// coarse_x[1] for b_bot (highest coarse bin whose inclusive count reaches hi_target);
+// 0xFFFFFFFF = no crossing.  coarse_incl[c] = samples in coarse bins >= c is kept for kernel B.
+__global__ void __launch_bounds__(1024) sample_coarse_kernel(const uint32_t* __restrict__ keys, uint64_t n,
+                                                             uint32_t k, WsHeader* hdr,
+                                                             uint32_t* __restrict__ sample,
+                                                             uint32_t* __restrict__ coarse_hist,
+                                                             uint32_t* __restrict__ coarse_incl) {
+    __shared__ unsigned long long smem[33];
+    __shared__ uint32_t sh_coarse[256];
+    __shared__ long long s_incl[257];
+    const uint32_t t = threadIdx.x;
+    if (t < 256) sh_coarse[t] = 0;
+    __syncthreads();
+    const uint32_t j = blockIdx.x * 1024 + t;   // sample number, < 2^18
+    const uint32_t key = __ldg(keys + (((uint64_t)j * n) >> kSampleBits));
+    sample[j] = key;
+    atomicAdd(&sh_coarse[key >> 24], 1u);
+    __syncthreads();
+    if (t < 256 && sh_coarse[t]) atomicAdd(&coarse_hist[t], sh_coarse[t]);
+    if (!last_cta_done(&hdr->ticket[6])) return;
+    long long lo_target, hi_target;
+    bracket_targets(k, n, &lo_target, &hi_target);
     // coarse bins from the top down: thread t < 256 owns coarse bin 255 - t
     unsigned long long total;
-    const unsigned long long c = (t < 256) ? coarse[255 - t] : 0ull;
+    const unsigned long long c = (t < 256) ? __ldcg(coarse_hist + 255 - t) : 0ull;
     const long long c_above = (long long)block_exclusive_scan64<32>(c, smem, &total);
-    if (t < 256) s_incl[255 - t] = c_above + (long long)c;   // samples in coarse bins >= 255 - t
-    if (t < 2) s_val[t] = 0xFFFFFFFFu;
+    if (t < 256) s_incl[255 - t] = c_above + (long long)c;
+    if (t == 0) {
+        s_incl[256] = 0;
+        hdr->coarse_x[0] = 0xFFFFFFFFu;
+        hdr->coarse_x[1] = 0xFFFFFFFFu;
+    }
     __syncthreads();
-    // b_top: lowest fine bin b with (samples in bins >= b) <= lo_target; 65536 if there is none.
-    // b_bot: highest fine bin b with (samples in bins >= b) >= hi_target; 0 if there is none.
-    // which = 0 resolves b_top, which = 1 resolves b_bot; both walk one coarse bin's 256 fine bins.
+    if (t < 256) {
+        const long long incl = s_incl[t], above = s_incl[t + 1];
+        coarse_incl[t] = (uint32_t)incl;
+        if (incl > lo_target && above <= lo_target) hdr->coarse_x[0] = t;
+        if (incl >= hi_target && above < hi_target) hdr->coarse_x[1] = t;
+    }
+}
+
+// Sample kernel B: the members of the two crossing coarse bins are counted by their top 16 bits
+// (2 x 256 fine bins); the last CTA resolves each crossing to a 16-bit bin:
+// b_top = lowest bin b with (samples in bins >= b) <= lo_target, 65536 if there is none;
+// b_bot = highest bin b with (samples in bins >= b) >= hi_target, 0 if there is none.
+__global__ void __launch_bounds__(1024) sample_fine_kernel(const uint32_t* __restrict__ sample, uint64_t n,
+                                                           uint32_t k, WsHeader* hdr,
+                                                           uint32_t* __restrict__ fine_hist,
+                                                           const uint32_t* __restrict__ coarse_incl) {
+    __shared__ unsigned long long smem[33];
+    __shared__ uint32_t sh_fine[2][256];
+    __shared__ uint32_t s_val[2];
+    const uint32_t t = threadIdx.x;
+    const uint32_t cx0 = hdr->coarse_x[0], cx1 = hdr->coarse_x[1];
+    if (t < 512) sh_fine[t >> 8][t & 255u] = 0;
+    __syncthreads();
+    const uint32_t key = sample[blockIdx.x * 1024 + t];
+    const uint32_t cb = key >> 24, fb = (key >> 16) & 255u;
+    if (cb == cx0) atomicAdd(&sh_fine[0][fb], 1u);
+    if (cb == cx1) atomicAdd(&sh_fine[1][fb], 1u);
+    __syncthreads();
+    if (t < 512 && sh_fine[t >> 8][t & 255u]) atomicAdd(&fine_hist[t], sh_fine[t >> 8][t & 255u]);
+    if (!last_cta_done(&hdr->ticket[7])) return;
+    long long lo_target, hi_target;
+    bracket_targets(k, n, &lo_target, &hi_target);
     for (int which = 0; which < 2; ++which) {
         const long long target = which ? hi_target : lo_target;
-        // crossing coarse bin: the highest one whose inclusive count exceeds (which = 0) / reaches (which = 1) the target
-        if (t < 256) {
-            const long long incl = s_incl[t], above = (t == 255) ? 0 : s_incl[t + 1];
-            const bool here = which ? (incl >= target && above < target) : (incl > target && above <= target);
-            if (here) s_val[which] = t;
-        }
-        __syncthreads();
-        const uint32_t cx = s_val[which];
-        __syncthreads();
-        uint32_t result;
+        const uint32_t cx = which ? cx1 : cx0;
         if (cx == 0xFFFFFFFFu) {
-            // no crossing: which = 0: target < 0 (nothing certain, 65536) or every bin qualifies (0);
-            //              which = 1: target above the sample size, or target <= 0: every bin may hold T
-            result = which ? 0u : ((target < 0) ? 65536u : 0u);
-            if (t == 0) s_val[which] = result;
+            // no crossing: which = 0: target < 0 (nothing is certain: 65536) or every bin qualifies (0);
+            //              which = 1: target above the sample size: every bin may hold T (0)
+            if (t == 0) s_val[which] = which ? 0u : ((target < 0) ? 65536u : 0u);
             __syncthreads();
             continue;
         }
-        const long long above_cx = (cx == 255) ? 0 : s_incl[cx + 1];
+        const long long above_cx = (cx == 255) ? 0 : (long long)coarse_incl[cx + 1];
         // fine bins of coarse bin cx from the top down: thread t < 256 owns fine bin cx * 256 + 255 - t
-        const unsigned long long f = (t < 256) ? fine[cx * 256 + 255 - t] : 0ull;
+        unsigned long long total;
+        const unsigned long long f = (t < 256) ? __ldcg(fine_hist + which * 256 + 255 - t) : 0ull;
         const long long f_above = (long long)block_exclusive_scan64<32>(f, smem, &total);
         if (t == 0) s_val[which] = which ? 0u : (cx + 1) * 256u;   // default when no fine bin of cx qualifies
         __syncthreads();
@@ -189,35 +229,47 @@ __global__ void __launch_bounds__(256) bracket_pass_kernel(const uint32_t* __res
         }
         __syncwarp();
     };
+    // keys >= top_key are certainly in the core; keys in [bot_key, top_key) are candidates
+    const bool has_top = b_top < 65536u;
+    const uint32_t top_key = has_top ? (b_top << 16) : 0xFFFFFFFFu;
+    const uint32_t bot_key = b_bot << 16;
     const uint64_t warps = (uint64_t)gridDim.x * (blockDim.x >> 5);
     for (uint64_t blk = (uint64_t)blockIdx.x * (blockDim.x >> 5) + wid; blk < nb; blk += warps) {
         const uint64_t base = blk * kBlock;
-        const bool full = base + kBlock <= n;
+        const uint32_t valid = (base + kBlock <= n) ? kBlock : (uint32_t)(n - base);   // parameters in this block
+        const uint32_t* src = keys + base + lane;
+        const uint32_t idx0 = (uint32_t)base + lane;
         uint32_t myG = 0;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             uint32_t key[8];
+            if (valid == kBlock) {
 #pragma unroll
-            for (int wd = 0; wd < 8; ++wd) {
-                const uint64_t i = base + (q * 8 + wd) * 32 + lane;
-                key[wd] = (full || i < n) ? __ldcs(keys + i) : 0u;
+                for (int wd = 0; wd < 8; ++wd) key[wd] = __ldcs(src + (q * 8 + wd) * 32);
+            } else {
+                // ragged last block: positions past the end read as key 0 and are masked out below
+#pragma unroll
+                for (int wd = 0; wd < 8; ++wd)
+                    key[wd] = ((q * 8 + wd) * 32 + lane < valid) ? __ldcs(src + (q * 8 + wd) * 32) : 0u;
             }
             uint32_t place = staged;
 #pragma unroll
             for (int wd = 0; wd < 8; ++wd) {
-                const uint32_t off = (q * 8 + wd) * 32 + lane;
-                const bool in = full || (base + off < n);
-                const uint32_t bin = key[wd] >> 16;
-                const bool cand = in && bin >= b_bot && bin < b_top;
-                const uint32_t bg = __ballot_sync(0xFFFFFFFFu, in && bin >= b_top);
+                const uint32_t off = (q * 8 + wd) * 32;
+                const bool in = off + lane < valid;
+                const bool def = has_top && key[wd] >= top_key && in;
+                const bool cand = key[wd] >= bot_key && !def && in;
+                const uint32_t bg = __ballot_sync(0xFFFFFFFFu, def);
                 const uint32_t bc = __ballot_sync(0xFFFFFFFFu, cand);
                 if (lane == (uint32_t)(q * 8 + wd)) myG = bg;
-                if (cand) {
-                    const uint32_t slot = place + __popc(bc & lt_mask);
-                    my_key[slot] = key[wd];
-                    my_idx[slot] = (uint32_t)(base + off);
+                if (bc) {   // warp-uniform: most rows hold no candidate
+                    if (cand) {
+                        const uint32_t slot = place + __popc(bc & lt_mask);
+                        my_key[slot] = key[wd];
+                        my_idx[slot] = idx0 + off;
+                    }
+                    place += __popc(bc);
                 }
-                place += __popc(bc);
             }
             staged = place;
             __syncwarp();
@@ -263,7 +315,6 @@ __global__ void __launch_bounds__(kHistThreads) hist_kernel(const uint32_t* __re
     constexpr uint32_t SHIFT = (PASS == 0) ? 20 : (PASS == 1 ? 10 : 0);
     __shared__ uint32_t sh[NB];
     __shared__ unsigned long long smem[33];
-    __shared__ bool last;
     if (!mode_runs(mode, hdr, k, cap)) return;
     const uint32_t* keys = (mode == kCandidates) ? cand_key : all_keys;
     const uint64_t n = (mode == kCandidates) ? hdr->n_cand : n_all;
@@ -294,12 +345,7 @@ __global__ void __launch_bounds__(kHistThreads) hist_kernel(const uint32_t* __re
         uint32_t c = sh[b];
         if (c) atomicAdd(&hist[b], c);
     }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) last = atomicAdd(&hdr->ticket[PASS + (mode == kCandidates ? 0 : 3)], 1u) == gridDim.x - 1;
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
+    if (!last_cta_done(&hdr->ticket[PASS + (mode == kCandidates ? 0 : 3)])) return;
 
     // rank wanted inside the current prefix
     uint32_t want;
@@ -500,7 +546,7 @@ slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, ui
     const uint32_t k = (uint32_t)k_core;
     const uint32_t cap = (uint32_t)L.cand_cap;
 
-    // header, radix histograms and sample histogram are contiguous: one clear
+    // header, radix histograms and sample histograms are contiguous: one clear
     if (cudaMemsetAsync(L.hdr, 0, L.zero_bytes, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
     select_init_kernel<<<1, 1, 0, st>>>(L.hdr, k);
     SLIMDP_LAUNCHED(1);
@@ -509,8 +555,10 @@ slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, ui
     const unsigned hgrid = (unsigned)sms * 4;
     const bool bracketed = k_core > 0 && n >= kBracketMinN;
     if (bracketed) {
-        sample_bracket_kernel<<<(1u << kSampleBits) / 1024, 1024, 0, st>>>(keys, n, k, L.hdr, L.sample_hist,
-                                                                              L.coarse_hist);
+        sample_coarse_kernel<<<(1u << kSampleBits) / 1024, 1024, 0, st>>>(keys, n, k, L.hdr, L.sample, L.coarse_hist,
+                                                                          L.coarse_incl);
+        sample_fine_kernel<<<(1u << kSampleBits) / 1024, 1024, 0, st>>>(L.sample, n, k, L.hdr, L.fine_hist,
+                                                                        L.coarse_incl);
         bracket_pass_kernel<<<(unsigned)cgrid, 256, 0, st>>>(keys, n, nb, L.hdr, cap, L.G, L.E, L.cnt, L.cand_key,
                                                              L.cand_idx);
         // T and r from the candidates (these return at once if the bracket failed) ...
@@ -523,7 +571,7 @@ slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, ui
                                                            kCandidates);
         mark_candidates_kernel<<<(unsigned)sms * 4, 256, 0, st>>>(L.cand_key, L.cand_idx, L.hdr, k, cap, L.G, L.E,
                                                                   L.cnt);
-        SLIMDP_LAUNCHED(6);
+        SLIMDP_LAUNCHED(7);
     }
     if (k_core > 0) {
         // ... or from all keys (these return at once if the bracket held)
