@@ -65,7 +65,18 @@ __device__ __forceinline__ void find_bounds(uint32_t (*bound)[kMergeWarps + 1], 
     __syncthreads();
 }
 
-__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+// Sparse 4-byte accesses: ask L2 for the smallest fetch it offers (64 B) instead of a whole 128-byte line.
+__device__ __forceinline__ float ld_sparse(const float* p) {
+    float v;
+    asm volatile("ld.global.L2::64B.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+    return v;
+}
+// Early request of a location that a later phase reads: a real load whose value only feeds `sink`.
+__device__ __forceinline__ void touch(const float* p, uint32_t& sink) {
+    uint32_t v;
+    asm volatile("ld.global.L2::64B.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    sink ^= v;
+}
 
 // One CTA owns 8 consecutive ranges of 2^range_shift parameters, one per warp.  Every warp, on
 // its own, first requests all lines it is going to touch (L2 prefetch), then applies worker 0's
@@ -77,10 +88,11 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* 
     __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
     find_bounds(bound, exp, k_exp, K, range_shift);
     const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
+    uint32_t sink = 0;
     for (int k = 0; k < K; ++k) {
         const uint32_t* __restrict__ idx = exp.p[k];
         const uint32_t b = bound[k][wid + 1];
-        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) prefetch_l2(w + __ldg(idx + e));
+        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) touch(w + __ldg(idx + e), sink);
     }
     for (int k = 0; k < K; ++k) {
         const uint32_t* __restrict__ idx = exp.p[k];
@@ -88,10 +100,11 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* 
         const uint32_t b = bound[k][wid + 1];
         for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) {
             const uint32_t i = __ldg(idx + e);
-            w[i] = __fmaf_rn(neg_eta, __ldcs(v + e), w[i]);
+            w[i] = __fmaf_rn(neg_eta, __ldcs(v + e), ld_sparse(w + i));
         }
         __syncwarp();   // worker k's updates are visible to the whole warp before worker k+1 starts
     }
+    if (sink == 0x9E3779B9u && lane >= 32) w[0] = 0.0f;   // never true: keeps the early requests alive
 }
 
 // ---- push + server update + pull in one pass (slimdp_exchange) -----------------------------
@@ -139,14 +152,15 @@ __global__ void __launch_bounds__(kMergeWarps * 32) exchange_explore_kernel(
     __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
     find_bounds(bound, exp, k_exp, K, range_shift);
     const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
+    uint32_t sink = 0;
     for (int k = 0; k < K; ++k) {
         const uint32_t* __restrict__ idx = exp.p[k];
         const float* __restrict__ d = delta.p[k];
         const uint32_t b = bound[k][wid + 1];
         for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) {
             const uint32_t i = __ldg(idx + e);
-            prefetch_l2(w + i);
-            prefetch_l2(d + i);
+            touch(w + i, sink);
+            touch(d + i, sink);
         }
     }
     for (int k = 0; k < K; ++k) {
@@ -156,9 +170,9 @@ __global__ void __launch_bounds__(kMergeWarps * 32) exchange_explore_kernel(
         const uint32_t b = bound[k][wid + 1];
         for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) {
             const uint32_t i = __ldg(idx + e);
-            const float u = __ldg(d + i);
+            const float u = ld_sparse(d + i);
             __stcs(v + e, u);
-            w[i] = __fmaf_rn(neg_eta, u, w[i]);
+            w[i] = __fmaf_rn(neg_eta, u, ld_sparse(w + i));
         }
         __syncwarp();   // worker k's updates are visible to the whole warp before worker k+1 starts
     }
@@ -166,8 +180,9 @@ __global__ void __launch_bounds__(kMergeWarps * 32) exchange_explore_kernel(
         const uint32_t* __restrict__ idx = exp.p[k];
         float* __restrict__ o = pulled.p[k] + k_core;
         const uint32_t b = bound[k][wid + 1];
-        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) __stcs(o + e, w[__ldg(idx + e)]);
+        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) __stcs(o + e, ld_sparse(w + __ldg(idx + e)));
     }
+    if (sink == 0x9E3779B9u && lane >= 32) w[0] = 0.0f;   // never true: keeps the early requests alive
 }
 
 // Range per warp: a power of two with 16 to 32 entries per worker on average, at least 32 parameters.
