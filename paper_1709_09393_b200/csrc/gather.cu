@@ -13,6 +13,13 @@ namespace slimdp {
 
 namespace {
 
+// Sparse 4-byte reads: ask L2 for its smallest fetch (64 B) instead of a whole 128-byte line.
+__device__ __forceinline__ float ld_sparse(const float* p) {
+    float v;
+    asm volatile("ld.global.L2::64B.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+
 // out[k][j] = src[k][core_idx[j]] for every worker k.  SAME: all workers read the same source.
 template <bool SAME>
 __global__ void __launch_bounds__(256) gather_core_kernel(PtrArray<const float> src,
@@ -58,7 +65,7 @@ __global__ void __launch_bounds__(256) gather_explore_kernel(PtrArray<const floa
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const uint64_t j = j0 + (uint64_t)q * blockDim.x;
-            if (j < k_exp) v[q] = __ldg(s + idx[q]);
+            if (j < k_exp) v[q] = ld_sparse(s + idx[q]);
         }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {

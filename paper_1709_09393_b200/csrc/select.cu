@@ -240,23 +240,19 @@ __global__ void __launch_bounds__(256) bracket_pass_kernel(const uint32_t* __res
         const uint32_t* src = keys + base + lane;
         const uint32_t idx0 = (uint32_t)base + lane;
         uint32_t myG = 0;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        // a quarter block (8 rows of 32 keys) at a time; `full` blocks skip the end-of-vector tests
+        auto quarter = [&](const int q, const bool full) {
             uint32_t key[8];
-            if (valid == kBlock) {
 #pragma unroll
-                for (int wd = 0; wd < 8; ++wd) key[wd] = __ldcs(src + (q * 8 + wd) * 32);
-            } else {
-                // ragged last block: positions past the end read as key 0 and are masked out below
-#pragma unroll
-                for (int wd = 0; wd < 8; ++wd)
-                    key[wd] = ((q * 8 + wd) * 32 + lane < valid) ? __ldcs(src + (q * 8 + wd) * 32) : 0u;
+            for (int wd = 0; wd < 8; ++wd) {
+                const uint32_t off = (q * 8 + wd) * 32;
+                key[wd] = (full || off + lane < valid) ? __ldcs(src + off) : 0u;
             }
             uint32_t place = staged;
 #pragma unroll
             for (int wd = 0; wd < 8; ++wd) {
                 const uint32_t off = (q * 8 + wd) * 32;
-                const bool in = off + lane < valid;
+                const bool in = full || off + lane < valid;
                 const bool def = has_top && key[wd] >= top_key && in;
                 const bool cand = key[wd] >= bot_key && !def && in;
                 const uint32_t bg = __ballot_sync(0xFFFFFFFFu, def);
@@ -277,6 +273,13 @@ __global__ void __launch_bounds__(256) bracket_pass_kernel(const uint32_t* __res
                 flush(staged);
                 staged = 0;
             }
+        };
+        if (valid == kBlock) {
+#pragma unroll 1
+            for (int q = 0; q < 4; ++q) quarter(q, true);
+        } else {
+#pragma unroll 1
+            for (int q = 0; q < 4; ++q) quarter(q, false);
         }
         G[blk * kWordsPerBlock + lane] = myG;
         E[blk * kWordsPerBlock + lane] = 0u;
