@@ -29,6 +29,7 @@ namespace slimdp {
 namespace {
 
 constexpr int kBucketThreads = 256;
+constexpr size_t kGroupSmemMax = 200 * 1024;   // shared memory the scatter step may use to group a chunk
 
 
 __device__ __forceinline__ void philox4x32_10(uint32_t k0, uint32_t k1, uint32_t c0, uint32_t c1, uint32_t c2,
@@ -169,15 +170,21 @@ __global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, 
 // grid = (chunks, workers).  Move every rank of the chunk into its bucket's slice of `sorted`.
 // SMEM: with the chunk's histogram from the rank step the CTA reserves one contiguous piece of
 // every bucket's slice (a single global atomic per bucket) and hands out places inside it from
-// shared memory.
-template <bool SMEM>
+// shared memory.  GROUP (needs SMEM): the chunk is first grouped by bucket in shared memory and
+// then copied out, so that a warp's stores fall into a few runs instead of 32 separate sectors.
+template <bool SMEM, bool GROUP>
 __global__ void __launch_bounds__(1024) scatter_kernel(uint32_t k_exp, uint32_t chunk, uint32_t s, uint32_t buckets,
                                                        const uint32_t* __restrict__ rho, uint64_t rho_stride,
                                                        const unsigned long long* __restrict__ pref,
                                                        uint64_t cnt_stride, uint32_t* __restrict__ cursor,
                                                        const uint32_t* __restrict__ cta_hist,
                                                        uint32_t* __restrict__ sorted) {
-    extern __shared__ uint32_t sh_place[];   // per bucket: next free place of this CTA's piece
+    extern __shared__ uint32_t sh[];
+    __shared__ unsigned long long scan_smem[33];
+    uint32_t* sh_place = sh;                  // per bucket: first / next free global place of this CTA's piece
+    uint32_t* sh_first = sh + buckets;        // GROUP: first local place of the bucket's run
+    uint32_t* sh_next = sh + 2 * buckets;     // GROUP: next free local place
+    uint32_t* sh_sorted = sh + 3 * buckets;   // GROUP: the chunk, grouped by bucket
     const uint32_t worker = blockIdx.y;
     const uint32_t* my_rho = rho + (uint64_t)worker * rho_stride;
     uint32_t* my_sorted = sorted + (uint64_t)worker * rho_stride;
@@ -187,9 +194,30 @@ __global__ void __launch_bounds__(1024) scatter_kernel(uint32_t k_exp, uint32_t 
     const uint64_t c1 = (c0 + chunk < k_exp) ? c0 + chunk : k_exp;
     if (SMEM) {
         const uint32_t* mine = cta_hist + ((uint64_t)worker * gridDim.x + blockIdx.x) * buckets;
-        for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) {
-            const uint32_t c = mine[b];
-            sh_place[b] = c ? (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], c) : 0u;
+        if (GROUP) {
+            // local run offsets: exclusive scan of the chunk's histogram, consecutive buckets per thread
+            const uint32_t per = (buckets + blockDim.x - 1) / blockDim.x;
+            const uint32_t b0 = threadIdx.x * per;
+            unsigned long long sum = 0;
+            for (uint32_t q = 0; q < per; ++q)
+                if (b0 + q < buckets) sum += mine[b0 + q];
+            unsigned long long total;
+            uint32_t run = (uint32_t)block_exclusive_scan64<32>(sum, scan_smem, &total);
+            for (uint32_t q = 0; q < per; ++q) {
+                const uint32_t b = b0 + q;
+                if (b < buckets) {
+                    const uint32_t c = mine[b];
+                    sh_first[b] = run;
+                    sh_next[b] = run;
+                    sh_place[b] = c ? (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], c) : 0u;
+                    run += c;
+                }
+            }
+        } else {
+            for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) {
+                const uint32_t c = mine[b];
+                sh_place[b] = c ? (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], c) : 0u;
+            }
         }
         __syncthreads();
     }
@@ -205,13 +233,31 @@ __global__ void __launch_bounds__(1024) scatter_kernel(uint32_t k_exp, uint32_t 
             const uint64_t j = j0 + (uint64_t)q * blockDim.x;
             if (j < c1) {
                 const uint32_t b = x[q] >> s;
-                const uint32_t pos =
-                    SMEM ? atomicAdd(&sh_place[b], 1u) : (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], 1u);
-                if (pos < k_exp) my_sorted[pos] = x[q];
+                if (GROUP) {
+                    sh_sorted[atomicAdd(&sh_next[b], 1u)] = x[q];
+                } else {
+                    const uint32_t pos =
+                        SMEM ? atomicAdd(&sh_place[b], 1u) : (uint32_t)my_pref[b] + atomicAdd(&my_cur[b], 1u);
+                    if (pos < k_exp) my_sorted[pos] = x[q];
+                }
             }
         }
     }
+    if (GROUP) {
+        __syncthreads();
+        const uint32_t len = (c1 > c0) ? (uint32_t)(c1 - c0) : 0u;
+        for (uint32_t p = threadIdx.x; p < len; p += blockDim.x) {
+            const uint32_t x = sh_sorted[p];
+            const uint32_t b = x >> s;
+            const uint32_t pos = sh_place[b] + (p - sh_first[b]);
+            if (pos < k_exp) my_sorted[pos] = x;
+        }
+    }
 }
+
+// Shared-memory index of bitmap word w: one pad word per 32 keeps a thread's run of
+// consecutive words (stride 2, 4 or 8 across lanes) free of bank conflicts.
+__device__ __forceinline__ uint32_t sw(uint32_t w) { return w + (w >> 5); }
 
 constexpr uint32_t kDirCache = 2048;
 constexpr uint32_t kListCap = 4096;
@@ -222,7 +268,7 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
     uint32_t k_exp, uint32_t s, const uint32_t* __restrict__ sorted, uint64_t rho_stride,
     const unsigned long long* __restrict__ cnt, const unsigned long long* __restrict__ pref,
     const unsigned long long* __restrict__ totals, uint64_t cnt_stride, PtrArray<uint32_t> out, WsHeader* hdr) {
-    __shared__ uint32_t bm[2048];                // up to 2^16 rank bits
+    __shared__ uint32_t bm[2048 + 64];           // up to 2^16 rank bits, padded (see sw)
     __shared__ uint32_t dir_sh[kDirCache + 1];   // directory entries of the bucket's 256-parameter groups (+1)
     __shared__ uint16_t list[kListCap];          // sorted ranks (low s bits) of the current round
     __shared__ uint32_t warp_sums[kBucketThreads / 32];
@@ -233,7 +279,7 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
     const uint32_t offset = (uint32_t)pref[(uint64_t)worker * cnt_stride + bucket];
     if (bucket == 0 && t == 0 && totals[worker] != k_exp) hdr->status = SLIMDP_ERR_INTERNAL;
     if (count == 0) return;
-    for (uint32_t i = t; i < words; i += kBucketThreads) bm[i] = 0;
+    for (uint32_t i = t; i < words + (words >> 5); i += kBucketThreads) bm[i] = 0;
     // the bucket's ranks live in directory groups [grp_lo, grp_hi]
     const uint32_t grp_lo = __ldg(bounds + bucket), grp_hi = __ldg(bounds + bucket + 1);
     const uint32_t ngrp = grp_hi - grp_lo + 1;
@@ -245,12 +291,12 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
     const uint32_t low_mask = (1u << s) - 1u;
     for (uint32_t e = t; e < count; e += kBucketThreads) {
         const uint32_t r = my_sorted[e] & low_mask;
-        atomicOr(&bm[r >> 5], 1u << (r & 31u));
+        atomicOr(&bm[sw(r >> 5)], 1u << (r & 31u));
     }
     __syncthreads();
     // place of this thread's first rank in the sorted order: exclusive scan of the popcounts
     uint32_t mine = 0;
-    for (uint32_t q = 0; q < per; ++q) mine += __popc(bm[t * per + q]);
+    for (uint32_t q = 0; q < per; ++q) mine += __popc(bm[sw(t * per + q)]);
     const uint32_t inc = warp_inclusive_scan(mine);
     if ((t & 31u) == 31u) warp_sums[t >> 5] = inc;
     __syncthreads();
@@ -266,7 +312,7 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
         if (base < r0 + kListCap && base + mine > r0) {
             uint32_t p = base;
             for (uint32_t q = 0; q < per; ++q) {
-                uint32_t word = bm[t * per + q];
+                uint32_t word = bm[sw(t * per + q)];
                 while (word) {
                     const uint32_t bit = __ffs(word) - 1;
                     word &= word - 1;
@@ -394,12 +440,21 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
     slimdp_status rc =
         launch_block_scan(L.cnt, L.pref, L.tile_sums, L.totals, buckets, workers, L.cnt_stride, L.tile_stride, st);
     if (rc != SLIMDP_OK) return rc;
-    if (smem) {
-        scatter_kernel<true><<<grid, 1024, buckets * 4, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets, L.rho,
-                                                              L.rho_stride, L.pref, L.cnt_stride, L.cursor,
-                                                              L.cta_hist, L.sorted);
+    const size_t group_smem = (3 * buckets + chunk) * 4;
+    if (smem && group_smem <= kGroupSmemMax) {
+        if (group_smem > 48 * 1024 &&
+            cudaFuncSetAttribute(scatter_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)group_smem) != cudaSuccess)
+            return SLIMDP_ERR_CUDA;
+        scatter_kernel<true, true><<<grid, 1024, group_smem, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets,
+                                                                   L.rho, L.rho_stride, L.pref, L.cnt_stride,
+                                                                   L.cursor, L.cta_hist, L.sorted);
+    } else if (smem) {
+        scatter_kernel<true, false><<<grid, 1024, buckets * 4, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets,
+                                                                     L.rho, L.rho_stride, L.pref, L.cnt_stride,
+                                                                     L.cursor, L.cta_hist, L.sorted);
     } else {
-        scatter_kernel<false><<<grid, 1024, 0, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets, L.rho,
+        scatter_kernel<false, false><<<grid, 1024, 0, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets, L.rho,
                                                      L.rho_stride, L.pref, L.cnt_stride, L.cursor, L.cta_hist,
                                                      L.sorted);
     }
