@@ -71,11 +71,52 @@ __device__ __forceinline__ float ld_sparse(const float* p) {
     asm volatile("ld.global.L2::64B.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
     return v;
 }
-// Early request of a location that a later phase reads: a real load whose value only feeds `sink`.
-__device__ __forceinline__ void touch(const float* p, uint32_t& sink) {
+// Early request of a location that a later phase reads: a real load whose value is only
+// folded into a sink.  The caller folds a whole batch after issuing it, so that the loads of a
+// batch are all in flight together.
+__device__ __forceinline__ uint32_t touch(const float* p) {
     uint32_t v;
     asm volatile("ld.global.L2::64B.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    sink ^= v;
+    return v;
+}
+
+// Requests, for every worker, the model values (and, if delta is given, the update values) of
+// this warp's range ahead of the ordered phases: 8 workers' loads are issued back to back.
+template <bool WITH_DELTA>
+__device__ __forceinline__ uint32_t touch_range(const float* w, const PtrArray<const uint32_t>& exp,
+                                                const PtrArray<const float>& delta,
+                                                uint32_t (*bound)[kMergeWarps + 1], int K, uint32_t wid,
+                                                uint32_t lane) {
+    uint32_t sink = 0;
+    for (int k0 = 0; k0 < K; k0 += 8) {
+        uint32_t i[8], v[16];
+        bool ok[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int k = k0 + q;
+            const uint32_t e = (k < K) ? bound[k][wid] + lane : 0u;
+            ok[q] = k < K && e < bound[k][wid + 1];
+            i[q] = ok[q] ? __ldg(exp.p[k] + e) : 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            v[2 * q] = ok[q] ? touch(w + i[q]) : 0u;
+            v[2 * q + 1] = (WITH_DELTA && ok[q]) ? touch(delta.p[k0 + q] + i[q]) : 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < 16; ++q) sink ^= v[q];
+        // the rare worker with more than 32 entries in this range
+        for (int q = 0; q < 8 && k0 + q < K; ++q) {
+            const int k = k0 + q;
+            const uint32_t b = bound[k][wid + 1];
+            for (uint32_t e = bound[k][wid] + lane + 32; e < b; e += 32) {
+                const uint32_t j = __ldg(exp.p[k] + e);
+                sink ^= touch(w + j);
+                if (WITH_DELTA) sink ^= touch(delta.p[k] + j);
+            }
+        }
+    }
+    return sink;
 }
 
 // One CTA owns 8 consecutive ranges of 2^range_shift parameters, one per warp.  Every warp, on
@@ -88,12 +129,8 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* 
     __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
     find_bounds(bound, exp, k_exp, K, range_shift);
     const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
-    uint32_t sink = 0;
-    for (int k = 0; k < K; ++k) {
-        const uint32_t* __restrict__ idx = exp.p[k];
-        const uint32_t b = bound[k][wid + 1];
-        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) touch(w + __ldg(idx + e), sink);
-    }
+    PtrArray<const float> none;
+    const uint32_t sink = touch_range<false>(w, exp, none, bound, K, wid, lane);
     for (int k = 0; k < K; ++k) {
         const uint32_t* __restrict__ idx = exp.p[k];
         const float* __restrict__ v = val.p[k] + k_core;
@@ -152,17 +189,7 @@ __global__ void __launch_bounds__(kMergeWarps * 32) exchange_explore_kernel(
     __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
     find_bounds(bound, exp, k_exp, K, range_shift);
     const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
-    uint32_t sink = 0;
-    for (int k = 0; k < K; ++k) {
-        const uint32_t* __restrict__ idx = exp.p[k];
-        const float* __restrict__ d = delta.p[k];
-        const uint32_t b = bound[k][wid + 1];
-        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) {
-            const uint32_t i = __ldg(idx + e);
-            touch(w + i, sink);
-            touch(d + i, sink);
-        }
-    }
+    const uint32_t sink = touch_range<true>(w, exp, delta, bound, K, wid, lane);
     for (int k = 0; k < K; ++k) {
         const uint32_t* __restrict__ idx = exp.p[k];
         const float* __restrict__ d = delta.p[k];
