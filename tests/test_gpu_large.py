@@ -1,0 +1,76 @@
+"""The 10^9-parameter flat sweep (core 1 / 5 / 10 / 30 %, explorer 1 %, K = 4) at full size.
+
+Takes several minutes and about 40 GB of host memory, so it only runs when SLIMDP_RUN_LARGE=1.
+Scores, explorers, packed values, merged model and pulled values are compared with the CPU
+oracle element by element.  For the core, sorting 10^9 keys on one host thread is replaced by
+the property that defines the same set: the threshold is the k-th largest score (np.partition),
+everything above it is in, and the equal scores with the smallest indices fill the rest.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from workloads import CONFIGS, all_inputs
+from workloads.configs import LARGE_CORE_PCTS
+
+pytestmark = [pytest.mark.gpu, pytest.mark.slow]
+
+
+def _bits(a):
+    return np.ascontiguousarray(a).view(np.uint32)
+
+
+def _same(t: torch.Tensor, a: np.ndarray) -> bool:
+    return np.array_equal(t.cpu().numpy().view(np.uint32), _bits(a))
+
+
+@pytest.mark.skipif(os.environ.get("SLIMDP_RUN_LARGE") != "1", reason="set SLIMDP_RUN_LARGE=1 (minutes, ~40 GB host)")
+def test_large_flat_sweep_full_size():
+    import paper_1709_09393_b200 as P
+    base = CONFIGS["large"]
+    n, K = base.N, base.K
+    w, gs = all_inputs(base)
+    d_w0 = torch.from_numpy(w).cuda()
+    d_gs = [torch.from_numpy(g).cuda() for g in gs]
+    scores = torch.empty(n, dtype=torch.float32, device="cuda")
+    P.slimdp_score(d_w0, d_gs, base.c, scores)
+    S = oracle.score(w, gs, base.c)
+    assert _same(scores, S), "scores"
+    aux = torch.empty(P.core_aux_bytes(n), dtype=torch.uint8, device="cuda")
+    sel_ws = torch.empty(P.select_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    for pct in LARGE_CORE_PCTS:
+        cfg = base.with_core_pct(pct)
+        k_core, k_exp, m = cfg.k_core, cfg.k_exp, cfg.m
+        core_idx = torch.empty(k_core, dtype=torch.int32, device="cuda")
+        P.slimdp_select_core(scores, k_core, core_idx, aux, sel_ws)
+        P.read_status(sel_ws)
+        # the core by its definition, without a sort
+        T = np.partition(S, n - k_core)[n - k_core]
+        above = np.flatnonzero(S > T)
+        ties = np.flatnonzero(S == T)[:k_core - above.size]
+        core = np.sort(np.concatenate([above, ties])).astype(np.uint32)
+        del above, ties
+        assert core.size == k_core
+        assert np.array_equal(core_idx.cpu().numpy().view(np.uint32), core), f"core at {pct} %"
+        exp_ws = torch.empty(P.explore_workspace_bytes(n, k_exp, K), dtype=torch.uint8, device="cuda")
+        exp_idx = [torch.empty(k_exp, dtype=torch.int32, device="cuda") for _ in range(K)]
+        P.slimdp_sample_explore_batched(aux, n, k_core, k_exp, cfg.seed, 0, pct, exp_idx, exp_ws)
+        P.read_status(exp_ws)
+        exps = [oracle.sample_explore(core, n, k_exp, cfg.seed, k, pct) for k in range(K)]
+        for k in range(K):
+            assert np.array_equal(exp_idx[k].cpu().numpy().view(np.uint32), exps[k]), f"explorer {k} at {pct} %"
+        d_w = d_w0.clone()
+        val = [torch.empty(m, dtype=torch.float32, device="cuda") for _ in range(K)]
+        pulled = [torch.empty(m, dtype=torch.float32, device="cuda") for _ in range(K)]
+        P.slimdp_exchange(d_w, d_gs, core_idx, exp_idx, cfg.eta, val, pulled)
+        vals = [oracle.pack(gs[k], core, exps[k]) for k in range(K)]
+        merged = oracle.merge(w, core, exps, vals, cfg.eta)
+        assert _same(d_w, merged), f"merged model at {pct} %"
+        for k in range(K):
+            assert _same(val[k], vals[k]), f"packed values {k} at {pct} %"
+            assert _same(pulled[k], oracle.pull(merged, core, exps[k])), f"pulled values {k} at {pct} %"
+        del d_w, val, pulled, exp_idx, exp_ws, core_idx, vals, merged, exps, core
+        torch.cuda.empty_cache()
