@@ -1,6 +1,7 @@
 """The 10^9-parameter flat sweep (core 1 / 5 / 10 / 30 %, explorer 1 %, K = 4) at full size.
 
-Takes several minutes and about 40 GB of host memory, so it only runs when SLIMDP_RUN_LARGE=1.
+Takes two to three minutes, about 40 GB of host memory and 45 GB on the device; it is skipped
+on smaller machines and when SLIMDP_SKIP_LARGE=1.
 Scores, explorers, packed values, merged model and pulled values are compared with the CPU
 oracle element by element.  For the core, sorting 10^9 keys on one host thread is replaced by
 the property that defines the same set: the threshold is the k-th largest score (np.partition),
@@ -27,8 +28,18 @@ def _same(t: torch.Tensor, a: np.ndarray) -> bool:
     return np.array_equal(t.cpu().numpy().view(np.uint32), _bits(a))
 
 
-@pytest.mark.skipif(os.environ.get("SLIMDP_RUN_LARGE") != "1", reason="set SLIMDP_RUN_LARGE=1 (minutes, ~40 GB host)")
+def _enough_memory() -> bool:
+    import psutil
+    if psutil.virtual_memory().available < 64 << 30:
+        return False
+    return torch.cuda.is_available() and torch.cuda.mem_get_info()[0] > (60 << 30)
+
+
 def test_large_flat_sweep_full_size():
+    if os.environ.get("SLIMDP_SKIP_LARGE") == "1":
+        pytest.skip("SLIMDP_SKIP_LARGE=1")
+    if not _enough_memory():
+        pytest.skip("needs 64 GB of free host memory and 60 GB of free device memory")
     import paper_1709_09393_b200 as P
     base = CONFIGS["large"]
     n, K = base.N, base.K
