@@ -61,7 +61,7 @@ enum {
 
 /* Parameters per bitmap block (32 words), and per directory entry of core_aux. */
 #define SLIMDP_BLOCK 1024
-#define SLIMDP_DIR_STRIDE 256
+#define SLIMDP_DIR_STRIDE 64
 
 const char* slimdp_status_string(slimdp_status s);
 
@@ -70,9 +70,9 @@ const char* slimdp_status_string(slimdp_status s);
  * sampler reads.  Layout (all uint32_t, little-endian bit order):
  *   bitmap    [nb * 32] words, nb = ceil(n / 1024): bit (i & 31) of word (i >> 5)
  *             is 1 iff parameter i is in the core; bits at i >= n are 0;
- *   directory [nd + 1] words, nd = 4 nb, starting at byte offset slimdp_core_aux_dir_offset(n):
- *             directory[d] = 256 d - (number of core parameters with index < 256 d) for d < nd,
- *             i.e. the number of NON-core parameters below 256 d wherever 256 d <= n;
+ *   directory [nd + 1] words, nd = 16 nb, starting at byte offset slimdp_core_aux_dir_offset(n):
+ *             directory[d] = 64 d - (number of core parameters with index < 64 d) for d < nd,
+ *             i.e. the number of NON-core parameters below 64 d wherever 64 d <= n;
  *             directory[nd] = n - k_core.
  */
 size_t slimdp_core_aux_bytes(uint64_t n);

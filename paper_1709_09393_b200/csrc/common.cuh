@@ -11,8 +11,9 @@ namespace slimdp {
 constexpr uint32_t kBlock = SLIMDP_BLOCK;        // parameters per bitmap block
 constexpr uint32_t kWordsPerBlock = kBlock / 32; // 32 bitmap words per block
 constexpr uint32_t kDirStride = SLIMDP_DIR_STRIDE;      // parameters per directory entry
-constexpr uint32_t kDirPerBlock = kBlock / kDirStride;  // 4 directory entries per bitmap block
-constexpr uint32_t kWordsPerDir = kDirStride / 32;      // 8 bitmap words per directory entry
+constexpr uint32_t kDirPerBlock = kBlock / kDirStride;  // 16 directory entries per bitmap block
+constexpr uint32_t kWordsPerDir = kDirStride / 32;      // 2 bitmap words per directory entry
+static_assert(kWordsPerDir == 2, "select0 walks exactly two bitmap words per directory entry");
 constexpr uint32_t kScanTile = 1024;             // bitmap blocks per scan tile
 constexpr uint32_t kSampleBits = 18;             // the selection's bracket is estimated from 2^18 sampled keys
 constexpr uint64_t kBracketMinN = 1ull << 21;    // below this the selection reads the keys three more times instead

@@ -16,8 +16,8 @@
 //   5. bucket: one CTA per (bucket, worker) marks its ranks in a 2^s-bit
 //      shared-memory bitmap, which sorts them; a block scan of the popcounts
 //      gives each rank its output position, and a select0 query (binary
-//      search of the per-256 non-core directory inside the bucket's range,
-//      then a popcount walk over the group's 8 bitmap words, skipped when
+//      search of the per-64 non-core directory inside the bucket's range,
+//      seeded by interpolation, then the group's 2 bitmap words, skipped when
 //      the group holds no core parameter) turns it into the parameter index.
 // No global bitmap, no inter-CTA waiting; the result does not depend on the
 // order in which atomics land.
@@ -68,7 +68,7 @@ __device__ __forceinline__ uint32_t find_block(const uint32_t* __restrict__ dir,
     return lo;
 }
 
-// Round keys per worker, and per rank bucket the directory entry (256-parameter group) that holds
+// Round keys per worker, and per rank bucket the directory entry (64-parameter group) that holds
 // the bucket's first rank (bounds[buckets] = the group of the last rank M - 1).  The bounds
 // depend on the core only.
 __global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, uint32_t seed_lo, uint32_t seed_hi,
@@ -269,7 +269,7 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
     const unsigned long long* __restrict__ cnt, const unsigned long long* __restrict__ pref,
     const unsigned long long* __restrict__ totals, uint64_t cnt_stride, PtrArray<uint32_t> out, WsHeader* hdr) {
     __shared__ uint32_t bm[2048 + 64];           // up to 2^16 rank bits, padded (see sw)
-    __shared__ uint32_t dir_sh[kDirCache + 1];   // directory entries of the bucket's 256-parameter groups (+1)
+    __shared__ uint32_t dir_sh[kDirCache + 1];   // directory entries of the bucket's 64-parameter groups (+1)
     __shared__ uint16_t list[kListCap];          // sorted ranks (low s bits) of the current round
     __shared__ uint32_t warp_sums[kBucketThreads / 32];
     const uint32_t worker = blockIdx.y, bucket = blockIdx.x, t = threadIdx.x;
@@ -287,6 +287,9 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
     if (cached)
         for (uint32_t i = t; i <= ngrp; i += kBucketThreads) dir_sh[i] = __ldg(dir + grp_lo + i);
     __syncthreads();
+    // groups per rank inside this bucket, for the interpolated first guess of select0
+    const uint32_t dir_first = cached ? dir_sh[0] : 0u;
+    const float groups_per_rank = cached ? (float)ngrp / (float)(dir_sh[ngrp] - dir_sh[0] + 1u) : 0.0f;
     const uint32_t* my_sorted = sorted + (uint64_t)worker * rho_stride + offset;
     const uint32_t low_mask = (1u << s) - 1u;
     for (uint32_t e = t; e < count; e += kBucketThreads) {
@@ -326,10 +329,20 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
         uint32_t rel = 0;     // group relative to grp_lo; ranks ascend inside a thread, so it only moves up
         for (uint32_t e = t; e < m; e += kBucketThreads) {
             const uint32_t rank = first_rank + list[e];
-            // select0(rank): the 256-parameter group by binary search of the directory ...
+            // select0(rank): the 64-parameter group from the directory ...
             uint32_t d0, d1;
             if (cached) {
                 uint32_t lo = rel, hi = ngrp - 1;
+                // the directory is close to linear inside one bucket: try a small window around the
+                // interpolated group first, and search the whole range only if the window misses
+                const uint32_t guess = (uint32_t)((float)(rank - dir_first) * groups_per_rank);
+                const uint32_t wl = (guess > 8u) ? guess - 8u : 0u;
+                const uint32_t win_lo = (wl > lo) ? wl : lo;
+                const uint32_t win_hi = (guess + 8u < hi) ? guess + 8u : hi;
+                if (win_lo <= win_hi && dir_sh[win_lo] <= rank && dir_sh[win_hi + 1] > rank) {
+                    lo = win_lo;
+                    hi = win_hi;
+                }
                 while (lo < hi) {
                     const uint32_t mid = lo + ((hi - lo + 1) >> 1);
                     if (dir_sh[mid] <= rank)
@@ -351,25 +364,15 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
             if (d1 - d0 == kDirStride) {
                 idx = grp * kDirStride + rem;   // no core parameter in this group
             } else {
-                // ... then the word holding the rem-th zero bit of the group, then the bit
-                const uint32_t* grp_words = bitmap + (uint64_t)grp * kWordsPerDir;
-                const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(grp_words));
-                const uint4 v1 = __ldg(reinterpret_cast<const uint4*>(grp_words) + 1);
-                const uint32_t w8[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-                uint32_t zeros = 0, wsel = 0, before = 0, zword = 0;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const uint32_t z = ~w8[q];
-                    const uint32_t after = zeros + __popc(z);
-                    const bool passed = after <= rem;          // the whole word lies before the wanted zero
-                    const bool here = !passed && zeros <= rem;  // the wanted zero is in this word
-                    wsel += passed ? 1u : 0u;
-                    before = passed ? after : before;
-                    zword = here ? z : zword;
-                    zeros = after;
-                }
-                idx = (wsel < kWordsPerDir) ? grp * kDirStride + wsel * 32u + nth_set_bit(zword, rem - before)
-                                            : 0xFFFFFFFFu;
+                // ... then the rem-th zero bit of the group's two bitmap words
+                const uint2 v = __ldg(reinterpret_cast<const uint2*>(bitmap + (uint64_t)grp * kWordsPerDir));
+                const uint32_t z0 = ~v.x, z1 = ~v.y;
+                const uint32_t c0 = __popc(z0);
+                const bool second = rem >= c0;
+                const uint32_t z = second ? z1 : z0;
+                const uint32_t r = second ? rem - c0 : rem;
+                idx = (r < (uint32_t)__popc(z)) ? grp * kDirStride + (second ? 32u : 0u) + nth_set_bit(z, r)
+                                                : 0xFFFFFFFFu;
             }
             if (idx == 0xFFFFFFFFu || offset + r0 + e >= k_exp) {
                 hdr->status = SLIMDP_ERR_INTERNAL;   // directory and bitmap disagree

@@ -499,7 +499,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const uint32_t* __restrict__ 
         const uint32_t ps_incl = warp_inclusive_scan(ps);
         const uint32_t out_base = sel_before + ps_incl - ps;
         bitmap[blk * kWordsPerBlock + lane] = sel;
-        if ((lane & (kWordsPerDir - 1)) == 0)   // one directory entry per 256 parameters (8 words)
+        if ((lane & (kWordsPerDir - 1)) == 0)   // one directory entry per 64 parameters (2 words)
             dir[blk * kDirPerBlock + lane / kWordsPerDir] = (uint32_t)(blk * kBlock + lane * 32 - out_base);
         const uint32_t in_block = __shfl_sync(0xFFFFFFFFu, ps_incl, 31);
         if (in_block == 0) continue;

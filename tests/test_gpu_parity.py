@@ -13,6 +13,8 @@ from workloads import CONFIGS, all_inputs, scaled_config
 
 pytestmark = pytest.mark.gpu
 
+DIR_STRIDE = 64      # parameters per directory entry of core_aux (SLIMDP_DIR_STRIDE)
+
 
 @pytest.fixture(scope="module")
 def P():
@@ -41,15 +43,15 @@ def bits(a) -> np.ndarray:
 
 
 def expected_aux(P, core: np.ndarray, n: int):
-    """core_aux by its definition: bitmap of the core, non-core counts before each 1024-block."""
+    """core_aux by its definition: bitmap of the core, non-core counts before each 64-parameter group."""
     nb = (n + 1023) // 1024
     member = np.zeros(nb * 1024, np.uint8)
     member[core] = 1
     words = np.packbits(member.reshape(-1, 8), axis=1, bitorder="little").reshape(-1).view(np.uint32)
-    nd = nb * 4
-    per_group = member.reshape(nd, 256).sum(axis=1, dtype=np.int64)
+    nd = nb * (1024 // DIR_STRIDE)
+    per_group = member.reshape(nd, DIR_STRIDE).sum(axis=1, dtype=np.int64)
     directory = np.zeros(nd + 1, np.int64)
-    directory[1:] = np.cumsum(256 - per_group)       # 256 d minus the core members below 256 d
+    directory[1:] = np.cumsum(DIR_STRIDE - per_group)       # 64 d minus the core members below 64 d
     directory[nd] = n - core.size
     return words, directory.astype(np.uint32)
 
@@ -71,7 +73,7 @@ def check_aux(P, aux: torch.Tensor, core: np.ndarray, n: int):
     words, directory = expected_aux(P, core, n)
     assert np.array_equal(raw[:nb * 128].view(np.uint32), words)
     off = P.core_aux_dir_offset(n)
-    assert np.array_equal(raw[off:off + 4 * (4 * nb + 1)].view(np.uint32), directory)
+    assert np.array_equal(raw[off:off + 4 * directory.size].view(np.uint32), directory)
 
 
 # --------------------------------------------------------------------- score
@@ -367,7 +369,8 @@ def test_round_is_deterministic(P):
     nb = (cfg.N + 1023) // 1024
     off = P.core_aux_dir_offset(cfg.N)
     assert torch.equal(a.core_aux[:nb * 128], b.core_aux[:nb * 128])                      # bitmap
-    assert torch.equal(a.core_aux[off:off + 4 * (4 * nb + 1)], b.core_aux[off:off + 4 * (4 * nb + 1)])   # directory
+    nd = nb * (1024 // DIR_STRIDE)
+    assert torch.equal(a.core_aux[off:off + 4 * (nd + 1)], b.core_aux[off:off + 4 * (nd + 1)])   # directory
     for k in range(cfg.K):
         assert torch.equal(a.exp_idx[k], b.exp_idx[k]) and torch.equal(a.pulled[k], b.pulled[k])
 
