@@ -130,10 +130,11 @@ slimdp_status slimdp_select_core(const float* scores, uint64_t n, uint64_t k_cor
  * reproduced bit for bit:
  *   round keys rk[0..11] = three Philox-4x32-10 blocks with key
  *       (seed low word, seed high word) and counters (b, worker, round, 0x534C494D), b = 0, 1, 2;
- *   pi = a 10-round balanced Feistel network on 2h bits, h = ceil(b/2) with b the least
- *       integer >= 1 such that 2^b >= M; round r maps (L, R) to (R, (L ^ F) & (2^h - 1)),
- *       F = hi32(p) ^ lo32(p), p = (uint64)(R ^ rk[r]) * (r even ? 0xD2511F53 : 0xCD9E8D57);
- *       images >= M are fed through the network again (cycle walking);
+ *   pi = a 10-round alternating Feistel network on b bits, b the least integer >= 2 with
+ *       2^b >= M: x = A * 2^c + B with A of a = floor(b/2) bits and B of c = b - a bits;
+ *       even round r: A = (A ^ F(B ^ rk[r])) & (2^a - 1); odd round r: B = (B ^ F(A ^ rk[r])) & (2^c - 1);
+ *       F(v) = hi32(p) ^ lo32(p), p = (uint64)v * (r even ? 0xD2511F53 : 0xCD9E8D57);
+ *       images >= M are fed through the network again (cycle walking, fewer than 2 passes on average);
  *   explorer = { the pi(j)-th non-core parameter (0-based, ascending) : j < k_exp }.
  *   core_aux  as written by slimdp_select_core for the same n and k_core (read)
  *   k_exp     0 <= k_exp <= n - k_core

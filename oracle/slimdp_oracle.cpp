@@ -25,7 +25,8 @@
 //     the parameters outside the core, drawn anew per worker and per
 //     communication) is an exact-size uniform subset: the first k_exp images
 //     of a keyed pseudo-random permutation of the M = n - k_core non-core
-//     ranks.  The paper fixes only "random, outside the core"; the generator
+//     ranks (an alternating Feistel network on the smallest power-of-two
+//     domain that holds M, with cycle walking).  The paper fixes only "random, outside the core"; the generator
 //     (Philox-4x32-10 round keys feeding a cycle-walking Feistel network) is
 //     this library's own definition.  It is pinned by the generator's
 //     published known answers, by exhaustive bijection checks, by an
@@ -87,32 +88,42 @@ void round_keys(uint64_t seed, uint32_t worker, uint32_t round, uint32_t rk[12])
     }
 }
 
-// Half-width h of the Feistel domain for M ranks: b = least integer >= 1 with
-// 2^b >= M, h = ceil(b / 2); the network permutes [0, 2^(2h)).
-int half_bits(uint64_t M) {
-    int b = 1;
+// Width of the Feistel domain for M ranks: b = least integer >= 2 with 2^b >= M.
+// The network permutes [0, 2^b): x = A * 2^c + B with A of a = floor(b / 2) bits
+// and B of c = b - a bits.
+int domain_bits(uint64_t M) {
+    int b = 2;
     while (((uint64_t)1 << b) < M) ++b;
-    return (b + 1) / 2;
+    return b;
 }
 
-// pi(j) on [0, M): apply the balanced Feistel network to j, and while the
-// image falls outside [0, M) apply it again (cycle walking).
+// Round function: both halves of the 64-bit product of v with the round's multiplier, folded.
+uint32_t round_function(uint32_t v, int r) {
+    const uint64_t mult = (r % 2 == 0) ? 0xD2511F53u : 0xCD9E8D57u;
+    const uint64_t p = (uint64_t)v * mult;
+    return (uint32_t)(p >> 32) ^ (uint32_t)p;
+}
+
+// pi(j) on [0, M): apply the alternating Feistel network to j (even rounds change A by a
+// function of B, odd rounds change B by a function of A; each round is invertible, so the
+// network is a bijection of [0, 2^b) for any split), and while the image falls outside
+// [0, M) apply it again (cycle walking).
 uint64_t feistel_perm(uint64_t j, uint64_t M, const uint32_t rk[12]) {
-    const int h = half_bits(M);
-    const uint32_t mask = (uint32_t)(((uint64_t)1 << h) - 1);
+    const int b = domain_bits(M);
+    const int a = b / 2, c = b - a;
+    const uint32_t maskA = (uint32_t)(((uint64_t)1 << a) - 1);
+    const uint32_t maskB = (uint32_t)(((uint64_t)1 << c) - 1);
     uint64_t x = j;
     do {
-        uint32_t L = (uint32_t)(x >> h);
-        uint32_t R = (uint32_t)(x & mask);
+        uint32_t A = (uint32_t)(x >> c);
+        uint32_t B = (uint32_t)(x & maskB);
         for (int r = 0; r < FEISTEL_ROUNDS; ++r) {
-            const uint64_t mult = (r % 2 == 0) ? 0xD2511F53u : 0xCD9E8D57u;
-            uint64_t p = (uint64_t)(uint32_t)(R ^ rk[r]) * mult;
-            uint32_t F = (uint32_t)(p >> 32) ^ (uint32_t)p;
-            uint32_t newR = (L ^ F) & mask;
-            L = R;
-            R = newR;
+            if (r % 2 == 0)
+                A = (A ^ round_function(B ^ rk[r], r)) & maskA;
+            else
+                B = (B ^ round_function(A ^ rk[r], r)) & maskB;
         }
-        x = ((uint64_t)L << h) | R;
+        x = ((uint64_t)A << c) | B;
     } while (x >= M);
     return x;
 }

@@ -8,8 +8,8 @@
 // the ranks are uniform on [0, M), so a bucket sort by the ranks' high bits
 // is balanced:
 //   1. setup: round keys (three Philox-4x32-10 blocks per worker);
-//   2. rank: thread j evaluates pi(j) (10-round Feistel network with cycle
-//      walking), stores it and counts it into its bucket (rank >> s);
+//   2. rank: thread j evaluates pi(j) (10-round alternating Feistel network
+//      with cycle walking), stores it and counts it into its bucket (rank >> s);
 //   3. two-kernel exclusive scan of the bucket counts;
 //   4. scatter: every rank goes to its bucket's slice (order inside a bucket
 //      is arbitrary here and is fixed by the next step);
@@ -95,7 +95,7 @@ __global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, u
 // Lanes whose walk has ended take the next j of their warp's range at once, so a
 // long cycle walk in one lane does not idle the other 31.
 template <bool SMEM_HIST>
-__global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, uint32_t chunk, uint32_t h,
+__global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, uint32_t chunk, uint32_t bits,
                                                     uint32_t s, uint32_t buckets,
                                                     const uint32_t* __restrict__ rk_all, uint32_t* __restrict__ rho,
                                                     uint64_t rho_stride, unsigned long long* __restrict__ cnt,
@@ -109,7 +109,9 @@ __global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, 
     uint32_t rk[10];
 #pragma unroll
     for (int r = 0; r < 10; ++r) rk[r] = rk_all[worker * 12 + r];
-    const uint32_t mask = (1u << h) - 1u;
+    // x = A * 2^c + B, A of a = floor(bits / 2) bits, B of c = bits - a bits
+    const uint32_t a = bits >> 1, c = bits - a;
+    const uint32_t maskA = (1u << a) - 1u, maskB = (1u << c) - 1u;
     uint32_t* my_rho = rho + (uint64_t)worker * rho_stride;
     unsigned long long* my_cnt = cnt + (uint64_t)worker * cnt_stride;
     // this warp's contiguous range of j
@@ -134,17 +136,20 @@ __global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, 
         next += __popc(want);
         if (__ballot_sync(0xFFFFFFFFu, have) == 0) break;
         if (have) {
-            uint32_t L = x >> h, R = x & mask;
+            uint32_t A = x >> c, B = x & maskB;
 #pragma unroll
             for (int r = 0; r < 10; ++r) {
+                // even rounds change A by a function of B, odd rounds change B by a function of A
                 const unsigned long long mult = (r & 1) ? 0xCD9E8D57ull : 0xD2511F53ull;
-                const unsigned long long prod = (unsigned long long)(R ^ rk[r]) * mult;   // one 32x32->64 multiply
+                const uint32_t v = ((r & 1) ? A : B) ^ rk[r];
+                const unsigned long long prod = (unsigned long long)v * mult;   // one 32x32->64 multiply
                 const uint32_t F = (uint32_t)(prod >> 32) ^ (uint32_t)prod;
-                const uint32_t nr = (L ^ F) & mask;
-                L = R;
-                R = nr;
+                if (r & 1)
+                    B = (B ^ F) & maskB;
+                else
+                    A = (A ^ F) & maskA;
             }
-            x = (L << h) | R;
+            x = (A << c) | B;
             if (x < M) {          // the walk ends at the first image inside [0, M)
                 my_rho[j] = x;
                 if (SMEM_HIST)
@@ -418,9 +423,8 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
     if (k_exp == 0) return SLIMDP_OK;
     if (cudaMemsetAsync(L.cnt, 0, L.zero_bytes, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
 
-    int b = 1;
-    while (((uint64_t)1 << b) < M) ++b;
-    const uint32_t h = (uint32_t)((b + 1) / 2);
+    uint32_t bits = 2;   // the permutation's domain is [0, 2^bits), the smallest that holds M (at least 4)
+    while (((uint64_t)1 << bits) < M) ++bits;
 
     // about two 1024-thread CTAs per SM over all workers; every CTA owns one contiguous chunk of j
     uint64_t chunks = ((uint64_t)sms * 2 + workers - 1) / workers;
@@ -431,11 +435,11 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
     const dim3 grid((unsigned)chunks, workers);
     const bool smem = buckets <= kMaxSmemBuckets;
     if (smem) {
-        rank_kernel<true><<<grid, 1024, buckets * 4, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, h, s,
+        rank_kernel<true><<<grid, 1024, buckets * 4, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, bits, s,
                                                            (uint32_t)buckets, L.round_keys, L.rho, L.rho_stride,
                                                            L.cnt, L.cnt_stride, L.cta_hist);
     } else {
-        rank_kernel<false><<<grid, 1024, 0, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, h, s, (uint32_t)buckets,
+        rank_kernel<false><<<grid, 1024, 0, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, bits, s, (uint32_t)buckets,
                                                   L.round_keys, L.rho, L.rho_stride, L.cnt, L.cnt_stride,
                                                   L.cta_hist);
     }

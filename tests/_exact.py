@@ -65,19 +65,24 @@ def round_keys_py(seed, worker, rnd):
 
 
 def perm_py(j, M, rk):
-    b = 1
+    b = 2
     while (1 << b) < M:
         b += 1
-    h = (b + 1) // 2
-    mask = (1 << h) - 1
+    a = b // 2
+    c = b - a
+    mask_a, mask_b = (1 << a) - 1, (1 << c) - 1
     x = j
     while True:
-        L, R = x >> h, x & mask
+        A, B = x >> c, x & mask_b
         for r in range(10):
-            p = ((R ^ rk[r]) & M32) * (0xD2511F53 if r % 2 == 0 else 0xCD9E8D57)
+            v = ((B if r % 2 == 0 else A) ^ rk[r]) & M32
+            p = v * (0xD2511F53 if r % 2 == 0 else 0xCD9E8D57)
             F = ((p >> 32) ^ p) & M32
-            L, R = R, (L ^ F) & mask
-        x = (L << h) | R
+            if r % 2 == 0:
+                A = (A ^ F) & mask_a
+            else:
+                B = (B ^ F) & mask_b
+        x = (A << c) | B
         if x < M:
             return x
 
