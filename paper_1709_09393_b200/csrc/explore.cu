@@ -84,10 +84,23 @@ __global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, u
 #pragma unroll
         for (int q = 0; q < 4; ++q) rk[w * 12 + b * 4 + q] = out[q];
     }
-    if (M > 0 && t <= buckets) {
-        const uint64_t first = (uint64_t)t << s;
+    // one warp per bucket boundary: a 32-way search (5 probes for 2^25 entries instead of 25)
+    const uint32_t bnd = t >> 5, lane = t & 31u;
+    if (M > 0 && bnd <= buckets) {
+        const uint64_t first = (uint64_t)bnd << s;
         const uint32_t rank = (first < M) ? (uint32_t)first : M - 1;
-        bounds[t] = find_block(dir, 0, nd - 1, rank);
+        uint32_t lo = 0, hi = nd - 1;   // the answer is the largest d in [lo, hi] with dir[d] <= rank; dir[lo] <= rank
+        while (hi > lo) {
+            const uint32_t step = (hi - lo) / 32u + 1u;              // lane probes lo + lane * step
+            const uint64_t p = (uint64_t)lo + (uint64_t)lane * step;
+            const bool le = p <= hi && __ldg(dir + p) <= rank;       // true for a prefix of the lanes (lane 0 always)
+            const uint32_t c = __popc(__ballot_sync(0xFFFFFFFFu, le));
+            const uint32_t nlo = lo + (c - 1u) * step;
+            const uint64_t nhi = (uint64_t)nlo + step - 1u;
+            lo = nlo;
+            hi = (nhi < hi) ? (uint32_t)nhi : hi;
+        }
+        if (lane == 0) bounds[bnd] = lo;
     }
 }
 
@@ -414,7 +427,8 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
     const uint32_t s = explore_bucket_shift(M);
     const uint64_t buckets = (M + (1ull << s) - 1) >> s;
 
-    const unsigned setup_threads = (unsigned)((buckets + 1 > 3ull * workers) ? buckets + 1 : 3ull * workers);
+    const unsigned setup_threads =
+        (unsigned)(((buckets + 1) * 32 > 3ull * workers) ? (buckets + 1) * 32 : 3ull * workers);
     explore_setup_kernel<<<(setup_threads + 255) / 256, 256, 0, st>>>(L.hdr, L.round_keys, (uint32_t)seed,
                                                                       (uint32_t)(seed >> 32), first_worker, workers,
                                                                       round, dir, (uint32_t)nd, (uint32_t)M, s,

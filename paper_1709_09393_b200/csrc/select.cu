@@ -201,7 +201,7 @@ constexpr uint32_t kStage = kFlushAt + 256;    // staging capacity: below kFlush
 // Warp per 1024-parameter block, a quarter block (8 words) at a time.  Candidates are staged per
 // warp in shared memory and appended to the global list at least kFlushAt at a time, so the
 // list cursor sees one atomic per kFlushAt candidates or more.
-__global__ void __launch_bounds__(256) bracket_pass_kernel(const uint32_t* __restrict__ keys, uint64_t n, uint64_t nb,
+__global__ void __launch_bounds__(256, 8) bracket_pass_kernel(const uint32_t* __restrict__ keys, uint64_t n, uint64_t nb,
                                                            WsHeader* hdr, uint32_t cap, uint32_t* __restrict__ G,
                                                            uint32_t* __restrict__ E,
                                                            unsigned long long* __restrict__ cnt,
