@@ -267,10 +267,14 @@ def run_ours(args):
     # ---- per-call breakdown (untimed for the headline; 5 more rounds) -------
     # "exchange" is the fused pack + merge + pull the timed rounds use; the three separate calls
     # are timed after it for comparison (they repeat the exchange's work on the next model state)
-    names = ["score", "select", "explore", "exchange", "pack_alone", "merge_alone", "pull_alone"]
+    # after them the two steps either side of the path: the worker-side merge and the dense push
+    # (+ scoring) of a reselection boundary
+    names = ["score", "select", "explore", "exchange", "pack_alone", "merge_alone", "pull_alone", "worker_merge",
+             "dense_merge_score"]
     acc = {nm: [] for nm in names}
+    local = [w.clone() for _ in range(K)]
     for _ in range(5):
-        marks = [torch.cuda.Event(enable_timing=True) for _ in range(8)]
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(10)]
         marks[0].record()
         P.slimdp_score(w, grads, cfg.c, buf.scores); marks[1].record()
         P.slimdp_select_core(buf.scores, k_core, buf.core_idx, buf.core_aux, buf.select_ws); marks[2].record()
@@ -280,11 +284,14 @@ def run_ours(args):
         P.slimdp_pack_batched(grads, buf.core_idx, buf.exp_idx, buf.val); marks[5].record()
         P.slimdp_merge(w, buf.core_idx, buf.exp_idx, buf.val, cfg.eta); marks[6].record()
         P.slimdp_pull_batched(w, buf.core_idx, buf.exp_idx, buf.pulled); marks[7].record()
+        P.slimdp_worker_merge_batched(local, buf.core_idx, buf.exp_idx, buf.pulled); marks[8].record()
+        P.slimdp_dense_merge_score(w, grads, cfg.eta, cfg.c, buf.scores); marks[9].record()
         torch.cuda.synchronize()
         t += 1
         for i, nm in enumerate(names):
             acc[nm].append(marks[i].elapsed_time(marks[i + 1]) * 1e3)
     breakdown_us = {nm: round(statistics.median(v), 1) for nm, v in acc.items()}
+    del local
 
     peak, peak_src = measured_peak()
     achieved = bytes_model["score"] / (score_ms * 1e-3) / 1e9

@@ -242,6 +242,33 @@ slimdp_status slimdp_exchange(float* w_global, uint64_t n, uint32_t K, const flo
                               const uint32_t* core_idx, uint64_t k_core, const uint32_t* const* exp_idx,
                               uint64_t k_exp, float eta, float* const* val, float* const* pulled, void* stream);
 
+/* ------------------------------------------ the steps either side of the path ---
+ * Dense push at a reselection boundary (Algorithm 1, worker: "if (t+1) % q == 0
+ * Push(delta)"; server: Update, t <- t+1, "if t % q == 0 Core-Selection(w-bar^t,
+ * delta^t, beta)"; Section 3.3 steps 3 and 6).  One pass applies every worker's
+ * WHOLE update to the global model in ascending worker order (this is also
+ * Plump-DP's update, Section 2.1) and, if scores is not NULL, scores the
+ * UPDATED model with the updates just pushed:
+ *     x = w[i];  g = grads[0][i];  x = fma(-eta, grads[0][i], x);
+ *     for k = 1..K-1:  g = g + grads[k][i];  x = fma(-eta, grads[k][i], x);
+ *     w[i] = x;  scores[i] = fma(c, |g|, |x|)   (NaN stored as 0x7FC00000)
+ * Bit-identical to slimdp_merge with everything in the communication set
+ * followed by slimdp_score.
+ *   w_global [n] (updated in place); grads HOST array of K device pointers [n]; scores [n] or NULL
+ */
+slimdp_status slimdp_dense_merge_score(float* w_global, const float* const* grads, uint32_t K, float eta, float c,
+                                       uint64_t n, float* scores, void* stream);
+
+/* Worker-side Merge (Algorithm 1 "Merge(w_k, w~_k)", Section 3.3 step 5): the
+ * values a worker pulled replace its local model's values on its communication
+ * set; the rest of the local model is left as local training made it.
+ *     w_local[k][core_idx[j]] = pulled[k][j];  w_local[k][exp_idx[k][j]] = pulled[k][k_core + j]
+ *   w_local, exp_idx, pulled: HOST arrays of K device pointers ([n], [k_exp], [k_core + k_exp])
+ */
+slimdp_status slimdp_worker_merge_batched(float* const* w_local, uint32_t K, uint64_t n, const uint32_t* core_idx,
+                                          uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
+                                          const float* const* pulled, void* stream);
+
 /* --------------------------------------------------------------- status ---
  * Synchronises `stream`, then returns the sticky status word kept in the first
  * 4 bytes of a workspace used by slimdp_select_core / slimdp_sample_explore*:

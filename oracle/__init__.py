@@ -40,6 +40,7 @@ _merge = _sig("oracle_merge", None, _f32p, ctypes.c_uint32, _u32p, ctypes.c_uint
               _pp, ctypes.c_float)
 _pull = _sig("oracle_pull", None, _f32p, _u32p, ctypes.c_uint64, _u32p, ctypes.c_uint64, _f32p)
 _dense = _sig("oracle_dense_merge", None, _f32p, ctypes.c_uint64, ctypes.c_uint32, _pp, ctypes.c_float)
+_wmerge = _sig("oracle_worker_merge", None, _f32p, _u32p, ctypes.c_uint64, _u32p, ctypes.c_uint64, _f32p)
 
 
 def _f32(a) -> np.ndarray:
@@ -133,6 +134,15 @@ def dense_merge(w, grads: Sequence[np.ndarray], eta: float) -> np.ndarray:
     out = _f32(w).copy()
     gs = [_f32(g) for g in grads]
     _dense(_ptr(out, _f32p), out.size, len(gs), _ptr_array(gs), eta)
+    return out
+
+
+def worker_merge(w_local, core_idx, exp_idx, pulled) -> np.ndarray:
+    """Returns the merged copy of the local model (the input is left untouched)."""
+    out = _f32(w_local).copy()
+    c, e, p = _u32(core_idx), _u32(exp_idx), _f32(pulled)
+    assert p.size == c.size + e.size
+    _wmerge(_ptr(out, _f32p), _ptr(c, _u32p), c.size, _ptr(e, _u32p), e.size, _ptr(p, _f32p))
     return out
 
 

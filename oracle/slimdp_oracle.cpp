@@ -15,6 +15,7 @@
 //   merge   Section 3.3 step 3: w <- w - eta' * T_C(delta_k), every worker, k ascending
 //   pull    Section 3.3 step 4: T_C(w) = the merged values on core U explorer
 //   dense   Section 2.1: Plump-DP pushes and merges every parameter
+//   worker merge  Section 3.3 step 5: pulled values overwrite the local model on T_C
 // Readings the paper leaves open (all also listed in the design notes):
 //   * g_i is the fp32 sum of the K workers' dense updates, k ascending
 //     (Section 3.3 step 6 scores with the updates pushed densely before reselection);
@@ -224,6 +225,14 @@ void oracle_pull(const float* w, const uint32_t* core_idx, uint64_t k_core,
                  const uint32_t* exp_idx, uint64_t k_exp, float* out) {
     for (uint64_t j = 0; j < k_core; ++j) out[j] = w[core_idx[j]];
     for (uint64_t j = 0; j < k_exp; ++j) out[k_core + j] = w[exp_idx[j]];
+}
+
+// Worker-side Merge (Algorithm 1; Section 3.3 step 5), read as: the pulled values replace the
+// local model's values on the communication set, the rest of the local model is untouched.
+void oracle_worker_merge(float* w_local, const uint32_t* core_idx, uint64_t k_core, const uint32_t* exp_idx,
+                         uint64_t k_exp, const float* pulled) {
+    for (uint64_t j = 0; j < k_core; ++j) w_local[core_idx[j]] = pulled[j];
+    for (uint64_t j = 0; j < k_exp; ++j) w_local[exp_idx[j]] = pulled[k_core + j];
 }
 
 // Plump-DP (Section 2.1): every worker pushes its whole update.

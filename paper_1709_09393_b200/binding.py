@@ -47,6 +47,8 @@ EXPORTS = {
     "slimdp_pull": (ctypes.c_int32, [_vp, _u64, _vp, _u64, _vp, _u64, _vp, _vp]),
     "slimdp_pull_batched": (ctypes.c_int32, [_vp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _vp]),
     "slimdp_exchange": (ctypes.c_int32, [_vp, _u64, _u32, _pp, _vp, _u64, _pp, _u64, _f32, _pp, _pp, _vp]),
+    "slimdp_dense_merge_score": (ctypes.c_int32, [_vp, _pp, _u32, _f32, _f32, _u64, _vp, _vp]),
+    "slimdp_worker_merge_batched": (ctypes.c_int32, [_pp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _vp]),
     "slimdp_read_status": (ctypes.c_int32, [_vp, _vp]),
     "slimdp_launch_count": (_u64, []),
     "slimdp_round_arena_bytes": (_sz, [_u64, _u32, _u64, _u64]),
@@ -271,6 +273,38 @@ def slimdp_exchange(w_global: torch.Tensor, deltas: Sequence[torch.Tensor], core
            lib.slimdp_exchange(w_global.data_ptr(), w_global.numel(), K, _ptr_array(deltas), _ptr(core_idx),
                                core_idx.numel(), _ptr_array(exp_idx), exp_idx[0].numel(), eta, _ptr_array(val),
                                _ptr_array(pulled), _stream(stream)))
+
+
+def slimdp_dense_merge_score(w_global: torch.Tensor, grads: Sequence[torch.Tensor], eta: float, c: float,
+                             scores: Optional[torch.Tensor] = None, stream=None):
+    """Dense push of all workers at a reselection boundary; optionally scores the updated model."""
+    n = w_global.numel()
+    _dev(w_global, torch.float32, "w_global")
+    for g in grads:
+        if _dev(g, torch.float32, "grads").numel() != n:
+            raise ValueError("grads: length differs from w_global")
+    if scores is not None and _dev(scores, torch.float32, "scores").numel() != n:
+        raise ValueError("scores: length differs from w_global")
+    _check("slimdp_dense_merge_score",
+           lib.slimdp_dense_merge_score(w_global.data_ptr(), _ptr_array(grads), len(grads), eta, c, n, _ptr(scores),
+                                        _stream(stream)))
+
+
+def slimdp_worker_merge_batched(w_local: Sequence[torch.Tensor], core_idx: torch.Tensor,
+                                exp_idx: Sequence[torch.Tensor], pulled: Sequence[torch.Tensor], stream=None):
+    """Worker-side Merge: pulled values overwrite each local model on its communication set."""
+    K = len(w_local)
+    if len(exp_idx) != K or len(pulled) != K:
+        raise ValueError("w_local, exp_idx and pulled must have K entries each")
+    n = w_local[0].numel()
+    for wl, e, p in zip(w_local, exp_idx, pulled):
+        if _dev(wl, torch.float32, "w_local").numel() != n:
+            raise ValueError("w_local: lengths differ")
+        _check_sets(core_idx, e, p, "pulled")
+    _check("slimdp_worker_merge_batched",
+           lib.slimdp_worker_merge_batched(_ptr_array(w_local), K, n, _ptr(core_idx), core_idx.numel(),
+                                           _ptr_array(exp_idx), exp_idx[0].numel(), _ptr_array(pulled),
+                                           _stream(stream)))
 
 
 def _host(t: torch.Tensor, dtype, name: str) -> torch.Tensor:

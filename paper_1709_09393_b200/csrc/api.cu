@@ -37,6 +37,12 @@ slimdp_status launch_explore_static(const void* core_aux, uint64_t n, uint64_t k
                                     uint32_t worker, uint32_t round, uint32_t* exp_idx, int32_t* status_out,
                                     cudaStream_t st);
 
+slimdp_status launch_dense_merge_score(float* w, const PtrArray<const float>& g, uint32_t K, float eta, float c,
+                                       uint64_t n, float* S, bool vec, cudaStream_t st);
+slimdp_status launch_worker_merge(const PtrArray<float>& w_local, uint32_t workers, const uint32_t* core_idx,
+                                  uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp,
+                                  const PtrArray<const float>& pulled, cudaStream_t st);
+
 int sm_count() {
     static int cached[64];
     int dev = 0;
@@ -247,6 +253,31 @@ slimdp_status slimdp_exchange(float* w_global, uint64_t n, uint32_t K, const flo
     if (!fill<float>(o, pulled, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (k_core + k_exp == 0) return SLIMDP_OK;
     return launch_exchange(w_global, n, K, d, core_idx, k_core, exp, k_exp, eta, v, o, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_dense_merge_score(float* w_global, const float* const* grads, uint32_t K, float eta, float c,
+                                       uint64_t n, float* scores, void* stream) {
+    if (!n_ok(n) || !k_ok(K) || !w_global || !grads || !isfinite(c) || !isfinite(eta)) return SLIMDP_ERR_INVALID_ARG;
+    if (!aligned4(w_global) || (scores && !aligned4(scores))) return SLIMDP_ERR_INVALID_ARG;
+    PtrArray<const float> g;
+    if (!fill<const float>(g, grads, K, true, 4)) return SLIMDP_ERR_INVALID_ARG;
+    bool vec = aligned16(w_global) && (!scores || aligned16(scores));
+    for (uint32_t k = 0; k < K; ++k) vec = vec && aligned16(g.p[k]);
+    return launch_dense_merge_score(w_global, g, K, eta, c, n, scores, vec, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_worker_merge_batched(float* const* w_local, uint32_t K, uint64_t n, const uint32_t* core_idx,
+                                          uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
+                                          const float* const* pulled, void* stream) {
+    if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !w_local) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    PtrArray<float> w;
+    PtrArray<const uint32_t> exp;
+    PtrArray<const float> v;
+    if (!fill<float>(w, w_local, K, true, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const float>(v, pulled, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
+    return launch_worker_merge(w, K, core_idx, k_core, exp, k_exp, v, (cudaStream_t)stream);
 }
 
 uint64_t slimdp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

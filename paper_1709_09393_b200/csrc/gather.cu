@@ -75,7 +75,40 @@ __global__ void __launch_bounds__(256) gather_explore_kernel(PtrArray<const floa
     }
 }
 
+// Worker-side Merge (Algorithm 1; Section 3.3 step 5): the pulled values replace the local
+// model's values on the communication set.  grid.y = worker.
+__global__ void __launch_bounds__(256) worker_merge_kernel(PtrArray<float> w_local,
+                                                           const uint32_t* __restrict__ core_idx, uint64_t k_core,
+                                                           PtrArray<const uint32_t> exp, uint64_t k_exp,
+                                                           PtrArray<const float> pulled) {
+    const uint32_t worker = blockIdx.y;
+    float* __restrict__ w = w_local.p[worker];
+    const uint32_t* __restrict__ e = exp.p[worker];
+    const float* __restrict__ v = pulled.p[worker];
+    const uint64_t m = k_core + k_exp;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < m; j += stride) {
+        const uint32_t i = (j < k_core) ? __ldg(core_idx + j) : __ldg(e + (j - k_core));
+        w[i] = __ldcs(v + j);
+    }
+}
+
 }  // namespace
+
+slimdp_status launch_worker_merge(const PtrArray<float>& w_local, uint32_t workers, const uint32_t* core_idx,
+                                  uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp,
+                                  const PtrArray<const float>& pulled, cudaStream_t st) {
+    const uint64_t m = k_core + k_exp;
+    if (m == 0) return SLIMDP_OK;
+    const int sms = sm_count();
+    if (sms <= 0) return SLIMDP_ERR_CUDA;
+    uint64_t grid = (m + 255) / 256;
+    const uint64_t cap = ((uint64_t)sms * 32 + workers - 1) / workers;
+    if (grid > cap) grid = cap;
+    worker_merge_kernel<<<dim3((unsigned)grid, workers), 256, 0, st>>>(w_local, core_idx, k_core, exp, k_exp, pulled);
+    SLIMDP_LAUNCHED(1);
+    return SLIMDP_OK;
+}
 
 slimdp_status launch_gather(const PtrArray<const float>& src, bool same_src, uint32_t workers,
                             const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,

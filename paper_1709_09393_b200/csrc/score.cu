@@ -74,7 +74,79 @@ __global__ void __launch_bounds__(256) score_scalar_kernel(const float* __restri
     }
 }
 
+// Dense push at a reselection boundary (Algorithm 1: Push(delta) when (t + 1) % q == 0, then
+// Update, then Core-Selection on the updated model with the updates just pushed): one streaming
+// pass applies every worker's whole update in worker order and, if S is given, scores the result.
+template <bool VEC>
+__global__ void __launch_bounds__(256) dense_merge_score_kernel(float* __restrict__ w, PtrArray<const float> g, int K,
+                                                                float neg_eta, float c, uint64_t n,
+                                                                float* __restrict__ S) {
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    if (VEC) {
+        const uint64_t n4 = n / 4;
+        float4* w4 = reinterpret_cast<float4*>(w);
+        for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+            float4 x = w4[i];
+            float4 a = __ldcs(reinterpret_cast<const float4*>(g.p[0]) + i);
+            x.x = __fmaf_rn(neg_eta, a.x, x.x);
+            x.y = __fmaf_rn(neg_eta, a.y, x.y);
+            x.z = __fmaf_rn(neg_eta, a.z, x.z);
+            x.w = __fmaf_rn(neg_eta, a.w, x.w);
+#pragma unroll 4
+            for (int k = 1; k < K; ++k) {
+                const float4 b = __ldcs(reinterpret_cast<const float4*>(g.p[k]) + i);
+                a.x = __fadd_rn(a.x, b.x);
+                a.y = __fadd_rn(a.y, b.y);
+                a.z = __fadd_rn(a.z, b.z);
+                a.w = __fadd_rn(a.w, b.w);
+                x.x = __fmaf_rn(neg_eta, b.x, x.x);
+                x.y = __fmaf_rn(neg_eta, b.y, x.y);
+                x.z = __fmaf_rn(neg_eta, b.z, x.z);
+                x.w = __fmaf_rn(neg_eta, b.w, x.w);
+            }
+            w4[i] = x;
+            if (S) {
+                float4 s;
+                s.x = score_one(c, a.x, x.x);
+                s.y = score_one(c, a.y, x.y);
+                s.z = score_one(c, a.z, x.z);
+                s.w = score_one(c, a.w, x.w);
+                reinterpret_cast<float4*>(S)[i] = s;
+            }
+        }
+    }
+    // scalar path: everything when not vectorised, else the ragged tail
+    const uint64_t first = VEC ? (n / 4) * 4 : 0;
+    for (uint64_t i = first + (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        float x = w[i];
+        float a = g.p[0][i];
+        x = __fmaf_rn(neg_eta, a, x);
+        for (int k = 1; k < K; ++k) {
+            const float b = g.p[k][i];
+            a = __fadd_rn(a, b);
+            x = __fmaf_rn(neg_eta, b, x);
+        }
+        w[i] = x;
+        if (S) S[i] = score_one(c, a, x);
+    }
+}
+
 }  // namespace
+
+slimdp_status launch_dense_merge_score(float* w, const PtrArray<const float>& g, uint32_t K, float eta, float c,
+                                       uint64_t n, float* S, bool vec, cudaStream_t st) {
+    const int sms = sm_count();
+    if (sms <= 0) return SLIMDP_ERR_CUDA;
+    uint64_t blocks = ((vec ? n / 4 : n) + 255) / 256;
+    if (blocks > (uint64_t)sms * 32) blocks = (uint64_t)sms * 32;
+    if (blocks == 0) blocks = 1;
+    if (vec)
+        dense_merge_score_kernel<true><<<(unsigned)blocks, 256, 0, st>>>(w, g, (int)K, -eta, c, n, S);
+    else
+        dense_merge_score_kernel<false><<<(unsigned)blocks, 256, 0, st>>>(w, g, (int)K, -eta, c, n, S);
+    SLIMDP_LAUNCHED(1);
+    return SLIMDP_OK;
+}
 
 slimdp_status launch_score(const float* w, const PtrArray<const float>& g, uint32_t K, float c, uint64_t n,
                            float* S, bool vec, cudaStream_t st) {

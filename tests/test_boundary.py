@@ -101,6 +101,11 @@ def test_invalid_arguments_are_rejected_on_the_host(P):
     assert lib.slimdp_exchange(fake, 10, 2, arr, fake, 5, arr, 5, 0.5, arr, null_in, None) == INVALID
     assert lib.slimdp_exchange(fake, 10, 2, null_in, fake, 5, arr, 5, 0.5, arr, arr, None) == INVALID
     assert lib.slimdp_exchange(fake, 10, 2, arr, fake, 5, arr, 6, 0.5, arr, arr, None) == INVALID
+    assert lib.slimdp_dense_merge_score(fake, arr, 2, float("nan"), 1.0, 10, fake, None) == INVALID
+    assert lib.slimdp_dense_merge_score(fake, null_in, 2, 0.5, 1.0, 10, None, None) == INVALID
+    assert lib.slimdp_dense_merge_score(None, arr, 2, 0.5, 1.0, 10, None, None) == INVALID
+    assert lib.slimdp_worker_merge_batched(arr, 2, 10, fake, 5, arr, 6, arr, None) == INVALID
+    assert lib.slimdp_worker_merge_batched(null_in, 2, 10, fake, 5, arr, 5, arr, None) == INVALID
     # whole round on host buffers
     assert lib.slimdp_round_host(fake, arr, 2, 10, 1.0, 5, 5, 0, 0, 0.5, fake, arr, arr, None, 0, None) == INVALID
     assert lib.slimdp_round_host(fake, arr, 2, 10, 1.0, 5, 5, 0, 0, 0.5, fake, arr, arr, fake, 16, None) == WORKSPACE
