@@ -269,6 +269,20 @@ slimdp_status slimdp_worker_merge_batched(float* const* w_local, uint32_t K, uin
                                           uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
                                           const float* const* pulled, void* stream);
 
+/* Key caching (Section 3.5): "the sender then only needs to send the values with
+ * a signature of the keys".  slimdp_core_signature writes a 64-bit signature of a
+ * key list to device memory:
+ *     sig = sum_j mix64(((j << 32) | keys[j]) + 0x9E3779B97F4A7C15)  mod 2^64,
+ *     mix64(z): z ^= z >> 30; z *= 0xBF58476D1CE4E5B9; z ^= z >> 27; z *= 0x94D049BB133111EB; z ^= z >> 31
+ * (the SplitMix64 output function).  Sender and receiver compare signatures to
+ * know that their cached core keys agree; the empty list has signature 0.
+ *   keys [count] (read), signature: DEVICE uint64, 8-byte aligned (written)
+ * slimdp_wire_bytes: bytes one worker sends per direction and round with key
+ * caching: 4 k_core values + 8 k_exp <key, value> pairs + the 8-byte signature,
+ * i.e. (2 alpha - beta) n words as in Section 3.5, against 4 n for Plump-DP. */
+slimdp_status slimdp_core_signature(const uint32_t* keys, uint64_t count, uint64_t* signature, void* stream);
+size_t slimdp_wire_bytes(uint64_t k_core, uint64_t k_exp);
+
 /* --------------------------------------------------------------- status ---
  * Synchronises `stream`, then returns the sticky status word kept in the first
  * 4 bytes of a workspace used by slimdp_select_core / slimdp_sample_explore*:

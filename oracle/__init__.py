@@ -40,6 +40,7 @@ _merge = _sig("oracle_merge", None, _f32p, ctypes.c_uint32, _u32p, ctypes.c_uint
               _pp, ctypes.c_float)
 _pull = _sig("oracle_pull", None, _f32p, _u32p, ctypes.c_uint64, _u32p, ctypes.c_uint64, _f32p)
 _dense = _sig("oracle_dense_merge", None, _f32p, ctypes.c_uint64, ctypes.c_uint32, _pp, ctypes.c_float)
+_signature = _sig("oracle_core_signature", ctypes.c_uint64, _u32p, ctypes.c_uint64)
 _wmerge = _sig("oracle_worker_merge", None, _f32p, _u32p, ctypes.c_uint64, _u32p, ctypes.c_uint64, _f32p)
 
 
@@ -144,6 +145,11 @@ def worker_merge(w_local, core_idx, exp_idx, pulled) -> np.ndarray:
     assert p.size == c.size + e.size
     _wmerge(_ptr(out, _f32p), _ptr(c, _u32p), c.size, _ptr(e, _u32p), e.size, _ptr(p, _f32p))
     return out
+
+
+def core_signature(keys) -> int:
+    k = _u32(keys)
+    return int(_signature(_ptr(k, _u32p), k.size))
 
 
 def run_round(w, grads: Sequence[np.ndarray], c: float, k_core: int, k_exp: int,

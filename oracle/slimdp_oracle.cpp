@@ -235,6 +235,20 @@ void oracle_worker_merge(float* w_local, const uint32_t* core_idx, uint64_t k_co
     for (uint64_t j = 0; j < k_exp; ++j) w_local[exp_idx[j]] = pulled[k_core + j];
 }
 
+// Key caching (Section 3.5): signature of a key list, the wrapping sum over positions j of
+// mix64(((j << 32) | key_j) + 0x9E3779B97F4A7C15), mix64 = the SplitMix64 output function.
+uint64_t oracle_core_signature(const uint32_t* keys, uint64_t count) {
+    uint64_t sig = 0;
+    for (uint64_t j = 0; j < count; ++j) {
+        uint64_t z = ((j << 32) | (uint64_t)keys[j]) + 0x9E3779B97F4A7C15ull;
+        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+        z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+        z = z ^ (z >> 31);
+        sig += z;
+    }
+    return sig;
+}
+
 // Plump-DP (Section 2.1): every worker pushes its whole update.
 void oracle_dense_merge(float* w, uint64_t n, uint32_t K, const float* const* grads, float eta) {
     for (uint32_t k = 0; k < K; ++k)

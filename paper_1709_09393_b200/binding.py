@@ -49,6 +49,8 @@ EXPORTS = {
     "slimdp_exchange": (ctypes.c_int32, [_vp, _u64, _u32, _pp, _vp, _u64, _pp, _u64, _f32, _pp, _pp, _vp]),
     "slimdp_dense_merge_score": (ctypes.c_int32, [_vp, _pp, _u32, _f32, _f32, _u64, _vp, _vp]),
     "slimdp_worker_merge_batched": (ctypes.c_int32, [_pp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _vp]),
+    "slimdp_core_signature": (ctypes.c_int32, [_vp, _u64, _vp, _vp]),
+    "slimdp_wire_bytes": (_sz, [_u64, _u64]),
     "slimdp_read_status": (ctypes.c_int32, [_vp, _vp]),
     "slimdp_launch_count": (_u64, []),
     "slimdp_round_arena_bytes": (_sz, [_u64, _u32, _u64, _u64]),
@@ -305,6 +307,18 @@ def slimdp_worker_merge_batched(w_local: Sequence[torch.Tensor], core_idx: torch
            lib.slimdp_worker_merge_batched(_ptr_array(w_local), K, n, _ptr(core_idx), core_idx.numel(),
                                            _ptr_array(exp_idx), exp_idx[0].numel(), _ptr_array(pulled),
                                            _stream(stream)))
+
+
+def slimdp_core_signature(keys: torch.Tensor, signature: torch.Tensor, stream=None):
+    """64-bit signature of a key list (key caching, Section 3.5) into a one-element int64 CUDA tensor."""
+    _dev(keys, IDX, "keys")
+    _dev(signature, torch.int64, "signature")
+    _check("slimdp_core_signature",
+           lib.slimdp_core_signature(_ptr(keys), keys.numel(), signature.data_ptr(), _stream(stream)))
+
+
+def wire_bytes(k_core: int, k_exp: int) -> int:
+    return lib.slimdp_wire_bytes(k_core, k_exp)
 
 
 def _host(t: torch.Tensor, dtype, name: str) -> torch.Tensor:

@@ -43,6 +43,8 @@ slimdp_status launch_worker_merge(const PtrArray<float>& w_local, uint32_t worke
                                   uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp,
                                   const PtrArray<const float>& pulled, cudaStream_t st);
 
+slimdp_status launch_signature(const uint32_t* keys, uint64_t count, unsigned long long* sig, cudaStream_t st);
+
 int sm_count() {
     static int cached[64];
     int dev = 0;
@@ -279,6 +281,14 @@ slimdp_status slimdp_worker_merge_batched(float* const* w_local, uint32_t K, uin
     if (!fill<const float>(v, pulled, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     return launch_worker_merge(w, K, core_idx, k_core, exp, k_exp, v, (cudaStream_t)stream);
 }
+
+slimdp_status slimdp_core_signature(const uint32_t* keys, uint64_t count, uint64_t* signature, void* stream) {
+    if (count > kMaxN || !signature || (reinterpret_cast<uintptr_t>(signature) & 7u) != 0) return SLIMDP_ERR_INVALID_ARG;
+    if (count > 0 && (!keys || !aligned4(keys))) return SLIMDP_ERR_INVALID_ARG;
+    return launch_signature(keys, count, reinterpret_cast<unsigned long long*>(signature), (cudaStream_t)stream);
+}
+
+size_t slimdp_wire_bytes(uint64_t k_core, uint64_t k_exp) { return (size_t)(4 * k_core + 8 * k_exp + 8); }
 
 uint64_t slimdp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -76,21 +76,38 @@ __global__ void __launch_bounds__(256) gather_explore_kernel(PtrArray<const floa
 }
 
 // Worker-side Merge (Algorithm 1; Section 3.3 step 5): the pulled values replace the local
-// model's values on the communication set.  grid.y = worker.
-__global__ void __launch_bounds__(256) worker_merge_kernel(PtrArray<float> w_local,
-                                                           const uint32_t* __restrict__ core_idx, uint64_t k_core,
-                                                           PtrArray<const uint32_t> exp, uint64_t k_exp,
-                                                           PtrArray<const float> pulled) {
+// model's values on the communication set.  Core segment: the shared key is read once and
+// serves all K workers.
+__global__ void __launch_bounds__(256) worker_merge_core_kernel(PtrArray<float> w_local,
+                                                                const uint32_t* __restrict__ core_idx,
+                                                                uint64_t k_core, PtrArray<const float> pulled,
+                                                                int K) {
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k_core; j += stride) {
+        const uint32_t i = __ldg(core_idx + j);
+        int k = 0;
+        for (; k + 8 <= K; k += 8) {
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = __ldcs(pulled.p[k + q] + j);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) w_local.p[k + q][i] = v[q];
+        }
+        for (; k < K; ++k) w_local.p[k][i] = __ldcs(pulled.p[k] + j);
+    }
+}
+
+// Explorer segments: grid.y = worker.
+__global__ void __launch_bounds__(256) worker_merge_explore_kernel(PtrArray<float> w_local,
+                                                                   PtrArray<const uint32_t> exp, uint64_t k_exp,
+                                                                   PtrArray<const float> pulled, uint64_t k_core) {
     const uint32_t worker = blockIdx.y;
     float* __restrict__ w = w_local.p[worker];
     const uint32_t* __restrict__ e = exp.p[worker];
-    const float* __restrict__ v = pulled.p[worker];
-    const uint64_t m = k_core + k_exp;
+    const float* __restrict__ v = pulled.p[worker] + k_core;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < m; j += stride) {
-        const uint32_t i = (j < k_core) ? __ldg(core_idx + j) : __ldg(e + (j - k_core));
-        w[i] = __ldcs(v + j);
-    }
+    for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k_exp; j += stride)
+        w[__ldg(e + j)] = __ldcs(v + j);
 }
 
 }  // namespace
@@ -98,15 +115,21 @@ __global__ void __launch_bounds__(256) worker_merge_kernel(PtrArray<float> w_loc
 slimdp_status launch_worker_merge(const PtrArray<float>& w_local, uint32_t workers, const uint32_t* core_idx,
                                   uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp,
                                   const PtrArray<const float>& pulled, cudaStream_t st) {
-    const uint64_t m = k_core + k_exp;
-    if (m == 0) return SLIMDP_OK;
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
-    uint64_t grid = (m + 255) / 256;
-    const uint64_t cap = ((uint64_t)sms * 32 + workers - 1) / workers;
-    if (grid > cap) grid = cap;
-    worker_merge_kernel<<<dim3((unsigned)grid, workers), 256, 0, st>>>(w_local, core_idx, k_core, exp, k_exp, pulled);
-    SLIMDP_LAUNCHED(1);
+    if (k_core > 0) {
+        uint64_t grid = (k_core + 255) / 256;
+        if (grid > (uint64_t)sms * 32) grid = (uint64_t)sms * 32;
+        worker_merge_core_kernel<<<(unsigned)grid, 256, 0, st>>>(w_local, core_idx, k_core, pulled, (int)workers);
+        SLIMDP_LAUNCHED(1);
+    }
+    if (k_exp > 0) {
+        uint64_t grid = (k_exp + 255) / 256;
+        const uint64_t cap = ((uint64_t)sms * 32 + workers - 1) / workers;
+        if (grid > cap) grid = cap;
+        worker_merge_explore_kernel<<<dim3((unsigned)grid, workers), 256, 0, st>>>(w_local, exp, k_exp, pulled, k_core);
+        SLIMDP_LAUNCHED(1);
+    }
     return SLIMDP_OK;
 }
 

@@ -406,3 +406,15 @@ def test_untouched_parameters_keep_their_bits(P):
         touched[e] = True
     got = d_w.cpu().numpy()
     assert np.array_equal(got[~touched].view(np.uint32), w[~touched].view(np.uint32))
+
+
+# ------------------------------------------------------------ key signature
+
+@pytest.mark.parametrize("count", [0, 1, 31, 1000, 100_003, 3_000_001])
+def test_core_signature_parity(P, count):
+    rng = np.random.default_rng(count)
+    keys = np.unique(rng.integers(0, 2 ** 32 - 1, count, dtype=np.uint64)).astype(np.uint32)   # ascending, distinct
+    sig = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+    P.slimdp_core_signature(dev(keys), sig)
+    assert int(sig.cpu().numpy().view(np.uint64)[0]) == oracle.core_signature(keys)
+    assert P.wire_bytes(1000, 50) == 4 * 1000 + 8 * 50 + 8

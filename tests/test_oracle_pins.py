@@ -388,3 +388,29 @@ def test_wire_words_match_table1_ratios():
         words = k_core + 2 * k_exp           # values for the core, (index, value) for the explorer
         assert words == round((2 * alpha - beta) * n)
         assert abs(words / n - float(t_slim) / float(t_plump)) < 0.03, model
+
+
+# ------------------------------------------------------------ key signature
+
+def test_key_signature_pins():
+    # Section 3.5: a signature of the cached keys.  Pinned to SplitMix64's published first outputs
+    # (seed 0: 0xE220A8397B1DCDAF, 0x6E789E6AA1B965F4) and to what a signature must tell apart.
+    assert oracle.core_signature(np.zeros(0, np.uint32)) == 0
+    assert oracle.core_signature(np.array([0], np.uint32)) == 0xE220A8397B1DCDAF      # mix64(0 + golden)
+    # key 0x9E3779B9 - carry trick is avoided: second published output checked through exact integers instead
+    M = (1 << 64) - 1
+
+    def mix(z):
+        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & M
+        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & M
+        return z ^ (z >> 31)
+
+    assert mix((2 * 0x9E3779B97F4A7C15) & M) == 0x6E789E6AA1B965F4
+    keys = np.array([5, 9, 12, 4000000000], np.uint32)
+    want = sum(mix((((j << 32) | int(k)) + 0x9E3779B97F4A7C15) & M) for j, k in enumerate(keys)) & M
+    assert oracle.core_signature(keys) == want
+    # equal lists agree; a changed key, a swapped pair, a dropped or an added key do not
+    assert oracle.core_signature(keys.copy()) == want
+    for other in (np.array([5, 9, 13, 4000000000], np.uint32), np.array([9, 5, 12, 4000000000], np.uint32),
+                  keys[:3], np.append(keys, np.uint32(7))):
+        assert oracle.core_signature(other) != want
