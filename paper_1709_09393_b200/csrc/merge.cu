@@ -56,8 +56,8 @@ __device__ __forceinline__ uint32_t lower_bound(const uint32_t* __restrict__ a, 
 
 // bound[k][r]: where the r-th of the CTA's 9 range boundaries falls in worker k's index list.
 __device__ __forceinline__ void find_bounds(uint32_t (*bound)[kMergeWarps + 1], const PtrArray<const uint32_t>& exp,
-                                            uint32_t k_exp, int K, uint32_t range_shift) {
-    const uint64_t first = ((uint64_t)blockIdx.x * kMergeWarps) << range_shift;
+                                            uint32_t k_exp, int K, uint32_t range_shift, uint64_t vblock) {
+    const uint64_t first = (vblock * kMergeWarps) << range_shift;
     for (int t = threadIdx.x; t < K * (kMergeWarps + 1); t += blockDim.x) {
         const int k = t / (kMergeWarps + 1), r = t % (kMergeWarps + 1);
         bound[k][r] = lower_bound(exp.p[k], k_exp, first + ((uint64_t)r << range_shift));
@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* 
                                                                          uint64_t k_core, int K, float neg_eta,
                                                                          uint32_t range_shift) {
     __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
-    find_bounds(bound, exp, k_exp, K, range_shift);
+    find_bounds(bound, exp, k_exp, K, range_shift, blockIdx.x);
     const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
     PtrArray<const float> none;
     const uint32_t sink = touch_range<false>(w, exp, none, bound, K, wid, lane);
@@ -149,12 +149,12 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* 
 // Core segment: thread j gathers the K workers' updates of core parameter core_idx[j] (the
 // push), folds them into the parameter in worker order (the update) and hands the merged value
 // back to all K workers (the pull).  One read of the key, K gathers, one read-modify-write.
-__global__ void __launch_bounds__(256) exchange_core_kernel(float* __restrict__ w,
-                                                            const uint32_t* __restrict__ core_idx, uint64_t k_core,
-                                                            PtrArray<const float> delta, PtrArray<float> val,
-                                                            PtrArray<float> pulled, int K, float neg_eta) {
-    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k_core; j += stride) {
+__device__ __forceinline__ void exchange_core_body(float* __restrict__ w, const uint32_t* __restrict__ core_idx,
+                                                   uint64_t k_core, const PtrArray<const float>& delta,
+                                                   const PtrArray<float>& val, const PtrArray<float>& pulled, int K,
+                                                   float neg_eta, uint64_t vblock, uint64_t vgrid) {
+    const uint64_t stride = vgrid * blockDim.x;
+    for (uint64_t j = vblock * blockDim.x + threadIdx.x; j < k_core; j += stride) {
         const uint32_t i = __ldg(core_idx + j);
         float x = w[i];
         int k = 0;
@@ -183,11 +183,12 @@ __global__ void __launch_bounds__(256) exchange_core_kernel(float* __restrict__ 
 // order, the warp gathers the worker's updates inside its range, stores them as the pushed
 // values and applies them; after the last worker it reads the merged values back for every
 // worker's pull (they are still in cache).
-__global__ void __launch_bounds__(kMergeWarps * 32) exchange_explore_kernel(
-    float* w, PtrArray<const uint32_t> exp, uint32_t k_exp, PtrArray<const float> delta, PtrArray<float> val,
-    PtrArray<float> pulled, uint64_t k_core, int K, float neg_eta, uint32_t range_shift) {
-    __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
-    find_bounds(bound, exp, k_exp, K, range_shift);
+__device__ __forceinline__ void exchange_explore_body(float* w, const PtrArray<const uint32_t>& exp, uint32_t k_exp,
+                                                      const PtrArray<const float>& delta, const PtrArray<float>& val,
+                                                      const PtrArray<float>& pulled, uint64_t k_core, int K,
+                                                      float neg_eta, uint32_t range_shift, uint64_t vblock,
+                                                      uint32_t (*bound)[kMergeWarps + 1]) {
+    find_bounds(bound, exp, k_exp, K, range_shift, vblock);
     const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
     const uint32_t sink = touch_range<true>(w, exp, delta, bound, K, wid, lane);
     for (int k = 0; k < K; ++k) {
@@ -210,6 +211,27 @@ __global__ void __launch_bounds__(kMergeWarps * 32) exchange_explore_kernel(
         for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) __stcs(o + e, ld_sparse(w + __ldg(idx + e)));
     }
     if (sink == 0x9E3779B9u && lane >= 32) w[0] = 0.0f;   // never true: keeps the early requests alive
+}
+
+// One launch for both segments.  The core segment streams whole lines of the dense layers and is
+// bound by DRAM bandwidth; the explorer segments issue sparse accesses and are bound by their
+// latency and rate.  CTAs of both kinds are interleaved in the grid (core_ctas of every
+// total_ctas, evenly spread), so both kinds are resident together and fill each other's gaps.
+// The two segments touch disjoint parameters and disjoint parts of val / pulled.
+__global__ void __launch_bounds__(256) exchange_kernel(float* w, const uint32_t* __restrict__ core_idx,
+                                                       uint64_t k_core, PtrArray<const uint32_t> exp, uint32_t k_exp,
+                                                       PtrArray<const float> delta, PtrArray<float> val,
+                                                       PtrArray<float> pulled, int K, float neg_eta,
+                                                       uint32_t range_shift, uint64_t core_ctas, uint64_t total_ctas) {
+    __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
+    const uint64_t b = blockIdx.x;
+    const uint64_t core_before = b * core_ctas / total_ctas;            // core CTAs among blocks [0, b)
+    const bool is_core = (b + 1) * core_ctas / total_ctas > core_before;
+    if (is_core)
+        exchange_core_body(w, core_idx, k_core, delta, val, pulled, K, neg_eta, core_before, core_ctas);
+    else
+        exchange_explore_body(w, exp, k_exp, delta, val, pulled, k_core, K, neg_eta, range_shift, b - core_before,
+                              bound);
 }
 
 // Range per warp: a power of two with 16 to 32 entries per worker on average, at least 32 parameters.
@@ -248,23 +270,25 @@ slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<c
                               const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,
                               uint64_t k_exp, float eta, const PtrArray<float>& val, const PtrArray<float>& pulled,
                               cudaStream_t st) {
+    static_assert(kMergeWarps * 32 == 256, "both kinds of CTA have 256 threads");
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
-    const float neg_eta = -eta;
+    uint64_t core_ctas = 0, explore_ctas = 0;
+    uint32_t shift = 0;
     if (k_core > 0) {
-        uint64_t grid = (k_core + 255) / 256;
-        if (grid > (uint64_t)sms * 32) grid = (uint64_t)sms * 32;
-        exchange_core_kernel<<<(unsigned)grid, 256, 0, st>>>(w, core_idx, k_core, delta, val, pulled, (int)K, neg_eta);
-        SLIMDP_LAUNCHED(1);
+        core_ctas = (k_core + 255) / 256;
+        if (core_ctas > (uint64_t)sms * 32) core_ctas = (uint64_t)sms * 32;
     }
     if (k_exp > 0) {
-        const uint32_t shift = explore_range_shift(n, k_exp);
+        shift = explore_range_shift(n, k_exp);
         const uint64_t per_cta = (uint64_t)kMergeWarps << shift;
-        const uint64_t ctas = (n + per_cta - 1) / per_cta;
-        exchange_explore_kernel<<<(unsigned)ctas, kMergeWarps * 32, 0, st>>>(w, exp, (uint32_t)k_exp, delta, val, pulled,
-                                                                             k_core, (int)K, neg_eta, shift);
-        SLIMDP_LAUNCHED(1);
+        explore_ctas = (n + per_cta - 1) / per_cta;
     }
+    const uint64_t total = core_ctas + explore_ctas;
+    if (total == 0) return SLIMDP_OK;
+    exchange_kernel<<<(unsigned)total, 256, 0, st>>>(w, core_idx, k_core, exp, (uint32_t)k_exp, delta, val, pulled,
+                                                     (int)K, -eta, shift, core_ctas, total);
+    SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }
 
