@@ -276,8 +276,7 @@ slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<c
     uint64_t core_ctas = 0, explore_ctas = 0;
     uint32_t shift = 0;
     if (k_core > 0) {
-        core_ctas = (k_core + 255) / 256;
-        if (core_ctas > (uint64_t)sms * 32) core_ctas = (uint64_t)sms * 32;
+        core_ctas = (k_core + 255) / 256;   // one core parameter per thread: short CTAs interleave best
     }
     if (k_exp > 0) {
         shift = explore_range_shift(n, k_exp);
