@@ -20,8 +20,9 @@
  *     host-side array whose K entries are device pointers; it is read during
  *     the call and may be freed as soon as the call returns.
  *   - The caller owns every buffer.  The library allocates no device memory,
- *     creates no stream, and never synchronises except in slimdp_read_status
- *     and slimdp_round_host.  All work is enqueued on `stream` (a cudaStream_t
+ *     creates no stream (slimdp_round and slimdp_round_host excepted, see
+ *     there), and never synchronises except in slimdp_read_status and
+ *     slimdp_round_host.  All work is enqueued on `stream` (a cudaStream_t
  *     passed as void*; NULL is the legacy default stream) and is ordered with
  *     other work on that stream.
  *   - Arguments are validated on the host before anything is enqueued.  A
@@ -295,10 +296,58 @@ slimdp_status slimdp_read_status(const void* ws, void* stream);
  * after a timed region.  The paper has no counterpart. */
 uint64_t slimdp_launch_count(void);
 
+/* --------------------------------------------------- whole round, device ---
+ * One whole round on device buffers (Algorithm 1's communication step; Section
+ * 3.3 steps 1 to 4, with the server's Core-Selection(w-bar, delta, beta) taking
+ * the model and the updates directly, as Algorithm 1 writes it): the results
+ * core_idx, core_aux, exp_idx, val, pulled and the updated w_global are
+ * bit-identical to slimdp_score with grads, slimdp_select_core,
+ * slimdp_sample_explore_batched for workers 0..K-1 and slimdp_exchange with
+ * deltas = grads, called in that order.  What differs is how the device gets
+ * there:
+ *   - Scoring is folded into the selection's single pass over all parameters
+ *     (n >= 2^21, k_core > 0 and 16-byte aligned w_global / grads / scores;
+ *     otherwise the two calls above run): each score is computed in registers
+ *     and classified on the spot, so the n scores are neither written nor read
+ *     back.  `scores` is then only scratch: it holds the scores if the
+ *     selection had to fall back to its full path (e.g. millions of equal
+ *     scores around the threshold) and is left untouched otherwise.  Callers
+ *     that want the scores call slimdp_score.
+ *   - The steps of a round depend on one another as a graph, not a chain: the
+ *     explorer's ranks need the sizes only, so they run beside scoring and
+ *     selection.  For that this call keeps, per device, ONE non-blocking stream
+ *     and two events of its own, created on the first call on that device and
+ *     kept for the life of the process (the one exception to "creates no
+ *     stream").  The side branch forks from `stream` at the start of the call
+ *     and is joined back into it inside the call, so for the caller the whole
+ *     round is ordered on `stream` as usual.  Calls on one device are
+ *     serialised on the host by a lock while they enqueue.
+ *   w_global [n] (updated in place); grads HOST array of K device pointers [n] (read)
+ *   scores [n] scratch (see above); core_idx [k_core], core_aux (written; as slimdp_select_core)
+ *   exp_idx HOST array of K device pointers [k_exp] (written)
+ *   val, pulled HOST arrays of K device pointers [k_core + k_exp] (written)
+ *   select_ws, explore_ws: two workspaces that do NOT overlap (both are in use
+ *   at once), of at least slimdp_select_workspace_bytes(n) and
+ *   slimdp_explore_workspace_bytes(n, k_exp, K) bytes; each keeps the status
+ *   word of its step (slimdp_read_status). */
+slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t K, uint64_t n, float c,
+                           uint64_t k_core, uint64_t k_exp, uint64_t seed, uint32_t round, float eta, float* scores,
+                           uint32_t* core_idx, void* core_aux, uint32_t* const* exp_idx, float* const* val,
+                           float* const* pulled, void* select_ws, size_t select_ws_bytes, void* explore_ws,
+                           size_t explore_ws_bytes, void* stream);
+
+/* Measurement aid (the paper has no counterpart).  The next slimdp_round called
+ * from this host thread records `begin_event` just before and `end_event` just
+ * after its pass over all parameters (the fused scoring + classification
+ * kernel, or slimdp_score's kernel on the unfused path) on the round's stream;
+ * the request is used up by that call.  Both are cudaEvent_t handles, passed
+ * as void*, created by the caller with timing enabled; NULL cancels. */
+void slimdp_mark_dominant_kernel(void* begin_event, void* end_event);
+
 /* ----------------------------------------------------- whole round, host ---
  * One whole round (score, select, K x explore, then the exchange: K x pack,
- * merge, K x pull) on HOST buffers: copies w and the K updates to the device, runs the round
- * above, copies the results back, and synchronises before returning.
+ * merge, K x pull) on HOST buffers: copies w and the K updates to the device, runs
+ * slimdp_round, copies the results back, and synchronises before returning.
  *   w_host       HOST [n]: global model, replaced by the merged model
  *   grads_host   HOST array of K HOST pointers, each [n]
  *   core_idx_host HOST [k_core] (written)

@@ -1,9 +1,9 @@
 """Slim-DP communication round on B200: thin Python binding of the C ABI in
 include/slimdp.h.  Every step runs in the CUDA library; this package only
 marshals torch tensors (device pointers, sizes, the current stream)."""
-from .binding import (SlimDPError, core_aux_bytes, core_aux_dir_offset, explore_workspace_bytes, launch_count, lib,
+from .binding import (SlimDPError, core_aux_bytes, core_aux_dir_offset, explore_workspace_bytes, launch_count, lib, mark_dominant_kernel,
                       read_status, round_arena_bytes, select_workspace_bytes, slimdp_core_signature, wire_bytes, slimdp_dense_merge_score, slimdp_exchange, slimdp_merge, slimdp_pack,
-                      slimdp_pack_batched, slimdp_pull, slimdp_pull_batched, slimdp_round_host,
+                      slimdp_pack_batched, slimdp_pull, slimdp_pull_batched, slimdp_round, slimdp_round_host,
                       slimdp_sample_explore, slimdp_sample_explore_batched, slimdp_sample_explore_static,
                       slimdp_worker_merge_batched, slimdp_score, slimdp_select_core,
                       workspace_bytes)
@@ -11,9 +11,9 @@ from .driver import SlimDPDriver
 from .round import RoundBuffers, run_round
 
 __all__ = [
-    "SlimDPError", "lib", "launch_count", "core_aux_bytes", "core_aux_dir_offset", "select_workspace_bytes",
+    "SlimDPError", "lib", "launch_count", "mark_dominant_kernel", "core_aux_bytes", "core_aux_dir_offset", "select_workspace_bytes",
     "explore_workspace_bytes", "workspace_bytes", "round_arena_bytes", "read_status", "slimdp_score",
     "slimdp_select_core", "slimdp_sample_explore", "slimdp_sample_explore_batched", "slimdp_sample_explore_static", "slimdp_pack",
-    "slimdp_core_signature", "wire_bytes", "slimdp_pack_batched", "slimdp_exchange", "slimdp_dense_merge_score", "slimdp_worker_merge_batched", "slimdp_merge", "slimdp_pull", "slimdp_pull_batched", "slimdp_round_host",
+    "slimdp_core_signature", "wire_bytes", "slimdp_pack_batched", "slimdp_exchange", "slimdp_dense_merge_score", "slimdp_worker_merge_batched", "slimdp_merge", "slimdp_pull", "slimdp_pull_batched", "slimdp_round", "slimdp_round_host",
     "RoundBuffers", "run_round", "SlimDPDriver",
 ]

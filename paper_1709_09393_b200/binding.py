@@ -54,6 +54,9 @@ EXPORTS = {
     "slimdp_read_status": (ctypes.c_int32, [_vp, _vp]),
     "slimdp_launch_count": (_u64, []),
     "slimdp_round_arena_bytes": (_sz, [_u64, _u32, _u64, _u64]),
+    "slimdp_round": (ctypes.c_int32, [_vp, _pp, _u32, _u64, _f32, _u64, _u64, _u64, _u32, _f32, _vp, _vp, _vp, _pp, _pp,
+                                      _pp, _vp, ctypes.c_size_t, _vp, ctypes.c_size_t, _vp]),
+    "slimdp_mark_dominant_kernel": (None, [_vp, _vp]),
     "slimdp_round_host": (ctypes.c_int32, [_vp, _pp, _u32, _u64, _f32, _u64, _u64, _u64, _u32, _f32, _vp, _pp, _pp,
                                            _vp, _sz, _vp]),
 }
@@ -275,6 +278,40 @@ def slimdp_exchange(w_global: torch.Tensor, deltas: Sequence[torch.Tensor], core
            lib.slimdp_exchange(w_global.data_ptr(), w_global.numel(), K, _ptr_array(deltas), _ptr(core_idx),
                                core_idx.numel(), _ptr_array(exp_idx), exp_idx[0].numel(), eta, _ptr_array(val),
                                _ptr_array(pulled), _stream(stream)))
+
+
+def slimdp_round(w_global: torch.Tensor, grads: Sequence[torch.Tensor], c: float, seed: int, rnd: int, eta: float,
+                 scores: torch.Tensor, core_idx: torch.Tensor, core_aux: torch.Tensor,
+                 exp_idx: Sequence[torch.Tensor], val: Sequence[torch.Tensor], pulled: Sequence[torch.Tensor],
+                 select_ws: torch.Tensor, explore_ws: torch.Tensor, stream=None):
+    """One whole round on device buffers; same results as score, select_core, sample_explore_batched,
+    exchange, except that `scores` is scratch (written only if the selection falls back to its full path)."""
+    n = w_global.numel()
+    _dev(w_global, torch.float32, "w_global")
+    K = len(grads)
+    if len(exp_idx) != K or len(val) != K or len(pulled) != K:
+        raise ValueError("grads, exp_idx, val and pulled must have K entries each")
+    if _dev(scores, torch.float32, "scores").numel() != n:
+        raise ValueError("scores: length differs from w_global")
+    for g, e, v, o in zip(grads, exp_idx, val, pulled):
+        if _dev(g, torch.float32, "grads").numel() != n:
+            raise ValueError("grads: length differs from w_global")
+        _check_sets(core_idx, e, v, "val")
+        _check_sets(core_idx, e, o, "pulled")
+    for t, name in ((core_aux, "core_aux"), (select_ws, "select_ws"), (explore_ws, "explore_ws")):
+        _dev(t, torch.uint8, name)
+    _check("slimdp_round",
+           lib.slimdp_round(w_global.data_ptr(), _ptr_array(grads), K, n, c, core_idx.numel(), exp_idx[0].numel(),
+                            seed, rnd, eta, _ptr(scores), _ptr(core_idx), _ptr(core_aux), _ptr_array(exp_idx),
+                            _ptr_array(val), _ptr_array(pulled), _ptr(select_ws), select_ws.numel(),
+                            _ptr(explore_ws), explore_ws.numel(), _stream(stream)))
+
+
+def mark_dominant_kernel(begin: Optional[torch.cuda.Event], end: Optional[torch.cuda.Event]) -> None:
+    """The next slimdp_round records the two events around its pass over all parameters.  Both
+    events must have been recorded once already (torch creates the CUDA event lazily)."""
+    lib.slimdp_mark_dominant_kernel(begin.cuda_event if begin is not None else None,
+                                    end.cuda_event if end is not None else None)
 
 
 def slimdp_dense_merge_score(w_global: torch.Tensor, grads: Sequence[torch.Tensor], eta: float, c: float,

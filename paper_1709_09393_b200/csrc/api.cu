@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <mutex>
 
 #include "common.cuh"
 #include "layout.cuh"
@@ -32,6 +33,14 @@ slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<c
                               const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,
                               uint64_t k_exp, float eta, const PtrArray<float>& val, const PtrArray<float>& pulled,
                               cudaStream_t st);
+
+slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
+                                   uint32_t first_worker, uint32_t workers, uint32_t round,
+                                   const PtrArray<uint32_t>& out, void* ws, int parts, cudaStream_t st);
+bool score_select_fusable(uint64_t n, uint64_t k_core, bool vec);
+slimdp_status launch_score_select(const float* w, const PtrArray<const float>& g, uint32_t K, float c, uint64_t n,
+                                  float* scores, uint64_t k_core, uint32_t* core_idx, void* core_aux, void* ws,
+                                  cudaEvent_t mark_begin, cudaEvent_t mark_end, cudaStream_t st);
 
 slimdp_status launch_explore_static(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                     uint32_t worker, uint32_t round, uint32_t* exp_idx, int32_t* status_out,
@@ -301,6 +310,119 @@ slimdp_status slimdp_read_status(const void* ws, void* stream) {
     return (s == SLIMDP_OK) ? SLIMDP_OK : SLIMDP_ERR_INTERNAL;
 }
 
+// ---- whole round on device buffers ----------------------------------------
+//
+// The round's steps form a small graph rather than a chain: the explorer's
+// ranks depend on the sizes alone, so they run beside scoring and selection,
+// on a stream the library owns, one per device.  The join is the wait on
+// ranks_done, which every path through the call reaches.  Scoring is folded
+// into the selection's one pass over all parameters, so the scores are never
+// written unless the selection has to fall back to its full path.
+
+namespace {
+struct SideStream {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, ranks_done = nullptr;
+    bool ready = false;
+};
+std::mutex g_side_mutex;
+thread_local cudaEvent_t t_mark_begin = nullptr, t_mark_end = nullptr;
+SideStream g_side[64];
+
+SideStream* side_stream_locked() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    SideStream& s = g_side[dev];
+    if (!s.ready) {
+        int lo = 0, hi = 0;
+        if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) return nullptr;
+        if (cudaStreamCreateWithPriority(&s.stream, cudaStreamNonBlocking, hi) != cudaSuccess) return nullptr;
+        cudaEvent_t* ev[2] = {&s.fork, &s.ranks_done};
+        for (auto e : ev)
+            if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        s.ready = true;
+    }
+    return &s;
+}
+}  // namespace
+
+slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t K, uint64_t n, float c,
+                           uint64_t k_core, uint64_t k_exp, uint64_t seed, uint32_t round, float eta, float* scores,
+                           uint32_t* core_idx, void* core_aux, uint32_t* const* exp_idx, float* const* val,
+                           float* const* pulled, void* select_ws, size_t select_ws_bytes, void* explore_ws,
+                           size_t explore_ws_bytes, void* stream) {
+    if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !w_global || !grads || !scores || !core_aux || !select_ws ||
+        !explore_ws || !isfinite(c) || !isfinite(eta))
+        return SLIMDP_ERR_INVALID_ARG;
+    if (!aligned4(w_global) || !aligned4(scores) || !aligned16(core_aux) || !aligned16(select_ws) ||
+        !aligned16(explore_ws))
+        return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    PtrArray<const float> g;
+    PtrArray<uint32_t> exp_out;
+    PtrArray<const uint32_t> exp_in;
+    PtrArray<float> v, o;
+    if (!fill<const float>(g, grads, K, true, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<uint32_t>(exp_out, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<float>(v, val, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<float>(o, pulled, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
+    memset(&exp_in, 0, sizeof(exp_in));
+    for (uint32_t k = 0; k < K; ++k) exp_in.p[k] = exp_out.p[k];
+    if (select_ws_bytes < slimdp_select_workspace_bytes(n)) return SLIMDP_ERR_WORKSPACE;
+    if (explore_ws_bytes < slimdp_explore_workspace_bytes(n, k_exp, K)) return SLIMDP_ERR_WORKSPACE;
+    {
+        const char* a = static_cast<const char*>(select_ws);
+        const char* b = static_cast<const char*>(explore_ws);
+        if (a < b + explore_ws_bytes && b < a + select_ws_bytes) return SLIMDP_ERR_INVALID_ARG;
+    }
+    bool vec = aligned16(w_global) && aligned16(scores);
+    for (uint32_t k = 0; k < K; ++k) vec = vec && aligned16(g.p[k]);
+
+    cudaStream_t st = (cudaStream_t)stream;
+    std::lock_guard<std::mutex> lock(g_side_mutex);
+    SideStream* side = side_stream_locked();
+    if (!side) return SLIMDP_ERR_CUDA;
+    cudaStream_t sd = side->stream;
+
+    if (cudaEventRecord(side->fork, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
+    if (cudaStreamWaitEvent(sd, side->fork, 0) != cudaSuccess) return SLIMDP_ERR_CUDA;
+    // From here on the side stream is joined back into `st` whatever happens.
+    slimdp_status rc = SLIMDP_OK;
+    auto step = [&](slimdp_status s) {
+        if (rc == SLIMDP_OK) rc = s;
+    };
+    auto cuda = [&](cudaError_t e) { step(e == cudaSuccess ? SLIMDP_OK : SLIMDP_ERR_CUDA); };
+    cudaEvent_t mark0 = t_mark_begin, mark1 = t_mark_end;
+    t_mark_begin = t_mark_end = nullptr;
+
+    // side: ranks and bucket grouping of every worker's explorer (they need the sizes only)
+    step(launch_explore_parts(core_aux, n, k_core, k_exp, seed, 0, K, round, exp_out, explore_ws, 1, sd));
+    cuda(cudaEventRecord(side->ranks_done, sd));
+    // main: the core, scored and selected in one pass where sizes and alignment allow
+    if (score_select_fusable(n, k_core, vec)) {
+        if (rc == SLIMDP_OK)
+            step(launch_score_select(w_global, g, K, c, n, scores, k_core, core_idx, core_aux, select_ws, mark0,
+                                     mark1, st));
+    } else {
+        if (rc == SLIMDP_OK && mark0) cuda(cudaEventRecord(mark0, st));
+        if (rc == SLIMDP_OK) step(launch_score(w_global, g, K, c, n, scores, vec, st));
+        if (rc == SLIMDP_OK && mark1) cuda(cudaEventRecord(mark1, st));
+        if (rc == SLIMDP_OK) step(launch_select(scores, n, k_core, core_idx, core_aux, select_ws, st));
+    }
+    // main: explorer indices from the ranks and the core, then the exchange
+    cuda(cudaStreamWaitEvent(st, side->ranks_done, 0));
+    if (rc == SLIMDP_OK)
+        step(launch_explore_parts(core_aux, n, k_core, k_exp, seed, 0, K, round, exp_out, explore_ws, 2, st));
+    if (rc == SLIMDP_OK && k_core + k_exp > 0)
+        step(launch_exchange(w_global, n, K, g, core_idx, k_core, exp_in, k_exp, eta, v, o, st));
+    return rc;
+}
+
+void slimdp_mark_dominant_kernel(void* begin_event, void* end_event) {
+    t_mark_begin = (cudaEvent_t)begin_event;
+    t_mark_end = (cudaEvent_t)end_event;
+}
+
 // ---- whole round on host buffers ------------------------------------------
 
 namespace {
@@ -382,13 +504,9 @@ slimdp_status slimdp_round_host(float* w_host, const float* const* grads_host, u
     SLIMDP_CUDA(cudaMemcpyAsync(A.w, w_host, n * 4, cudaMemcpyHostToDevice, st));
     for (uint32_t k = 0; k < K; ++k)
         SLIMDP_CUDA(cudaMemcpyAsync(A.delta[k], grads_host[k], n * 4, cudaMemcpyHostToDevice, st));
-    SLIMDP_TRY(slimdp_score(A.w, A.delta, K, c, n, A.scores, stream));
-    SLIMDP_TRY(slimdp_select_core(A.scores, n, k_core, A.core_idx, A.core_aux, A.select_ws, A.select_ws_bytes,
-                                  stream));
-    SLIMDP_TRY(slimdp_sample_explore_batched(A.core_aux, n, k_core, k_exp, seed, 0, K, round, A.exp_idx,
-                                             A.explore_ws, A.explore_ws_bytes, stream));
-    SLIMDP_TRY(slimdp_exchange(A.w, n, K, A.delta, A.core_idx, k_core, A.exp_idx, k_exp, eta, A.val, A.pulled,
-                               stream));
+    SLIMDP_TRY(slimdp_round(A.w, A.delta, K, n, c, k_core, k_exp, seed, round, eta, A.scores, A.core_idx, A.core_aux,
+                            A.exp_idx, A.val, A.pulled, A.select_ws, A.select_ws_bytes, A.explore_ws,
+                            A.explore_ws_bytes, stream));
     SLIMDP_CUDA(cudaMemcpyAsync(w_host, A.w, n * 4, cudaMemcpyDeviceToHost, st));
     if (k_core) SLIMDP_CUDA(cudaMemcpyAsync(core_idx_host, A.core_idx, k_core * 4, cudaMemcpyDeviceToHost, st));
     for (uint32_t k = 0; k < K; ++k) {

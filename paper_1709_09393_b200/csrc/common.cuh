@@ -129,6 +129,12 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan64_1024(unsign
     return block_exclusive_scan64<32>(v, smem, total);
 }
 
+// Significance of one parameter (Eq. 1): |w| + c |g| with one rounding, every NaN as the canonical quiet NaN.
+__device__ __forceinline__ float score_one(float c, float g, float w) {
+    float s = __fmaf_rn(c, fabsf(g), fabsf(w));
+    return (s != s) ? __uint_as_float(0x7FC00000u) : s;
+}
+
 // ---- internal launchers (each enqueues on `st`, returns a slimdp_status) ---
 
 // Exclusive scan over bitmap blocks of 64-bit counters: cnt[y][nb] -> pref[y][nb],

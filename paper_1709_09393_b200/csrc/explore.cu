@@ -74,10 +74,10 @@ __device__ __forceinline__ uint32_t find_block(const uint32_t* __restrict__ dir,
 __global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, uint32_t seed_lo, uint32_t seed_hi,
                                      uint32_t first_worker, uint32_t workers, uint32_t round,
                                      const uint32_t* __restrict__ dir, uint32_t nd, uint32_t M, uint32_t s,
-                                     uint32_t buckets, uint32_t* __restrict__ bounds) {
+                                     uint32_t buckets, uint32_t* __restrict__ bounds, int parts) {
     const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
-    if (t == 0) hdr->status = SLIMDP_OK;
-    if (t < workers * 3) {
+    if ((parts & 1) && t == 0) hdr->status = SLIMDP_OK;
+    if ((parts & 1) && t < workers * 3) {
         const uint32_t w = t / 3, b = t % 3;
         uint32_t out[4];
         philox4x32_10(seed_lo, seed_hi, b, first_worker + w, round, 0x534C494Du, out);
@@ -86,7 +86,7 @@ __global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, u
     }
     // one warp per bucket boundary: a 32-way search (5 probes for 2^25 entries instead of 25)
     const uint32_t bnd = t >> 5, lane = t & 31u;
-    if (M > 0 && bnd <= buckets) {
+    if ((parts & 2) && M > 0 && bnd <= buckets) {
         const uint64_t first = (uint64_t)bnd << s;
         const uint32_t rank = (first < M) ? (uint32_t)first : M - 1;
         uint32_t lo = 0, hi = nd - 1;   // the answer is the largest d in [lo, hi] with dir[d] <= rank; dir[lo] <= rank
@@ -413,9 +413,11 @@ uint32_t explore_bucket_shift(uint64_t M) {
     return (uint32_t)(13 + extra);
 }
 
-slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
-                             uint32_t first_worker, uint32_t workers, uint32_t round,
-                             const PtrArray<uint32_t>& out, void* ws, cudaStream_t st) {
+// parts: 1 = the steps that need only the sizes (round keys, ranks, bucket grouping),
+//        2 = the steps that need the core (bucket bounds, parameter indices), 3 = everything.
+slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
+                                   uint32_t first_worker, uint32_t workers, uint32_t round,
+                                   const PtrArray<uint32_t>& out, void* ws, int parts, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
     const ExploreWs L = explore_ws_layout(ws, n, k_exp, workers);
@@ -432,9 +434,10 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
     explore_setup_kernel<<<(setup_threads + 255) / 256, 256, 0, st>>>(L.hdr, L.round_keys, (uint32_t)seed,
                                                                       (uint32_t)(seed >> 32), first_worker, workers,
                                                                       round, dir, (uint32_t)nd, (uint32_t)M, s,
-                                                                      (uint32_t)buckets, L.bounds);
+                                                                      (uint32_t)buckets, L.bounds, parts);
     SLIMDP_LAUNCHED(1);
     if (k_exp == 0) return SLIMDP_OK;
+    if (parts & 1) {
     if (cudaMemsetAsync(L.cnt, 0, L.zero_bytes, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
 
     uint32_t bits = 2;   // the permutation's domain is [0, 2^bits), the smallest that holds M (at least 4)
@@ -480,11 +483,19 @@ slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, 
                                                      L.sorted);
     }
     SLIMDP_LAUNCHED(1);
+    }   // parts & 1
+    if (!(parts & 2)) return SLIMDP_OK;
     bucket_kernel<<<dim3((unsigned)buckets, workers), kBucketThreads, 0, st>>>(
         bitmap, dir, L.bounds, (uint32_t)k_exp, s, L.sorted, L.rho_stride, L.cnt, L.pref, L.totals, L.cnt_stride,
         out, L.hdr);
     SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
+}
+
+slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
+                             uint32_t first_worker, uint32_t workers, uint32_t round,
+                             const PtrArray<uint32_t>& out, void* ws, cudaStream_t st) {
+    return launch_explore_parts(core_aux, n, k_core, k_exp, seed, first_worker, workers, round, out, ws, 3, st);
 }
 
 // ---- explorer sampling without a caller-supplied workspace ---------------------------------

@@ -9,11 +9,6 @@ namespace slimdp {
 
 namespace {
 
-__device__ __forceinline__ float score_one(float c, float g, float w) {
-    float s = __fmaf_rn(c, fabsf(g), fabsf(w));
-    return (s != s) ? __uint_as_float(0x7FC00000u) : s;
-}
-
 // KT > 0: K known at compile time (all loads of one element group are issued
 // before the first add).  KT == 0: K from the argument.
 template <int KT>

@@ -293,6 +293,226 @@ __global__ void __launch_bounds__(256, 8) bracket_pass_kernel(const uint32_t* __
     if (threadIdx.x == 0 && cta_def) atomicAdd(&hdr->n_def, cta_def);
 }
 
+// ---- scoring fused into the bracketed path -----------------------------------------------
+//
+// When a whole round is enqueued at once the scores need not exist in memory: the sample is
+// scored straight from the model and the updates, and the one pass over all parameters computes
+// each score in registers and sorts it into "certainly core" / candidate / neither on the spot.
+// The score array is written only if the bracket fails and the full path has to read it.
+
+// Left-to-right fp32 sum of the K updates of four consecutive parameters, then their scores.
+template <int KT>
+__device__ __forceinline__ void score4(const float* __restrict__ w, const PtrArray<const float>& g, int K, float c,
+                                       uint64_t i4, uint32_t key[4]) {
+    const int kk = (KT > 0) ? KT : K;
+    float4 a = __ldcs(reinterpret_cast<const float4*>(g.p[0]) + i4);
+    if (KT > 0) {
+        float4 b[KT > 1 ? KT - 1 : 1];
+#pragma unroll
+        for (int k = 1; k < KT; ++k) b[k - 1] = __ldcs(reinterpret_cast<const float4*>(g.p[k]) + i4);
+#pragma unroll
+        for (int k = 1; k < KT; ++k) {
+            a.x = __fadd_rn(a.x, b[k - 1].x);
+            a.y = __fadd_rn(a.y, b[k - 1].y);
+            a.z = __fadd_rn(a.z, b[k - 1].z);
+            a.w = __fadd_rn(a.w, b[k - 1].w);
+        }
+    } else {
+#pragma unroll 4
+        for (int k = 1; k < kk; ++k) {
+            const float4 b = __ldcs(reinterpret_cast<const float4*>(g.p[k]) + i4);
+            a.x = __fadd_rn(a.x, b.x);
+            a.y = __fadd_rn(a.y, b.y);
+            a.z = __fadd_rn(a.z, b.z);
+            a.w = __fadd_rn(a.w, b.w);
+        }
+    }
+    const float4 ww = __ldcs(reinterpret_cast<const float4*>(w) + i4);
+    key[0] = __float_as_uint(score_one(c, a.x, ww.x));
+    key[1] = __float_as_uint(score_one(c, a.y, ww.y));
+    key[2] = __float_as_uint(score_one(c, a.z, ww.z));
+    key[3] = __float_as_uint(score_one(c, a.w, ww.w));
+}
+
+__device__ __forceinline__ uint32_t score1(const float* __restrict__ w, const PtrArray<const float>& g, int K,
+                                           float c, uint64_t i) {
+    float a = g.p[0][i];
+    for (int k = 1; k < K; ++k) a = __fadd_rn(a, g.p[k][i]);
+    return __float_as_uint(score_one(c, a, w[i]));
+}
+
+// Sample kernel A of the fused path: 2^16 evenly spaced groups of four consecutive parameters
+// are scored (2^18 sampled keys, one 16-byte load per tensor and group); the rest is
+// sample_coarse_kernel's.  Needs n >= 4 and 16-byte aligned tensors.
+__global__ void __launch_bounds__(1024) sample_score_coarse_kernel(const float* __restrict__ w,
+                                                                   PtrArray<const float> g, int K, float c,
+                                                                   uint64_t n, uint32_t k, WsHeader* hdr,
+                                                                   uint32_t* __restrict__ sample,
+                                                                   uint32_t* __restrict__ coarse_hist,
+                                                                   uint32_t* __restrict__ coarse_incl) {
+    __shared__ unsigned long long smem[33];
+    __shared__ uint32_t sh_coarse[256];
+    __shared__ long long s_incl[257];
+    const uint32_t t = threadIdx.x;
+    if (t < 256) sh_coarse[t] = 0;
+    __syncthreads();
+    const uint32_t j = blockIdx.x * 1024 + t;   // group number, < 2^16
+    uint32_t key[4];
+    score4<0>(w, g, K, c, ((uint64_t)j * (n / 4)) >> (kSampleBits - 2), key);
+    reinterpret_cast<uint4*>(sample)[j] = make_uint4(key[0], key[1], key[2], key[3]);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) atomicAdd(&sh_coarse[key[q] >> 24], 1u);
+    __syncthreads();
+    if (t < 256 && sh_coarse[t]) atomicAdd(&coarse_hist[t], sh_coarse[t]);
+    if (!last_cta_done(&hdr->ticket[6])) return;
+    long long lo_target, hi_target;
+    bracket_targets(k, n, &lo_target, &hi_target);
+    unsigned long long total;
+    const unsigned long long cc = (t < 256) ? __ldcg(coarse_hist + 255 - t) : 0ull;
+    const long long c_above = (long long)block_exclusive_scan64<32>(cc, smem, &total);
+    if (t < 256) s_incl[255 - t] = c_above + (long long)cc;
+    if (t == 0) {
+        s_incl[256] = 0;
+        hdr->coarse_x[0] = 0xFFFFFFFFu;
+        hdr->coarse_x[1] = 0xFFFFFFFFu;
+    }
+    __syncthreads();
+    if (t < 256) {
+        const long long incl = s_incl[t], above = s_incl[t + 1];
+        coarse_incl[t] = (uint32_t)incl;
+        if (incl > lo_target && above <= lo_target) hdr->coarse_x[0] = t;
+        if (incl >= hi_target && above < hi_target) hdr->coarse_x[1] = t;
+    }
+}
+
+constexpr uint32_t kFusedStage = kFlushAt + 128;   // below kFlushAt before a row of 128 parameters, +128 in it
+
+// The bracket pass with the scores computed in place of being read.  Warp per 1024-parameter
+// block, a row of 128 parameters (one 16-byte load per lane and tensor) at a time; lane l holds
+// parameters 4l .. 4l+3 of the row, so eight neighbouring lanes make one bitmap word.
+template <int KT>
+__global__ void __launch_bounds__(256, 4) score_bracket_kernel(const float* __restrict__ w, PtrArray<const float> g,
+                                                               int K, float c, uint64_t n, uint64_t nb,
+                                                               WsHeader* hdr, uint32_t cap,
+                                                               uint32_t* __restrict__ G, uint32_t* __restrict__ E,
+                                                               unsigned long long* __restrict__ cnt,
+                                                               uint32_t* __restrict__ cand_key,
+                                                               uint32_t* __restrict__ cand_idx) {
+    __shared__ uint32_t st_key[8][kFusedStage], st_idx[8][kFusedStage];
+    __shared__ uint32_t cta_def;
+    const uint32_t b_top = hdr->b_top, b_bot = hdr->b_bot;
+    const uint32_t lane = lane_id(), wid = threadIdx.x >> 5;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    uint32_t* my_key = st_key[wid];
+    uint32_t* my_idx = st_idx[wid];
+    if (threadIdx.x == 0) cta_def = 0;
+    __syncthreads();
+    uint32_t staged = 0, def_acc = 0;
+    auto flush = [&](uint32_t m) {
+        uint32_t base = 0;
+        if (lane == 0) base = atomicAdd(&hdr->n_cand, m);
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        if ((uint64_t)base + m <= cap) {   // else: overflow, n_cand > cap sends the call down the full path
+            for (uint32_t e = lane; e < m; e += 32) {
+                cand_key[base + e] = my_key[e];
+                cand_idx[base + e] = my_idx[e];
+            }
+        }
+        __syncwarp();
+    };
+    const bool has_top = b_top < 65536u;
+    const uint32_t top_key = has_top ? (b_top << 16) : 0xFFFFFFFFu;
+    const uint32_t bot_key = b_bot << 16;
+    const uint64_t warps = (uint64_t)gridDim.x * (blockDim.x >> 5);
+    for (uint64_t blk = (uint64_t)blockIdx.x * (blockDim.x >> 5) + wid; blk < nb; blk += warps) {
+        const uint64_t base = blk * kBlock;
+        const bool full = base + kBlock <= n;
+        uint32_t myG = 0;
+#pragma unroll 1
+        for (uint32_t r = 0; r < 8; ++r) {
+            const uint64_t e0 = base + r * 128 + 4 * lane;   // this lane's first parameter of the row
+            uint32_t key[4];
+            uint32_t in = 0xFu;                               // which of the four exist
+            if (full || e0 + 4 <= n) {
+                score4<KT>(w, g, K, c, e0 / 4, key);
+            } else {
+                in = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    key[q] = 0;
+                    if (e0 + q < n) {
+                        key[q] = score1(w, g, K, c, e0 + q);
+                        in |= 1u << q;
+                    }
+                }
+            }
+            uint32_t nib = 0, cm = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const bool ex = (in >> q) & 1u;
+                const bool def = has_top && key[q] >= top_key && ex;
+                const bool cand = key[q] >= bot_key && !def && ex;
+                nib |= (uint32_t)def << q;
+                cm |= (uint32_t)cand << q;
+            }
+            // the row's four bitmap words: lanes 8j .. 8j+7 assemble word j, lane 4r + j keeps it
+            uint32_t word = nib << (4 * (lane & 7u));
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
+            const uint32_t got = __shfl_sync(0xFFFFFFFFu, word, (lane & 3u) * 8);
+            if ((lane >> 2) == r) myG = got;
+            if (__any_sync(0xFFFFFFFFu, cm != 0)) {   // warp-uniform: most rows hold no candidate
+                uint32_t place = staged;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const bool cand = (cm >> q) & 1u;
+                    const uint32_t bc = __ballot_sync(0xFFFFFFFFu, cand);
+                    if (cand) {
+                        const uint32_t slot = place + __popc(bc & lt_mask);
+                        my_key[slot] = key[q];
+                        my_idx[slot] = (uint32_t)e0 + q;
+                    }
+                    place += __popc(bc);
+                }
+                staged = place;
+                __syncwarp();
+                if (staged >= kFlushAt) {
+                    flush(staged);
+                    staged = 0;
+                }
+            }
+        }
+        G[blk * kWordsPerBlock + lane] = myG;
+        E[blk * kWordsPerBlock + lane] = 0u;
+        const uint32_t cg = __reduce_add_sync(0xFFFFFFFFu, __popc(myG));
+        if (lane == 0) cnt[blk] = cg;
+        def_acc += cg;
+    }
+    if (staged) flush(staged);
+    if (lane == 0 && def_acc) atomicAdd(&cta_def, def_acc);
+    __syncthreads();
+    if (threadIdx.x == 0 && cta_def) atomicAdd(&hdr->n_def, cta_def);
+}
+
+// The scores for the full path, written only when the bracket failed.
+__global__ void __launch_bounds__(256) score_if_bracket_failed_kernel(const float* __restrict__ w,
+                                                                      PtrArray<const float> g, int K, float c,
+                                                                      uint64_t n, const WsHeader* __restrict__ hdr,
+                                                                      uint32_t k, uint32_t cap,
+                                                                      uint32_t* __restrict__ S) {
+    if (bracket_ok(hdr, k, cap)) return;
+    const uint64_t n4 = n / 4;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    const uint64_t gid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (uint64_t i = gid; i < n4; i += stride) {
+        uint32_t key[4];
+        score4<0>(w, g, K, c, i, key);
+        reinterpret_cast<uint4*>(S)[i] = make_uint4(key[0], key[1], key[2], key[3]);
+    }
+    if (gid < n - 4 * n4) S[4 * n4 + gid] = score1(w, g, K, c, 4 * n4 + gid);
+}
+
 // ---- radix histogram passes (over all keys, or over the candidates) -----------------------
 
 template <int PASS>
@@ -537,8 +757,19 @@ __global__ void __launch_bounds__(256) emit_kernel(const uint32_t* __restrict__ 
 
 }  // namespace
 
-slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx, void* core_aux,
-                            void* ws, cudaStream_t st) {
+// One selection.  `fused` non-null: the scores are not in memory yet; they are computed from the
+// model and the updates inside the bracketed path (which the caller has checked applies), and
+// `scores` is written only if the full path has to run.
+struct FusedScore {
+    const float* w;
+    const PtrArray<const float>* g;
+    uint32_t K;
+    float c;
+    cudaEvent_t mark_begin, mark_end;   // recorded around the pass over all parameters when not null
+};
+
+static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx,
+                                        void* core_aux, void* ws, const FusedScore* fused, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
     const SelectWs L = select_ws_layout(ws, n);
@@ -558,12 +789,32 @@ slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, ui
     const unsigned hgrid = (unsigned)sms * 4;
     const bool bracketed = k_core > 0 && n >= kBracketMinN;
     if (bracketed) {
-        sample_coarse_kernel<<<(1u << kSampleBits) / 1024, 1024, 0, st>>>(keys, n, k, L.hdr, L.sample, L.coarse_hist,
-                                                                          L.coarse_incl);
+        if (fused)
+            sample_score_coarse_kernel<<<(1u << (kSampleBits - 2)) / 1024, 1024, 0, st>>>(
+                fused->w, *fused->g, (int)fused->K, fused->c, n, k, L.hdr, L.sample, L.coarse_hist, L.coarse_incl);
+        else
+            sample_coarse_kernel<<<(1u << kSampleBits) / 1024, 1024, 0, st>>>(keys, n, k, L.hdr, L.sample,
+                                                                              L.coarse_hist, L.coarse_incl);
         sample_fine_kernel<<<(1u << kSampleBits) / 1024, 1024, 0, st>>>(L.sample, n, k, L.hdr, L.fine_hist,
                                                                         L.coarse_incl);
-        bracket_pass_kernel<<<(unsigned)cgrid, 256, 0, st>>>(keys, n, nb, L.hdr, cap, L.G, L.E, L.cnt, L.cand_key,
-                                                             L.cand_idx);
+        if (fused) {
+            if (fused->mark_begin && cudaEventRecord(fused->mark_begin, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
+            uint64_t fgrid = (nb + 7) / 8;
+            if (fgrid > (uint64_t)sms * 4) fgrid = (uint64_t)sms * 4;
+#define SLIMDP_FUSED_CASE(KK)                                                                                     \
+    score_bracket_kernel<KK><<<(unsigned)fgrid, 256, 0, st>>>(fused->w, *fused->g, (int)fused->K, fused->c, n, nb, \
+                                                              L.hdr, cap, L.G, L.E, L.cnt, L.cand_key, L.cand_idx)
+            switch (fused->K) {
+                case 4: SLIMDP_FUSED_CASE(4); break;
+                case 8: SLIMDP_FUSED_CASE(8); break;
+                default: SLIMDP_FUSED_CASE(0);
+            }
+#undef SLIMDP_FUSED_CASE
+            if (fused->mark_end && cudaEventRecord(fused->mark_end, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
+        } else {
+            bracket_pass_kernel<<<(unsigned)cgrid, 256, 0, st>>>(keys, n, nb, L.hdr, cap, L.G, L.E, L.cnt, L.cand_key,
+                                                                 L.cand_idx);
+        }
         // T and r from the candidates (these return at once if the bracket failed) ...
         const unsigned cand_grid = (unsigned)sms;
         hist_kernel<0><<<cand_grid, kHistThreads, 0, st>>>(keys, n, L.cand_key, L.hdr, L.hist + 3 * kBins0, k, cap,
@@ -575,6 +826,12 @@ slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, ui
         mark_candidates_kernel<<<(unsigned)sms * 4, 256, 0, st>>>(L.cand_key, L.cand_idx, L.hdr, k, cap, L.G, L.E,
                                                                   L.cnt);
         SLIMDP_LAUNCHED(7);
+    }
+    if (fused) {
+        score_if_bracket_failed_kernel<<<(unsigned)sms * 8, 256, 0, st>>>(fused->w, *fused->g, (int)fused->K, fused->c,
+                                                                          n, L.hdr, k, cap,
+                                                                          reinterpret_cast<uint32_t*>(scores));
+        SLIMDP_LAUNCHED(1);
     }
     if (k_core > 0) {
         // ... or from all keys (these return at once if the bracket held)
@@ -592,6 +849,21 @@ slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, ui
     emit_kernel<<<(unsigned)cgrid, 256, 0, st>>>(L.G, L.E, L.pref, L.totals, n, nb, k, L.hdr, core_idx, bitmap, dir);
     SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
+}
+
+slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx, void* core_aux,
+                            void* ws, cudaStream_t st) {
+    return launch_select_impl(const_cast<float*>(scores), n, k_core, core_idx, core_aux, ws, nullptr, st);
+}
+
+// Whether scoring can be folded into the selection for these sizes and alignments.
+bool score_select_fusable(uint64_t n, uint64_t k_core, bool vec) { return vec && k_core > 0 && n >= kBracketMinN; }
+
+slimdp_status launch_score_select(const float* w, const PtrArray<const float>& g, uint32_t K, float c, uint64_t n,
+                                  float* scores, uint64_t k_core, uint32_t* core_idx, void* core_aux, void* ws,
+                                  cudaEvent_t mark_begin, cudaEvent_t mark_end, cudaStream_t st) {
+    const FusedScore f{w, &g, K, c, mark_begin, mark_end};
+    return launch_select_impl(scores, n, k_core, core_idx, core_aux, ws, &f, st);
 }
 
 }  // namespace slimdp

@@ -29,10 +29,18 @@ class RoundBuffers:
 
 
 def run_round(w: torch.Tensor, grads: Sequence[torch.Tensor], c: float, seed: int, rnd: int, eta: float,
-              buf: RoundBuffers, with_score: bool = True, fused_exchange: bool = True) -> None:
+              buf: RoundBuffers, with_score: bool = True, fused_exchange: bool = True,
+              overlapped: bool = False) -> None:
     """Enqueue one round on the current stream; w is merged in place.  fused_exchange selects
-    slimdp_exchange over the three separate calls (identical results)."""
+    slimdp_exchange over the three separate calls, overlapped the single slimdp_round call
+    over the sequence of calls (identical results in every case)."""
     n, k_core, k_exp = buf.n, buf.k_core, buf.k_exp
+    if overlapped:
+        if not with_score:
+            raise ValueError("slimdp_round always scores")
+        B.slimdp_round(w, grads, c, seed, rnd, eta, buf.scores, buf.core_idx, buf.core_aux, buf.exp_idx, buf.val,
+                       buf.pulled, buf.select_ws, buf.explore_ws)
+        return
     if with_score:
         B.slimdp_score(w, grads, c, buf.scores)
     B.slimdp_select_core(buf.scores, k_core, buf.core_idx, buf.core_aux, buf.select_ws)

@@ -292,33 +292,44 @@ def test_merge_collisions_follow_worker_order(P):
 
 # --------------------------------------------------------------- whole round
 
-def gpu_round(P, w, gs, cfg_c, k_core, k_exp, seed, rnd, eta, fused=True):
+def gpu_round(P, w, gs, cfg_c, k_core, k_exp, seed, rnd, eta, fused=True, one_call=False):
     n, K = w.size, len(gs)
     buf = P.RoundBuffers(n, K, k_core, k_exp)
     d_w, d_gs = dev(w), [dev(g) for g in gs]
-    P.run_round(d_w, d_gs, cfg_c, seed, rnd, eta, buf, fused_exchange=fused)
+    P.run_round(d_w, d_gs, cfg_c, seed, rnd, eta, buf, fused_exchange=fused, overlapped=one_call)
     P.read_status(buf.select_ws)
     P.read_status(buf.explore_ws)
     return d_w, buf
 
 
-def assert_round_equal(P, d_w, buf, ref, n):
-    assert np.array_equal(host_bits(buf.scores), bits(ref["scores"])), "scores"
+def same_bits_or_both_nan(got_bits, want):
+    """Bit equality, except that any NaN matches any NaN: IEEE 754 leaves the payload of a NaN that an
+    operation passes on to the implementation, and the merge's fma passes a NaN model value on."""
+    want_bits = bits(want)
+    nan = np.isnan(want)
+    return np.array_equal(np.isnan(got_bits.view(np.float32)), nan) and np.array_equal(got_bits[~nan], want_bits[~nan])
+
+
+def assert_round_equal(P, d_w, buf, ref, n, scores=True, merged_nans=False):
+    same = same_bits_or_both_nan if merged_nans else (lambda got, want: np.array_equal(got, bits(want)))
+    if scores:      # slimdp_round keeps its scores in registers: the buffer is scratch there
+        assert np.array_equal(host_bits(buf.scores), bits(ref["scores"])), "scores"
     assert np.array_equal(host_u32(buf.core_idx), ref["core_idx"]), "core_idx"
     check_aux(P, buf.core_aux, ref["core_idx"], n)
     for k in range(buf.K):
         assert np.array_equal(host_u32(buf.exp_idx[k]), ref["exp_idx"][k]), f"exp_idx[{k}]"
         assert np.array_equal(host_bits(buf.val[k]), bits(ref["val"][k])), f"val[{k}]"
-        assert np.array_equal(host_bits(buf.pulled[k]), bits(ref["pulled"][k])), f"pulled[{k}]"
-    assert np.array_equal(host_bits(d_w), bits(ref["w"])), "merged model"
+        assert same(host_bits(buf.pulled[k]), ref["pulled"][k]), f"pulled[{k}]"
+    assert same(host_bits(d_w), ref["w"]), "merged model"
 
 
 def _round_case(P, cfg, rnd=0):
     w, gs = all_inputs(cfg)
     ref = oracle.run_round(w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta)
-    for fused in (True, False):      # slimdp_exchange, and the three separate calls
-        d_w, buf = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta, fused)
-        assert_round_equal(P, d_w, buf, ref, cfg.N)
+    # slimdp_exchange, the three separate calls, and the whole round as one call
+    for fused, one_call in ((True, False), (False, False), (True, True)):
+        d_w, buf = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta, fused, one_call)
+        assert_round_equal(P, d_w, buf, ref, cfg.N, scores=not one_call)
         del d_w, buf
     return w, gs, ref
 
@@ -354,10 +365,97 @@ def test_round_degenerate_ratios(P, case):
     k_core, k_exp = {"beta_zero": (0, 30_000), "beta_equals_alpha": (30_000, 0), "everything_core": (n, 0),
                      "everything_explored": (0, n), "core_plus_rest": (12_345, n - 12_345)}[case]
     ref = oracle.run_round(w, gs, 1.0, k_core, k_exp, 5, 1, cfg.eta)
-    d_w, buf = gpu_round(P, w, gs, 1.0, k_core, k_exp, 5, 1, cfg.eta)
-    assert_round_equal(P, d_w, buf, ref, n)
-    if k_core + k_exp == n:       # 100 % communication ratio: the dense Plump-DP merge
-        assert np.array_equal(host_bits(d_w), bits(oracle.dense_merge(w, gs, cfg.eta)))
+    for one_call in (False, True):
+        d_w, buf = gpu_round(P, w, gs, 1.0, k_core, k_exp, 5, 1, cfg.eta, one_call=one_call)
+        assert_round_equal(P, d_w, buf, ref, n, scores=not one_call)
+        if k_core + k_exp == n:       # 100 % communication ratio: the dense Plump-DP merge
+            assert np.array_equal(host_bits(d_w), bits(oracle.dense_merge(w, gs, cfg.eta)))
+
+
+# slimdp_round folds scoring into the selection's pass over all parameters from n = 2^21 up.
+FUSED_N = (1 << 21) + 1061      # several thousand bitmap blocks, a ragged last block, n % 4 == 1
+
+
+@pytest.mark.parametrize("case", ["ragged", "k_core_one", "everything_core", "all_scores_equal", "two_values",
+                                  "nan_and_inf"])
+def test_round_one_call_fused_cases(P, case):
+    cfg = scaled_config(CONFIGS["vgg16"], FUSED_N)
+    w, gs = all_inputs(cfg)
+    w, gs = w.copy(), [g.copy() for g in gs]
+    n, k_core, k_exp = cfg.N, cfg.k_core, cfg.k_exp
+    if case == "k_core_one":
+        k_core = 1
+    elif case == "everything_core":
+        k_core, k_exp = n, 0
+    elif case == "all_scores_equal":      # the bracket cannot hold: the full path scores into the scratch
+        w[:] = 0.25
+        for g in gs:
+            g[:] = 0.0
+    elif case == "two_values":            # threshold inside a tie group of about n / 2 parameters
+        w[:] = np.where(np.arange(n) % 2 == 0, np.float32(0.5), np.float32(0.125))
+        for g in gs:
+            g[:] = 0.0
+        k_core = n // 2 + 12_345
+        k_exp = 1000
+    elif case == "nan_and_inf":
+        w[7::1001] = np.nan
+        gs[1][3::2003] = np.inf
+        gs[2][5::3001] = -np.inf
+        w[11::4001] = np.float32(-0.0)
+    ref = oracle.run_round(w, gs, cfg.c, k_core, k_exp, cfg.seed, 2, cfg.eta)
+    d_w, buf = gpu_round(P, w, gs, cfg.c, k_core, k_exp, cfg.seed, 2, cfg.eta, one_call=True)
+    assert_round_equal(P, d_w, buf, ref, n, scores=False, merged_nans=(case == "nan_and_inf"))
+    if case == "all_scores_equal":        # and there the scratch does hold the scores
+        assert np.array_equal(host_bits(buf.scores), bits(ref["scores"]))
+
+
+def test_round_one_call_any_alignment(P):
+    # tensors that start 4 bytes off a 16-byte boundary: the round scores and selects in two steps
+    cfg = scaled_config(CONFIGS["vgg16"], FUSED_N)
+    w, gs = all_inputs(cfg)
+    ref = oracle.run_round(w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 0, cfg.eta)
+    n, K = cfg.N, cfg.K
+    buf = P.RoundBuffers(n, K, cfg.k_core, cfg.k_exp)
+    off = lambda a: torch.cat([torch.zeros(1, dtype=torch.float32), torch.from_numpy(a)]).cuda()[1:]
+    d_w, d_gs = off(w), [off(g) for g in gs]
+    assert d_w.data_ptr() % 16 == 4
+    P.run_round(d_w, d_gs, cfg.c, cfg.seed, 0, cfg.eta, buf, overlapped=True)
+    P.read_status(buf.select_ws)
+    P.read_status(buf.explore_ws)
+    assert_round_equal(P, d_w, buf, ref, n, scores=True)      # unfused: the scores are there
+
+
+def test_round_one_call_repeats_and_marks(P):
+    cfg = scaled_config(CONFIGS["vgg16"], FUSED_N)
+    w, gs = all_inputs(cfg)
+    d_w, d_gs = dev(w), [dev(g) for g in gs]
+    a_w = d_w.clone()
+    buf = P.RoundBuffers(cfg.N, cfg.K, cfg.k_core, cfg.k_exp)
+    ref_buf = P.RoundBuffers(cfg.N, cfg.K, cfg.k_core, cfg.k_exp)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(); e1.record()
+    for rnd in range(3):      # successive rounds on the evolving model, buffers reused
+        if rnd == 1:
+            P.mark_dominant_kernel(e0, e1)
+        P.run_round(d_w, d_gs, cfg.c, cfg.seed, rnd, cfg.eta, buf, overlapped=True)
+        P.run_round(a_w, d_gs, cfg.c, cfg.seed, rnd, cfg.eta, ref_buf)
+        torch.cuda.synchronize()
+        assert torch.equal(d_w.view(torch.int32), a_w.view(torch.int32))
+        assert torch.equal(buf.core_idx, ref_buf.core_idx)
+        for k in range(cfg.K):
+            assert torch.equal(buf.exp_idx[k], ref_buf.exp_idx[k])
+            assert torch.equal(buf.pulled[k].view(torch.int32), ref_buf.pulled[k].view(torch.int32))
+    assert 0.0 < e0.elapsed_time(e1) < 50.0      # ms: one pass over two million parameters
+
+
+def test_round_one_call_rejects_overlapping_workspaces(P):
+    cfg = CONFIGS["tiny"]
+    w, gs = all_inputs(cfg)
+    buf = P.RoundBuffers(cfg.N, cfg.K, cfg.k_core, cfg.k_exp)
+    both = torch.empty(max(buf.select_ws.numel(), buf.explore_ws.numel()), dtype=torch.uint8, device="cuda")
+    with pytest.raises(P.SlimDPError):
+        P.slimdp_round(dev(w), [dev(g) for g in gs], cfg.c, cfg.seed, 0, cfg.eta, buf.scores, buf.core_idx,
+                       buf.core_aux, buf.exp_idx, buf.val, buf.pulled, both, both)
 
 
 def test_round_is_deterministic(P):
