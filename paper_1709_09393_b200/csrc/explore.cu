@@ -68,39 +68,17 @@ __device__ __forceinline__ uint32_t find_block(const uint32_t* __restrict__ dir,
     return lo;
 }
 
-// Round keys per worker, and per rank bucket the directory entry (64-parameter group) that holds
-// the bucket's first rank (bounds[buckets] = the group of the last rank M - 1).  The bounds
-// depend on the core only.
+// Round keys of every worker of the call.
 __global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, uint32_t seed_lo, uint32_t seed_hi,
-                                     uint32_t first_worker, uint32_t workers, uint32_t round,
-                                     const uint32_t* __restrict__ dir, uint32_t nd, uint32_t M, uint32_t s,
-                                     uint32_t buckets, uint32_t* __restrict__ bounds, int parts) {
+                                     uint32_t first_worker, uint32_t workers, uint32_t round) {
     const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
-    if ((parts & 1) && t == 0) hdr->status = SLIMDP_OK;
-    if ((parts & 1) && t < workers * 3) {
+    if (t == 0) hdr->status = SLIMDP_OK;
+    if (t < workers * 3) {
         const uint32_t w = t / 3, b = t % 3;
         uint32_t out[4];
         philox4x32_10(seed_lo, seed_hi, b, first_worker + w, round, 0x534C494Du, out);
 #pragma unroll
         for (int q = 0; q < 4; ++q) rk[w * 12 + b * 4 + q] = out[q];
-    }
-    // one warp per bucket boundary: a 32-way search (5 probes for 2^25 entries instead of 25)
-    const uint32_t bnd = t >> 5, lane = t & 31u;
-    if ((parts & 2) && M > 0 && bnd <= buckets) {
-        const uint64_t first = (uint64_t)bnd << s;
-        const uint32_t rank = (first < M) ? (uint32_t)first : M - 1;
-        uint32_t lo = 0, hi = nd - 1;   // the answer is the largest d in [lo, hi] with dir[d] <= rank; dir[lo] <= rank
-        while (hi > lo) {
-            const uint32_t step = (hi - lo) / 32u + 1u;              // lane probes lo + lane * step
-            const uint64_t p = (uint64_t)lo + (uint64_t)lane * step;
-            const bool le = p <= hi && __ldg(dir + p) <= rank;       // true for a prefix of the lanes (lane 0 always)
-            const uint32_t c = __popc(__ballot_sync(0xFFFFFFFFu, le));
-            const uint32_t nlo = lo + (c - 1u) * step;
-            const uint64_t nhi = (uint64_t)nlo + step - 1u;
-            lo = nlo;
-            hi = (nhi < hi) ? (uint32_t)nhi : hi;
-        }
-        if (lane == 0) bounds[bnd] = lo;
     }
 }
 
@@ -277,17 +255,16 @@ __global__ void __launch_bounds__(1024) scatter_kernel(uint32_t k_exp, uint32_t 
 // consecutive words (stride 2, 4 or 8 across lanes) free of bank conflicts.
 __device__ __forceinline__ uint32_t sw(uint32_t w) { return w + (w >> 5); }
 
-constexpr uint32_t kDirCache = 2048;
 constexpr uint32_t kListCap = 4096;
 
-// grid = (buckets, workers).  Sort the bucket's ranks through a shared bitmap and emit parameter indices.
-__global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
-    const uint32_t* __restrict__ bitmap, const uint32_t* __restrict__ dir, const uint32_t* __restrict__ bounds,
-    uint32_t k_exp, uint32_t s, const uint32_t* __restrict__ sorted, uint64_t rho_stride,
-    const unsigned long long* __restrict__ cnt, const unsigned long long* __restrict__ pref,
-    const unsigned long long* __restrict__ totals, uint64_t cnt_stride, PtrArray<uint32_t> out, WsHeader* hdr) {
+// grid = (buckets, workers).  Sorts one bucket's ranks through a shared bitmap and writes them,
+// ascending, to the worker's row of `ranks`: buckets are rank ranges, so the row ends up sorted
+// as a whole.  Needs the sizes only, not the core.
+__global__ void __launch_bounds__(kBucketThreads) bucket_sort_kernel(
+    uint32_t k_exp, uint32_t s, const uint32_t* __restrict__ grouped, uint32_t* __restrict__ ranks,
+    uint64_t rho_stride, const unsigned long long* __restrict__ cnt, const unsigned long long* __restrict__ pref,
+    const unsigned long long* __restrict__ totals, uint64_t cnt_stride, WsHeader* hdr) {
     __shared__ uint32_t bm[2048 + 64];           // up to 2^16 rank bits, padded (see sw)
-    __shared__ uint32_t dir_sh[kDirCache + 1];   // directory entries of the bucket's 64-parameter groups (+1)
     __shared__ uint16_t list[kListCap];          // sorted ranks (low s bits) of the current round
     __shared__ uint32_t warp_sums[kBucketThreads / 32];
     const uint32_t worker = blockIdx.y, bucket = blockIdx.x, t = threadIdx.x;
@@ -297,21 +274,16 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
     const uint32_t offset = (uint32_t)pref[(uint64_t)worker * cnt_stride + bucket];
     if (bucket == 0 && t == 0 && totals[worker] != k_exp) hdr->status = SLIMDP_ERR_INTERNAL;
     if (count == 0) return;
+    if ((uint64_t)offset + count > k_exp) {
+        if (t == 0) hdr->status = SLIMDP_ERR_INTERNAL;
+        return;
+    }
     for (uint32_t i = t; i < words + (words >> 5); i += kBucketThreads) bm[i] = 0;
-    // the bucket's ranks live in directory groups [grp_lo, grp_hi]
-    const uint32_t grp_lo = __ldg(bounds + bucket), grp_hi = __ldg(bounds + bucket + 1);
-    const uint32_t ngrp = grp_hi - grp_lo + 1;
-    const bool cached = ngrp <= kDirCache;
-    if (cached)
-        for (uint32_t i = t; i <= ngrp; i += kBucketThreads) dir_sh[i] = __ldg(dir + grp_lo + i);
     __syncthreads();
-    // groups per rank inside this bucket, for the interpolated first guess of select0
-    const uint32_t dir_first = cached ? dir_sh[0] : 0u;
-    const float groups_per_rank = cached ? (float)ngrp / (float)(dir_sh[ngrp] - dir_sh[0] + 1u) : 0.0f;
-    const uint32_t* my_sorted = sorted + (uint64_t)worker * rho_stride + offset;
+    const uint32_t* src = grouped + (uint64_t)worker * rho_stride + offset;
     const uint32_t low_mask = (1u << s) - 1u;
     for (uint32_t e = t; e < count; e += kBucketThreads) {
-        const uint32_t r = my_sorted[e] & low_mask;
+        const uint32_t r = src[e] & low_mask;
         atomicOr(&bm[sw(r >> 5)], 1u << (r & 31u));
     }
     __syncthreads();
@@ -326,9 +298,9 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
     uint32_t total = 0;
     for (uint32_t wdx = 0; wdx < kBucketThreads / 32; ++wdx) total += warp_sums[wdx];
     if (t == 0 && total != count) hdr->status = SLIMDP_ERR_INTERNAL;   // two ranks collided: pi is not injective
-    uint32_t* dst = out.p[worker] + offset;
+    uint32_t* dst = ranks + (uint64_t)worker * rho_stride + offset;
     const uint32_t first_rank = bucket << s;
-    // rounds of up to kListCap ranks: write them to `list` in sorted order, then share them out evenly
+    // rounds of up to kListCap ranks: into `list` in sorted order, then out with coalesced stores
     for (uint32_t r0 = 0; r0 < count; r0 += kListCap) {
         if (base < r0 + kListCap && base + mine > r0) {
             uint32_t p = base;
@@ -344,61 +316,167 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_kernel(
         }
         __syncthreads();
         const uint32_t m = (count - r0 < kListCap) ? count - r0 : kListCap;
-        uint32_t rel = 0;     // group relative to grp_lo; ranks ascend inside a thread, so it only moves up
-        for (uint32_t e = t; e < m; e += kBucketThreads) {
-            const uint32_t rank = first_rank + list[e];
-            // select0(rank): the 64-parameter group from the directory ...
-            uint32_t d0, d1;
-            if (cached) {
-                uint32_t lo = rel, hi = ngrp - 1;
-                // the directory is close to linear inside one bucket: try a small window around the
-                // interpolated group first, and search the whole range only if the window misses
-                const uint32_t guess = (uint32_t)((float)(rank - dir_first) * groups_per_rank);
-                const uint32_t wl = (guess > 8u) ? guess - 8u : 0u;
-                const uint32_t win_lo = (wl > lo) ? wl : lo;
-                const uint32_t win_hi = (guess + 8u < hi) ? guess + 8u : hi;
-                if (win_lo <= win_hi && dir_sh[win_lo] <= rank && dir_sh[win_hi + 1] > rank) {
-                    lo = win_lo;
-                    hi = win_hi;
-                }
-                while (lo < hi) {
-                    const uint32_t mid = lo + ((hi - lo + 1) >> 1);
-                    if (dir_sh[mid] <= rank)
-                        lo = mid;
-                    else
-                        hi = mid - 1;
-                }
-                rel = lo;
-                d0 = dir_sh[rel];
-                d1 = dir_sh[rel + 1];
-            } else {
-                rel = find_block(dir, grp_lo + rel, grp_hi, rank) - grp_lo;
-                d0 = __ldg(dir + grp_lo + rel);
-                d1 = __ldg(dir + grp_lo + rel + 1);
-            }
-            const uint32_t grp = grp_lo + rel;
-            const uint32_t rem = rank - d0;
-            uint32_t idx;
-            if (d1 - d0 == kDirStride) {
-                idx = grp * kDirStride + rem;   // no core parameter in this group
-            } else {
-                // ... then the rem-th zero bit of the group's two bitmap words
-                const uint2 v = __ldg(reinterpret_cast<const uint2*>(bitmap + (uint64_t)grp * kWordsPerDir));
-                const uint32_t z0 = ~v.x, z1 = ~v.y;
-                const uint32_t c0 = __popc(z0);
-                const bool second = rem >= c0;
-                const uint32_t z = second ? z1 : z0;
-                const uint32_t r = second ? rem - c0 : rem;
-                idx = (r < (uint32_t)__popc(z)) ? grp * kDirStride + (second ? 32u : 0u) + nth_set_bit(z, r)
-                                                : 0xFFFFFFFFu;
-            }
-            if (idx == 0xFFFFFFFFu || offset + r0 + e >= k_exp) {
-                hdr->status = SLIMDP_ERR_INTERNAL;   // directory and bitmap disagree
-            } else {
-                dst[r0 + e] = idx;
-            }
-        }
+        for (uint32_t e = t; e < m; e += kBucketThreads) dst[r0 + e] = first_rank + list[e];
         __syncthreads();
+    }
+}
+
+constexpr uint32_t kSelThreads = 256;
+constexpr uint32_t kSelPer = 8;                          // consecutive sorted ranks per thread
+constexpr uint32_t kSelTile = kSelThreads * kSelPer;     // per CTA
+constexpr uint32_t kDirCache = 6144;                     // directory entries a CTA keeps in shared memory
+
+// cell_group[c] = the 64-parameter group that holds non-core rank c * 4096, c < cells;
+// cell_group[cells] = the last group.  A group holds at most 64 ranks, so it contains at most
+// one cell boundary, and every boundary below M lies in exactly one group: no search, no races.
+__global__ void __launch_bounds__(256) cell_table_kernel(const uint32_t* __restrict__ dir, uint32_t nd,
+                                                         uint32_t cells, uint32_t* __restrict__ cell_group) {
+    const uint32_t stride = gridDim.x * blockDim.x;
+    for (uint32_t d = blockIdx.x * blockDim.x + threadIdx.x; d < nd; d += stride) {
+        const uint32_t a = __ldg(dir + d), b = __ldg(dir + d + 1);
+        const uint64_t c = ((uint64_t)a + (1u << kCellShift) - 1u) >> kCellShift;   // first boundary at or after a
+        if ((c << kCellShift) < b && c < cells) cell_group[c] = d;
+        if (d == 0) cell_group[cells] = nd - 1;
+    }
+}
+
+// grid = (tiles, workers).  idx = select0(core bitmap, rank) for one tile of a worker's sorted
+// ranks: the tile's ranks lie in a contiguous run of directory groups, bounded through the cell
+// table and kept in shared memory; each thread then walks its consecutive ranks forward
+// through that run.  Ascending ranks give ascending indices, so the output is the sorted set.
+__global__ void __launch_bounds__(kSelThreads, 5) select0_kernel(const uint32_t* __restrict__ bitmap,
+                                                                 const uint32_t* __restrict__ dir, uint32_t nd,
+                                                                 const uint32_t* __restrict__ cell_group,
+                                                                 uint32_t cells, uint32_t k_exp,
+                                                                 const uint32_t* __restrict__ ranks,
+                                                                 uint64_t rho_stride, PtrArray<uint32_t> out,
+                                                                 WsHeader* hdr) {
+    __shared__ uint32_t dir_sh[kDirCache + 1];
+    __shared__ uint32_t grp_bounds[2];
+    const uint32_t worker = blockIdx.y, t = threadIdx.x;
+    const uint32_t tile0 = blockIdx.x * kSelTile;
+    if (tile0 >= k_exp) return;
+    const uint32_t m = (k_exp - tile0 < kSelTile) ? k_exp - tile0 : kSelTile;
+    const uint32_t* src = ranks + (uint64_t)worker * rho_stride + tile0;
+    uint32_t* dst = out.p[worker] + tile0;
+    if (t < 2) {   // the group of the first cell the tile touches, and of the cell after its last
+        const uint32_t cell = (__ldg(src + (t ? m - 1u : 0u)) >> kCellShift) + t;
+        grp_bounds[t] = __ldg(cell_group + (cell < cells ? cell : cells));
+    }
+    // this thread's ranks (the row is 256-byte aligned and tile0, kSelPer are multiples of 4)
+    const uint32_t e0 = t * kSelPer;
+    uint32_t rank[kSelPer];
+    if (e0 + kSelPer <= m) {
+#pragma unroll
+        for (uint32_t q = 0; q < kSelPer; q += 4) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + e0 + q));
+            rank[q] = v.x;
+            rank[q + 1] = v.y;
+            rank[q + 2] = v.z;
+            rank[q + 3] = v.w;
+        }
+    } else {
+#pragma unroll
+        for (uint32_t q = 0; q < kSelPer; ++q) rank[q] = (e0 + q < m) ? __ldg(src + e0 + q) : 0u;
+    }
+    __syncthreads();
+    const uint32_t grp_lo = grp_bounds[0], grp_hi = grp_bounds[1];
+    if (grp_hi < grp_lo) {
+        if (t == 0) hdr->status = SLIMDP_ERR_INTERNAL;   // the ranks are not ascending
+        return;
+    }
+    const uint32_t ngrp = grp_hi - grp_lo + 1;
+    const bool cached = ngrp <= kDirCache;
+    if (cached)
+        for (uint32_t i = t; i <= ngrp; i += kSelThreads) dir_sh[i] = __ldg(dir + grp_lo + i);
+    __syncthreads();
+    // first every rank's group and its place in the group (shared memory only), then all bitmap
+    // words of the thread at once, so that their latencies overlap
+    uint32_t grp[kSelPer], rem[kSelPer];
+    bool plain[kSelPer];   // no core parameter in the group
+    bool bad = false;
+    if (cached) {
+        // groups per rank inside this tile, for the interpolated first guess
+        const uint32_t dir_first = dir_sh[0];
+        const float groups_per_rank = (float)ngrp / (float)(dir_sh[ngrp] - dir_first + 1u);
+        uint32_t rel = 0;
+        if (e0 < m) {
+            const uint32_t r = rank[0];
+            uint32_t lo = 0, hi = ngrp - 1;
+            const uint32_t guess = (uint32_t)((float)(r - dir_first) * groups_per_rank);
+            const uint32_t win_lo = (guess > 8u) ? guess - 8u : 0u;
+            const uint32_t win_hi = (guess + 8u < hi) ? guess + 8u : hi;
+            if (win_lo <= win_hi && dir_sh[win_lo] <= r && dir_sh[win_hi + 1] > r) {
+                lo = win_lo;
+                hi = win_hi;
+            }
+            while (lo < hi) {
+                const uint32_t mid = lo + ((hi - lo + 1) >> 1);
+                if (dir_sh[mid] <= r)
+                    lo = mid;
+                else
+                    hi = mid - 1;
+            }
+            rel = lo;
+        }
+#pragma unroll
+        for (uint32_t q = 0; q < kSelPer; ++q) {
+            const uint32_t r = rank[q];
+            if (e0 + q < m)
+                while (rel + 1 < ngrp && dir_sh[rel + 1] <= r) ++rel;   // ranks ascend: the group only moves up
+            const uint32_t d0 = dir_sh[rel], d1 = dir_sh[rel + 1];
+            grp[q] = grp_lo + rel;
+            rem[q] = r - d0;
+            plain[q] = d1 - d0 == kDirStride;
+            bad |= e0 + q < m && !(r >= d0 && r < d1);
+        }
+    } else {
+        // a tile that spans more groups than the cache holds (few ranks over many parameters)
+        uint32_t g = grp_lo;
+#pragma unroll
+        for (uint32_t q = 0; q < kSelPer; ++q) {
+            const uint32_t r = rank[q];
+            if (e0 + q < m) g = find_block(dir, g, grp_hi, r);
+            const uint32_t d0 = __ldg(dir + g), d1 = __ldg(dir + g + 1);
+            grp[q] = g;
+            rem[q] = r - d0;
+            plain[q] = d1 - d0 == kDirStride;
+            bad |= e0 + q < m && !(r >= d0 && r < d1);
+        }
+    }
+    uint2 words[kSelPer];
+#pragma unroll
+    for (uint32_t q = 0; q < kSelPer; ++q)
+        words[q] = (e0 + q < m && !plain[q] && !bad)
+                       ? __ldg(reinterpret_cast<const uint2*>(bitmap + (uint64_t)grp[q] * kWordsPerDir))
+                       : make_uint2(0u, 0u);
+    uint32_t idx[kSelPer];
+#pragma unroll
+    for (uint32_t q = 0; q < kSelPer; ++q) {
+        if (plain[q]) {
+            idx[q] = grp[q] * kDirStride + rem[q];
+        } else {
+            const uint32_t z0 = ~words[q].x, z1 = ~words[q].y;
+            const uint32_t c0 = __popc(z0);
+            const bool second = rem[q] >= c0;
+            const uint32_t z = second ? z1 : z0;
+            const uint32_t r = second ? rem[q] - c0 : rem[q];
+            idx[q] = grp[q] * kDirStride + (second ? 32u : 0u) + nth_set_bit(z, r);
+            bad |= e0 + q < m && r >= (uint32_t)__popc(z);
+        }
+    }
+    if (bad) {
+        hdr->status = SLIMDP_ERR_INTERNAL;   // directory and bitmap disagree, or the ranks are not sorted
+        return;
+    }
+    if (e0 + kSelPer <= m) {
+#pragma unroll
+        for (uint32_t q = 0; q < kSelPer; q += 4)
+            *reinterpret_cast<uint4*>(dst + e0 + q) = make_uint4(idx[q], idx[q + 1], idx[q + 2], idx[q + 3]);
+    } else {
+#pragma unroll
+        for (uint32_t q = 0; q < kSelPer; ++q)
+            if (e0 + q < m) dst[e0 + q] = idx[q];
     }
 }
 
@@ -413,8 +491,8 @@ uint32_t explore_bucket_shift(uint64_t M) {
     return (uint32_t)(13 + extra);
 }
 
-// parts: 1 = the steps that need only the sizes (round keys, ranks, bucket grouping),
-//        2 = the steps that need the core (bucket bounds, parameter indices), 3 = everything.
+// parts: 1 = the steps that need only the sizes (round keys, ranks, their sort),
+//        2 = the step that needs the core (parameter indices from sorted ranks), 3 = everything.
 slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                    uint32_t first_worker, uint32_t workers, uint32_t round,
                                    const PtrArray<uint32_t>& out, void* ws, int parts, cudaStream_t st) {
@@ -429,13 +507,12 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
     const uint32_t s = explore_bucket_shift(M);
     const uint64_t buckets = (M + (1ull << s) - 1) >> s;
 
-    const unsigned setup_threads =
-        (unsigned)(((buckets + 1) * 32 > 3ull * workers) ? (buckets + 1) * 32 : 3ull * workers);
-    explore_setup_kernel<<<(setup_threads + 255) / 256, 256, 0, st>>>(L.hdr, L.round_keys, (uint32_t)seed,
-                                                                      (uint32_t)(seed >> 32), first_worker, workers,
-                                                                      round, dir, (uint32_t)nd, (uint32_t)M, s,
-                                                                      (uint32_t)buckets, L.bounds, parts);
-    SLIMDP_LAUNCHED(1);
+    if (parts & 1) {
+        explore_setup_kernel<<<(3 * workers + 255) / 256, 256, 0, st>>>(L.hdr, L.round_keys, (uint32_t)seed,
+                                                                        (uint32_t)(seed >> 32), first_worker,
+                                                                        workers, round);
+        SLIMDP_LAUNCHED(1);
+    }
     if (k_exp == 0) return SLIMDP_OK;
     if (parts & 1) {
     if (cudaMemsetAsync(L.cnt, 0, L.zero_bytes, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
@@ -483,12 +560,18 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
                                                      L.sorted);
     }
     SLIMDP_LAUNCHED(1);
+    bucket_sort_kernel<<<dim3((unsigned)buckets, workers), kBucketThreads, 0, st>>>(
+        (uint32_t)k_exp, s, L.sorted, L.rho, L.rho_stride, L.cnt, L.pref, L.totals, L.cnt_stride, L.hdr);
+    SLIMDP_LAUNCHED(1);
     }   // parts & 1
     if (!(parts & 2)) return SLIMDP_OK;
-    bucket_kernel<<<dim3((unsigned)buckets, workers), kBucketThreads, 0, st>>>(
-        bitmap, dir, L.bounds, (uint32_t)k_exp, s, L.sorted, L.rho_stride, L.cnt, L.pref, L.totals, L.cnt_stride,
-        out, L.hdr);
-    SLIMDP_LAUNCHED(1);
+    const uint32_t cells = (uint32_t)((M + (1u << kCellShift) - 1) >> kCellShift);
+    uint64_t tgrid = (nd + 255) / 256;
+    if (tgrid > (uint64_t)sms * 8) tgrid = (uint64_t)sms * 8;
+    cell_table_kernel<<<(unsigned)tgrid, 256, 0, st>>>(dir, (uint32_t)nd, cells, L.cell_group);
+    select0_kernel<<<dim3((unsigned)((k_exp + kSelTile - 1) / kSelTile), workers), kSelThreads, 0, st>>>(
+        bitmap, dir, (uint32_t)nd, L.cell_group, cells, (uint32_t)k_exp, L.rho, L.rho_stride, out, L.hdr);
+    SLIMDP_LAUNCHED(2);
     return SLIMDP_OK;
 }
 

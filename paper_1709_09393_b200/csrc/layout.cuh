@@ -58,12 +58,12 @@ inline SelectWs select_ws_layout(void* ws, uint64_t n) {
 struct ExploreWs {
     WsHeader* hdr;
     uint32_t* round_keys;           // 12 words per worker
-    uint32_t* bounds;               // per bucket: bitmap block of its first rank (+1 entry)
-    uint32_t* rho;                  // per worker: pi(j), j < k_exp
-    uint32_t* sorted;               // per worker: the same ranks grouped by bucket
+    uint32_t* rho;                  // per worker: pi(j), j < k_exp; later the same ranks in ascending order
+    uint32_t* sorted;               // per worker: the ranks grouped by bucket
     unsigned long long* cnt;        // per worker: ranks per bucket
     uint32_t* cursor;               // per worker: scatter cursors per bucket
     uint32_t* cta_hist;             // per rank-step CTA: its chunk's ranks per bucket
+    uint32_t* cell_group;           // per 4096 non-core ranks: the 64-parameter group that holds the cell's first rank
     unsigned long long* pref;       // per worker: exclusive scan of cnt
     unsigned long long* tile_sums;  // per worker: per scan tile
     unsigned long long* totals;     // per worker: 1
@@ -74,6 +74,7 @@ struct ExploreWs {
     size_t bytes;
 };
 
+constexpr uint32_t kCellShift = 12;          // ranks per cell of the rank -> group table
 constexpr uint64_t kMaxSmemBuckets = 5120;   // bucket histograms up to this size live in shared memory (20 KB)
 constexpr uint64_t kMaxExploreCtas = 1024;   // rank / scatter CTAs over all workers of one call
 
@@ -98,7 +99,6 @@ inline ExploreWs explore_ws_layout(void* ws, uint64_t n, uint64_t k_exp, uint32_
     L.tile_stride = align_up((L.cnt_stride + kScanTile - 1) / kScanTile, 32);
     L.hdr = reinterpret_cast<WsHeader*>(take(sizeof(WsHeader)));
     L.round_keys = reinterpret_cast<uint32_t*>(take((size_t)workers * 12 * 4));
-    L.bounds = reinterpret_cast<uint32_t*>(take((L.cnt_stride + 1) * 4));
     L.rho = reinterpret_cast<uint32_t*>(take((size_t)workers * L.rho_stride * 4));
     L.sorted = reinterpret_cast<uint32_t*>(take((size_t)workers * L.rho_stride * 4));
     const size_t zero_begin = off;
@@ -110,6 +110,7 @@ inline ExploreWs explore_ws_layout(void* ws, uint64_t n, uint64_t k_exp, uint32_
     L.totals = reinterpret_cast<unsigned long long*>(take((size_t)workers * 8));
     const uint64_t hist_buckets = explore_max_buckets(n) < kMaxSmemBuckets ? explore_max_buckets(n) : kMaxSmemBuckets;
     L.cta_hist = reinterpret_cast<uint32_t*>(take((size_t)kMaxExploreCtas * hist_buckets * 4));
+    L.cell_group = reinterpret_cast<uint32_t*>(take(((n >> kCellShift) + 2) * 4));
     L.bytes = off;
     return L;
 }

@@ -800,7 +800,11 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
         if (fused) {
             if (fused->mark_begin && cudaEventRecord(fused->mark_begin, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
             uint64_t fgrid = (nb + 7) / 8;
-            if (fgrid > (uint64_t)sms * 4) fgrid = (uint64_t)sms * 4;
+            // The pass is bound by memory bandwidth, which four fifths of the SMs saturate; its CTAs
+            // stay resident from start to end, so the SMs it leaves free are what lets the explorer's
+            // rank kernels (queued beside it on the round's side stream) run at the same time.
+            const uint64_t fmax = 4ull * (uint64_t)(sms - sms / 5);
+            if (fgrid > fmax) fgrid = fmax;
 #define SLIMDP_FUSED_CASE(KK)                                                                                     \
     score_bracket_kernel<KK><<<(unsigned)fgrid, 256, 0, st>>>(fused->w, *fused->g, (int)fused->K, fused->c, n, nb, \
                                                               L.hdr, cap, L.G, L.E, L.cnt, L.cand_key, L.cand_idx)
