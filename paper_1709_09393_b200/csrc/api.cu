@@ -40,7 +40,9 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
 bool score_select_fusable(uint64_t n, uint64_t k_core, bool vec);
 slimdp_status launch_score_select(const float* w, const PtrArray<const float>& g, uint32_t K, float c, uint64_t n,
                                   float* scores, uint64_t k_core, uint32_t* core_idx, void* core_aux, void* ws,
-                                  cudaEvent_t mark_begin, cudaEvent_t mark_end, cudaStream_t st);
+                                  cudaEvent_t mark_begin, cudaEvent_t mark_end, cudaStream_t gate_stream,
+                                  cudaEvent_t gate_fork, cudaEvent_t gate_join, slimdp_status (*after_pass)(void*),
+                                  void* after_arg, cudaStream_t st);
 
 slimdp_status launch_explore_static(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                     uint32_t worker, uint32_t round, uint32_t* exp_idx, int32_t* status_out,
@@ -321,8 +323,8 @@ slimdp_status slimdp_read_status(const void* ws, void* stream) {
 
 namespace {
 struct SideStream {
-    cudaStream_t stream = nullptr;
-    cudaEvent_t fork = nullptr, ranks_done = nullptr;
+    cudaStream_t stream = nullptr, gate = nullptr;
+    cudaEvent_t fork = nullptr, ranks_done = nullptr, gate_fork = nullptr, gate_join = nullptr;
     bool ready = false;
 };
 std::mutex g_side_mutex;
@@ -337,7 +339,8 @@ SideStream* side_stream_locked() {
         int lo = 0, hi = 0;
         if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) return nullptr;
         if (cudaStreamCreateWithPriority(&s.stream, cudaStreamNonBlocking, hi) != cudaSuccess) return nullptr;
-        cudaEvent_t* ev[2] = {&s.fork, &s.ranks_done};
+        if (cudaStreamCreateWithPriority(&s.gate, cudaStreamNonBlocking, hi) != cudaSuccess) return nullptr;
+        cudaEvent_t* ev[4] = {&s.fork, &s.ranks_done, &s.gate_fork, &s.gate_join};
         for (auto e : ev)
             if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         s.ready = true;
@@ -377,6 +380,7 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
     }
     bool vec = aligned16(w_global) && aligned16(scores);
     for (uint32_t k = 0; k < K; ++k) vec = vec && aligned16(g.p[k]);
+    const bool fusable = score_select_fusable(n, k_core, vec);
 
     cudaStream_t st = (cudaStream_t)stream;
     std::lock_guard<std::mutex> lock(g_side_mutex);
@@ -395,15 +399,32 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
     cudaEvent_t mark0 = t_mark_begin, mark1 = t_mark_end;
     t_mark_begin = t_mark_end = nullptr;
 
-    // side: ranks and bucket grouping of every worker's explorer (they need the sizes only)
-    step(launch_explore_parts(core_aux, n, k_core, k_exp, seed, 0, K, round, exp_out, explore_ws, 1, sd));
-    cuda(cudaEventRecord(side->ranks_done, sd));
+    // side: ranks of every worker's explorer, sorted (they need the sizes only).  On the fused path
+    // they are enqueued right after the pass over all parameters, so that the pass has its CTAs
+    // placed before the rank kernels look for room.
+    struct SideWork {
+        const void* core_aux;
+        uint64_t n, k_core, k_exp, seed;
+        uint32_t K, round;
+        const PtrArray<uint32_t>* out;
+        void* ws;
+        cudaStream_t sd;
+        cudaEvent_t done;
+    } side_work{core_aux, n, k_core, k_exp, seed, K, round, &exp_out, explore_ws, sd, side->ranks_done};
+    auto enqueue_side = [](void* p) -> slimdp_status {
+        const SideWork& s = *static_cast<const SideWork*>(p);
+        const slimdp_status r =
+            launch_explore_parts(s.core_aux, s.n, s.k_core, s.k_exp, s.seed, 0, s.K, s.round, *s.out, s.ws, 1, s.sd);
+        if (cudaEventRecord(s.done, s.sd) != cudaSuccess) return SLIMDP_ERR_CUDA;
+        return r;
+    };
     // main: the core, scored and selected in one pass where sizes and alignment allow
-    if (score_select_fusable(n, k_core, vec)) {
-        if (rc == SLIMDP_OK)
-            step(launch_score_select(w_global, g, K, c, n, scores, k_core, core_idx, core_aux, select_ws, mark0,
-                                     mark1, st));
+    if (fusable) {
+        step(launch_score_select(w_global, g, K, c, n, scores, k_core, core_idx, core_aux, select_ws, mark0, mark1,
+                                 side->gate, side->gate_fork, side->gate_join, enqueue_side, &side_work, st));
+        // (if the call failed before it reached the hook, ranks_done keeps an earlier record: nothing to wait for)
     } else {
+        step(enqueue_side(&side_work));
         if (rc == SLIMDP_OK && mark0) cuda(cudaEventRecord(mark0, st));
         if (rc == SLIMDP_OK) step(launch_score(w_global, g, K, c, n, scores, vec, st));
         if (rc == SLIMDP_OK && mark1) cuda(cudaEventRecord(mark1, st));

@@ -36,7 +36,8 @@ struct WsHeader {
     uint32_t b_bot;      // lowest 16-bit bin that may hold T
     uint32_t ticket[8];  // "last CTA done" counters, one per kernel that needs one
     uint32_t coarse_x[2];  // sample: coarse bins in which the two target ranks are crossed
-    uint32_t reserved[46];
+    uint32_t next_block;   // fused scoring pass: the next 1024-parameter block to hand out
+    uint32_t reserved[45];
 };
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 

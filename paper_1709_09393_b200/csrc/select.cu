@@ -344,7 +344,7 @@ __device__ __forceinline__ uint32_t score1(const float* __restrict__ w, const Pt
 // Sample kernel A of the fused path: 2^16 evenly spaced groups of four consecutive parameters
 // are scored (2^18 sampled keys, one 16-byte load per tensor and group); the rest is
 // sample_coarse_kernel's.  Needs n >= 4 and 16-byte aligned tensors.
-__global__ void __launch_bounds__(1024) sample_score_coarse_kernel(const float* __restrict__ w,
+__global__ void __launch_bounds__(256) sample_score_coarse_kernel(const float* __restrict__ w,
                                                                    PtrArray<const float> g, int K, float c,
                                                                    uint64_t n, uint32_t k, WsHeader* hdr,
                                                                    uint32_t* __restrict__ sample,
@@ -354,35 +354,33 @@ __global__ void __launch_bounds__(1024) sample_score_coarse_kernel(const float* 
     __shared__ uint32_t sh_coarse[256];
     __shared__ long long s_incl[257];
     const uint32_t t = threadIdx.x;
-    if (t < 256) sh_coarse[t] = 0;
+    sh_coarse[t] = 0;   // 256 threads
     __syncthreads();
-    const uint32_t j = blockIdx.x * 1024 + t;   // group number, < 2^16
+    const uint32_t j = blockIdx.x * 256 + t;   // group number, < 2^16
     uint32_t key[4];
     score4<0>(w, g, K, c, ((uint64_t)j * (n / 4)) >> (kSampleBits - 2), key);
     reinterpret_cast<uint4*>(sample)[j] = make_uint4(key[0], key[1], key[2], key[3]);
 #pragma unroll
     for (int q = 0; q < 4; ++q) atomicAdd(&sh_coarse[key[q] >> 24], 1u);
     __syncthreads();
-    if (t < 256 && sh_coarse[t]) atomicAdd(&coarse_hist[t], sh_coarse[t]);
+    if (sh_coarse[t]) atomicAdd(&coarse_hist[t], sh_coarse[t]);
     if (!last_cta_done(&hdr->ticket[6])) return;
     long long lo_target, hi_target;
     bracket_targets(k, n, &lo_target, &hi_target);
     unsigned long long total;
-    const unsigned long long cc = (t < 256) ? __ldcg(coarse_hist + 255 - t) : 0ull;
-    const long long c_above = (long long)block_exclusive_scan64<32>(cc, smem, &total);
-    if (t < 256) s_incl[255 - t] = c_above + (long long)cc;
+    const unsigned long long cc = __ldcg(coarse_hist + 255 - t);
+    const long long c_above = (long long)block_exclusive_scan64<8>(cc, smem, &total);
+    s_incl[255 - t] = c_above + (long long)cc;
     if (t == 0) {
         s_incl[256] = 0;
         hdr->coarse_x[0] = 0xFFFFFFFFu;
         hdr->coarse_x[1] = 0xFFFFFFFFu;
     }
     __syncthreads();
-    if (t < 256) {
-        const long long incl = s_incl[t], above = s_incl[t + 1];
-        coarse_incl[t] = (uint32_t)incl;
-        if (incl > lo_target && above <= lo_target) hdr->coarse_x[0] = t;
-        if (incl >= hi_target && above < hi_target) hdr->coarse_x[1] = t;
-    }
+    const long long incl = s_incl[t], above = s_incl[t + 1];
+    coarse_incl[t] = (uint32_t)incl;
+    if (incl > lo_target && above <= lo_target) hdr->coarse_x[0] = t;
+    if (incl >= hi_target && above < hi_target) hdr->coarse_x[1] = t;
 }
 
 constexpr uint32_t kFusedStage = kFlushAt + 128;   // below kFlushAt before a row of 128 parameters, +128 in it
@@ -423,8 +421,19 @@ __global__ void __launch_bounds__(256, 4) score_bracket_kernel(const float* __re
     const bool has_top = b_top < 65536u;
     const uint32_t top_key = has_top ? (b_top << 16) : 0xFFFFFFFFu;
     const uint32_t bot_key = b_bot << 16;
-    const uint64_t warps = (uint64_t)gridDim.x * (blockDim.x >> 5);
-    for (uint64_t blk = (uint64_t)blockIdx.x * (blockDim.x >> 5) + wid; blk < nb; blk += warps) {
+    // Blocks are handed out on request, one at a time per warp: other kernels share the SMs while
+    // this pass runs, so CTAs start at different times and a fixed split would leave a long tail.
+    // The request for the block after this one is issued before the work on this one starts.
+    auto next_block = [&]() {
+        uint32_t b = 0;
+        if (lane == 0) b = atomicAdd(&hdr->next_block, 1u);
+        return b;
+    };
+    uint32_t ahead = next_block();
+    for (;;) {
+        const uint64_t blk = __shfl_sync(0xFFFFFFFFu, ahead, 0);
+        if (blk >= nb) break;
+        ahead = next_block();
         const uint64_t base = blk * kBlock;
         const bool full = base + kBlock <= n;
         uint32_t myG = 0;
@@ -766,10 +775,23 @@ struct FusedScore {
     uint32_t K;
     float c;
     cudaEvent_t mark_begin, mark_end;   // recorded around the pass over all parameters when not null
+    // called once the pass over all parameters is enqueued: what the caller enqueues on other
+    // streams from here on finds the pass's CTAs already placed
+    slimdp_status (*after_pass)(void*);
+    void* after_arg;
+};
+
+// A second stream for the full path's kernels.  After the bracket pass exactly one of the two
+// paths does any work (the other's kernels return at once), and the two write disjoint state, so
+// they may run side by side; the idle one then costs no time on the critical path.
+struct GateStream {
+    cudaStream_t stream;
+    cudaEvent_t fork, join;
 };
 
 static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx,
-                                        void* core_aux, void* ws, const FusedScore* fused, cudaStream_t st) {
+                                        void* core_aux, void* ws, const FusedScore* fused, const GateStream* gate,
+                                        cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
     const SelectWs L = select_ws_layout(ws, n);
@@ -788,9 +810,10 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
     if (cgrid > (uint64_t)sms * 8) cgrid = (uint64_t)sms * 8;
     const unsigned hgrid = (unsigned)sms * 4;
     const bool bracketed = k_core > 0 && n >= kBracketMinN;
+    cudaStream_t fs = st;   // the stream of the full path's kernels
     if (bracketed) {
         if (fused)
-            sample_score_coarse_kernel<<<(1u << (kSampleBits - 2)) / 1024, 1024, 0, st>>>(
+            sample_score_coarse_kernel<<<(1u << (kSampleBits - 2)) / 256, 256, 0, st>>>(
                 fused->w, *fused->g, (int)fused->K, fused->c, n, k, L.hdr, L.sample, L.coarse_hist, L.coarse_incl);
         else
             sample_coarse_kernel<<<(1u << kSampleBits) / 1024, 1024, 0, st>>>(keys, n, k, L.hdr, L.sample,
@@ -815,9 +838,19 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
             }
 #undef SLIMDP_FUSED_CASE
             if (fused->mark_end && cudaEventRecord(fused->mark_end, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
+            if (fused->after_pass) {
+                const slimdp_status hs = fused->after_pass(fused->after_arg);
+                if (hs != SLIMDP_OK) return hs;
+            }
         } else {
             bracket_pass_kernel<<<(unsigned)cgrid, 256, 0, st>>>(keys, n, nb, L.hdr, cap, L.G, L.E, L.cnt, L.cand_key,
                                                                  L.cand_idx);
+        }
+        if (gate) {   // the full path's kernels go to the second stream from here on
+            if (cudaEventRecord(gate->fork, st) != cudaSuccess ||
+                cudaStreamWaitEvent(gate->stream, gate->fork, 0) != cudaSuccess)
+                return SLIMDP_ERR_CUDA;
+            fs = gate->stream;
         }
         // T and r from the candidates (these return at once if the bracket failed) ...
         const unsigned cand_grid = (unsigned)sms;
@@ -832,7 +865,7 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
         SLIMDP_LAUNCHED(7);
     }
     if (fused) {
-        score_if_bracket_failed_kernel<<<(unsigned)sms * 8, 256, 0, st>>>(fused->w, *fused->g, (int)fused->K, fused->c,
+        score_if_bracket_failed_kernel<<<(unsigned)sms * 8, 256, 0, fs>>>(fused->w, *fused->g, (int)fused->K, fused->c,
                                                                           n, L.hdr, k, cap,
                                                                           reinterpret_cast<uint32_t*>(scores));
         SLIMDP_LAUNCHED(1);
@@ -840,14 +873,18 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
     if (k_core > 0) {
         // ... or from all keys (these return at once if the bracket held)
         const int mode = bracketed ? kFullIfBracketFailed : kFullAlways;
-        hist_kernel<0><<<hgrid, kHistThreads, 0, st>>>(keys, n, L.cand_key, L.hdr, L.hist, k, cap, mode);
-        hist_kernel<1><<<hgrid, kHistThreads, 0, st>>>(keys, n, L.cand_key, L.hdr, L.hist + kBins0, k, cap, mode);
-        hist_kernel<2><<<hgrid, kHistThreads, 0, st>>>(keys, n, L.cand_key, L.hdr, L.hist + 2 * kBins0, k, cap, mode);
+        hist_kernel<0><<<hgrid, kHistThreads, 0, fs>>>(keys, n, L.cand_key, L.hdr, L.hist, k, cap, mode);
+        hist_kernel<1><<<hgrid, kHistThreads, 0, fs>>>(keys, n, L.cand_key, L.hdr, L.hist + kBins0, k, cap, mode);
+        hist_kernel<2><<<hgrid, kHistThreads, 0, fs>>>(keys, n, L.cand_key, L.hdr, L.hist + 2 * kBins0, k, cap, mode);
         SLIMDP_LAUNCHED(3);
     }
-    classify_kernel<<<(unsigned)cgrid, 256, 0, st>>>(keys, n, nb, L.hdr, k, cap,
+    classify_kernel<<<(unsigned)cgrid, 256, 0, fs>>>(keys, n, nb, L.hdr, k, cap,
                                                      bracketed ? kFullIfBracketFailed : kFullAlways, L.G, L.E, L.cnt);
     SLIMDP_LAUNCHED(1);
+    if (fs != st) {   // join: the scan needs whichever path ran
+        if (cudaEventRecord(gate->join, fs) != cudaSuccess || cudaStreamWaitEvent(st, gate->join, 0) != cudaSuccess)
+            return SLIMDP_ERR_CUDA;
+    }
     slimdp_status s = launch_block_scan(L.cnt, L.pref, L.tile_sums, L.totals, nb, 1, nb, num_scan_tiles(n), st);
     if (s != SLIMDP_OK) return s;
     emit_kernel<<<(unsigned)cgrid, 256, 0, st>>>(L.G, L.E, L.pref, L.totals, n, nb, k, L.hdr, core_idx, bitmap, dir);
@@ -857,7 +894,7 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
 
 slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx, void* core_aux,
                             void* ws, cudaStream_t st) {
-    return launch_select_impl(const_cast<float*>(scores), n, k_core, core_idx, core_aux, ws, nullptr, st);
+    return launch_select_impl(const_cast<float*>(scores), n, k_core, core_idx, core_aux, ws, nullptr, nullptr, st);
 }
 
 // Whether scoring can be folded into the selection for these sizes and alignments.
@@ -865,9 +902,12 @@ bool score_select_fusable(uint64_t n, uint64_t k_core, bool vec) { return vec &&
 
 slimdp_status launch_score_select(const float* w, const PtrArray<const float>& g, uint32_t K, float c, uint64_t n,
                                   float* scores, uint64_t k_core, uint32_t* core_idx, void* core_aux, void* ws,
-                                  cudaEvent_t mark_begin, cudaEvent_t mark_end, cudaStream_t st) {
-    const FusedScore f{w, &g, K, c, mark_begin, mark_end};
-    return launch_select_impl(scores, n, k_core, core_idx, core_aux, ws, &f, st);
+                                  cudaEvent_t mark_begin, cudaEvent_t mark_end, cudaStream_t gate_stream,
+                                  cudaEvent_t gate_fork, cudaEvent_t gate_join, slimdp_status (*after_pass)(void*),
+                                  void* after_arg, cudaStream_t st) {
+    const FusedScore f{w, &g, K, c, mark_begin, mark_end, after_pass, after_arg};
+    const GateStream gs{gate_stream, gate_fork, gate_join};
+    return launch_select_impl(scores, n, k_core, core_idx, core_aux, ws, &f, gate_stream ? &gs : nullptr, st);
 }
 
 }  // namespace slimdp
