@@ -149,6 +149,8 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* 
 // Core segment: thread j gathers the K workers' updates of core parameter core_idx[j] (the
 // push), folds them into the parameter in worker order (the update) and hands the merged value
 // back to all K workers (the pull).  One read of the key, K gathers, one read-modify-write.
+// The gathers ask for 64-byte fetches: where the core is dense both halves of a line are asked
+// for anyway, where it is thin (one member per line) half the line stays in DRAM.
 __device__ __forceinline__ void exchange_core_body(float* __restrict__ w, const uint32_t* __restrict__ core_idx,
                                                    uint64_t k_core, const PtrArray<const float>& delta,
                                                    const PtrArray<float>& val, const PtrArray<float>& pulled, int K,
@@ -156,12 +158,12 @@ __device__ __forceinline__ void exchange_core_body(float* __restrict__ w, const 
     const uint64_t stride = vgrid * blockDim.x;
     for (uint64_t j = vblock * blockDim.x + threadIdx.x; j < k_core; j += stride) {
         const uint32_t i = __ldg(core_idx + j);
-        float x = w[i];
+        float x = ld_sparse(w + i);
         int k = 0;
         for (; k + 8 <= K; k += 8) {
             float v[8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = __ldg(delta.p[k + q] + i);
+            for (int q = 0; q < 8; ++q) v[q] = ld_sparse(delta.p[k + q] + i);
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
                 __stcs(val.p[k + q] + j, v[q]);
@@ -169,7 +171,7 @@ __device__ __forceinline__ void exchange_core_body(float* __restrict__ w, const 
             }
         }
         for (; k < K; ++k) {
-            const float v = __ldg(delta.p[k] + i);
+            const float v = ld_sparse(delta.p[k] + i);
             __stcs(val.p[k] + j, v);
             x = __fmaf_rn(neg_eta, v, x);
         }
