@@ -53,6 +53,19 @@ def model_bytes(N: int, K: int, k_core: int, k_exp: int) -> dict:
     return b
 
 
+def fused_pass_kernel_name(K: int) -> str:
+    """Which kernel slimdp_round's pass over all parameters is for K workers (the library's own rule:
+    a ring of 2..8 stages of 8 x (K + 1) x 512 bytes within 112 KB, or two stages within 176 KB)."""
+    stage = 8 * (K + 1) * 512
+    stages = (112 * 1024) // stage
+    if stages < 2 and 2 * stage <= 176 * 1024:
+        stages = 2
+    stages = min(stages, 8)
+    if stages >= 2 and stages * stage >= 64 * 1024:
+        return f"score_bracket_async_kernel<{stages}, 8>"
+    return f"score_bracket_kernel<{K if K in (4, 8) else 0}>"
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -302,7 +315,7 @@ def run_ours(args):
     if fused:
         # per parameter: K + 1 fp32 values read, one bit in each of the two bitmaps written (the
         # candidates, about 1 % of the parameters at 8 B each, are not counted)
-        dominant = {"kernel": f"score_bracket_kernel<{K if K in (4, 8) else 0}>",
+        dominant = {"kernel": fused_pass_kernel_name(K),
                     "bytes": 4 * N * (K + 1) + 2 * (N // 8), "traffic": TRAFFIC_DOMINANT_BYTES.get(cfg.name)}
     else:
         dominant = {"kernel": f"score_vec4_kernel<{K}>", "bytes": bytes_model["score"], "traffic": None}

@@ -36,13 +36,13 @@ slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<c
 
 slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                    uint32_t first_worker, uint32_t workers, uint32_t round,
-                                   const PtrArray<uint32_t>& out, void* ws, int parts, cudaStream_t st);
+                                   const PtrArray<uint32_t>& out, void* ws, int parts, bool lean, cudaStream_t st);
 bool score_select_fusable(uint64_t n, uint64_t k_core, bool vec);
 slimdp_status launch_score_select(const float* w, const PtrArray<const float>& g, uint32_t K, float c, uint64_t n,
                                   float* scores, uint64_t k_core, uint32_t* core_idx, void* core_aux, void* ws,
                                   cudaEvent_t mark_begin, cudaEvent_t mark_end, cudaStream_t gate_stream,
                                   cudaEvent_t gate_fork, cudaEvent_t gate_join, slimdp_status (*after_pass)(void*),
-                                  void* after_arg, cudaStream_t st);
+                                  void* after_arg, cudaEvent_t pass_ready, cudaStream_t st);
 
 slimdp_status launch_explore_static(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                     uint32_t worker, uint32_t round, uint32_t* exp_idx, int32_t* status_out,
@@ -314,17 +314,24 @@ slimdp_status slimdp_read_status(const void* ws, void* stream) {
 
 // ---- whole round on device buffers ----------------------------------------
 //
-// The round's steps form a small graph rather than a chain: the explorer's
-// ranks depend on the sizes alone, so they run beside scoring and selection,
-// on a stream the library owns, one per device.  The join is the wait on
-// ranks_done, which every path through the call reaches.  Scoring is folded
-// into the selection's one pass over all parameters, so the scores are never
-// written unless the selection has to fall back to its full path.
+// The round's steps form a small graph rather than a chain.  The chain that
+// decides the round's time (sampling, the pass over all parameters, the
+// threshold, the core, the explorers' indices, the exchange) runs on a stream
+// of the highest priority that the library owns, one per device.  The
+// explorer's ranks depend on the sizes alone: they are computed and sorted on
+// a second stream of the lowest priority, released when the pass starts, in the
+// part of each SM that the pass leaves free.  Whenever a kernel of the chain
+// becomes ready its CTAs are placed ahead of those of the rank kernels.  The
+// caller's stream only forks into the chain at the start of the call and
+// waits for it at the end (chain_done), on every path through the call.
+// Scoring is folded into the selection's one pass over all parameters, so the
+// scores are never written unless the selection has to fall back to its full path.
 
 namespace {
 struct SideStream {
-    cudaStream_t stream = nullptr, gate = nullptr;
-    cudaEvent_t fork = nullptr, ranks_done = nullptr, gate_fork = nullptr, gate_join = nullptr;
+    cudaStream_t chain = nullptr, ranks = nullptr, gate = nullptr;
+    cudaEvent_t fork = nullptr, pass_ready = nullptr, ranks_done = nullptr, chain_done = nullptr, gate_fork = nullptr,
+                gate_join = nullptr;
     bool ready = false;
 };
 std::mutex g_side_mutex;
@@ -336,11 +343,12 @@ SideStream* side_stream_locked() {
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     SideStream& s = g_side[dev];
     if (!s.ready) {
-        int lo = 0, hi = 0;
+        int lo = 0, hi = 0;   // numerically, hi <= lo: hi is the highest priority
         if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) return nullptr;
-        if (cudaStreamCreateWithPriority(&s.stream, cudaStreamNonBlocking, hi) != cudaSuccess) return nullptr;
+        if (cudaStreamCreateWithPriority(&s.chain, cudaStreamNonBlocking, hi) != cudaSuccess) return nullptr;
         if (cudaStreamCreateWithPriority(&s.gate, cudaStreamNonBlocking, hi) != cudaSuccess) return nullptr;
-        cudaEvent_t* ev[4] = {&s.fork, &s.ranks_done, &s.gate_fork, &s.gate_join};
+        if (cudaStreamCreateWithPriority(&s.ranks, cudaStreamNonBlocking, lo) != cudaSuccess) return nullptr;
+        cudaEvent_t* ev[6] = {&s.fork, &s.pass_ready, &s.ranks_done, &s.chain_done, &s.gate_fork, &s.gate_join};
         for (auto e : ev)
             if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         s.ready = true;
@@ -386,11 +394,11 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
     std::lock_guard<std::mutex> lock(g_side_mutex);
     SideStream* side = side_stream_locked();
     if (!side) return SLIMDP_ERR_CUDA;
-    cudaStream_t sd = side->stream;
+    cudaStream_t ch = side->chain, rk = side->ranks;
 
     if (cudaEventRecord(side->fork, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
-    if (cudaStreamWaitEvent(sd, side->fork, 0) != cudaSuccess) return SLIMDP_ERR_CUDA;
-    // From here on the side stream is joined back into `st` whatever happens.
+    if (cudaStreamWaitEvent(ch, side->fork, 0) != cudaSuccess) return SLIMDP_ERR_CUDA;
+    // From here on the chain is joined back into `st` whatever happens.
     slimdp_status rc = SLIMDP_OK;
     auto step = [&](slimdp_status s) {
         if (rc == SLIMDP_OK) rc = s;
@@ -399,43 +407,50 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
     cudaEvent_t mark0 = t_mark_begin, mark1 = t_mark_end;
     t_mark_begin = t_mark_end = nullptr;
 
-    // side: ranks of every worker's explorer, sorted (they need the sizes only).  On the fused path
-    // they are enqueued right after the pass over all parameters, so that the pass has its CTAs
-    // placed before the rank kernels look for room.
-    struct SideWork {
+    // ranks stream: ranks of every worker's explorer, sorted (they need the sizes only).  The stream
+    // waits for `after`, an event of the chain: the moment from which the ranks may take SM room.
+    struct RankWork {
         const void* core_aux;
         uint64_t n, k_core, k_exp, seed;
         uint32_t K, round;
         const PtrArray<uint32_t>* out;
         void* ws;
-        cudaStream_t sd;
-        cudaEvent_t done;
-    } side_work{core_aux, n, k_core, k_exp, seed, K, round, &exp_out, explore_ws, sd, side->ranks_done};
-    auto enqueue_side = [](void* p) -> slimdp_status {
-        const SideWork& s = *static_cast<const SideWork*>(p);
-        const slimdp_status r =
-            launch_explore_parts(s.core_aux, s.n, s.k_core, s.k_exp, s.seed, 0, s.K, s.round, *s.out, s.ws, 1, s.sd);
-        if (cudaEventRecord(s.done, s.sd) != cudaSuccess) return SLIMDP_ERR_CUDA;
+        cudaStream_t rk;
+        cudaEvent_t after, done;
+        bool lean;
+    } rank_work{core_aux, n, k_core, k_exp, seed, K, round, &exp_out, explore_ws, rk, side->fork, side->ranks_done,
+                false};
+    auto enqueue_ranks = [](void* p) -> slimdp_status {
+        const RankWork& s = *static_cast<const RankWork*>(p);
+        if (cudaStreamWaitEvent(s.rk, s.after, 0) != cudaSuccess) return SLIMDP_ERR_CUDA;
+        const slimdp_status r = launch_explore_parts(s.core_aux, s.n, s.k_core, s.k_exp, s.seed, 0, s.K, s.round,
+                                                     *s.out, s.ws, 1, s.lean, s.rk);
+        if (cudaEventRecord(s.done, s.rk) != cudaSuccess) return SLIMDP_ERR_CUDA;
         return r;
     };
-    // main: the core, scored and selected in one pass where sizes and alignment allow
+    // chain: the core, scored and selected in one pass where sizes and alignment allow
     if (fusable) {
+        rank_work.after = side->pass_ready;   // recorded by the call below just before its pass
+        rank_work.lean = true;
         step(launch_score_select(w_global, g, K, c, n, scores, k_core, core_idx, core_aux, select_ws, mark0, mark1,
-                                 side->gate, side->gate_fork, side->gate_join, enqueue_side, &side_work, st));
+                                 side->gate, side->gate_fork, side->gate_join, enqueue_ranks, &rank_work,
+                                 side->pass_ready, ch));
         // (if the call failed before it reached the hook, ranks_done keeps an earlier record: nothing to wait for)
     } else {
-        step(enqueue_side(&side_work));
-        if (rc == SLIMDP_OK && mark0) cuda(cudaEventRecord(mark0, st));
-        if (rc == SLIMDP_OK) step(launch_score(w_global, g, K, c, n, scores, vec, st));
-        if (rc == SLIMDP_OK && mark1) cuda(cudaEventRecord(mark1, st));
-        if (rc == SLIMDP_OK) step(launch_select(scores, n, k_core, core_idx, core_aux, select_ws, st));
+        step(enqueue_ranks(&rank_work));
+        if (rc == SLIMDP_OK && mark0) cuda(cudaEventRecord(mark0, ch));
+        if (rc == SLIMDP_OK) step(launch_score(w_global, g, K, c, n, scores, vec, ch));
+        if (rc == SLIMDP_OK && mark1) cuda(cudaEventRecord(mark1, ch));
+        if (rc == SLIMDP_OK) step(launch_select(scores, n, k_core, core_idx, core_aux, select_ws, ch));
     }
-    // main: explorer indices from the ranks and the core, then the exchange
-    cuda(cudaStreamWaitEvent(st, side->ranks_done, 0));
+    // chain: explorer indices from the sorted ranks and the core, then the exchange
+    cuda(cudaStreamWaitEvent(ch, side->ranks_done, 0));
     if (rc == SLIMDP_OK)
-        step(launch_explore_parts(core_aux, n, k_core, k_exp, seed, 0, K, round, exp_out, explore_ws, 2, st));
+        step(launch_explore_parts(core_aux, n, k_core, k_exp, seed, 0, K, round, exp_out, explore_ws, 2, false, ch));
     if (rc == SLIMDP_OK && k_core + k_exp > 0)
-        step(launch_exchange(w_global, n, K, g, core_idx, k_core, exp_in, k_exp, eta, v, o, st));
+        step(launch_exchange(w_global, n, K, g, core_idx, k_core, exp_in, k_exp, eta, v, o, ch));
+    if (cudaEventRecord(side->chain_done, ch) != cudaSuccess || cudaStreamWaitEvent(st, side->chain_done, 0) != cudaSuccess)
+        step(SLIMDP_ERR_CUDA);
     return rc;
 }
 

@@ -54,6 +54,14 @@ void count_launches(unsigned n);
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
+// Asks for the largest shared-memory share of the SM's L1 for `kernel`.  An SM keeps one split
+// at a time, so kernels that are to run side by side on one SM ask for the same split.
+template <typename Kernel>
+inline bool prefer_max_shared(Kernel kernel) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+}
+
 // After a group of `count` kernel launches: fail on a launch error, else count them.
 #define SLIMDP_LAUNCHED(count)                                          \
     do {                                                                \

@@ -30,6 +30,7 @@ namespace {
 
 constexpr int kBucketThreads = 256;
 constexpr size_t kGroupSmemMax = 200 * 1024;   // shared memory the scatter step may use to group a chunk
+constexpr size_t kGroupSmemLean = 80 * 1024;   // the same when it has to fit beside another kernel's CTA
 
 
 __device__ __forceinline__ void philox4x32_10(uint32_t k0, uint32_t k1, uint32_t c0, uint32_t c1, uint32_t c2,
@@ -493,9 +494,11 @@ uint32_t explore_bucket_shift(uint64_t M) {
 
 // parts: 1 = the steps that need only the sizes (round keys, ranks, their sort),
 //        2 = the step that needs the core (parameter indices from sorted ranks), 3 = everything.
+// lean: part 1 runs beside a kernel that holds most of every SM's shared memory, so its
+// kernels keep to small shared-memory footprints (the scatter step does not group its chunk).
 slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                    uint32_t first_worker, uint32_t workers, uint32_t round,
-                                   const PtrArray<uint32_t>& out, void* ws, int parts, cudaStream_t st) {
+                                   const PtrArray<uint32_t>& out, void* ws, int parts, bool lean, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
     const ExploreWs L = explore_ws_layout(ws, n, k_exp, workers);
@@ -525,9 +528,22 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
     if (chunks * workers > kMaxExploreCtas) chunks = kMaxExploreCtas / workers;
     if (chunks > (k_exp + 1023) / 1024) chunks = (k_exp + 1023) / 1024;
     if (chunks == 0) chunks = 1;
+    if (lean && buckets <= kMaxSmemBuckets && 3 * buckets * 4 + 4096 < kGroupSmemLean) {
+        // more, smaller chunks, so that the scatter step can still group a chunk in the shared memory it gets
+        const uint64_t fit = (kGroupSmemLean - 3 * buckets * 4) / 4;
+        uint64_t need = (k_exp + fit - 1) / fit;
+        if (need * workers > kMaxExploreCtas) need = kMaxExploreCtas / workers;
+        if (need > chunks) chunks = need;
+    }
     const uint32_t chunk = (uint32_t)((k_exp + chunks - 1) / chunks);
     const dim3 grid((unsigned)chunks, workers);
     const bool smem = buckets <= kMaxSmemBuckets;
+    // part 1 may run beside another kernel's CTAs on the same SMs: one shared-memory split for all
+    if (!prefer_max_shared(rank_kernel<true>) || !prefer_max_shared(rank_kernel<false>) ||
+        !prefer_max_shared(scatter_kernel<true, true>) || !prefer_max_shared(scatter_kernel<true, false>) ||
+        !prefer_max_shared(scatter_kernel<false, false>) || !prefer_max_shared(bucket_sort_kernel) ||
+        !prefer_max_shared(explore_setup_kernel))
+        return SLIMDP_ERR_CUDA;
     if (smem) {
         rank_kernel<true><<<grid, 1024, buckets * 4, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, bits, s,
                                                            (uint32_t)buckets, L.round_keys, L.rho, L.rho_stride,
@@ -542,7 +558,7 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
         launch_block_scan(L.cnt, L.pref, L.tile_sums, L.totals, buckets, workers, L.cnt_stride, L.tile_stride, st);
     if (rc != SLIMDP_OK) return rc;
     const size_t group_smem = (3 * buckets + chunk) * 4;
-    if (smem && group_smem <= kGroupSmemMax) {
+    if (smem && group_smem <= (lean ? kGroupSmemLean : kGroupSmemMax)) {
         if (group_smem > 48 * 1024 &&
             cudaFuncSetAttribute(scatter_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)group_smem) != cudaSuccess)
@@ -578,7 +594,8 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
 slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                              uint32_t first_worker, uint32_t workers, uint32_t round,
                              const PtrArray<uint32_t>& out, void* ws, cudaStream_t st) {
-    return launch_explore_parts(core_aux, n, k_core, k_exp, seed, first_worker, workers, round, out, ws, 3, st);
+    return launch_explore_parts(core_aux, n, k_core, k_exp, seed, first_worker, workers, round, out, ws, 3, false,
+                                st);
 }
 
 // ---- explorer sampling without a caller-supplied workspace ---------------------------------

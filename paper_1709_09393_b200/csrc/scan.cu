@@ -45,6 +45,7 @@ slimdp_status launch_block_scan(const unsigned long long* cnt, unsigned long lon
                                 uint32_t batch, uint64_t stride, uint64_t tile_stride, cudaStream_t st) {
     const uint32_t tiles = (uint32_t)((nb + kScanTile - 1) / kScanTile);
     dim3 grid(tiles, batch);
+    if (!prefer_max_shared(tile_sum_kernel) || !prefer_max_shared(tile_scan_kernel)) return SLIMDP_ERR_CUDA;
     tile_sum_kernel<<<grid, 1024, 0, st>>>(cnt, tile_sums, nb, stride, tile_stride);
     tile_scan_kernel<<<grid, 1024, 0, st>>>(cnt, tile_sums, pref, totals, nb, stride, tile_stride);
     SLIMDP_LAUNCHED(2);

@@ -504,6 +504,214 @@ __global__ void __launch_bounds__(256, 4) score_bracket_kernel(const float* __re
     if (threadIdx.x == 0 && cta_def) atomicAdd(&hdr->n_def, cta_def);
 }
 
+// ---- the same pass with its loads kept in flight in shared memory ---------------------------
+//
+// The pass above keeps a row's 16-byte loads in registers, so the bytes in flight per SM are
+// bounded by the registers of its 32 resident warps, and it leaves other kernels no room on the
+// SM.  Here every lane copies its 16 bytes of each tensor straight into a per-warp ring in
+// shared memory (cp.async, no registers) and reads them back S rows later: 8 warps per SM keep
+// S rows each in flight, which saturates the memory system with one CTA per SM and a fraction
+// of the register file.  The rest of the SM is free for the kernels that run beside the pass.
+// A lane reads only what it copied itself, so waiting for its own copy groups is all the
+// synchronisation the ring needs.
+
+// 16 bytes from global to shared memory without a register in between.  `policy` marks the line
+// as the first to leave L2 (the pass reads every byte once), and the copy asks for whole 128-byte lines.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, uint64_t policy) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint.L2::128B [%0], [%1], 16, %2;" ::"r"(d), "l"(gmem_src),
+                 "l"(policy)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
+}
+
+// Ring bytes per CTA: as many stages as fit the first budget, which leaves the kernels beside the
+// pass about 100 KB of the SM's shared memory; with many workers, two stages within the second.
+constexpr uint32_t kAsyncRingBudget = 112u * 1024u, kAsyncRingBudgetMax = 176u * 1024u;
+
+// Candidate staging of a CTA of `warps` warps, as in the pass above.
+inline uint32_t async_cand_bytes(uint32_t warps) { return warps * 2u * kFusedStage * 4u; }
+// Bytes of one ring stage of a CTA: a row of 128 parameters of the model and the K updates per warp.
+inline uint32_t async_stage_bytes(uint32_t K, uint32_t warps) { return warps * (K + 1u) * 512u; }
+// Stages the ring gets for K workers and `warps` warps per CTA (0: this pass does not apply:
+// a stage is too large, or the rows are too short to keep enough bytes in flight).
+inline int async_stages(uint32_t K, uint32_t warps) {
+    const uint32_t stage = async_stage_bytes(K, warps);
+    uint32_t s = kAsyncRingBudget / stage;
+    if (s < 2 && 2 * stage <= kAsyncRingBudgetMax) s = 2;
+    if (s > 8) s = 8;   // the copies run at most one block ahead of the arithmetic
+    if (s < 2 || s * stage < 64u * 1024u) return 0;
+    return (int)s;
+}
+
+// S ring stages per warp, W warps per CTA.
+template <int S, int W>
+__global__ void __launch_bounds__(W * 32, 2)
+    score_bracket_async_kernel(const float* __restrict__ w, PtrArray<const float> g, int K, float c, uint64_t n,
+                               uint64_t nb, WsHeader* hdr, uint32_t cap, uint32_t* __restrict__ G,
+                               uint32_t* __restrict__ E, unsigned long long* __restrict__ cnt,
+                               uint32_t* __restrict__ cand_key, uint32_t* __restrict__ cand_idx) {
+    static_assert(S >= 2 && S <= 8, "the copies stay within the block after the one being processed");
+    extern __shared__ __align__(16) uint32_t async_smem[];
+    __shared__ uint32_t cta_def;
+    const uint32_t b_top = hdr->b_top, b_bot = hdr->b_bot;
+    const uint32_t lane = lane_id(), wid = threadIdx.x >> 5;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    uint32_t* my_key = async_smem + wid * kFusedStage;
+    uint32_t* my_idx = async_smem + (W + wid) * kFusedStage;
+    const uint32_t stage_f4 = (uint32_t)(K + 1) * 32u;   // 16-byte words of one stage of one warp
+    float4* ring = reinterpret_cast<float4*>(async_smem + 2 * W * kFusedStage) + (size_t)wid * S * stage_f4;
+    if (threadIdx.x == 0) cta_def = 0;
+    __syncthreads();
+    uint32_t staged = 0, def_acc = 0;
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    auto flush = [&](uint32_t m) {
+        uint32_t base = 0;
+        if (lane == 0) base = atomicAdd(&hdr->n_cand, m);
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        if ((uint64_t)base + m <= cap) {   // else: overflow, n_cand > cap sends the call down the full path
+            for (uint32_t e = lane; e < m; e += 32) {
+                cand_key[base + e] = my_key[e];
+                cand_idx[base + e] = my_idx[e];
+            }
+        }
+        __syncwarp();
+    };
+    const bool has_top = b_top < 65536u;
+    const uint32_t top_key = has_top ? (b_top << 16) : 0xFFFFFFFFu;
+    const uint32_t bot_key = b_bot << 16;
+    // Blocks are handed out on request, one at a time per warp (other kernels share the SMs, so
+    // warps advance at different speeds).  A warp knows the block it works on and the next one;
+    // the request for the one after that is in flight meanwhile.
+    auto request_block = [&]() {
+        uint32_t b = 0;
+        if (lane == 0) b = atomicAdd(&hdr->next_block, 1u);
+        return b;
+    };
+    uint64_t blk = __shfl_sync(0xFFFFFFFFu, request_block(), 0);
+    uint64_t blk_next = __shfl_sync(0xFFFFFFFFu, request_block(), 0);
+    uint32_t requested = request_block();
+    // the copies: row `copy_row` of block (copy_ahead ? blk_next : blk) goes to stage `copy_slot`
+    uint32_t copy_ahead = 0, copy_row = 0, copy_slot = 0, slot = 0;
+    auto copy_next_row = [&]() {
+        const uint64_t b = copy_ahead ? blk_next : blk;
+        if (b < nb && (b + 1) * kBlock <= n) {   // whole blocks only; the ragged last block is loaded directly
+            const uint64_t i4 = (b * kBlock + copy_row * 128u) / 4u + lane;
+            float4* dst = ring + copy_slot * stage_f4 + lane;
+            for (int k = 0; k < K; ++k)
+                cp_async16(dst + k * 32, reinterpret_cast<const float4*>(g.p[k]) + i4, policy);
+            cp_async16(dst + K * 32, reinterpret_cast<const float4*>(w) + i4, policy);
+        }
+        cp_async_commit();   // one group per row, empty or not, so that the group count tells the row
+        copy_slot = (copy_slot + 1 == S) ? 0 : copy_slot + 1;
+        if (++copy_row == 8) {
+            copy_row = 0;
+            ++copy_ahead;
+        }
+    };
+#pragma unroll 1
+    for (int s0 = 0; s0 < S; ++s0) copy_next_row();
+    while (blk < nb) {
+        const uint64_t base = blk * kBlock;
+        const bool full = base + kBlock <= n;
+        uint32_t myG = 0;
+#pragma unroll 1
+        for (uint32_t r = 0; r < 8; ++r) {
+            const uint64_t e0 = base + r * 128 + 4 * lane;   // this lane's first parameter of the row
+            uint32_t key[4];
+            uint32_t in = 0xFu;                               // which of the four exist
+            cp_async_wait<S - 1>();                           // this row's copies have landed
+            if (full) {
+                const float4* src = ring + slot * stage_f4 + lane;
+                float4 a = src[0];
+#pragma unroll 4
+                for (int k = 1; k < K; ++k) {
+                    const float4 b = src[k * 32];
+                    a.x = __fadd_rn(a.x, b.x);
+                    a.y = __fadd_rn(a.y, b.y);
+                    a.z = __fadd_rn(a.z, b.z);
+                    a.w = __fadd_rn(a.w, b.w);
+                }
+                const float4 ww = src[K * 32];
+                key[0] = __float_as_uint(score_one(c, a.x, ww.x));
+                key[1] = __float_as_uint(score_one(c, a.y, ww.y));
+                key[2] = __float_as_uint(score_one(c, a.z, ww.z));
+                key[3] = __float_as_uint(score_one(c, a.w, ww.w));
+            } else if (e0 + 4 <= n) {
+                score4<0>(w, g, K, c, e0 / 4, key);
+            } else {
+                in = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    key[q] = 0;
+                    if (e0 + q < n) {
+                        key[q] = score1(w, g, K, c, e0 + q);
+                        in |= 1u << q;
+                    }
+                }
+            }
+            slot = (slot + 1 == S) ? 0 : slot + 1;
+            copy_next_row();   // into the stage just read
+            uint32_t nib = 0, cm = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const bool ex = (in >> q) & 1u;
+                const bool def = has_top && key[q] >= top_key && ex;
+                const bool cand = key[q] >= bot_key && !def && ex;
+                nib |= (uint32_t)def << q;
+                cm |= (uint32_t)cand << q;
+            }
+            // the row's four bitmap words: lanes 8j .. 8j+7 assemble word j, lane 4r + j keeps it
+            uint32_t word = nib << (4 * (lane & 7u));
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
+            const uint32_t got = __shfl_sync(0xFFFFFFFFu, word, (lane & 3u) * 8);
+            if ((lane >> 2) == r) myG = got;
+            if (__any_sync(0xFFFFFFFFu, cm != 0)) {   // warp-uniform: most rows hold no candidate
+                uint32_t place = staged;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const bool cand = (cm >> q) & 1u;
+                    const uint32_t bc = __ballot_sync(0xFFFFFFFFu, cand);
+                    if (cand) {
+                        const uint32_t at = place + __popc(bc & lt_mask);
+                        my_key[at] = key[q];
+                        my_idx[at] = (uint32_t)e0 + q;
+                    }
+                    place += __popc(bc);
+                }
+                staged = place;
+                __syncwarp();
+                if (staged >= kFlushAt) {
+                    flush(staged);
+                    staged = 0;
+                }
+            }
+        }
+        G[blk * kWordsPerBlock + lane] = myG;
+        E[blk * kWordsPerBlock + lane] = 0u;
+        const uint32_t cg = __reduce_add_sync(0xFFFFFFFFu, __popc(myG));
+        if (lane == 0) cnt[blk] = cg;
+        def_acc += cg;
+        // on to the next block; the copies are S rows into it already
+        blk = blk_next;
+        blk_next = __shfl_sync(0xFFFFFFFFu, requested, 0);
+        requested = request_block();
+        --copy_ahead;
+    }
+    cp_async_wait<0>();
+    if (staged) flush(staged);
+    if (lane == 0 && def_acc) atomicAdd(&cta_def, def_acc);
+    __syncthreads();
+    if (threadIdx.x == 0 && cta_def) atomicAdd(&hdr->n_def, cta_def);
+}
+
 // The scores for the full path, written only when the bracket failed.
 __global__ void __launch_bounds__(256) score_if_bracket_failed_kernel(const float* __restrict__ w,
                                                                       PtrArray<const float> g, int K, float c,
@@ -779,6 +987,8 @@ struct FusedScore {
     // streams from here on finds the pass's CTAs already placed
     slimdp_status (*after_pass)(void*);
     void* after_arg;
+    cudaEvent_t pass_ready;   // recorded just before the pass is enqueued when not null: work that is to run
+                              // beside the pass, not before it, waits for this
 };
 
 // A second stream for the full path's kernels.  After the bracket pass exactly one of the two
@@ -822,21 +1032,49 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
                                                                         L.coarse_incl);
         if (fused) {
             if (fused->mark_begin && cudaEventRecord(fused->mark_begin, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
-            uint64_t fgrid = (nb + 7) / 8;
-            // The pass is bound by memory bandwidth, which four fifths of the SMs saturate; its CTAs
-            // stay resident from start to end, so the SMs it leaves free are what lets the explorer's
-            // rank kernels (queued beside it on the round's side stream) run at the same time.
-            const uint64_t fmax = 4ull * (uint64_t)(sms - sms / 5);
-            if (fgrid > fmax) fgrid = fmax;
+            if (fused->pass_ready && cudaEventRecord(fused->pass_ready, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
+            constexpr uint32_t warps = 8;
+            const int stages = async_stages(fused->K, warps);
+            if (stages > 0) {
+                // one CTA per SM, its loads in flight in shared memory (see score_bracket_async_kernel)
+                const uint32_t smem = async_cand_bytes(warps) + (uint32_t)stages * async_stage_bytes(fused->K, warps);
+                uint64_t agrid = (nb + warps - 1) / warps;
+                if (agrid > (uint64_t)sms) agrid = (uint64_t)sms;
+#define SLIMDP_ASYNC_CASE(SS)                                                                                       \
+    case SS: {                                                                                                      \
+        auto kern = score_bracket_async_kernel<SS, warps>;                                                          \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||    \
+            !prefer_max_shared(kern))                                                                               \
+            return SLIMDP_ERR_CUDA;                                                                                 \
+        kern<<<(unsigned)agrid, warps * 32, smem, st>>>(fused->w, *fused->g, (int)fused->K, fused->c, n, nb, L.hdr, \
+                                                        cap, L.G, L.E, L.cnt, L.cand_key, L.cand_idx);              \
+    } break
+                switch (stages) {
+                    SLIMDP_ASYNC_CASE(2);
+                    SLIMDP_ASYNC_CASE(3);
+                    SLIMDP_ASYNC_CASE(4);
+                    SLIMDP_ASYNC_CASE(5);
+                    SLIMDP_ASYNC_CASE(6);
+                    SLIMDP_ASYNC_CASE(7);
+                    SLIMDP_ASYNC_CASE(8);
+                    default: return SLIMDP_ERR_INTERNAL;
+                }
+#undef SLIMDP_ASYNC_CASE
+            } else {
+                // very many workers (a ring stage would not fit) or very few (too few bytes per row)
+                uint64_t fgrid = (nb + 7) / 8;
+                const uint64_t fmax = 4ull * (uint64_t)sms;
+                if (fgrid > fmax) fgrid = fmax;
 #define SLIMDP_FUSED_CASE(KK)                                                                                     \
     score_bracket_kernel<KK><<<(unsigned)fgrid, 256, 0, st>>>(fused->w, *fused->g, (int)fused->K, fused->c, n, nb, \
                                                               L.hdr, cap, L.G, L.E, L.cnt, L.cand_key, L.cand_idx)
-            switch (fused->K) {
-                case 4: SLIMDP_FUSED_CASE(4); break;
-                case 8: SLIMDP_FUSED_CASE(8); break;
-                default: SLIMDP_FUSED_CASE(0);
-            }
+                switch (fused->K) {
+                    case 4: SLIMDP_FUSED_CASE(4); break;
+                    case 8: SLIMDP_FUSED_CASE(8); break;
+                    default: SLIMDP_FUSED_CASE(0);
+                }
 #undef SLIMDP_FUSED_CASE
+            }
             if (fused->mark_end && cudaEventRecord(fused->mark_end, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
             if (fused->after_pass) {
                 const slimdp_status hs = fused->after_pass(fused->after_arg);
@@ -904,8 +1142,8 @@ slimdp_status launch_score_select(const float* w, const PtrArray<const float>& g
                                   float* scores, uint64_t k_core, uint32_t* core_idx, void* core_aux, void* ws,
                                   cudaEvent_t mark_begin, cudaEvent_t mark_end, cudaStream_t gate_stream,
                                   cudaEvent_t gate_fork, cudaEvent_t gate_join, slimdp_status (*after_pass)(void*),
-                                  void* after_arg, cudaStream_t st) {
-    const FusedScore f{w, &g, K, c, mark_begin, mark_end, after_pass, after_arg};
+                                  void* after_arg, cudaEvent_t pass_ready, cudaStream_t st) {
+    const FusedScore f{w, &g, K, c, mark_begin, mark_end, after_pass, after_arg, pass_ready};
     const GateStream gs{gate_stream, gate_fork, gate_join};
     return launch_select_impl(scores, n, k_core, core_idx, core_aux, ws, &f, gate_stream ? &gs : nullptr, st);
 }
