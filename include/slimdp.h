@@ -314,17 +314,21 @@ uint64_t slimdp_launch_count(void);
  *     scores around the threshold) and is left untouched otherwise.  Callers
  *     that want the scores call slimdp_score.
  *   - The steps of a round depend on one another as a graph, not a chain: the
- *     explorer's ranks need the sizes only, so they run beside scoring and
- *     selection; and of the selection's two ways to the threshold (from the
- *     candidates, or from all scores when the bracket failed) only one does
- *     any work, so the idle one's kernels run beside the other's.  For that
- *     this call keeps, per device, TWO non-blocking streams and four events of
- *     its own, created on the first call on that device and kept for the life
- *     of the process (the one exception to "creates no stream").  Both side
- *     branches fork from `stream` inside the call and are joined back into it
- *     inside the call, so for the caller the whole round is ordered on
- *     `stream` as usual.  Calls on one device are serialised on the host by a
- *     lock while they enqueue.
+ *     explorer's ranks need the sizes only, so they are computed and sorted
+ *     beside the pass over all parameters, in the part of every SM that the
+ *     pass leaves free (the pass keeps its loads in flight in shared memory,
+ *     one CTA per SM, and so needs few registers and threads); and of the
+ *     selection's two ways to the threshold (from the candidates, or from all
+ *     scores when the bracket failed) only one does any work, so the idle
+ *     one's kernels run beside the other's.  For that this call keeps, per
+ *     device, THREE non-blocking streams and six events of its own, created on
+ *     the first call on that device and kept for the life of the process (the
+ *     one exception to "creates no stream"): one of the highest priority for
+ *     the chain of kernels that decides the round's time, one of the lowest
+ *     for the ranks, one for the idle way.  `stream` forks into them at the
+ *     start of the call and waits for them at the end, inside the call, so
+ *     for the caller the whole round is ordered on `stream` as usual.  Calls
+ *     on one device are serialised on the host by a lock while they enqueue.
  *   w_global [n] (updated in place); grads HOST array of K device pointers [n] (read)
  *   scores [n] scratch (see above); core_idx [k_core], core_aux (written; as slimdp_select_core)
  *   exp_idx HOST array of K device pointers [k_exp] (written)

@@ -913,10 +913,22 @@ __global__ void __launch_bounds__(256) emit_kernel(const uint32_t* __restrict__ 
         if (ng + min(ne, ties) != k_core) hdr->status = SLIMDP_ERR_INTERNAL;
         dir[nb * kDirPerBlock] = (uint32_t)(n - k_core);
     }
+    // the next block's words are requested before this block's are worked on
+    uint32_t Gn = 0, En = 0;
+    unsigned long long pn = 0;
+    if (warp0 < nb) {
+        Gn = __ldcs(G + warp0 * kWordsPerBlock + lane);
+        En = __ldcs(E + warp0 * kWordsPerBlock + lane);
+        pn = __ldcs(pref + warp0);
+    }
     for (uint64_t blk = warp0; blk < nb; blk += warps) {
-        const uint32_t Gw = G[blk * kWordsPerBlock + lane];
-        const uint32_t Ew = E[blk * kWordsPerBlock + lane];
-        const unsigned long long p = pref[blk];
+        const uint32_t Gw = Gn, Ew = En;
+        const unsigned long long p = pn;
+        if (blk + warps < nb) {
+            Gn = __ldcs(G + (blk + warps) * kWordsPerBlock + lane);
+            En = __ldcs(E + (blk + warps) * kWordsPerBlock + lane);
+            pn = __ldcs(pref + blk + warps);
+        }
         const uint32_t g_before = (uint32_t)p, e_before = (uint32_t)(p >> 32);
         // equal keys: admit those whose rank among all equal keys (index order) is below r
         const uint32_t pe = __popc(Ew);
