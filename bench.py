@@ -394,9 +394,10 @@ def run_ours(args):
         torch.distributed.destroy_process_group()
 
 
-# DRAM bytes (read + write) of one score launch, per workload, from an ncu capture of the same
-# kernel on the leading 40 M parameters (38.88 B per parameter), scaled to the full launch.
-TRAFFIC_DOMINANT_BYTES: dict = {}
+# DRAM bytes (read + write) of one launch of the fused pass, per workload: from an ncu capture of the
+# same kernel on the leading 40 M parameters of the workload (1448.0 MB = 36.20 B per parameter;
+# traffic grows in proportion to n), scaled to the full launch of 138 357 544 parameters.
+TRAFFIC_DOMINANT_BYTES: dict = {"vgg16": 5_008_632_000}
 
 
 def main():

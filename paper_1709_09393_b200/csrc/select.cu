@@ -343,44 +343,54 @@ __device__ __forceinline__ uint32_t score1(const float* __restrict__ w, const Pt
 
 // Sample kernel A of the fused path: 2^16 evenly spaced groups of four consecutive parameters
 // are scored (2^18 sampled keys, one 16-byte load per tensor and group); the rest is
-// sample_coarse_kernel's.  Needs n >= 4 and 16-byte aligned tensors.
-__global__ void __launch_bounds__(256) sample_score_coarse_kernel(const float* __restrict__ w,
-                                                                   PtrArray<const float> g, int K, float c,
-                                                                   uint64_t n, uint32_t k, WsHeader* hdr,
-                                                                   uint32_t* __restrict__ sample,
-                                                                   uint32_t* __restrict__ coarse_hist,
-                                                                   uint32_t* __restrict__ coarse_incl) {
+// sample_coarse_kernel's.  Needs n >= 4 and 16-byte aligned tensors.  1024 groups per CTA: the
+// sampled keys fall into a handful of coarse bins, and every CTA adds to those few global
+// counters, so few large CTAs queue up less there than many small ones.
+__global__ void __launch_bounds__(1024) sample_score_coarse_kernel(const float* __restrict__ w,
+                                                                    PtrArray<const float> g, int K, float c,
+                                                                    uint64_t n, uint32_t k, WsHeader* hdr,
+                                                                    uint32_t* __restrict__ sample,
+                                                                    uint32_t* __restrict__ coarse_hist,
+                                                                    uint32_t* __restrict__ coarse_incl) {
     __shared__ unsigned long long smem[33];
     __shared__ uint32_t sh_coarse[256];
     __shared__ long long s_incl[257];
     const uint32_t t = threadIdx.x;
-    sh_coarse[t] = 0;   // 256 threads
+    if (t < 256) sh_coarse[t] = 0;
     __syncthreads();
-    const uint32_t j = blockIdx.x * 256 + t;   // group number, < 2^16
+    const uint32_t j = blockIdx.x * 1024 + t;   // group number, < 2^16
     uint32_t key[4];
     score4<0>(w, g, K, c, ((uint64_t)j * (n / 4)) >> (kSampleBits - 2), key);
     reinterpret_cast<uint4*>(sample)[j] = make_uint4(key[0], key[1], key[2], key[3]);
+    // most of a warp's keys share a coarse bin: one shared-memory atomic per distinct bin and warp
 #pragma unroll
-    for (int q = 0; q < 4; ++q) atomicAdd(&sh_coarse[key[q] >> 24], 1u);
+    for (int q = 0; q < 4; ++q) {
+        const uint32_t bin = key[q] >> 24;
+        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, bin);
+        if ((peers & ((1u << lane_id()) - 1u)) == 0) atomicAdd(&sh_coarse[bin], (uint32_t)__popc(peers));
+    }
     __syncthreads();
-    if (sh_coarse[t]) atomicAdd(&coarse_hist[t], sh_coarse[t]);
+    if (t < 256 && sh_coarse[t]) atomicAdd(&coarse_hist[t], sh_coarse[t]);
     if (!last_cta_done(&hdr->ticket[6])) return;
     long long lo_target, hi_target;
     bracket_targets(k, n, &lo_target, &hi_target);
+    // coarse bins from the top down: thread t < 256 owns coarse bin 255 - t
     unsigned long long total;
-    const unsigned long long cc = __ldcg(coarse_hist + 255 - t);
-    const long long c_above = (long long)block_exclusive_scan64<8>(cc, smem, &total);
-    s_incl[255 - t] = c_above + (long long)cc;
+    const unsigned long long cc = (t < 256) ? __ldcg(coarse_hist + 255 - t) : 0ull;
+    const long long c_above = (long long)block_exclusive_scan64<32>(cc, smem, &total);
+    if (t < 256) s_incl[255 - t] = c_above + (long long)cc;
     if (t == 0) {
         s_incl[256] = 0;
         hdr->coarse_x[0] = 0xFFFFFFFFu;
         hdr->coarse_x[1] = 0xFFFFFFFFu;
     }
     __syncthreads();
-    const long long incl = s_incl[t], above = s_incl[t + 1];
-    coarse_incl[t] = (uint32_t)incl;
-    if (incl > lo_target && above <= lo_target) hdr->coarse_x[0] = t;
-    if (incl >= hi_target && above < hi_target) hdr->coarse_x[1] = t;
+    if (t < 256) {
+        const long long incl = s_incl[t], above = s_incl[t + 1];
+        coarse_incl[t] = (uint32_t)incl;
+        if (incl > lo_target && above <= lo_target) hdr->coarse_x[0] = t;
+        if (incl >= hi_target && above < hi_target) hdr->coarse_x[1] = t;
+    }
 }
 
 constexpr uint32_t kFusedStage = kFlushAt + 128;   // below kFlushAt before a row of 128 parameters, +128 in it
@@ -1035,7 +1045,7 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
     cudaStream_t fs = st;   // the stream of the full path's kernels
     if (bracketed) {
         if (fused)
-            sample_score_coarse_kernel<<<(1u << (kSampleBits - 2)) / 256, 256, 0, st>>>(
+            sample_score_coarse_kernel<<<(1u << (kSampleBits - 2)) / 1024, 1024, 0, st>>>(
                 fused->w, *fused->g, (int)fused->K, fused->c, n, k, L.hdr, L.sample, L.coarse_hist, L.coarse_incl);
         else
             sample_coarse_kernel<<<(1u << kSampleBits) / 1024, 1024, 0, st>>>(keys, n, k, L.hdr, L.sample,
