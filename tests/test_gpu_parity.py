@@ -409,6 +409,21 @@ def test_round_one_call_fused_cases(P, case):
         assert np.array_equal(host_bits(buf.scores), bits(ref["scores"]))
 
 
+# The pass keeps its loads in a shared-memory ring whose depth follows the number of workers
+# (8 stages for K <= 2 down to 2 for K = 12..17); from K = 18 a ring stage no longer fits and the
+# register version of the pass runs.  One case per depth, and one on the other side of the limit.
+@pytest.mark.parametrize("K", [1, 2, 3, 5, 7, 12, 17, 18, 33])
+def test_round_one_call_any_worker_count(P, K):
+    n = FUSED_N + 2 * K      # n % 4 in {1, 3}
+    rng = np.random.default_rng(1000 + K)
+    w = (rng.standard_normal(n) * 0.05).astype(np.float32)
+    gs = [(rng.standard_normal(n) * 1e-2).astype(np.float32) for _ in range(K)]
+    k_core, k_exp = n // 16, n // 200
+    ref = oracle.run_round(w, gs, 1.0, k_core, k_exp, 9, 3, 1.0 / K)
+    d_w, buf = gpu_round(P, w, gs, 1.0, k_core, k_exp, 9, 3, 1.0 / K, one_call=True)
+    assert_round_equal(P, d_w, buf, ref, n, scores=False)
+
+
 def test_round_one_call_any_alignment(P):
     # tensors that start 4 bytes off a 16-byte boundary: the round scores and selects in two steps
     cfg = scaled_config(CONFIGS["vgg16"], FUSED_N)
