@@ -32,7 +32,9 @@ void count_launches(unsigned n) { g_launches.fetch_add(n, std::memory_order_rela
 slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<const float>& delta,
                               const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,
                               uint64_t k_exp, float eta, const PtrArray<float>& val, const PtrArray<float>& pulled,
-                              cudaStream_t st);
+                              const uint32_t* ranks, uint64_t rank_stride, const uint32_t* core_bitmap,
+                              const uint32_t* core_dir, int32_t* explore_status, cudaStream_t st);
+bool exchange_takes_ranks(uint64_t n, uint64_t k_exp);
 
 slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                    uint32_t first_worker, uint32_t workers, uint32_t round,
@@ -265,7 +267,8 @@ slimdp_status slimdp_exchange(float* w_global, uint64_t n, uint32_t K, const flo
     if (!fill<float>(v, val, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (!fill<float>(o, pulled, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (k_core + k_exp == 0) return SLIMDP_OK;
-    return launch_exchange(w_global, n, K, d, core_idx, k_core, exp, k_exp, eta, v, o, (cudaStream_t)stream);
+    return launch_exchange(w_global, n, K, d, core_idx, k_core, exp, k_exp, eta, v, o, nullptr, 0, nullptr, nullptr,
+                           nullptr, (cudaStream_t)stream);
 }
 
 slimdp_status slimdp_dense_merge_score(float* w_global, const float* const* grads, uint32_t K, float eta, float c,
@@ -443,12 +446,25 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
         if (rc == SLIMDP_OK && mark1) cuda(cudaEventRecord(mark1, ch));
         if (rc == SLIMDP_OK) step(launch_select(scores, n, k_core, core_idx, core_aux, select_ws, ch));
     }
-    // chain: explorer indices from the sorted ranks and the core, then the exchange
+    // chain: explorer indices from the sorted ranks and the core, then the exchange; where the
+    // exchange's warp ranges line up with the core's directory it computes the indices itself
     cuda(cudaStreamWaitEvent(ch, side->ranks_done, 0));
-    if (rc == SLIMDP_OK)
-        step(launch_explore_parts(core_aux, n, k_core, k_exp, seed, 0, K, round, exp_out, explore_ws, 2, false, ch));
-    if (rc == SLIMDP_OK && k_core + k_exp > 0)
-        step(launch_exchange(w_global, n, K, g, core_idx, k_core, exp_in, k_exp, eta, v, o, ch));
+    if (exchange_takes_ranks(n, k_exp)) {
+        const ExploreWs EL = explore_ws_layout(explore_ws, n, k_exp, K);
+        if (rc == SLIMDP_OK)
+            step(launch_exchange(w_global, n, K, g, core_idx, k_core, exp_in, k_exp, eta, v, o, EL.rho, EL.rho_stride,
+                                 reinterpret_cast<const uint32_t*>(core_aux),
+                                 reinterpret_cast<const uint32_t*>(static_cast<const char*>(core_aux) +
+                                                                   slimdp_core_aux_dir_offset(n)),
+                                 &EL.hdr->status, ch));
+    } else {
+        if (rc == SLIMDP_OK)
+            step(launch_explore_parts(core_aux, n, k_core, k_exp, seed, 0, K, round, exp_out, explore_ws, 2, false,
+                                      ch));
+        if (rc == SLIMDP_OK && k_core + k_exp > 0)
+            step(launch_exchange(w_global, n, K, g, core_idx, k_core, exp_in, k_exp, eta, v, o, nullptr, 0, nullptr,
+                                 nullptr, nullptr, ch));
+    }
     if (cudaEventRecord(side->chain_done, ch) != cudaSuccess || cudaStreamWaitEvent(st, side->chain_done, 0) != cudaSuccess)
         step(SLIMDP_ERR_CUDA);
     return rc;

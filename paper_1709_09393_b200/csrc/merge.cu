@@ -215,6 +215,162 @@ __device__ __forceinline__ void exchange_explore_body(float* w, const PtrArray<c
     if (sink == 0x9E3779B9u && lane >= 32) w[0] = 0.0f;   // never true: keeps the early requests alive
 }
 
+// ---- explorer segments straight from the sorted ranks ---------------------------------------
+//
+// A worker's explorer is { select0(r) : r in its sorted ranks }, select0(r) the r-th parameter
+// outside the core.  A warp that owns the parameter range [a, a + 2^shift) owns exactly the ranks
+// in [dir(a), dir(a + 2^shift)), dir(x) the number of non-core parameters below x, which the
+// core's directory holds for every multiple of 64.  Inside the range select0 is local: the
+// range's directory entries (one per lane, at most 32 groups of 64 parameters) and bitmap words
+// (two per lane) are all it needs.  So the warp turns its ranks into indices itself, writes them
+// out as the explorer (ascending, since the ranks are) and goes on as exchange_explore_body; the
+// separate pass that turns all ranks into indices, and the wait for it, fall away.
+struct RankSource {
+    const uint32_t* ranks;    // worker k's sorted ranks at ranks + k * stride
+    uint64_t stride;
+    const uint32_t* bitmap;   // core bitmap, 32 words per 1024-parameter block
+    const uint32_t* dir;      // dir[d] = non-core parameters below 64 d, d <= nd; dir[nd] = n - k_core
+    uint32_t nd;
+    int32_t* status;          // the explorer workspace's status word
+};
+
+// First position in a[0, len) whose value is >= x (plain loads: `a` may have been written by this grid's predecessor only).
+__device__ __forceinline__ uint32_t lower_bound_ranks(const uint32_t* __restrict__ a, uint32_t len, uint32_t x) {
+    uint32_t lo = 0, hi = len;
+    while (lo < hi) {
+        const uint32_t mid = lo + ((hi - lo) >> 1);
+        if (__ldg(a + mid) < x)
+            lo = mid + 1;
+        else
+            hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ void exchange_explore_ranks_body(float* w, const RankSource& src,
+                                                            const PtrArray<const uint32_t>& exp, uint32_t k_exp,
+                                                            const PtrArray<const float>& delta,
+                                                            const PtrArray<float>& val, const PtrArray<float>& pulled,
+                                                            uint64_t k_core, int K, float neg_eta,
+                                                            uint32_t range_shift, uint64_t vblock,
+                                                            uint32_t (*bound)[kMergeWarps + 1]) {
+    const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
+    const uint32_t groups = 1u << (range_shift - 6);   // 64-parameter groups per warp range, 1 .. 32
+    const uint64_t first_group = (vblock * kMergeWarps) << (range_shift - 6);
+    // where the CTA's 9 range boundaries fall in every worker's sorted ranks
+    for (int t = threadIdx.x; t < K * (kMergeWarps + 1); t += blockDim.x) {
+        const int k = t / (kMergeWarps + 1), r = t % (kMergeWarps + 1);
+        const uint64_t d = first_group + (uint64_t)r * groups;
+        const uint32_t rank_lo = __ldg(src.dir + (d < src.nd ? d : src.nd));
+        bound[k][r] = lower_bound_ranks(src.ranks + (uint64_t)k * src.stride, k_exp, rank_lo);
+    }
+    __syncthreads();
+    // this warp's piece of the directory and of the bitmap: lane l holds group l of the range
+    const uint64_t my_group = first_group + (uint64_t)wid * groups + lane;
+    const bool have_group = lane < groups && my_group < src.nd;
+    const uint32_t dl = have_group ? __ldg(src.dir + my_group) : 0xFFFFFFFFu;
+    const uint2 words = have_group ? __ldg(reinterpret_cast<const uint2*>(src.bitmap) + my_group) : make_uint2(0u, 0u);
+    const uint32_t group0 = (uint32_t)(first_group + (uint64_t)wid * groups);
+    bool bad = false;
+    // rank -> parameter index inside this warp's range; every lane takes part (shuffles), `ok` says
+    // whether the lane's rank is real
+    auto select0_local = [&](uint32_t r, bool ok) -> uint32_t {
+        uint32_t lo = 0, hi = groups - 1;   // largest group g with dl[g] <= r
+#pragma unroll
+        for (int step = 0; step < 5; ++step) {
+            const uint32_t mid = lo + ((hi - lo + 1) >> 1);
+            const uint32_t v = __shfl_sync(0xFFFFFFFFu, dl, (int)mid);
+            if (lo < hi) {
+                if (v <= r)
+                    lo = mid;
+                else
+                    hi = mid - 1;
+            }
+        }
+        const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, dl, (int)lo);
+        const uint32_t w0 = __shfl_sync(0xFFFFFFFFu, words.x, (int)lo);
+        const uint32_t w1 = __shfl_sync(0xFFFFFFFFu, words.y, (int)lo);
+        const uint32_t rem = r - d0;
+        const uint32_t z0 = ~w0, z1 = ~w1;
+        const uint32_t c0 = __popc(z0);
+        const bool second = rem >= c0;
+        const uint32_t z = second ? z1 : z0;
+        const uint32_t rr = second ? rem - c0 : rem;
+        // the directory and the bitmap disagree, or the rank does not belong to this range
+        if (ok && (r < d0 || rr >= (uint32_t)__popc(z))) bad = true;
+        return (group0 + lo) * 64u + (second ? 32u : 0u) + nth_set_bit(z, (ok && !bad) ? rr : 0u);
+    };
+    // indices of every worker's entries in the range, written out as the explorer; early requests of
+    // the model and update values they name, 8 workers' worth in flight together
+    uint32_t sink = 0;
+    for (int k0 = 0; k0 < K; k0 += 8) {
+        uint32_t i[8], v[16];
+        bool ok[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int k = k0 + q;
+            ok[q] = false;
+            i[q] = 0;
+            if (k < K) {   // warp-uniform
+                const uint32_t e = bound[k][wid] + lane;
+                ok[q] = e < bound[k][wid + 1];
+                const uint32_t r = ok[q] ? __ldg(src.ranks + (uint64_t)k * src.stride + e) : 0u;
+                i[q] = select0_local(r, ok[q]);
+                ok[q] = ok[q] && !bad;
+                if (ok[q]) const_cast<uint32_t*>(exp.p[k])[e] = i[q];
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            v[2 * q] = ok[q] ? touch(w + i[q]) : 0u;
+            v[2 * q + 1] = ok[q] ? touch(delta.p[k0 + q] + i[q]) : 0u;
+        }
+#pragma unroll
+        for (int q = 0; q < 16; ++q) sink ^= v[q];
+        // the rare worker with more than 32 entries in this range
+        for (int q = 0; q < 8 && k0 + q < K; ++q) {
+            const int k = k0 + q;
+            const uint32_t hi = bound[k][wid + 1];
+            for (uint32_t e0 = bound[k][wid] + 32; e0 < hi; e0 += 32) {   // warp-uniform bounds
+                const uint32_t e = e0 + lane;
+                const bool more = e < hi;
+                const uint32_t r = more ? __ldg(src.ranks + (uint64_t)k * src.stride + e) : 0u;
+                const uint32_t j = select0_local(r, more);
+                if (more && !bad) {
+                    const_cast<uint32_t*>(exp.p[k])[e] = j;
+                    sink ^= touch(w + j);
+                    sink ^= touch(delta.p[k] + j);
+                }
+            }
+        }
+    }
+    if (__any_sync(0xFFFFFFFFu, bad)) {
+        if (lane == 0) *src.status = SLIMDP_ERR_INTERNAL;
+        return;   // the whole warp: nothing of this range is exchanged
+    }
+    __syncwarp();
+    for (int k = 0; k < K; ++k) {
+        const uint32_t* idx = exp.p[k];   // plain loads: this thread reads back the entries it wrote itself
+        const float* __restrict__ d = delta.p[k];
+        float* __restrict__ v = val.p[k] + k_core;
+        const uint32_t b = bound[k][wid + 1];
+        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) {
+            const uint32_t i = idx[e];
+            const float u = ld_sparse(d + i);
+            __stcs(v + e, u);
+            w[i] = __fmaf_rn(neg_eta, u, ld_sparse(w + i));
+        }
+        __syncwarp();   // worker k's updates are visible to the whole warp before worker k+1 starts
+    }
+    for (int k = 0; k < K; ++k) {
+        const uint32_t* idx = exp.p[k];
+        float* __restrict__ o = pulled.p[k] + k_core;
+        const uint32_t b = bound[k][wid + 1];
+        for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) __stcs(o + e, ld_sparse(w + idx[e]));
+    }
+    if (sink == 0x9E3779B9u && lane >= 32) w[0] = 0.0f;   // never true: keeps the early requests alive
+}
+
 // One launch for both segments.  The core segment streams whole lines of the dense layers and is
 // bound by DRAM bandwidth; the explorer segments issue sparse accesses and are bound by their
 // latency and rate.  CTAs of both kinds are interleaved in the grid (core_ctas of every
@@ -224,16 +380,22 @@ __global__ void __launch_bounds__(256) exchange_kernel(float* w, const uint32_t*
                                                        uint64_t k_core, PtrArray<const uint32_t> exp, uint32_t k_exp,
                                                        PtrArray<const float> delta, PtrArray<float> val,
                                                        PtrArray<float> pulled, int K, float neg_eta,
-                                                       uint32_t range_shift, uint64_t core_ctas, uint64_t total_ctas) {
+                                                       uint32_t range_shift, uint64_t core_ctas, uint64_t total_ctas,
+                                                       RankSource from_ranks) {
     __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
     const uint64_t b = blockIdx.x;
     const uint64_t core_before = b * core_ctas / total_ctas;            // core CTAs among blocks [0, b)
     const bool is_core = (b + 1) * core_ctas / total_ctas > core_before;
-    if (is_core)
+    if (is_core) {
         exchange_core_body(w, core_idx, k_core, delta, val, pulled, K, neg_eta, core_before, core_ctas);
-    else
+    } else if (from_ranks.ranks != nullptr) {
+        // the explorers are not there yet: `exp` is where this launch writes them
+        exchange_explore_ranks_body(w, from_ranks, exp, k_exp, delta, val, pulled, k_core, K, neg_eta, range_shift,
+                                    b - core_before, bound);
+    } else {
         exchange_explore_body(w, exp, k_exp, delta, val, pulled, k_core, K, neg_eta, range_shift, b - core_before,
                               bound);
+    }
 }
 
 // Range per warp: a power of two with 16 to 32 entries per worker on average, at least 32 parameters.
@@ -268,10 +430,22 @@ slimdp_status launch_merge(float* w, uint64_t n, uint32_t K, const uint32_t* cor
     return SLIMDP_OK;
 }
 
+// Whether the exchange can turn sorted ranks into explorer indices itself: a warp's range must be
+// made of 1 to 32 whole 64-parameter groups of the core's directory.
+bool exchange_takes_ranks(uint64_t n, uint64_t k_exp) {
+    if (k_exp == 0) return false;
+    const uint32_t shift = explore_range_shift(n, k_exp);
+    return shift >= 6 && shift <= 11;
+}
+
+// ranks / rank_stride / core_aux_* / explore_status non-null: the explorers `exp` do not exist yet;
+// the launch computes them from every worker's sorted ranks and the core's bitmap and directory
+// (exchange_takes_ranks must hold) and writes them to `exp`.
 slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<const float>& delta,
                               const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,
                               uint64_t k_exp, float eta, const PtrArray<float>& val, const PtrArray<float>& pulled,
-                              cudaStream_t st) {
+                              const uint32_t* ranks, uint64_t rank_stride, const uint32_t* core_bitmap,
+                              const uint32_t* core_dir, int32_t* explore_status, cudaStream_t st) {
     static_assert(kMergeWarps * 32 == 256, "both kinds of CTA have 256 threads");
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
@@ -287,8 +461,14 @@ slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<c
     }
     const uint64_t total = core_ctas + explore_ctas;
     if (total == 0) return SLIMDP_OK;
+    RankSource src{};
+    if (ranks != nullptr) {
+        if (!exchange_takes_ranks(n, k_exp)) return SLIMDP_ERR_INTERNAL;
+        src = RankSource{ranks, rank_stride, core_bitmap, core_dir, (uint32_t)(num_blocks(n) * kDirPerBlock),
+                         explore_status};
+    }
     exchange_kernel<<<(unsigned)total, 256, 0, st>>>(w, core_idx, k_core, exp, (uint32_t)k_exp, delta, val, pulled,
-                                                     (int)K, -eta, shift, core_ctas, total);
+                                                     (int)K, -eta, shift, core_ctas, total, src);
     SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }
