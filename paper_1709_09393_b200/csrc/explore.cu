@@ -21,6 +21,8 @@
 //      the group holds no core parameter) turns it into the parameter index.
 // No global bitmap, no inter-CTA waiting; the result does not depend on the
 // order in which atomics land.
+#include <type_traits>
+
 #include "common.cuh"
 #include "layout.cuh"
 
@@ -260,17 +262,21 @@ constexpr uint32_t kListCap = 4096;
 
 // grid = (buckets, workers).  Sorts one bucket's ranks through a shared bitmap and writes them,
 // ascending, to the worker's row of `ranks`: buckets are rank ranges, so the row ends up sorted
-// as a whole.  Needs the sizes only, not the core.
+// as a whole.  Needs the sizes only, not the core.  WIDE: buckets of 2^17 ranks (s = 17), which
+// very long vectors use to keep the number of buckets within what the rank and scatter steps
+// count in shared memory.
+template <bool WIDE>
 __global__ void __launch_bounds__(kBucketThreads) bucket_sort_kernel(
     uint32_t k_exp, uint32_t s, const uint32_t* __restrict__ grouped, uint32_t* __restrict__ ranks,
     uint64_t rho_stride, const unsigned long long* __restrict__ cnt, const unsigned long long* __restrict__ pref,
     const unsigned long long* __restrict__ totals, uint64_t cnt_stride, WsHeader* hdr) {
-    __shared__ uint32_t bm[2048 + 64];           // up to 2^16 rank bits, padded (see sw)
-    __shared__ uint16_t list[kListCap];          // sorted ranks (low s bits) of the current round
+    using ListEntry = typename std::conditional<WIDE, uint32_t, uint16_t>::type;
+    __shared__ uint32_t bm[WIDE ? 4096 + 128 : 2048 + 64];   // up to 2^17 / 2^16 rank bits, padded (see sw)
+    __shared__ ListEntry list[kListCap];                     // sorted ranks (low s bits) of the current round
     __shared__ uint32_t warp_sums[kBucketThreads / 32];
     const uint32_t worker = blockIdx.y, bucket = blockIdx.x, t = threadIdx.x;
     const uint32_t words = 1u << (s - 5);
-    const uint32_t per = words / kBucketThreads;   // 1, 2, 4 or 8 words per thread
+    const uint32_t per = words / kBucketThreads;   // 1 .. 16 words per thread
     const uint32_t count = (uint32_t)cnt[(uint64_t)worker * cnt_stride + bucket];
     const uint32_t offset = (uint32_t)pref[(uint64_t)worker * cnt_stride + bucket];
     if (bucket == 0 && t == 0 && totals[worker] != k_exp) hdr->status = SLIMDP_ERR_INTERNAL;
@@ -310,7 +316,7 @@ __global__ void __launch_bounds__(kBucketThreads) bucket_sort_kernel(
                 while (word) {
                     const uint32_t bit = __ffs(word) - 1;
                     word &= word - 1;
-                    if (p >= r0 && p < r0 + kListCap) list[p - r0] = (uint16_t)((t * per + q) * 32u + bit);
+                    if (p >= r0 && p < r0 + kListCap) list[p - r0] = (ListEntry)((t * per + q) * 32u + bit);
                     ++p;
                 }
             }
@@ -489,6 +495,7 @@ uint32_t explore_bucket_shift(uint64_t M) {
     int extra = lg - 22;
     if (extra < 0) extra = 0;
     if (extra > 3) extra = 3;
+    if (lg >= 28) extra = 4;   // from 2^28 non-core parameters: 2^17 ranks per bucket, at most 8192 buckets up to 2^30
     return (uint32_t)(13 + extra);
 }
 
@@ -541,7 +548,8 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
     // part 1 may run beside another kernel's CTAs on the same SMs: one shared-memory split for all
     if (!prefer_max_shared(rank_kernel<true>) || !prefer_max_shared(rank_kernel<false>) ||
         !prefer_max_shared(scatter_kernel<true, true>) || !prefer_max_shared(scatter_kernel<true, false>) ||
-        !prefer_max_shared(scatter_kernel<false, false>) || !prefer_max_shared(bucket_sort_kernel) ||
+        !prefer_max_shared(scatter_kernel<false, false>) || !prefer_max_shared(bucket_sort_kernel<false>) ||
+        !prefer_max_shared(bucket_sort_kernel<true>) ||
         !prefer_max_shared(explore_setup_kernel))
         return SLIMDP_ERR_CUDA;
     if (smem) {
@@ -576,8 +584,12 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
                                                      L.sorted);
     }
     SLIMDP_LAUNCHED(1);
-    bucket_sort_kernel<<<dim3((unsigned)buckets, workers), kBucketThreads, 0, st>>>(
-        (uint32_t)k_exp, s, L.sorted, L.rho, L.rho_stride, L.cnt, L.pref, L.totals, L.cnt_stride, L.hdr);
+    if (s > 16)
+        bucket_sort_kernel<true><<<dim3((unsigned)buckets, workers), kBucketThreads, 0, st>>>(
+            (uint32_t)k_exp, s, L.sorted, L.rho, L.rho_stride, L.cnt, L.pref, L.totals, L.cnt_stride, L.hdr);
+    else
+        bucket_sort_kernel<false><<<dim3((unsigned)buckets, workers), kBucketThreads, 0, st>>>(
+            (uint32_t)k_exp, s, L.sorted, L.rho, L.rho_stride, L.cnt, L.pref, L.totals, L.cnt_stride, L.hdr);
     SLIMDP_LAUNCHED(1);
     }   // parts & 1
     if (!(parts & 2)) return SLIMDP_OK;

@@ -75,11 +75,11 @@ struct ExploreWs {
 };
 
 constexpr uint32_t kCellShift = 12;          // ranks per cell of the rank -> group table
-constexpr uint64_t kMaxSmemBuckets = 5120;   // bucket histograms up to this size live in shared memory (20 KB)
+constexpr uint64_t kMaxSmemBuckets = 8192;   // bucket histograms up to this size live in shared memory (32 KB)
 constexpr uint64_t kMaxExploreCtas = 1024;   // rank / scatter CTAs over all workers of one call
 
 // Upper bound on the number of rank buckets for any core size: buckets hold
-// 2^13 .. 2^16 ranks, 2^16 once there are at least 2^25 non-core parameters.
+// 2^13 .. 2^17 ranks, at least 2^16 once there are 2^25 non-core parameters.
 inline uint64_t explore_max_buckets(uint64_t n) {
     const uint64_t big = (n + 65535) / 65536;
     return big > 1024 ? big : 1024;
