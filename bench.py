@@ -395,9 +395,9 @@ def run_ours(args):
 
 
 # DRAM bytes (read + write) of one launch of the fused pass, per workload: from an ncu capture of the
-# same kernel on the leading 40 M parameters of the workload (1448.0 MB = 36.20 B per parameter;
+# same kernel on the leading 40 M parameters of the workload (1447.6 MB = 36.19 B per parameter;
 # traffic grows in proportion to n), scaled to the full launch of 138 357 544 parameters.
-TRAFFIC_DOMINANT_BYTES: dict = {"vgg16": 5_008_632_000}
+TRAFFIC_DOMINANT_BYTES: dict = {"vgg16": 5_007_158_000}
 
 
 def main():
