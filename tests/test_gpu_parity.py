@@ -424,6 +424,38 @@ def test_round_one_call_any_worker_count(P, K):
     assert_round_equal(P, d_w, buf, ref, n, scores=False)
 
 
+# In the one-call round the exchange's explorer warps compute the indices from the sorted ranks where
+# a warp's parameter range is 1 to 32 groups of 64 parameters, i.e. for explorers of about 0.8 % to 50 % of
+# the vector per worker; denser and thinner explorers take the separate index kernels.  One case per
+# range size on either side of both limits.
+@pytest.mark.parametrize("per_mille", [600, 300, 100, 30, 12, 6, 1])
+def test_round_one_call_explorer_densities(P, per_mille):
+    K, n = 3, FUSED_N
+    rng = np.random.default_rng(per_mille)
+    w = (rng.standard_normal(n) * 0.05).astype(np.float32)
+    gs = [(rng.standard_normal(n) * 1e-2).astype(np.float32) for _ in range(K)]
+    k_core = n // 33
+    k_exp = (n - k_core) * per_mille // 1000
+    ref = oracle.run_round(w, gs, 1.0, k_core, k_exp, 11, 5, 0.25)
+    d_w, buf = gpu_round(P, w, gs, 1.0, k_core, k_exp, 11, 5, 0.25, one_call=True)
+    assert_round_equal(P, d_w, buf, ref, n, scores=False)
+
+
+# Short vectors through the one-call round: a single bitmap block or a few, the last directory groups
+# partly or wholly beyond the end of the vector.
+@pytest.mark.parametrize("n,k_core,k_exp", [(1, 0, 1), (1, 1, 0), (5, 2, 2), (63, 6, 3), (64, 6, 3), (65, 7, 58),
+                                            (100, 10, 3), (1000, 100, 45), (1025, 1, 512), (4097, 400, 200),
+                                            (70_001, 3000, 900)])
+def test_round_one_call_short_vectors(P, n, k_core, k_exp):
+    K = 2
+    rng = np.random.default_rng(n)
+    w = rng.standard_normal(n).astype(np.float32)
+    gs = [(rng.standard_normal(n) * 0.1).astype(np.float32) for _ in range(K)]
+    ref = oracle.run_round(w, gs, 0.5, k_core, k_exp, 3, 1, 0.5)
+    d_w, buf = gpu_round(P, w, gs, 0.5, k_core, k_exp, 3, 1, 0.5, one_call=True)
+    assert_round_equal(P, d_w, buf, ref, n, scores=True)      # below 2^21 parameters the scores are written
+
+
 def test_round_one_call_any_alignment(P):
     # tensors that start 4 bytes off a 16-byte boundary: the round scores and selects in two steps
     cfg = scaled_config(CONFIGS["vgg16"], FUSED_N)
