@@ -4,7 +4,8 @@ Checks the 64-bit offset arithmetic of every call at the top of the index range.
 are mostly zero with a few hundred distinct non-zero values at chosen positions (the very
 first and very last indices among them), so the expected core, packed values, merged model
 and pulled values follow from the definitions without sorting 4.3 G keys; the explorer is
-checked against the CPU oracle.  Needs about 75 GB on the device and 60 GB of host memory.
+checked against the CPU oracle; the one-call round is then compared with the separate calls on the
+same inputs.  Needs about 110 GB on the device and 60 GB of host memory.
 """
 import os
 
@@ -23,14 +24,14 @@ def _enough_memory() -> bool:
     import psutil
     if psutil.virtual_memory().available < 70 << 30:
         return False
-    return torch.cuda.is_available() and torch.cuda.mem_get_info()[0] > (90 << 30)
+    return torch.cuda.is_available() and torch.cuda.mem_get_info()[0] > (130 << 30)
 
 
 def test_maximum_vector_length():
     if os.environ.get("SLIMDP_SKIP_LARGE") == "1":
         pytest.skip("SLIMDP_SKIP_LARGE=1")
     if not _enough_memory():
-        pytest.skip("needs 70 GB of free host memory and 90 GB of free device memory")
+        pytest.skip("needs 70 GB of free host memory and 130 GB of free device memory")
     import paper_1709_09393_b200 as P
     rng = np.random.default_rng(2 ** 32 - 1)
     # 600 marked parameters: both ends of the vector, block / directory boundaries, random places
@@ -124,3 +125,39 @@ def test_maximum_vector_length():
         assert np.array_equal(val[k].cpu().numpy().view(np.uint32), vals_ref[k].view(np.uint32))
         ref_pull = oracle.pull(merged_small, pos(core), pos(exps[k]))
         assert np.array_equal(pulled[k].cpu().numpy().view(np.uint32), ref_pull.view(np.uint32))
+
+    # the whole round as one call at this length: same bytes as the separate calls on the same inputs
+    del val, pulled, exp_idx, ews, aux, core_idx, g
+    torch.cuda.empty_cache()
+    w.uniform_(-1.0, 1.0)      # a model without the zeros, so that the selection's bracket holds at this length too
+    k_core, k_exp = 30_000_001, 40_000_003      # 0.7 % core, ~1 % explorers
+    m = k_core + k_exp
+
+    def buffers():
+        return dict(core=torch.empty(k_core, dtype=torch.int32, device="cuda"),
+                    aux=torch.empty(P.core_aux_bytes(N), dtype=torch.uint8, device="cuda"),
+                    exp=[torch.empty(k_exp, dtype=torch.int32, device="cuda") for _ in range(K)],
+                    val=[torch.empty(m, dtype=torch.float32, device="cuda") for _ in range(K)],
+                    pulled=[torch.empty(m, dtype=torch.float32, device="cuda") for _ in range(K)])
+
+    sel_ws = torch.empty(P.select_workspace_bytes(N), dtype=torch.uint8, device="cuda")
+    exp_ws = torch.empty(P.explore_workspace_bytes(N, k_exp, K), dtype=torch.uint8, device="cuda")
+    scores = torch.empty(N, dtype=torch.float32, device="cuda")
+    a, b = buffers(), buffers()
+    w_a = w.clone()
+    P.slimdp_score(w_a, deltas, c, scores)
+    P.slimdp_select_core(scores, k_core, a["core"], a["aux"], sel_ws)
+    P.slimdp_sample_explore_batched(a["aux"], N, k_core, k_exp, 78, 0, 4, a["exp"], exp_ws)
+    P.slimdp_exchange(w_a, deltas, a["core"], a["exp"], eta, a["val"], a["pulled"])
+    P.read_status(sel_ws)
+    P.read_status(exp_ws)
+    P.slimdp_round(w, deltas, c, 78, 4, eta, scores, b["core"], b["aux"], b["exp"], b["val"], b["pulled"], sel_ws,
+                   exp_ws)
+    P.read_status(sel_ws)
+    P.read_status(exp_ws)
+    assert torch.equal(a["core"], b["core"])
+    assert torch.equal(w_a.view(torch.int32), w.view(torch.int32))
+    for k in range(K):
+        assert torch.equal(a["exp"][k], b["exp"][k])
+        assert torch.equal(a["val"][k].view(torch.int32), b["val"][k].view(torch.int32))
+        assert torch.equal(a["pulled"][k].view(torch.int32), b["pulled"][k].view(torch.int32))
