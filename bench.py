@@ -278,6 +278,28 @@ def run_ours(args):
     dominant_ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
     value = aggregate_value(N, world, ms_per_step)
 
+    # ---- optional: kernel timeline of three more rounds (CUPTI through torch.profiler) ----
+    # Start, duration and stream of every kernel, relative to the first: shows which kernels of the
+    # one-call round run side by side, which a serialising profiler cannot.  Not a timing source.
+    if args.timeline and rank == 0:
+        from torch.profiler import ProfilerActivity, profile
+        with profile(activities=[ProfilerActivity.CUDA]) as prof:
+            for _ in range(3):
+                one_round(t)
+                t += 1
+            torch.cuda.synchronize()
+        trace = args.timeline + ".trace.json"
+        prof.export_chrome_trace(trace)
+        with open(trace) as f:
+            events = [e for e in json.load(f)["traceEvents"] if e.get("cat") in ("kernel", "gpu_memset")]
+        os.remove(trace)
+        events.sort(key=lambda e: e["ts"])
+        with open(args.timeline, "w") as f:
+            f.write("# start_us duration_us stream kernel   (three consecutive slimdp_round calls)\n")
+            for e in events:
+                name = e["name"].replace("slimdp::(anonymous namespace)::", "").split("(")[0]
+                f.write(f'{e["ts"] - events[0]["ts"]:10.1f} {e["dur"]:8.1f} s{e["args"].get("stream")} {name}\n')
+
     # ---- per-call breakdown (untimed for the headline; 5 more rounds) -------
     # "exchange" is the fused pack + merge + pull the timed rounds use; the three separate calls
     # are timed after it for comparison (they repeat the exchange's work on the next model state)
@@ -409,6 +431,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--timeline", default="",
+                    help="also write the kernel timeline of three extra rounds (start, duration, stream) to this file")
     ap.add_argument("--scale", type=int, default=0,
                     help="run on the leading SCALE parameters of the config (small case for profiler captures)")
     args = ap.parse_args()
