@@ -341,9 +341,9 @@ __device__ __forceinline__ uint32_t score1(const float* __restrict__ w, const Pt
     return __float_as_uint(score_one(c, a, w[i]));
 }
 
-// Sample kernel A of the fused path: 2^16 evenly spaced groups of four consecutive parameters
-// are scored (2^18 sampled keys, one 16-byte load per tensor and group); the rest is
-// sample_coarse_kernel's.  Needs n >= 4 and 16-byte aligned tensors.  1024 groups per CTA: the
+// Sample kernel A of the fused path: 2^14 evenly spaced groups of sixteen consecutive parameters
+// are scored (2^18 sampled keys, one 16-byte load per tensor and thread); the rest is
+// sample_coarse_kernel's.  Needs n >= 16 and 16-byte aligned tensors.  1024 groups per CTA: the
 // sampled keys fall into a handful of coarse bins, and every CTA adds to those few global
 // counters, so few large CTAs queue up less there than many small ones.
 __global__ void __launch_bounds__(1024) sample_score_coarse_kernel(const float* __restrict__ w,
@@ -358,9 +358,12 @@ __global__ void __launch_bounds__(1024) sample_score_coarse_kernel(const float* 
     const uint32_t t = threadIdx.x;
     if (t < 256) sh_coarse[t] = 0;
     __syncthreads();
-    const uint32_t j = blockIdx.x * 1024 + t;   // group number, < 2^16
+    // thread j scores four consecutive parameters; threads 4s .. 4s+3 together take sixteen consecutive
+    // ones at the s-th of 2^14 evenly spaced places: one 64-byte piece per tensor and place, the least
+    // DRAM hands out, so the sample costs a quarter of the fetches that 2^16 separate places would
+    const uint32_t j = blockIdx.x * 1024 + t;   // < 2^16
     uint32_t key[4];
-    score4<0>(w, g, K, c, ((uint64_t)j * (n / 4)) >> (kSampleBits - 2), key);
+    score4<0>(w, g, K, c, ((((uint64_t)(j >> 2) * (n / 16)) >> (kSampleBits - 4)) << 2) + (j & 3u), key);
     reinterpret_cast<uint4*>(sample)[j] = make_uint4(key[0], key[1], key[2], key[3]);
     // most of a warp's keys share a coarse bin: one shared-memory atomic per distinct bin and warp
 #pragma unroll
