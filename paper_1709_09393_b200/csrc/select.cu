@@ -6,7 +6,7 @@
 // to T that belong to the core (those with the smallest indices).
 //
 // Large inputs (n >= 2^21) take the bracketed path, which reads the scores once:
-//   1. sample (two small kernels): 2^18 evenly spaced keys are copied out and
+//   1. sample (two small kernels): 2^18 keys (sixteen at each of 2^14 evenly spaced places) are copied out and
 //      counted by their top 8 bits, then, around the two target ranks, by their
 //      top 16 bits; the last CTA of each kernel turns the counts into a
 //      bracket of 16-bit bins [b_bot, b_top) that holds T with overwhelming
@@ -90,7 +90,7 @@ __device__ __forceinline__ void bracket_targets(uint32_t k, uint64_t n, long lon
     *hi_target = (long long)ceil(r + margin);
 }
 
-// Sample kernel A: 2^18 evenly spaced keys are copied to `sample` and counted by their top 8
+// Sample kernel A: 2^18 keys, sixteen at each of 2^14 evenly spaced places, are copied to `sample` and counted by their top 8
 // bits (256 coarse bins: shared memory per CTA, then a few global atomics).  The last CTA finds
 // the two coarse bins in which the count from the top crosses the two target ranks:
 // coarse_x[0] for b_top (highest coarse bin whose inclusive count exceeds lo_target),
@@ -107,8 +107,9 @@ __global__ void __launch_bounds__(1024) sample_coarse_kernel(const uint32_t* __r
     const uint32_t t = threadIdx.x;
     if (t < 256) sh_coarse[t] = 0;
     __syncthreads();
+    // sixteen consecutive keys (one 64-byte piece, the least DRAM hands out) at each of 2^14 evenly spaced places
     const uint32_t j = blockIdx.x * 1024 + t;   // sample number, < 2^18
-    const uint32_t key = __ldg(keys + (((uint64_t)j * n) >> kSampleBits));
+    const uint32_t key = __ldg(keys + ((((uint64_t)(j >> 4) * (n / 16)) >> (kSampleBits - 4)) << 4) + (j & 15u));
     sample[j] = key;
     atomicAdd(&sh_coarse[key >> 24], 1u);
     __syncthreads();
