@@ -107,10 +107,9 @@ slimdp_status slimdp_score(const float* w, const float* const* grads, uint32_t K
                            float* scores, void* stream);
 
 /* --------------------------------------------------------------- select ---
- * Core selection T_S (Section 3.1 item 1, Section 3.2: "rank the parameters by
- * their significance, and select the top"): the k_core parameters that come
- * first when all n are ordered by (score bit pattern descending as unsigned
- * 32-bit, index ascending).  For scores from slimdp_score this is score
+ * Core selection T_S (Section 3.1 item 1; the ranking by significance of
+ * Section 3.2): the k_core parameters that come first when all n are ordered
+ * by (score bit pattern descending as unsigned 32-bit, index ascending).  For scores from slimdp_score this is score
  * descending with ties going to the smaller index and NaN ranking highest.
  *   scores    [n] (read)
  *   k_core    0 <= k_core <= n
@@ -127,7 +126,7 @@ slimdp_status slimdp_select_core(const float* scores, uint64_t n, uint64_t k_cor
  * Exploration operator T_R^k (Section 3.1 item 2, Section 3.3 step 2): worker
  * `worker` draws, for communication `round`, k_exp distinct parameters
  * uniformly from the M = n - k_core parameters outside the core.  The paper
- * fixes "random"; this library fixes the generator so that results can be
+ * asks only for a random choice; this library fixes the generator so that results can be
  * reproduced bit for bit:
  *   round keys rk[0..11] = three Philox-4x32-10 blocks with key
  *       (seed low word, seed high word) and counters (b, worker, round, 0x534C494D), b = 0, 1, 2;
@@ -185,7 +184,7 @@ slimdp_status slimdp_sample_explore_static(const void* core_aux, uint64_t n, uin
 
 /* ----------------------------------------------------------------- pack ---
  * Extraction of T_C(delta_k) = T_S(delta_k) U T_R^k(delta_k) (Section 3.1; the
- * "extract ... by scanning" cost of Section 3.5):
+ * extraction cost that Section 3.5 counts):
  *     val[j]          = delta[core_idx[j]]   j < k_core
  *     val[k_core + j] = delta[exp_idx[j]]    j < k_exp
  * The worker's <key, value> buffer (Section 3.5) is the pair
@@ -244,9 +243,9 @@ slimdp_status slimdp_exchange(float* w_global, uint64_t n, uint32_t K, const flo
                               uint64_t k_exp, float eta, float* const* val, float* const* pulled, void* stream);
 
 /* ------------------------------------------ the steps either side of the path ---
- * Dense push at a reselection boundary (Algorithm 1, worker: "if (t+1) % q == 0
- * Push(delta)"; server: Update, t <- t+1, "if t % q == 0 Core-Selection(w-bar^t,
- * delta^t, beta)"; Section 3.3 steps 3 and 6).  One pass applies every worker's
+ * Dense push at a reselection boundary (Algorithm 1: every q-th round the
+ * worker pushes its whole update, and the server, after its update, selects a
+ * new core; Section 3.3 steps 3 and 6).  One pass applies every worker's
  * WHOLE update to the global model in ascending worker order (this is also
  * Plump-DP's update, Section 2.1) and, if scores is not NULL, scores the
  * UPDATED model with the updates just pushed:
@@ -270,9 +269,9 @@ slimdp_status slimdp_worker_merge_batched(float* const* w_local, uint32_t K, uin
                                           uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
                                           const float* const* pulled, void* stream);
 
-/* Key caching (Section 3.5): "the sender then only needs to send the values with
- * a signature of the keys".  slimdp_core_signature writes a 64-bit signature of a
- * key list to device memory:
+/* Key caching (Section 3.5): both sides keep the core's keys, so a push carries
+ * the core's values and a signature of the keys instead of the keys themselves.
+ * slimdp_core_signature writes a 64-bit signature of a key list to device memory:
  *     sig = sum_j mix64(((j << 32) | keys[j]) + 0x9E3779B97F4A7C15)  mod 2^64,
  *     mix64(z): z ^= z >> 30; z *= 0xBF58476D1CE4E5B9; z ^= z >> 27; z *= 0x94D049BB133111EB; z ^= z >> 31
  * (the SplitMix64 output function).  Sender and receiver compare signatures to

@@ -21,6 +21,8 @@
 //     (Section 3.3 step 6 scores with the updates pushed densely before reselection);
 //   * score arithmetic is fp32: left-to-right sum, then one fused multiply-add;
 //     a NaN score is stored as 0x7FC00000 and ranks above +inf;
+//   * a NaN result of a server update is stored as 0x7FC00000 as well (pack and pull move
+//     bits and keep whatever payload they find);
 //   * ties in the ranking are broken by ascending parameter index;
 //   * the explorer (Section 3.1 item 2, Section 3.3 step 2: a random subset of
 //     the parameters outside the core, drawn anew per worker and per
@@ -129,6 +131,11 @@ uint64_t feistel_perm(uint64_t j, uint64_t M, const uint32_t rk[12]) {
     return x;
 }
 
+// A merged model value as stored: a NaN result of an update becomes the canonical quiet NaN
+// (IEEE 754 leaves the payload that an operation passes on to the implementation; Section 3.3
+// step 3 defines the value only), exactly as a NaN score does.
+inline float stored_model_value(float x) { return std::isnan(x) ? bits_f32(0x7FC00000u) : x; }
+
 struct Ranked {
     uint32_t key;   // bit pattern of the score
     uint32_t idx;   // parameter index
@@ -211,11 +218,11 @@ void oracle_merge(float* w, uint32_t K, const uint32_t* core_idx, uint64_t k_cor
     for (uint32_t k = 0; k < K; ++k) {
         for (uint64_t j = 0; j < k_core; ++j) {
             uint32_t i = core_idx[j];
-            w[i] = std::fmaf(-eta, val[k][j], w[i]);
+            w[i] = stored_model_value(std::fmaf(-eta, val[k][j], w[i]));
         }
         for (uint64_t j = 0; j < k_exp; ++j) {
             uint32_t i = exp_idx[k][j];
-            w[i] = std::fmaf(-eta, val[k][k_core + j], w[i]);
+            w[i] = stored_model_value(std::fmaf(-eta, val[k][k_core + j], w[i]));
         }
     }
 }
@@ -252,7 +259,7 @@ uint64_t oracle_core_signature(const uint32_t* keys, uint64_t count) {
 // Plump-DP (Section 2.1): every worker pushes its whole update.
 void oracle_dense_merge(float* w, uint64_t n, uint32_t K, const float* const* grads, float eta) {
     for (uint32_t k = 0; k < K; ++k)
-        for (uint64_t i = 0; i < n; ++i) w[i] = std::fmaf(-eta, grads[k][i], w[i]);
+        for (uint64_t i = 0; i < n; ++i) w[i] = stored_model_value(std::fmaf(-eta, grads[k][i], w[i]));
 }
 
 }  // extern "C"

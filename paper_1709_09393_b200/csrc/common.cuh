@@ -144,6 +144,12 @@ __device__ __forceinline__ float score_one(float c, float g, float w) {
     return (s != s) ? __uint_as_float(0x7FC00000u) : s;
 }
 
+// A merged model value as it is stored (Section 3.3 step 3 defines the value only): IEEE 754 leaves the
+// payload of a NaN that an operation passes on open, so every NaN result of an update is stored as the
+// canonical quiet NaN, as scores are.  Once NaN a parameter stays NaN, so one check after the last of a
+// chain of updates gives the same bits as a check after each.
+__device__ __forceinline__ float stored_model_value(float x) { return (x != x) ? __uint_as_float(0x7FC00000u) : x; }
+
 // ---- internal launchers (each enqueues on `st`, returns a slimdp_status) ---
 
 // Exclusive scan over bitmap blocks of 64-bit counters: cnt[y][nb] -> pref[y][nb],

@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(256) merge_core_kernel(float* __restrict__ w, 
             for (int q = 0; q < 8; ++q) x = __fmaf_rn(neg_eta, v[q], x);
         }
         for (; k < K; ++k) x = __fmaf_rn(neg_eta, __ldcs(val.p[k] + j), x);
-        w[i] = x;
+        w[i] = stored_model_value(x);
     }
 }
 
@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* 
         const uint32_t b = bound[k][wid + 1];
         for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) {
             const uint32_t i = __ldg(idx + e);
-            w[i] = __fmaf_rn(neg_eta, __ldcs(v + e), ld_sparse(w + i));
+            w[i] = stored_model_value(__fmaf_rn(neg_eta, __ldcs(v + e), ld_sparse(w + i)));
         }
         __syncwarp();   // worker k's updates are visible to the whole warp before worker k+1 starts
     }
@@ -175,6 +175,7 @@ __device__ __forceinline__ void exchange_core_body(float* __restrict__ w, const 
             __stcs(val.p[k] + j, v);
             x = __fmaf_rn(neg_eta, v, x);
         }
+        x = stored_model_value(x);
         w[i] = x;
 #pragma unroll 8
         for (int q = 0; q < K; ++q) __stcs(pulled.p[q] + j, x);
@@ -202,7 +203,7 @@ __device__ __forceinline__ void exchange_explore_body(float* w, const PtrArray<c
             const uint32_t i = __ldg(idx + e);
             const float u = ld_sparse(d + i);
             __stcs(v + e, u);
-            w[i] = __fmaf_rn(neg_eta, u, ld_sparse(w + i));
+            w[i] = stored_model_value(__fmaf_rn(neg_eta, u, ld_sparse(w + i)));
         }
         __syncwarp();   // worker k's updates are visible to the whole warp before worker k+1 starts
     }
@@ -358,7 +359,7 @@ __device__ __forceinline__ void exchange_explore_ranks_body(float* w, const Rank
             const uint32_t i = idx[e];
             const float u = ld_sparse(d + i);
             __stcs(v + e, u);
-            w[i] = __fmaf_rn(neg_eta, u, ld_sparse(w + i));
+            w[i] = stored_model_value(__fmaf_rn(neg_eta, u, ld_sparse(w + i)));
         }
         __syncwarp();   // worker k's updates are visible to the whole warp before worker k+1 starts
     }

@@ -99,6 +99,10 @@ __global__ void __launch_bounds__(256) dense_merge_score_kernel(float* __restric
                 x.z = __fmaf_rn(neg_eta, b.z, x.z);
                 x.w = __fmaf_rn(neg_eta, b.w, x.w);
             }
+            x.x = stored_model_value(x.x);
+            x.y = stored_model_value(x.y);
+            x.z = stored_model_value(x.z);
+            x.w = stored_model_value(x.w);
             w4[i] = x;
             if (S) {
                 float4 s;
@@ -121,6 +125,7 @@ __global__ void __launch_bounds__(256) dense_merge_score_kernel(float* __restric
             a = __fadd_rn(a, b);
             x = __fmaf_rn(neg_eta, b, x);
         }
+        x = stored_model_value(x);
         w[i] = x;
         if (S) S[i] = score_one(c, a, x);
     }

@@ -4,8 +4,11 @@ Checks the 64-bit offset arithmetic of every call at the top of the index range.
 are mostly zero with a few hundred distinct non-zero values at chosen positions (the very
 first and very last indices among them), so the expected core, packed values, merged model
 and pulled values follow from the definitions without sorting 4.3 G keys; the explorer is
-checked against the CPU oracle; the one-call round is then compared with the separate calls on the
-same inputs.  Needs about 110 GB on the device and 60 GB of host memory.
+checked against the CPU oracle.  The one-call round then runs on a model without zeros (so that
+its bracketed selection, not the fallback, is what runs): its outputs are compared with the separate
+calls on the same inputs and, on the host, with the definitions (threshold by np.partition plus the
+tie rule, the oracle's explorers, the oracle's merge and pull on the touched places).
+Needs about 110 GB on the device and 70 GB of host memory.
 """
 import os
 
@@ -144,6 +147,7 @@ def test_maximum_vector_length():
     exp_ws = torch.empty(P.explore_workspace_bytes(N, k_exp, K), dtype=torch.uint8, device="cuda")
     scores = torch.empty(N, dtype=torch.float32, device="cuda")
     a, b = buffers(), buffers()
+    w0 = w.cpu().numpy()                                           # the model before the round (host copy)
     w_a = w.clone()
     P.slimdp_score(w_a, deltas, c, scores)
     P.slimdp_select_core(scores, k_core, a["core"], a["aux"], sel_ws)
@@ -161,3 +165,49 @@ def test_maximum_vector_length():
         assert torch.equal(a["exp"][k], b["exp"][k])
         assert torch.equal(a["val"][k].view(torch.int32), b["val"][k].view(torch.int32))
         assert torch.equal(a["pulled"][k].view(torch.int32), b["pulled"][k].view(torch.int32))
+    del a, w_a, scores, sel_ws, exp_ws
+    torch.cuda.empty_cache()
+
+    # ... and the one-call round against the definitions, evaluated on the host without the library:
+    # the updates are zero outside a few hundred thousand places, so S = |w| there (Eq. 1 with g = 0) and
+    # the oracle scores the rest; the core is the threshold (k-th largest key) plus the tie rule.
+    nz = np.unique(np.concatenate([np.concatenate([core, e]).astype(np.int64) for e in exps]))
+    nz_t = torch.from_numpy(nz).cuda()
+    d_nz = [d[nz_t].cpu().numpy() for d in deltas]                 # the updates where they are not zero
+    assert all(int(torch.count_nonzero(d).item()) <= nz.size for d in deltas)
+    S = np.abs(w0)
+    S[nz] = oracle.score(w0[nz], d_nz, c)
+    keys = S.view(np.uint32)
+    part = keys.copy()
+    part.partition(N - k_core)
+    T = part[N - k_core]                                           # the k_core-th largest key
+    del part
+    greater = np.flatnonzero(keys > T)
+    equal = np.flatnonzero(keys == T)
+    del S, keys
+    core_ref = np.sort(np.concatenate([greater, equal[:k_core - greater.size]])).astype(np.uint32)
+    del greater, equal
+    assert core_ref.size == k_core
+    assert np.array_equal(b["core"].cpu().numpy().view(np.uint32), core_ref)
+    exps_ref = [oracle.sample_explore(core_ref, N, k_exp, 78, k, 4) for k in range(K)]
+    for k in range(K):
+        assert np.array_equal(b["exp"][k].cpu().numpy().view(np.uint32), exps_ref[k]), k
+    # pack by definition: the update's value where it has one, zero elsewhere
+    vals_ref = []
+    for k in range(K):
+        both = np.concatenate([core_ref, exps_ref[k]]).astype(np.int64)
+        at = np.minimum(np.searchsorted(nz, both), nz.size - 1)
+        vals_ref.append(np.where(nz[at] == both, d_nz[k][at], np.float32(0.0)).astype(np.float32))
+        assert np.array_equal(b["val"][k].cpu().numpy().view(np.uint32), vals_ref[k].view(np.uint32)), k
+    # merge and pull on the touched places (a compact copy of the model restricted to them) ...
+    touched = np.unique(np.concatenate([core_ref] + exps_ref).astype(np.int64))
+    pos = lambda x: np.searchsorted(touched, x.astype(np.int64)).astype(np.uint32)
+    merged_small = oracle.merge(w0[touched], pos(core_ref), [pos(e) for e in exps_ref], vals_ref, eta)
+    w1 = w.cpu().numpy()
+    assert np.array_equal(w1[touched].view(np.uint32), merged_small.view(np.uint32))
+    for k in range(K):
+        ref_pull = oracle.pull(merged_small, pos(core_ref), pos(exps_ref[k]))
+        assert np.array_equal(b["pulled"][k].cpu().numpy().view(np.uint32), ref_pull.view(np.uint32)), k
+    # ... and nothing else was written
+    changed = np.flatnonzero(w1.view(np.uint32) != w0.view(np.uint32))
+    assert np.isin(changed, touched, assume_unique=True).all()

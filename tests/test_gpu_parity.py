@@ -302,16 +302,9 @@ def gpu_round(P, w, gs, cfg_c, k_core, k_exp, seed, rnd, eta, fused=True, one_ca
     return d_w, buf
 
 
-def same_bits_or_both_nan(got_bits, want):
-    """Bit equality, except that any NaN matches any NaN: IEEE 754 leaves the payload of a NaN that an
-    operation passes on to the implementation, and the merge's fma passes a NaN model value on."""
-    want_bits = bits(want)
-    nan = np.isnan(want)
-    return np.array_equal(np.isnan(got_bits.view(np.float32)), nan) and np.array_equal(got_bits[~nan], want_bits[~nan])
-
-
-def assert_round_equal(P, d_w, buf, ref, n, scores=True, merged_nans=False):
-    same = same_bits_or_both_nan if merged_nans else (lambda got, want: np.array_equal(got, bits(want)))
+def assert_round_equal(P, d_w, buf, ref, n, scores=True):
+    # bit equality throughout, NaNs included: a NaN result of an update is stored as 0x7FC00000 on both sides
+    same = lambda got, want: np.array_equal(got, bits(want))
     if scores:      # slimdp_round keeps its scores in registers: the buffer is scratch there
         assert np.array_equal(host_bits(buf.scores), bits(ref["scores"])), "scores"
     assert np.array_equal(host_u32(buf.core_idx), ref["core_idx"]), "core_idx"
@@ -399,12 +392,14 @@ def test_round_one_call_fused_cases(P, case):
         k_exp = 1000
     elif case == "nan_and_inf":
         w[7::1001] = np.nan
+        w.view(np.uint32)[9::5003] = 0xFFC12345          # a NaN with a sign and a payload
+        gs[0].view(np.uint32)[13::7001] = 0x7F800001     # a signalling NaN in an update
         gs[1][3::2003] = np.inf
         gs[2][5::3001] = -np.inf
         w[11::4001] = np.float32(-0.0)
     ref = oracle.run_round(w, gs, cfg.c, k_core, k_exp, cfg.seed, 2, cfg.eta)
     d_w, buf = gpu_round(P, w, gs, cfg.c, k_core, k_exp, cfg.seed, 2, cfg.eta, one_call=True)
-    assert_round_equal(P, d_w, buf, ref, n, scores=False, merged_nans=(case == "nan_and_inf"))
+    assert_round_equal(P, d_w, buf, ref, n, scores=False)
     if case == "all_scores_equal":        # and there the scratch does hold the scores
         assert np.array_equal(host_bits(buf.scores), bits(ref["scores"]))
 

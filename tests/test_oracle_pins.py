@@ -307,6 +307,31 @@ def test_merge_applies_workers_in_ascending_order():
     assert bits(out[0]) == bits(first_b)
 
 
+def test_merge_stores_every_nan_result_as_the_canonical_quiet_nan():
+    # Section 3.3 step 3 defines the merged value; which NaN payload comes out of an update is open in
+    # IEEE 754, so the contract fixes it: any NaN result is stored as 0x7FC00000.  Pack and pull move bits.
+    odd_nans = np.array([0x7F800001, 0xFFC12345, 0x7FFFFFFF, 0xFF800001], np.uint32).view(np.float32)
+    inf = np.float32(np.inf)
+    #            NaN model x4 (signalling, negative, all-ones, negative signalling), inf - inf, finite
+    w = np.concatenate([odd_nans, np.array([inf, -inf, 1.0, 2.0], np.float32)])
+    d = np.array([1.0, 2.0, 3.0, 4.0, inf, -inf, odd_nans[1], 0.5], np.float32)
+    d.view(np.uint32)[6] = 0xFFC12345
+    n = w.size
+    core = np.array([0, 2, 4, 6], np.uint32)
+    exp = [np.array([1, 3, 5, 7], np.uint32)]
+    val = [oracle.pack(d, core, exp[0])]
+    assert bits(val[0]).tolist() == bits(d[[0, 2, 4, 6, 1, 3, 5, 7]]).tolist()      # payloads kept by pack
+    out = oracle.merge(w, core, exp, val, 0.5)
+    canon = 0x7FC00000
+    assert bits(out).tolist() == [canon] * 7 + [int(bits(np.float32(1.75)))]
+    assert bits(oracle.pull(out, core, exp[0])).tolist() == bits(out[[0, 2, 4, 6, 1, 3, 5, 7]]).tolist()
+    dense = oracle.dense_merge(w, [d], 0.5)
+    assert bits(dense).tolist() == bits(out).tolist()
+    # an untouched NaN keeps its payload: only results of updates are canonical
+    untouched = oracle.merge(w, np.array([7], np.uint32), [np.zeros(0, np.uint32)], [np.array([0.5], np.float32)], 0.5)
+    assert bits(untouched[:4]).tolist() == bits(odd_nans).tolist()
+
+
 def test_dense_merge_is_sequential_rounding_of_exact_updates():
     rng = np.random.default_rng(11)
     n, K = 200, 3
