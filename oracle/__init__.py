@@ -41,6 +41,12 @@ _merge = _sig("oracle_merge", None, _f32p, ctypes.c_uint32, _u32p, ctypes.c_uint
 _pull = _sig("oracle_pull", None, _f32p, _u32p, ctypes.c_uint64, _u32p, ctypes.c_uint64, _f32p)
 _dense = _sig("oracle_dense_merge", None, _f32p, ctypes.c_uint64, ctypes.c_uint32, _pp, ctypes.c_float)
 _signature = _sig("oracle_core_signature", ctypes.c_uint64, _u32p, ctypes.c_uint64)
+_u8p = ctypes.POINTER(ctypes.c_uint8)
+_wire_bytes = _sig("oracle_wire_message_bytes", ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int)
+_wire_pack = _sig("oracle_wire_pack", None, _u32p, ctypes.c_uint64, _u32p, ctypes.c_uint64, _f32p, ctypes.c_uint32,
+                  ctypes.c_uint32, ctypes.c_int, _u8p)
+_wire_unpack = _sig("oracle_wire_unpack", ctypes.c_int32, _u8p, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64,
+                    ctypes.c_uint64, _u32p, _u32p, _f32p, ctypes.POINTER(ctypes.c_uint64))
 _wmerge = _sig("oracle_worker_merge", None, _f32p, _u32p, ctypes.c_uint64, _u32p, ctypes.c_uint64, _f32p)
 
 
@@ -150,6 +156,34 @@ def worker_merge(w_local, core_idx, exp_idx, pulled) -> np.ndarray:
 def core_signature(keys) -> int:
     k = _u32(keys)
     return int(_signature(_ptr(k, _u32p), k.size))
+
+
+def wire_message_bytes(k_core: int, k_exp: int, with_keys: bool) -> int:
+    return int(_wire_bytes(k_core, k_exp, int(with_keys)))
+
+
+def wire_pack(core_idx, exp_idx, val, worker: int, rnd: int, with_keys: bool) -> np.ndarray:
+    """One worker's push as a byte message (Section 3.5)."""
+    c, e, v = _u32(core_idx), _u32(exp_idx), _f32(val)
+    assert v.size == c.size + e.size
+    msg = np.zeros(wire_message_bytes(c.size, e.size, with_keys), np.uint8)
+    _wire_pack(_ptr(c, _u32p), c.size, _ptr(e, _u32p), e.size, _ptr(v, _f32p), worker, rnd, int(with_keys),
+               _ptr(msg, _u8p))
+    return msg
+
+
+def wire_unpack(msg, cached_signature: int, k_core: int, k_exp: int):
+    """Takes a push message apart on the receiver's side.  Returns (status, core_idx or None, exp_idx, val,
+    signature): status 0 = taken, 1 = keys wanted (nothing else is meaningful), -1 = malformed."""
+    m = np.ascontiguousarray(msg, dtype=np.uint8)
+    core = np.zeros(k_core, np.uint32)
+    exp = np.zeros(k_exp, np.uint32)
+    val = np.zeros(k_core + k_exp, np.float32)
+    sig = ctypes.c_uint64(cached_signature)
+    st = int(_wire_unpack(_ptr(m, _u8p), m.size, cached_signature, k_core, k_exp, _ptr(core, _u32p), _ptr(exp, _u32p),
+                          _ptr(val, _f32p), ctypes.byref(sig)))
+    carried_keys = st == 0 and m.size >= 8 and (int(m[4]) & 1) == 1
+    return st, (core if carried_keys else None), exp, val, int(sig.value)
 
 
 def run_round(w, grads: Sequence[np.ndarray], c: float, k_core: int, k_exp: int,

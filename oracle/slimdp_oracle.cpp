@@ -256,6 +256,81 @@ uint64_t oracle_core_signature(const uint32_t* keys, uint64_t count) {
     return sig;
 }
 
+// ---- one worker's push as a message (Section 3.5: values + a signature of the cached keys for
+// the core, <key, value> pairs for the explorer) ------------------------------------------------
+// Layout, little-endian, every field 4-byte aligned:
+//    0 u32 magic 0x57504453 ("SDPW")      4 u32 flags (bit 0: the core's keys are included)
+//    8 u64 signature of the sender's core keys
+//   16 u32 k_core   20 u32 k_exp   24 u32 worker   28 u32 round
+//   32 [k_core x u32 keys, if flags bit 0]  k_core x f32 values  k_exp x (u32 key, f32 value)
+// so a push costs 32 + 4 k_core + 8 k_exp bytes = (2 alpha - beta) n words plus the header when the
+// receiver's cached keys are current, and 4 k_core more when they have to be sent again.
+uint64_t oracle_wire_message_bytes(uint64_t k_core, uint64_t k_exp, int with_keys) {
+    return 32 + 4 * k_core * (with_keys ? 2 : 1) + 8 * k_exp;
+}
+
+static void put_u32(uint8_t* p, uint32_t v) {
+    for (int b = 0; b < 4; ++b) p[b] = (uint8_t)(v >> (8 * b));
+}
+static uint32_t get_u32(const uint8_t* p) {
+    uint32_t v = 0;
+    for (int b = 0; b < 4; ++b) v |= (uint32_t)p[b] << (8 * b);
+    return v;
+}
+
+void oracle_wire_pack(const uint32_t* core_idx, uint64_t k_core, const uint32_t* exp_idx, uint64_t k_exp,
+                      const float* val, uint32_t worker, uint32_t round, int with_keys, uint8_t* msg) {
+    const uint64_t sig = oracle_core_signature(core_idx, k_core);
+    put_u32(msg + 0, 0x57504453u);
+    put_u32(msg + 4, with_keys ? 1u : 0u);
+    put_u32(msg + 8, (uint32_t)sig);
+    put_u32(msg + 12, (uint32_t)(sig >> 32));
+    put_u32(msg + 16, (uint32_t)k_core);
+    put_u32(msg + 20, (uint32_t)k_exp);
+    put_u32(msg + 24, worker);
+    put_u32(msg + 28, round);
+    uint8_t* p = msg + 32;
+    if (with_keys)
+        for (uint64_t j = 0; j < k_core; ++j, p += 4) put_u32(p, core_idx[j]);
+    for (uint64_t j = 0; j < k_core; ++j, p += 4) put_u32(p, f32_bits(val[j]));
+    for (uint64_t j = 0; j < k_exp; ++j, p += 8) {
+        put_u32(p, exp_idx[j]);
+        put_u32(p + 4, f32_bits(val[k_core + j]));
+    }
+}
+
+// The receiver's side.  Returns 0 when the message was taken apart (val, exp_idx and, if the
+// message carried the keys, core_idx and *signature_out written), 1 when the sender's keys are not
+// the ones the receiver has cached and the message does not carry them ("keys wanted": nothing is
+// written; the sender's next push includes the keys), -1 when the message is malformed (magic,
+// sizes, or included keys that do not give the signature in the header).
+int32_t oracle_wire_unpack(const uint8_t* msg, uint64_t msg_bytes, uint64_t cached_signature, uint64_t k_core,
+                           uint64_t k_exp, uint32_t* core_idx, uint32_t* exp_idx, float* val,
+                           uint64_t* signature_out) {
+    if (msg_bytes < 32 || get_u32(msg) != 0x57504453u) return -1;
+    const uint32_t flags = get_u32(msg + 4);
+    const uint64_t sig = (uint64_t)get_u32(msg + 8) | ((uint64_t)get_u32(msg + 12) << 32);
+    if (flags > 1u || get_u32(msg + 16) != k_core || get_u32(msg + 20) != k_exp) return -1;
+    if (msg_bytes != oracle_wire_message_bytes(k_core, k_exp, (int)flags)) return -1;
+    const uint8_t* p = msg + 32;
+    if (flags & 1u) {
+        std::vector<uint32_t> keys(k_core);
+        for (uint64_t j = 0; j < k_core; ++j) keys[j] = get_u32(p + 4 * j);
+        if (oracle_core_signature(keys.data(), k_core) != sig) return -1;
+        for (uint64_t j = 0; j < k_core; ++j) core_idx[j] = keys[j];
+        *signature_out = sig;
+        p += 4 * k_core;
+    } else if (sig != cached_signature) {
+        return 1;
+    }
+    for (uint64_t j = 0; j < k_core; ++j, p += 4) val[j] = bits_f32(get_u32(p));
+    for (uint64_t j = 0; j < k_exp; ++j, p += 8) {
+        exp_idx[j] = get_u32(p);
+        val[k_core + j] = bits_f32(get_u32(p + 4));
+    }
+    return 0;
+}
+
 // Plump-DP (Section 2.1): every worker pushes its whole update.
 void oracle_dense_merge(float* w, uint64_t n, uint32_t K, const float* const* grads, float eta) {
     for (uint32_t k = 0; k < K; ++k)

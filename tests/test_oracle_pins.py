@@ -439,3 +439,89 @@ def test_key_signature_pins():
     for other in (np.array([5, 9, 13, 4000000000], np.uint32), np.array([9, 5, 12, 4000000000], np.uint32),
                   keys[:3], np.append(keys, np.uint32(7))):
         assert oracle.core_signature(other) != want
+
+
+# ------------------------------------------------------------- wire message
+
+def _mix64(z):
+    M = (1 << 64) - 1
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & M
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & M
+    return z ^ (z >> 31)
+
+
+def _signature_py(keys):
+    M = (1 << 64) - 1
+    return sum(_mix64((((j << 32) | int(k)) + 0x9E3779B97F4A7C15) & M) for j, k in enumerate(keys)) & M
+
+
+def test_wire_message_layout_byte_for_byte():
+    # Section 3.5: the core travels as values plus a signature of the cached keys, the explorer as
+    # <key, value> pairs.  The expected bytes are assembled by hand here, field by field.
+    import struct
+    core, exp = [3, 9], [5]
+    val = [1.0, 2.0, -0.5]
+    sig = _signature_py(core)
+    head = struct.pack("<4sIQIIII", b"SDPW", 0, sig, 2, 1, 7, 11)
+    body = struct.pack("<ff", 1.0, 2.0) + struct.pack("<If", 5, -0.5)
+    msg = oracle.wire_pack(core, exp, val, 7, 11, False)
+    assert bytes(msg) == head + body
+    head_k = struct.pack("<4sIQIIII", b"SDPW", 1, sig, 2, 1, 7, 11)
+    msg_k = oracle.wire_pack(core, exp, val, 7, 11, True)
+    assert bytes(msg_k) == head_k + struct.pack("<II", 3, 9) + body
+    assert oracle.wire_message_bytes(2, 1, False) == 48 and oracle.wire_message_bytes(2, 1, True) == 56
+
+
+def test_wire_message_size_is_the_papers_amount_plus_a_header():
+    # (2 alpha - beta) n words per push (Section 3.5), checked against Table 1's time ratios above;
+    # the message adds a 32-byte header, and 4 k_core bytes when the keys have to travel again
+    n = 10 ** 6
+    for alpha, beta in ((0.2, 0.1), (0.3, 0.15), (0.5, 0.25)):
+        k_core, k_exp = round(beta * n), round((alpha - beta) * n)
+        assert oracle.wire_message_bytes(k_core, k_exp, False) == 4 * round((2 * alpha - beta) * n) + 32
+        assert oracle.wire_message_bytes(k_core, k_exp, True) == 4 * round((2 * alpha - beta) * n) + 32 + 4 * k_core
+
+
+def test_wire_round_trip_and_stale_keys():
+    rng = np.random.default_rng(21)
+    n, k_core, k_exp = 5000, 700, 333
+    idx = rng.permutation(n).astype(np.uint32)
+    core, exp = np.sort(idx[:k_core]), np.sort(idx[k_core:k_core + k_exp])
+    val = rng.standard_normal(k_core + k_exp).astype(np.float32)
+    val.view(np.uint32)[5] = 0x7FC12345          # a NaN payload must survive: the message moves bits
+    sig = _signature_py(core)
+    assert oracle.core_signature(core) == sig
+    # receiver with current keys: values and pairs come back bit for bit, the cache is left alone
+    st, got_core, got_exp, got_val, new_sig = oracle.wire_unpack(oracle.wire_pack(core, exp, val, 2, 9, False), sig,
+                                                                  k_core, k_exp)
+    assert st == 0 and got_core is None and new_sig == sig
+    assert np.array_equal(got_exp, exp) and np.array_equal(bits(got_val), bits(val))
+    # receiver whose cached keys are stale: "keys wanted", nothing is taken
+    stale = np.sort(idx[1:k_core + 1])
+    st, _, _, _, _ = oracle.wire_unpack(oracle.wire_pack(core, exp, val, 2, 9, False), _signature_py(stale), k_core, k_exp)
+    assert st == 1
+    # the next push carries the keys: taken whatever the cache held, keys and signature handed over
+    st, got_core, got_exp, got_val, new_sig = oracle.wire_unpack(oracle.wire_pack(core, exp, val, 2, 10, True),
+                                                                  _signature_py(stale), k_core, k_exp)
+    assert st == 0 and np.array_equal(got_core, core) and new_sig == sig
+    assert np.array_equal(got_exp, exp) and np.array_equal(bits(got_val), bits(val))
+    # unpack + merge is the same as merging what was packed
+    w = rng.standard_normal(n).astype(np.float32)
+    assert np.array_equal(bits(oracle.merge(w, got_core, [got_exp], [got_val], 0.25)),
+                          bits(oracle.merge(w, core, [exp], [val], 0.25)))
+
+
+def test_wire_malformed_messages_are_refused():
+    core, exp = np.array([1, 4, 6], np.uint32), np.array([2, 3], np.uint32)
+    val = np.arange(5, dtype=np.float32)
+    sig = _signature_py(core)
+    good = oracle.wire_pack(core, exp, val, 0, 0, True)
+    assert oracle.wire_unpack(good, 0, 3, 2)[0] == 0
+    bad = good.copy(); bad[0] ^= 1                       # magic
+    assert oracle.wire_unpack(bad, sig, 3, 2)[0] == -1
+    assert oracle.wire_unpack(good[:-4], sig, 3, 2)[0] == -1          # truncated
+    assert oracle.wire_unpack(good, sig, 4, 2)[0] == -1               # sizes other than agreed
+    bad = good.copy(); bad[32] ^= 1                      # an included key that the signature does not cover
+    assert oracle.wire_unpack(bad, sig, 3, 2)[0] == -1
+    bad = good.copy(); bad[4] = 2                        # unknown flag
+    assert oracle.wire_unpack(bad, sig, 3, 2)[0] == -1
