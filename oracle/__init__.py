@@ -47,6 +47,11 @@ _wire_pack = _sig("oracle_wire_pack", None, _u32p, ctypes.c_uint64, _u32p, ctype
                   ctypes.c_uint32, ctypes.c_int, _u8p)
 _wire_unpack = _sig("oracle_wire_unpack", ctypes.c_int32, _u8p, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64,
                     ctypes.c_uint64, _u32p, _u32p, _f32p, ctypes.POINTER(ctypes.c_uint64))
+_u64p = ctypes.POINTER(ctypes.c_uint64)
+_i8p = ctypes.POINTER(ctypes.c_int8)
+_select_seg = _sig("oracle_select_core_segmented", None, _f32p, ctypes.c_uint64, _u64p, _u64p, ctypes.c_uint32, _u32p)
+_quant = _sig("oracle_quantize_q8", None, _f32p, ctypes.c_uint64, ctypes.c_uint32, _i8p, _f32p)
+_dequant = _sig("oracle_dequantize_q8", None, _i8p, _f32p, ctypes.c_uint64, ctypes.c_uint32, _f32p)
 _wmerge = _sig("oracle_worker_merge", None, _f32p, _u32p, ctypes.c_uint64, _u32p, ctypes.c_uint64, _f32p)
 
 
@@ -156,6 +161,38 @@ def worker_merge(w_local, core_idx, exp_idx, pulled) -> np.ndarray:
 def core_signature(keys) -> int:
     k = _u32(keys)
     return int(_signature(_ptr(k, _u32p), k.size))
+
+
+def select_core_segmented(scores, seg_off: Sequence[int], seg_k: Sequence[int]) -> np.ndarray:
+    """Per-segment top-k: segment s = [seg_off[s], seg_off[s+1]) contributes its seg_k[s] largest scores."""
+    s = _f32(scores)
+    off = np.ascontiguousarray(seg_off, dtype=np.uint64)
+    ks = np.ascontiguousarray(seg_k, dtype=np.uint64)
+    assert off.size == ks.size + 1 and off[0] == 0 and off[-1] == s.size
+    assert all(int(ks[i]) <= int(off[i + 1]) - int(off[i]) for i in range(ks.size))
+    out = np.empty(int(ks.sum()), np.uint32)
+    _select_seg(_ptr(s, _f32p), s.size, _ptr(off, _u64p), _ptr(ks, _u64p), ks.size, _ptr(out, _u32p))
+    return out
+
+
+Q8_BUCKET = 256
+
+
+def quantize_q8(val, bucket: int = Q8_BUCKET):
+    """(codes int8[m], scales float32[ceil(m / bucket)]) of the packed values."""
+    v = _f32(val)
+    codes = np.zeros(v.size, np.int8)
+    scales = np.zeros((v.size + bucket - 1) // bucket, np.float32)
+    _quant(_ptr(v, _f32p), v.size, bucket, _ptr(codes, _i8p), _ptr(scales, _f32p))
+    return codes, scales
+
+
+def dequantize_q8(codes, scales, bucket: int = Q8_BUCKET) -> np.ndarray:
+    c = np.ascontiguousarray(codes, dtype=np.int8)
+    s = _f32(scales)
+    out = np.zeros(c.size, np.float32)
+    _dequant(_ptr(c, _i8p), _ptr(s, _f32p), c.size, bucket, _ptr(out, _f32p))
+    return out
 
 
 def wire_message_bytes(k_core: int, k_exp: int, with_keys: bool) -> int:

@@ -185,6 +185,31 @@ void oracle_select_core(const float* scores, uint64_t n, uint64_t k_core, uint32
     std::sort(core_idx, core_idx + k_core);
 }
 
+// A "model-specific significance measure" (Section 5) in its simplest form: the ranking of
+// Section 3.2 done per layer.  The vector is cut into segments [seg_off[s], seg_off[s+1]); segment
+// s contributes its seg_k[s] parameters of largest score (ties to the smaller index); the core is
+// the union, ascending.
+void oracle_select_core_segmented(const float* scores, uint64_t n, const uint64_t* seg_off, const uint64_t* seg_k,
+                                  uint32_t segments, uint32_t* core_idx) {
+    (void)n;
+    uint64_t out = 0;
+    for (uint32_t s = 0; s < segments; ++s) {
+        const uint64_t b = seg_off[s], e = seg_off[s + 1];
+        std::vector<Ranked> v(e - b);
+        for (uint64_t i = b; i < e; ++i) {
+            v[i - b].key = f32_bits(scores[i]);
+            v[i - b].idx = (uint32_t)i;
+        }
+        std::sort(v.begin(), v.end(), [](const Ranked& x, const Ranked& y) {
+            if (x.key != y.key) return x.key > y.key;
+            return x.idx < y.idx;
+        });
+        for (uint64_t j = 0; j < seg_k[s]; ++j) core_idx[out + j] = v[j].idx;
+        std::sort(core_idx + out, core_idx + out + seg_k[s]);
+        out += seg_k[s];
+    }
+}
+
 // Section 3.3 step 2: worker `worker`'s explorer for communication `round`.
 // core_idx ascending.  noncore = ascending complement; explorer =
 // { noncore[pi(j)] : j < k_exp }, ascending.
@@ -329,6 +354,40 @@ int32_t oracle_wire_unpack(const uint8_t* msg, uint64_t msg_bytes, uint64_t cach
         val[k_core + j] = bits_f32(get_u32(p + 4));
     }
     return 0;
+}
+
+// ---- 8-bit codes for the pushed values ---------------------------------------------------------
+// Section 2.2 ends by noting that the method combines with quantisation of what is sent; the paper
+// defines no quantiser, so this library fixes one (deterministic, so that both sides agree bit for
+// bit): the packed values are cut into buckets of `bucket` consecutive entries; a bucket's scale is
+// the largest finite magnitude in it; a value becomes the signed 8-bit code
+//     rint(v * (127 / scale)) clamped to [-127, 127]    (fp32 division, fp32 product, ties to even),
+// 0 if the scale is 0 or v is a NaN; an infinity gets +-127.  The receiver reads code * (scale / 127).
+void oracle_quantize_q8(const float* val, uint64_t m, uint32_t bucket, int8_t* codes, float* scales) {
+    for (uint64_t b0 = 0, b = 0; b0 < m; b0 += bucket, ++b) {
+        const uint64_t b1 = (b0 + bucket < m) ? b0 + bucket : m;
+        float amax = 0.0f;
+        for (uint64_t j = b0; j < b1; ++j) {
+            const float a = std::fabs(val[j]);
+            if (a <= 3.402823466e+38f && a > amax) amax = a;   // NaNs and infinities do not set the scale
+        }
+        scales[b] = amax;
+        const float inv = (amax > 0.0f) ? 127.0f / amax : 0.0f;
+        for (uint64_t j = b0; j < b1; ++j) {
+            const float v = val[j];
+            float q = std::isnan(v) ? 0.0f : std::rint(v * inv);
+            if (q > 127.0f) q = 127.0f;
+            if (q < -127.0f) q = -127.0f;
+            codes[j] = (int8_t)q;
+        }
+    }
+}
+
+void oracle_dequantize_q8(const int8_t* codes, const float* scales, uint64_t m, uint32_t bucket, float* val) {
+    for (uint64_t j = 0; j < m; ++j) {
+        const float step = scales[j / bucket] / 127.0f;
+        val[j] = (float)codes[j] * step;
+    }
 }
 
 // Plump-DP (Section 2.1): every worker pushes its whole update.

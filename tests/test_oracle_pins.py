@@ -525,3 +525,69 @@ def test_wire_malformed_messages_are_refused():
     assert oracle.wire_unpack(bad, sig, 3, 2)[0] == -1
     bad = good.copy(); bad[4] = 2                        # unknown flag
     assert oracle.wire_unpack(bad, sig, 3, 2)[0] == -1
+
+
+# ------------------------------------------------- per-segment selection (Section 5: model-specific significance)
+
+def test_segmented_select_brute_force_and_reductions():
+    rng = np.random.default_rng(30)
+    # brute force on tiny segments with many ties: the per-segment winners maximise the segment's sorted key tuple
+    for trial in range(40):
+        sizes = rng.integers(1, 6, 3)
+        off = np.concatenate([[0], np.cumsum(sizes)])
+        S = (rng.integers(0, 3, off[-1]) * 0.5).astype(np.float32)
+        ks = [int(rng.integers(0, sz + 1)) for sz in sizes]
+        got = oracle.select_core_segmented(S, off, ks)
+        want = []
+        for s in range(3):
+            idx = list(range(off[s], off[s + 1]))
+            best = max(itertools.combinations(idx, ks[s]),
+                       key=lambda c: (sorted((float(S[i]) for i in c), reverse=True), [-i for i in c]))
+            want += sorted(best)
+        assert got.tolist() == want, (S, off, ks)
+    # one segment = the global selection; and every segment is independent of the others
+    S = np.abs(rng.standard_normal(5000)).astype(np.float32)
+    assert np.array_equal(oracle.select_core_segmented(S, [0, 5000], [700]), oracle.select_core(S, 700))
+    off, ks = [0, 1000, 1001, 3500, 5000], [100, 1, 0, 1500]
+    got = oracle.select_core_segmented(S, off, ks)
+    parts = [oracle.select_core(S[off[s]:off[s + 1]], ks[s]).astype(np.int64) + off[s] for s in range(4)]
+    assert np.array_equal(got, np.concatenate(parts))
+    S2 = S.copy()
+    S2[:1000] = rng.random(1000).astype(np.float32)          # segment 0 changed: the others' choices stay
+    got2 = oracle.select_core_segmented(S2, off, ks)
+    assert np.array_equal(got2[got2 >= 1000], got[got >= 1000])
+
+
+# ---------------------------------------------------------------- 8-bit codes for the pushed values
+
+def test_q8_hand_example_and_special_values():
+    # one bucket, exact in binary: scale 1, inverse step 127; -0.5 * 127 = -63.5 rounds to the even -64
+    codes, scales = oracle.quantize_q8(np.array([1.0, -0.5, 0.25, 0.0], np.float32), bucket=4)
+    assert codes.tolist() == [127, -64, 32, 0] and scales.tolist() == [1.0]
+    deq = oracle.dequantize_q8(codes, scales, bucket=4)
+    step = np.float32(1.0) / np.float32(127.0)
+    assert bits(deq).tolist() == bits(np.array([127, -64, 32, 0], np.float32) * step).tolist()
+    # an all-zero bucket; NaN -> 0; infinities -> +-127 and do not set the scale; ragged last bucket
+    v = np.array([0, 0, 0, 0, np.nan, np.inf, -np.inf, 2.0, -3.0], np.float32)
+    codes, scales = oracle.quantize_q8(v, bucket=4)
+    assert scales.tolist() == [0.0, 2.0, 3.0]
+    assert codes.tolist() == [0, 0, 0, 0, 0, 127, -127, 127, -127]
+
+
+def test_q8_codes_are_one_rounding_of_the_scaled_value_and_the_error_is_half_a_step():
+    rng = np.random.default_rng(31)
+    v = (rng.standard_normal(5000) * np.exp(rng.uniform(-8, 2, 5000))).astype(np.float32)
+    codes, scales = oracle.quantize_q8(v)
+    assert scales.size == 20
+    for b in range(20):
+        seg = v[256 * b:256 * (b + 1)]
+        assert scales[b] == np.abs(seg).max()
+        inv = np.float32(127.0) / scales[b]                           # IEEE single division
+        want = np.clip(np.rint(seg * inv), -127, 127).astype(np.int8)  # IEEE single product, ties to even
+        assert np.array_equal(codes[256 * b:256 * (b + 1)], want), b
+    deq = oracle.dequantize_q8(codes, scales)
+    step = np.repeat(scales / np.float32(127.0), 256)[:v.size]
+    assert np.all(np.abs(deq.astype(np.float64) - v) <= 0.5 * step.astype(np.float64) * (1 + 1e-6))
+    # a second pass changes nothing: the codes of the decoded values are the codes
+    codes2, scales2 = oracle.quantize_q8(deq)
+    assert np.array_equal(codes2, codes)
