@@ -227,7 +227,7 @@ def run_ours(args):
     w_host, g_host = all_inputs(cfg)
     w = torch.from_numpy(w_host).to(device)
     grads = [torch.from_numpy(g).to(device) for g in g_host]
-    buf = P.RoundBuffers(N, K, k_core, k_exp, device)
+    buf = P.RoundBuffers(N, K, k_core, k_exp, device, staging=not args.no_staging)
     bytes_model = model_bytes(N, K, k_core, k_exp)
 
     def barrier():
@@ -238,7 +238,7 @@ def run_ours(args):
         # the whole round as ONE C-ABI call on device buffers (scoring folded into the selection's pass
         # over all parameters, explorer ranks beside it, then explorer indices and the exchange)
         P.slimdp_round(w, grads, cfg.c, cfg.seed, t, cfg.eta, buf.scores, buf.core_idx, buf.core_aux, buf.exp_idx,
-                       buf.val, buf.pulled, buf.select_ws, buf.explore_ws)
+                       buf.val, buf.pulled, buf.select_ws, buf.explore_ws, buf.stage)
 
     # warm-up: successive rounds t = 0, 1, ... on the evolving model, as in training
     t = 0
@@ -431,6 +431,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-staging", action="store_true",
+                    help="run slimdp_round without its staging area (the exchange then gathers the core's values)")
     ap.add_argument("--timeline", default="",
                     help="also write the kernel timeline of three extra rounds (start, duration, stream) to this file")
     ap.add_argument("--scale", type=int, default=0,

@@ -20,9 +20,8 @@
  *     host-side array whose K entries are device pointers; it is read during
  *     the call and may be freed as soon as the call returns.
  *   - The caller owns every buffer.  The library allocates no device memory,
- *     creates no stream (slimdp_round and slimdp_round_host excepted, see
- *     there), and never synchronises except in slimdp_read_status and
- *     slimdp_round_host.  All work is enqueued on `stream` (a cudaStream_t
+ *     creates no stream (round contexts excepted, see slimdp_round), and never
+ *     synchronises except in slimdp_read_status and slimdp_round_host.  All work is enqueued on `stream` (a cudaStream_t
  *     passed as void*; NULL is the legacy default stream) and is ordered with
  *     other work on that stream.
  *   - Arguments are validated on the host before anything is enqueued.  A
@@ -117,7 +116,9 @@ slimdp_status slimdp_score(const float* w, const float* const* grads, uint32_t K
  *   core_aux  [slimdp_core_aux_bytes(n)] (written): bitmap + directory, see above
  *   ws        [ws_bytes >= slimdp_select_workspace_bytes(n)] scratch, contents undefined after
  * Device-side consistency failures are recorded in the first word of ws; read
- * them with slimdp_read_status(ws, stream).
+ * them with slimdp_read_status(ws, stream).  The last kernel of the selection
+ * is a cooperative launch whose CTAs meet at a grid barrier; every wait there
+ * is bounded, and a wait that runs out is reported the same way.
  */
 slimdp_status slimdp_select_core(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx,
                                  void* core_aux, void* ws, size_t ws_bytes, void* stream);
@@ -283,6 +284,81 @@ slimdp_status slimdp_worker_merge_batched(float* const* w_local, uint32_t K, uin
 slimdp_status slimdp_core_signature(const uint32_t* keys, uint64_t count, uint64_t* signature, void* stream);
 size_t slimdp_wire_bytes(uint64_t k_core, uint64_t k_exp);
 
+/* ------------------------------------------ selection over a sharded model ---
+ * The parameter-server setting of Section 2.1 with the global model cut into
+ * contiguous shards, one per GPU.  Scoring, pack, merge and pull work shard by
+ * shard on local indices; the core does not, because Section 3.2 ranks all
+ * parameters.  These calls are the selection cut at its reduction points, so
+ * that the exact global core costs three all-reduces of 4096 counters and one
+ * all-gather of two counters per shard:
+ *   slimdp_select_shard_begin(k_total, state)         state <- (prefix 0, rank k_total), on every shard
+ *   for round = 0, 1, 2 (digits of 12, 10, 10 bits, most significant first):
+ *     clear hist; slimdp_select_hist(shard, round, state, hist)   hist[b] += keys of the shard with digit b
+ *                                                                 (and the prefix found so far)
+ *     sum hist over all shards (all-reduce)
+ *     slimdp_select_resolve(hist, round, state)      the digit that holds the wanted rank; the same on every shard
+ *   now state holds the threshold T (the k_total-th largest key of the whole model) and r, the
+ *   number of keys equal to T that belong to the core
+ *   clear counts; slimdp_select_count(shard, state, counts)   counts[0] += keys > T, counts[1] += keys == T
+ *   all-gather the counts: shard g admits quota_g = min(equal_g, max(0, r - sum of equal_h, h < g))
+ *   of its equal keys (ties go to the smaller global index, and shards are index ranges), and its
+ *   part of the core has k_g = greater_g + quota_g members
+ *   slimdp_select_emit(shard, T, quota_g, k_g, ...)  the shard's core_idx (shard-local indices,
+ *   ascending) and core_aux, exactly as slimdp_select_core writes them for a whole vector
+ * The concatenation of the shards' lists (local index + shard offset) is bit for bit the core that
+ * slimdp_select_core finds on the whole vector.  With one process per GPU the two reductions are
+ * NCCL calls on the device buffers `hist` and `counts`; nothing here waits on another GPU.
+ *   state   DEVICE record of 16 bytes, 8-byte aligned: uint32 prefix (after round 2: T), int32 status
+ *           (SLIMDP_OK, or SLIMDP_ERR_INTERNAL if the summed histogram held fewer keys than the rank),
+ *           uint64 remaining rank (after round 2: r)
+ *   hist    DEVICE uint64[4096] (rounds 1 and 2 use the first 1024), added to
+ *   counts  DEVICE uint64[2], added to
+ *   scores  the shard's scores [n_shard] (n_shard may be 0 in hist / count) */
+slimdp_status slimdp_select_shard_begin(uint64_t k_total, void* state, void* stream);
+slimdp_status slimdp_select_hist(const float* scores, uint64_t n_shard, uint32_t round, const void* state,
+                                 uint64_t* hist, void* stream);
+slimdp_status slimdp_select_resolve(const uint64_t* hist, uint32_t round, void* state, void* stream);
+slimdp_status slimdp_select_count(const float* scores, uint64_t n_shard, const void* state, uint64_t* counts,
+                                  void* stream);
+slimdp_status slimdp_select_emit(const float* scores, uint64_t n_shard, uint32_t threshold_bits, uint64_t tie_quota,
+                                 uint64_t k_shard, uint32_t* core_idx, void* core_aux, void* ws, size_t ws_bytes,
+                                 void* stream);
+
+/* One worker's push as a message (Section 3.5: the core as values plus the
+ * signature of its cached keys, the explorer as <key, value> pairs), built and
+ * taken apart on the device.  Layout, little-endian, every field 4-byte aligned:
+ *      0 u32 magic 0x57504453 ("SDPW")    4 u32 flags (bit 0: the core's keys are included)
+ *      8 u64 signature of the sender's core keys (slimdp_core_signature)
+ *     16 u32 k_core   20 u32 k_exp   24 u32 worker   28 u32 round
+ *     32 [k_core x u32 keys, if flags bit 0]  k_core x f32 values  k_exp x (u32 key, f32 value)
+ * i.e. 32 + 4 k_core + 8 k_exp bytes = (2 alpha - beta) n words plus the header
+ * while the receiver's cached keys are current, 4 k_core more when the keys
+ * travel again.  Values are moved as bits.
+ * slimdp_wire_pack:   core_idx [k_core], exp_idx [k_exp], val [k_core + k_exp] as written by
+ *   slimdp_pack (read); signature: DEVICE uint64 holding slimdp_core_signature(core_idx) (read);
+ *   msg [slimdp_wire_message_bytes(k_core, k_exp, with_keys)], 16-byte aligned (written).
+ * slimdp_wire_unpack: the receiver's side.  The verdict is reached on the device and left in
+ *   status[0]: 0 = taken apart (exp_idx, val and *signature_out written; core_idx too if the
+ *   message carried the keys, after their signature was checked against the header's);
+ *   SLIMDP_WIRE_KEYS_WANTED = the sender's keys are not the ones whose signature the receiver has
+ *   cached and the message does not carry them: nothing else is written, and the sender's next push
+ *   is to be packed with with_keys = 1; -1 = malformed (magic, sizes other than k_core / k_exp /
+ *   msg_bytes, unknown flags, keys that do not match the header's signature).
+ *   cached_signature: DEVICE uint64 (read); signature_out: DEVICE uint64 (may be the same word);
+ *   status: DEVICE scratch of 16 bytes, 8-byte aligned (status[0] is the verdict).
+ *   core_idx [k_core], exp_idx [k_exp], val [k_core + k_exp] (written as described).
+ * slimdp_wire_read_status synchronises `stream` and returns the verdict as SLIMDP_OK,
+ *   SLIMDP_WIRE_KEYS_WANTED or SLIMDP_ERR_INVALID_ARG (malformed). */
+#define SLIMDP_WIRE_KEYS_WANTED 1
+size_t slimdp_wire_message_bytes(uint64_t k_core, uint64_t k_exp, int with_keys);
+slimdp_status slimdp_wire_pack(const uint32_t* core_idx, uint64_t k_core, const uint32_t* exp_idx, uint64_t k_exp,
+                               const float* val, const uint64_t* signature, uint32_t worker, uint32_t round,
+                               int with_keys, void* msg, void* stream);
+slimdp_status slimdp_wire_unpack(const void* msg, size_t msg_bytes, const uint64_t* cached_signature,
+                                 uint64_t k_core, uint64_t k_exp, uint32_t* core_idx, uint32_t* exp_idx, float* val,
+                                 uint64_t* signature_out, int32_t* status, void* stream);
+slimdp_status slimdp_wire_read_status(const int32_t* status, void* stream);
+
 /* --------------------------------------------------------------- status ---
  * Synchronises `stream`, then returns the sticky status word kept in the first
  * 4 bytes of a workspace used by slimdp_select_core / slimdp_sample_explore*:
@@ -305,29 +381,40 @@ uint64_t slimdp_launch_count(void);
  * deltas = grads, called in that order.  What differs is how the device gets
  * there:
  *   - Scoring is folded into the selection's single pass over all parameters
- *     (n >= 2^21, k_core > 0 and 16-byte aligned w_global / grads / scores;
- *     otherwise the two calls above run): each score is computed in registers
- *     and classified on the spot, so the n scores are neither written nor read
- *     back.  `scores` is then only scratch: it holds the scores if the
- *     selection had to fall back to its full path (e.g. millions of equal
- *     scores around the threshold) and is left untouched otherwise.  Callers
- *     that want the scores call slimdp_score.
+ *     (n >= 2^21, k_core > 0, K <= 20 and 16-byte aligned w_global / grads /
+ *     scores; otherwise the calls above run one after the other): each score
+ *     is computed as the parameter streams by and classified on the spot, so
+ *     the n scores are neither written nor read back.  `scores` is then only
+ *     scratch: it holds the scores if the selection had to fall back to its
+ *     full path (e.g. millions of equal scores around the threshold) and is
+ *     left untouched otherwise.  Callers that want the scores call slimdp_score.
+ *   - With a staging area (`stage`, optional) that pass also sets aside the K
+ *     update values of every parameter that is certainly in the core or a
+ *     candidate for it, while it has them at hand; the exchange then streams
+ *     them instead of gathering K + 1 scattered lines per core parameter.
+ *     slimdp_round_stage_bytes gives the size (0: staging does not apply to
+ *     these sizes, e.g. a core of more than half the parameters); stage = NULL
+ *     or a smaller area simply turns staging off.  Results do not depend on it.
  *   - The steps of a round depend on one another as a graph, not a chain: the
  *     explorer's ranks need the sizes only, so they are computed and sorted
  *     beside the pass over all parameters, in the part of every SM that the
  *     pass leaves free (the pass keeps its loads in flight in shared memory,
- *     one CTA per SM, and so needs few registers and threads); and of the
- *     selection's two ways to the threshold (from the candidates, or from all
- *     scores when the bracket failed) only one does any work, so the idle
- *     one's kernels run beside the other's.  For that this call keeps, per
- *     device, THREE non-blocking streams and six events of its own, created on
- *     the first call on that device and kept for the life of the process (the
- *     one exception to "creates no stream"): one of the highest priority for
- *     the chain of kernels that decides the round's time, one of the lowest
- *     for the ranks, one for the idle way.  `stream` forks into them at the
- *     start of the call and waits for them at the end, inside the call, so
- *     for the caller the whole round is ordered on `stream` as usual.  Calls
- *     on one device are serialised on the host by a lock while they enqueue.
+ *     one CTA per SM, and so needs few registers and threads).  For that the
+ *     round runs on two streams of a round context: one of the highest
+ *     priority for the chain of kernels that decides the round's time, one of
+ *     the lowest for the ranks.  `stream` forks into them at the start of the
+ *     call and waits for them at the end, inside the call, so for the caller
+ *     the whole round is ordered on `stream` as usual.
+ * Round contexts: slimdp_round_ctx_create makes one on the current device (two
+ * non-blocking streams, four events; no device memory); the caller owns it,
+ * passes it to slimdp_round and destroys it with slimdp_round_ctx_destroy once
+ * the rounds that used it have completed.  Calls that share a context are
+ * serialised by a lock inside it while they enqueue and run one after the
+ * other on its streams; calls with different contexts are independent, on the
+ * host and on the device, as long as their buffers are.  ctx = NULL uses a
+ * context that the library creates for the device on first use and keeps
+ * until slimdp_round_release_default_ctx is called on that device (or the
+ * process ends): the one piece of state the library keeps by itself.
  *   w_global [n] (updated in place); grads HOST array of K device pointers [n] (read)
  *   scores [n] scratch (see above); core_idx [k_core], core_aux (written; as slimdp_select_core)
  *   exp_idx HOST array of K device pointers [k_exp] (written)
@@ -335,12 +422,19 @@ uint64_t slimdp_launch_count(void);
  *   select_ws, explore_ws: two workspaces that do NOT overlap (both are in use
  *   at once), of at least slimdp_select_workspace_bytes(n) and
  *   slimdp_explore_workspace_bytes(n, k_exp, K) bytes; each keeps the status
- *   word of its step (slimdp_read_status). */
+ *   word of its step (slimdp_read_status).
+ *   stage [stage_bytes] optional scratch, 256-byte aligned, overlapping nothing else */
+typedef struct slimdp_round_ctx slimdp_round_ctx;
+slimdp_status slimdp_round_ctx_create(slimdp_round_ctx** ctx);
+slimdp_status slimdp_round_ctx_destroy(slimdp_round_ctx* ctx);
+slimdp_status slimdp_round_release_default_ctx(void);
+size_t slimdp_round_stage_bytes(uint64_t n, uint32_t K, uint64_t k_core);
 slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t K, uint64_t n, float c,
                            uint64_t k_core, uint64_t k_exp, uint64_t seed, uint32_t round, float eta, float* scores,
                            uint32_t* core_idx, void* core_aux, uint32_t* const* exp_idx, float* const* val,
                            float* const* pulled, void* select_ws, size_t select_ws_bytes, void* explore_ws,
-                           size_t explore_ws_bytes, void* stream);
+                           size_t explore_ws_bytes, void* stage, size_t stage_bytes, slimdp_round_ctx* ctx,
+                           void* stream);
 
 /* Measurement aid (the paper has no counterpart).  The next slimdp_round called
  * from this host thread records `begin_event` just before and `end_event` just

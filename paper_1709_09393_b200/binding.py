@@ -51,11 +51,24 @@ EXPORTS = {
     "slimdp_worker_merge_batched": (ctypes.c_int32, [_pp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _vp]),
     "slimdp_core_signature": (ctypes.c_int32, [_vp, _u64, _vp, _vp]),
     "slimdp_wire_bytes": (_sz, [_u64, _u64]),
+    "slimdp_select_shard_begin": (ctypes.c_int32, [_u64, _vp, _vp]),
+    "slimdp_select_hist": (ctypes.c_int32, [_vp, _u64, _u32, _vp, _vp, _vp]),
+    "slimdp_select_resolve": (ctypes.c_int32, [_vp, _u32, _vp, _vp]),
+    "slimdp_select_count": (ctypes.c_int32, [_vp, _u64, _vp, _vp, _vp]),
+    "slimdp_select_emit": (ctypes.c_int32, [_vp, _u64, _u32, _u64, _u64, _vp, _vp, _vp, _sz, _vp]),
+    "slimdp_wire_message_bytes": (_sz, [_u64, _u64, ctypes.c_int]),
+    "slimdp_wire_pack": (ctypes.c_int32, [_vp, _u64, _vp, _u64, _vp, _vp, _u32, _u32, ctypes.c_int, _vp, _vp]),
+    "slimdp_wire_unpack": (ctypes.c_int32, [_vp, _sz, _vp, _u64, _u64, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "slimdp_wire_read_status": (ctypes.c_int32, [_vp, _vp]),
     "slimdp_read_status": (ctypes.c_int32, [_vp, _vp]),
     "slimdp_launch_count": (_u64, []),
     "slimdp_round_arena_bytes": (_sz, [_u64, _u32, _u64, _u64]),
     "slimdp_round": (ctypes.c_int32, [_vp, _pp, _u32, _u64, _f32, _u64, _u64, _u64, _u32, _f32, _vp, _vp, _vp, _pp, _pp,
-                                      _pp, _vp, ctypes.c_size_t, _vp, ctypes.c_size_t, _vp]),
+                                      _pp, _vp, _sz, _vp, _sz, _vp, _sz, _vp, _vp]),
+    "slimdp_round_ctx_create": (ctypes.c_int32, [_pp]),
+    "slimdp_round_ctx_destroy": (ctypes.c_int32, [_vp]),
+    "slimdp_round_release_default_ctx": (ctypes.c_int32, []),
+    "slimdp_round_stage_bytes": (_sz, [_u64, _u32, _u64]),
     "slimdp_mark_dominant_kernel": (None, [_vp, _vp]),
     "slimdp_round_host": (ctypes.c_int32, [_vp, _pp, _u32, _u64, _f32, _u64, _u64, _u64, _u32, _f32, _vp, _pp, _pp,
                                            _vp, _sz, _vp]),
@@ -283,9 +296,12 @@ def slimdp_exchange(w_global: torch.Tensor, deltas: Sequence[torch.Tensor], core
 def slimdp_round(w_global: torch.Tensor, grads: Sequence[torch.Tensor], c: float, seed: int, rnd: int, eta: float,
                  scores: torch.Tensor, core_idx: torch.Tensor, core_aux: torch.Tensor,
                  exp_idx: Sequence[torch.Tensor], val: Sequence[torch.Tensor], pulled: Sequence[torch.Tensor],
-                 select_ws: torch.Tensor, explore_ws: torch.Tensor, stream=None):
+                 select_ws: torch.Tensor, explore_ws: torch.Tensor, stage: Optional[torch.Tensor] = None,
+                 ctx: Optional["RoundContext"] = None, stream=None):
     """One whole round on device buffers; same results as score, select_core, sample_explore_batched,
-    exchange, except that `scores` is scratch (written only if the selection falls back to its full path)."""
+    exchange, except that `scores` is scratch (written only if the selection falls back to its full path).
+    `stage` (uint8, round_stage_bytes long) lets the round set the core's update values aside during its
+    pass; `ctx` is the round context whose streams the round runs on (None: the library's default one)."""
     n = w_global.numel()
     _dev(w_global, torch.float32, "w_global")
     K = len(grads)
@@ -300,11 +316,43 @@ def slimdp_round(w_global: torch.Tensor, grads: Sequence[torch.Tensor], c: float
         _check_sets(core_idx, e, o, "pulled")
     for t, name in ((core_aux, "core_aux"), (select_ws, "select_ws"), (explore_ws, "explore_ws")):
         _dev(t, torch.uint8, name)
+    if stage is not None:
+        _dev(stage, torch.uint8, "stage")
     _check("slimdp_round",
            lib.slimdp_round(w_global.data_ptr(), _ptr_array(grads), K, n, c, core_idx.numel(), exp_idx[0].numel(),
                             seed, rnd, eta, _ptr(scores), _ptr(core_idx), _ptr(core_aux), _ptr_array(exp_idx),
                             _ptr_array(val), _ptr_array(pulled), _ptr(select_ws), select_ws.numel(),
-                            _ptr(explore_ws), explore_ws.numel(), _stream(stream)))
+                            _ptr(explore_ws), explore_ws.numel(), _ptr(stage), stage.numel() if stage is not None else 0,
+                            ctx.handle if ctx is not None else None, _stream(stream)))
+
+
+def round_stage_bytes(n: int, K: int, k_core: int) -> int:
+    """Bytes of staging area for slimdp_round on the current device (0: staging does not apply)."""
+    return lib.slimdp_round_stage_bytes(n, K, k_core)
+
+
+class RoundContext:
+    """A round context on the current device (two streams, four events), owned by the caller."""
+
+    def __init__(self):
+        h = ctypes.c_void_p()
+        _check("slimdp_round_ctx_create", lib.slimdp_round_ctx_create(ctypes.byref(h)))
+        self.handle = h
+
+    def close(self) -> None:
+        if self.handle is not None:
+            _check("slimdp_round_ctx_destroy", lib.slimdp_round_ctx_destroy(self.handle))
+            self.handle = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+
+def release_default_round_ctx() -> None:
+    _check("slimdp_round_release_default_ctx", lib.slimdp_round_release_default_ctx())
 
 
 def mark_dominant_kernel(begin: Optional[torch.cuda.Event], end: Optional[torch.cuda.Event]) -> None:
@@ -356,6 +404,96 @@ def slimdp_core_signature(keys: torch.Tensor, signature: torch.Tensor, stream=No
 
 def wire_bytes(k_core: int, k_exp: int) -> int:
     return lib.slimdp_wire_bytes(k_core, k_exp)
+
+
+def slimdp_select_shard_begin(k_total: int, state: torch.Tensor, stream=None):
+    """state (int64[2] CUDA tensor) <- (prefix 0, rank k_total): start of a selection over a sharded model."""
+    _dev(state, torch.int64, "state")
+    _check("slimdp_select_shard_begin", lib.slimdp_select_shard_begin(k_total, state.data_ptr(), _stream(stream)))
+
+
+def slimdp_select_hist(scores: torch.Tensor, rnd: int, state: torch.Tensor, hist: torch.Tensor, stream=None):
+    """hist (int64[4096]) += this shard's keys by their digit of round rnd."""
+    _dev(scores, torch.float32, "scores")
+    if _dev(hist, torch.int64, "hist").numel() < 4096:
+        raise ValueError("hist: 4096 counters are needed")
+    _check("slimdp_select_hist", lib.slimdp_select_hist(_ptr(scores), scores.numel(), rnd, state.data_ptr(),
+                                                        hist.data_ptr(), _stream(stream)))
+
+
+def slimdp_select_resolve(hist: torch.Tensor, rnd: int, state: torch.Tensor, stream=None):
+    _dev(hist, torch.int64, "hist")
+    _check("slimdp_select_resolve", lib.slimdp_select_resolve(hist.data_ptr(), rnd, state.data_ptr(), _stream(stream)))
+
+
+def slimdp_select_count(scores: torch.Tensor, state: torch.Tensor, counts: torch.Tensor, stream=None):
+    """counts (int64[2]) += (keys above the threshold, keys equal to it) in this shard."""
+    _dev(scores, torch.float32, "scores")
+    _dev(counts, torch.int64, "counts")
+    _check("slimdp_select_count", lib.slimdp_select_count(_ptr(scores), scores.numel(), state.data_ptr(),
+                                                          counts.data_ptr(), _stream(stream)))
+
+
+def slimdp_select_emit(scores: torch.Tensor, threshold_bits: int, tie_quota: int, core_idx: torch.Tensor,
+                       core_aux: torch.Tensor, ws: torch.Tensor, stream=None):
+    """This shard's part of the core (shard-local indices) for a global threshold and the shard's tie quota."""
+    _dev(scores, torch.float32, "scores")
+    _dev(core_idx, IDX, "core_idx")
+    _check("slimdp_select_emit",
+           lib.slimdp_select_emit(scores.data_ptr(), scores.numel(), threshold_bits, tie_quota, core_idx.numel(),
+                                  _ptr(core_idx), core_aux.data_ptr(), ws.data_ptr(), ws.numel(), _stream(stream)))
+
+
+WIRE_KEYS_WANTED = 1
+
+
+def wire_message_bytes(k_core: int, k_exp: int, with_keys: bool) -> int:
+    return lib.slimdp_wire_message_bytes(k_core, k_exp, int(with_keys))
+
+
+def slimdp_wire_pack(core_idx: torch.Tensor, exp_idx: torch.Tensor, val: torch.Tensor, signature: torch.Tensor,
+                     worker: int, rnd: int, with_keys: bool, msg: torch.Tensor, stream=None):
+    """One worker's push as a message (Section 3.5) into the uint8 CUDA tensor `msg`."""
+    _dev(core_idx, IDX, "core_idx")
+    _dev(exp_idx, IDX, "exp_idx")
+    _dev(val, torch.float32, "val")
+    _dev(signature, torch.int64, "signature")
+    _dev(msg, torch.uint8, "msg")
+    if val.numel() != core_idx.numel() + exp_idx.numel():
+        raise ValueError("val: length differs from k_core + k_exp")
+    if msg.numel() != wire_message_bytes(core_idx.numel(), exp_idx.numel(), with_keys):
+        raise ValueError("msg: length differs from wire_message_bytes")
+    _check("slimdp_wire_pack",
+           lib.slimdp_wire_pack(_ptr(core_idx), core_idx.numel(), _ptr(exp_idx), exp_idx.numel(), _ptr(val),
+                                signature.data_ptr(), worker, rnd, int(with_keys), msg.data_ptr(), _stream(stream)))
+
+
+def slimdp_wire_unpack(msg: torch.Tensor, cached_signature: torch.Tensor, core_idx: torch.Tensor,
+                       exp_idx: torch.Tensor, val: torch.Tensor, signature_out: torch.Tensor, status: torch.Tensor,
+                       stream=None):
+    """Takes a push message apart; the verdict lands in status[0] (read it with wire_read_status)."""
+    _dev(msg, torch.uint8, "msg")
+    _dev(cached_signature, torch.int64, "cached_signature")
+    _dev(signature_out, torch.int64, "signature_out")
+    _dev(core_idx, IDX, "core_idx")
+    _dev(exp_idx, IDX, "exp_idx")
+    _dev(val, torch.float32, "val")
+    if _dev(status, torch.int32, "status").numel() < 4:
+        raise ValueError("status: four int32 words are needed")
+    if val.numel() != core_idx.numel() + exp_idx.numel():
+        raise ValueError("val: length differs from k_core + k_exp")
+    _check("slimdp_wire_unpack",
+           lib.slimdp_wire_unpack(msg.data_ptr(), msg.numel(), cached_signature.data_ptr(), core_idx.numel(),
+                                  exp_idx.numel(), _ptr(core_idx), _ptr(exp_idx), _ptr(val),
+                                  signature_out.data_ptr(), status.data_ptr(), _stream(stream)))
+
+
+def wire_read_status(status: torch.Tensor, stream=None) -> int:
+    """0 = taken apart, WIRE_KEYS_WANTED = the sender has to send its keys; malformed messages raise."""
+    st = lib.slimdp_wire_read_status(status.data_ptr(), _stream(stream))
+    if st not in (0, WIRE_KEYS_WANTED):
+        raise SlimDPError("slimdp_wire_unpack", st)
+    return st
 
 
 def _host(t: torch.Tensor, dtype, name: str) -> torch.Tensor:

@@ -33,18 +33,20 @@ slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<c
                               const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,
                               uint64_t k_exp, float eta, const PtrArray<float>& val, const PtrArray<float>& pulled,
                               const uint32_t* ranks, uint64_t rank_stride, const uint32_t* core_bitmap,
-                              const uint32_t* core_dir, int32_t* explore_status, cudaStream_t st);
+                              const uint32_t* core_dir, int32_t* explore_status, const ExchangeStage* stage,
+                              cudaStream_t st);
 bool exchange_takes_ranks(uint64_t n, uint64_t k_exp);
+size_t stage_bytes_for(uint64_t n, uint32_t K, uint64_t k_core);
 
 slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                    uint32_t first_worker, uint32_t workers, uint32_t round,
                                    const PtrArray<uint32_t>& out, void* ws, int parts, bool lean, cudaStream_t st);
-bool score_select_fusable(uint64_t n, uint64_t k_core, bool vec);
+bool score_select_fusable(uint64_t n, uint64_t k_core, uint32_t K, bool vec);
 slimdp_status launch_score_select(const float* w, const PtrArray<const float>& g, uint32_t K, float c, uint64_t n,
                                   float* scores, uint64_t k_core, uint32_t* core_idx, void* core_aux, void* ws,
-                                  cudaEvent_t mark_begin, cudaEvent_t mark_end, cudaStream_t gate_stream,
-                                  cudaEvent_t gate_fork, cudaEvent_t gate_join, slimdp_status (*after_pass)(void*),
-                                  void* after_arg, cudaEvent_t pass_ready, cudaStream_t st);
+                                  cudaEvent_t mark_begin, cudaEvent_t mark_end, slimdp_status (*after_pass)(void*),
+                                  void* after_arg, cudaEvent_t pass_ready, void* stage, size_t stage_bytes,
+                                  bool* staged, cudaStream_t st);
 
 slimdp_status launch_explore_static(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                     uint32_t worker, uint32_t round, uint32_t* exp_idx, int32_t* status_out,
@@ -56,18 +58,32 @@ slimdp_status launch_worker_merge(const PtrArray<float>& w_local, uint32_t worke
                                   uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp,
                                   const PtrArray<const float>& pulled, cudaStream_t st);
 
+slimdp_status launch_select_given(const float* scores, uint64_t n, uint32_t T, uint32_t ties, uint64_t k_shard,
+                                  uint32_t* core_idx, void* core_aux, void* ws, cudaStream_t st);
+slimdp_status launch_shard_state_init(void* state, uint64_t k, cudaStream_t st);
+slimdp_status launch_shard_hist(const float* scores, uint64_t n, uint32_t round, const void* state, uint64_t* hist,
+                                cudaStream_t st);
+slimdp_status launch_shard_resolve(const uint64_t* hist, uint32_t round, void* state, cudaStream_t st);
+slimdp_status launch_shard_count(const float* scores, uint64_t n, const void* state, uint64_t* counts,
+                                 cudaStream_t st);
 slimdp_status launch_signature(const uint32_t* keys, uint64_t count, unsigned long long* sig, cudaStream_t st);
+slimdp_status launch_wire_pack(const uint32_t* core_idx, uint64_t k_core, const uint32_t* exp_idx, uint64_t k_exp,
+                               const float* val, const unsigned long long* sig, uint32_t worker, uint32_t round,
+                               bool with_keys, void* msg, cudaStream_t st);
+slimdp_status launch_wire_unpack(const void* msg, size_t msg_bytes, const unsigned long long* cached_sig,
+                                 uint64_t k_core, uint64_t k_exp, uint32_t* core_idx, uint32_t* exp_idx, float* val,
+                                 unsigned long long* sig_out, int32_t* status, cudaStream_t st);
 
 int sm_count() {
-    static int cached[64];
+    static std::atomic<int> cached[64];   // 0 = not asked yet; every thread that asks stores the same value
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
-    if (cached[dev] == 0) {
-        int v = 0;
+    int v = cached[dev].load(std::memory_order_relaxed);
+    if (v == 0) {
         if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return -1;
-        cached[dev] = v;
+        cached[dev].store(v, std::memory_order_relaxed);
     }
-    return cached[dev];
+    return v;
 }
 
 namespace {
@@ -268,7 +284,7 @@ slimdp_status slimdp_exchange(float* w_global, uint64_t n, uint32_t K, const flo
     if (!fill<float>(o, pulled, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (k_core + k_exp == 0) return SLIMDP_OK;
     return launch_exchange(w_global, n, K, d, core_idx, k_core, exp, k_exp, eta, v, o, nullptr, 0, nullptr, nullptr,
-                           nullptr, (cudaStream_t)stream);
+                           nullptr, nullptr, (cudaStream_t)stream);
 }
 
 slimdp_status slimdp_dense_merge_score(float* w_global, const float* const* grads, uint32_t K, float eta, float c,
@@ -304,6 +320,98 @@ slimdp_status slimdp_core_signature(const uint32_t* keys, uint64_t count, uint64
 
 size_t slimdp_wire_bytes(uint64_t k_core, uint64_t k_exp) { return (size_t)(4 * k_core + 8 * k_exp + 8); }
 
+// ---- selection over a range-sharded model ---------------------------------
+
+slimdp_status slimdp_select_shard_begin(uint64_t k_total, void* state, void* stream) {
+    if (!state || (reinterpret_cast<uintptr_t>(state) & 7u) != 0) return SLIMDP_ERR_INVALID_ARG;
+    return launch_shard_state_init(state, k_total, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_select_hist(const float* scores, uint64_t n_shard, uint32_t round, const void* state,
+                                 uint64_t* hist, void* stream) {
+    if (n_shard > kMaxN || round > 2 || !state || !hist || (n_shard > 0 && (!scores || !aligned4(scores))))
+        return SLIMDP_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(state) | reinterpret_cast<uintptr_t>(hist)) & 7u) != 0)
+        return SLIMDP_ERR_INVALID_ARG;
+    return launch_shard_hist(scores, n_shard, round, state, hist, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_select_resolve(const uint64_t* hist, uint32_t round, void* state, void* stream) {
+    if (round > 2 || !state || !hist) return SLIMDP_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(state) | reinterpret_cast<uintptr_t>(hist)) & 7u) != 0)
+        return SLIMDP_ERR_INVALID_ARG;
+    return launch_shard_resolve(hist, round, state, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_select_count(const float* scores, uint64_t n_shard, const void* state, uint64_t* counts,
+                                  void* stream) {
+    if (n_shard > kMaxN || !state || !counts || (n_shard > 0 && (!scores || !aligned4(scores))))
+        return SLIMDP_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(state) | reinterpret_cast<uintptr_t>(counts)) & 7u) != 0)
+        return SLIMDP_ERR_INVALID_ARG;
+    return launch_shard_count(scores, n_shard, state, counts, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_select_emit(const float* scores, uint64_t n_shard, uint32_t threshold_bits, uint64_t tie_quota,
+                                 uint64_t k_shard, uint32_t* core_idx, void* core_aux, void* ws, size_t ws_bytes,
+                                 void* stream) {
+    if (!n_ok(n_shard) || k_shard > n_shard || tie_quota > k_shard || !scores || !core_aux || !ws)
+        return SLIMDP_ERR_INVALID_ARG;
+    if (k_shard > 0 && !core_idx) return SLIMDP_ERR_INVALID_ARG;
+    if (!aligned4(scores) || !aligned16(core_aux) || !aligned16(ws) || (core_idx && !aligned16(core_idx)))
+        return SLIMDP_ERR_INVALID_ARG;
+    if (ws_bytes < slimdp_select_workspace_bytes(n_shard)) return SLIMDP_ERR_WORKSPACE;
+    return launch_select_given(scores, n_shard, threshold_bits, (uint32_t)tie_quota, k_shard, core_idx, core_aux, ws,
+                               (cudaStream_t)stream);
+}
+
+size_t slimdp_wire_message_bytes(uint64_t k_core, uint64_t k_exp, int with_keys) {
+    if (k_core > kMaxN || k_exp > kMaxN) return 0;
+    return (size_t)(32 + 4 * k_core * (with_keys ? 2 : 1) + 8 * k_exp);
+}
+
+slimdp_status slimdp_wire_pack(const uint32_t* core_idx, uint64_t k_core, const uint32_t* exp_idx, uint64_t k_exp,
+                               const float* val, const uint64_t* signature, uint32_t worker, uint32_t round,
+                               int with_keys, void* msg, void* stream) {
+    if (k_core > kMaxN || k_exp > kMaxN || !signature || !msg || !aligned16(msg) ||
+        (reinterpret_cast<uintptr_t>(signature) & 7u) != 0)
+        return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned4(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_exp > 0 && (!exp_idx || !aligned4(exp_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core + k_exp > 0 && (!val || !aligned4(val))) return SLIMDP_ERR_INVALID_ARG;
+    return launch_wire_pack(core_idx, k_core, exp_idx, k_exp, val,
+                            reinterpret_cast<const unsigned long long*>(signature), worker, round, with_keys != 0, msg,
+                            (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_wire_unpack(const void* msg, size_t msg_bytes, const uint64_t* cached_signature,
+                                 uint64_t k_core, uint64_t k_exp, uint32_t* core_idx, uint32_t* exp_idx, float* val,
+                                 uint64_t* signature_out, int32_t* status, void* stream) {
+    if (k_core > kMaxN || k_exp > kMaxN || !msg || !aligned16(msg) || !cached_signature || !signature_out || !status)
+        return SLIMDP_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(cached_signature) | reinterpret_cast<uintptr_t>(signature_out) |
+          reinterpret_cast<uintptr_t>(status)) & 7u) != 0)
+        return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned4(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_exp > 0 && (!exp_idx || !aligned4(exp_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core + k_exp > 0 && (!val || !aligned4(val))) return SLIMDP_ERR_INVALID_ARG;
+    // the kernels read the header and the k_core words after it whatever the message turns out to be
+    if (msg_bytes < 32 + 4 * k_core) return SLIMDP_ERR_INVALID_ARG;
+    return launch_wire_unpack(msg, msg_bytes, reinterpret_cast<const unsigned long long*>(cached_signature), k_core,
+                              k_exp, core_idx, exp_idx, val, reinterpret_cast<unsigned long long*>(signature_out),
+                              status, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_wire_read_status(const int32_t* status, void* stream) {
+    if (!status) return SLIMDP_ERR_INVALID_ARG;
+    int32_t s = 0;
+    if (cudaMemcpyAsync(&s, status, sizeof(s), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+        return SLIMDP_ERR_CUDA;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return SLIMDP_ERR_CUDA;
+    if (s == 0) return SLIMDP_OK;
+    return (s == SLIMDP_WIRE_KEYS_WANTED) ? SLIMDP_WIRE_KEYS_WANTED : SLIMDP_ERR_INVALID_ARG;
+}
+
 uint64_t slimdp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 slimdp_status slimdp_read_status(const void* ws, void* stream) {
@@ -319,8 +427,8 @@ slimdp_status slimdp_read_status(const void* ws, void* stream) {
 //
 // The round's steps form a small graph rather than a chain.  The chain that
 // decides the round's time (sampling, the pass over all parameters, the
-// threshold, the core, the explorers' indices, the exchange) runs on a stream
-// of the highest priority that the library owns, one per device.  The
+// finishing kernel of the selection, the exchange incl. the explorers'
+// indices) runs on the context's stream of the highest priority.  The
 // explorer's ranks depend on the sizes alone: they are computed and sorted on
 // a second stream of the lowest priority, released when the pass starts, in the
 // part of each SM that the pass leaves free.  Whenever a kernel of the chain
@@ -330,47 +438,100 @@ slimdp_status slimdp_read_status(const void* ws, void* stream) {
 // Scoring is folded into the selection's one pass over all parameters, so the
 // scores are never written unless the selection has to fall back to its full path.
 
-namespace {
-struct SideStream {
-    cudaStream_t chain = nullptr, ranks = nullptr, gate = nullptr;
-    cudaEvent_t fork = nullptr, pass_ready = nullptr, ranks_done = nullptr, chain_done = nullptr, gate_fork = nullptr,
-                gate_join = nullptr;
-    bool ready = false;
-};
-std::mutex g_side_mutex;
-thread_local cudaEvent_t t_mark_begin = nullptr, t_mark_end = nullptr;
-SideStream g_side[64];
+}  // extern "C"
 
-SideStream* side_stream_locked() {
+struct slimdp_round_ctx {
+    std::mutex lock;
+    int device = -1;
+    cudaStream_t chain = nullptr, ranks = nullptr;
+    cudaEvent_t fork = nullptr, pass_ready = nullptr, ranks_done = nullptr, chain_done = nullptr;
+};
+
+namespace {
+thread_local cudaEvent_t t_mark_begin = nullptr, t_mark_end = nullptr;
+std::mutex g_default_mutex;
+slimdp_round_ctx* g_default_ctx[64];   // per device, guarded by g_default_mutex
+
+void ctx_release(slimdp_round_ctx* c) {
+    cudaEvent_t ev[4] = {c->fork, c->pass_ready, c->ranks_done, c->chain_done};
+    for (cudaEvent_t e : ev)
+        if (e) cudaEventDestroy(e);
+    if (c->chain) cudaStreamDestroy(c->chain);
+    if (c->ranks) cudaStreamDestroy(c->ranks);
+    delete c;
+}
+
+// A context on the current device; nullptr (nothing left behind) if any part of it cannot be created.
+slimdp_round_ctx* ctx_make() {
+    int dev = 0, lo = 0, hi = 0;   // numerically, hi <= lo: hi is the highest priority
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess)
+        return nullptr;
+    slimdp_round_ctx* c = new (std::nothrow) slimdp_round_ctx;
+    if (!c) return nullptr;
+    c->device = dev;
+    bool ok = cudaStreamCreateWithPriority(&c->chain, cudaStreamNonBlocking, hi) == cudaSuccess &&
+              cudaStreamCreateWithPriority(&c->ranks, cudaStreamNonBlocking, lo) == cudaSuccess;
+    cudaEvent_t* ev[4] = {&c->fork, &c->pass_ready, &c->ranks_done, &c->chain_done};
+    for (cudaEvent_t* e : ev) ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+        ctx_release(c);
+        return nullptr;
+    }
+    return c;
+}
+
+slimdp_round_ctx* default_ctx() {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    SideStream& s = g_side[dev];
-    if (!s.ready) {
-        int lo = 0, hi = 0;   // numerically, hi <= lo: hi is the highest priority
-        if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) return nullptr;
-        if (cudaStreamCreateWithPriority(&s.chain, cudaStreamNonBlocking, hi) != cudaSuccess) return nullptr;
-        if (cudaStreamCreateWithPriority(&s.gate, cudaStreamNonBlocking, hi) != cudaSuccess) return nullptr;
-        if (cudaStreamCreateWithPriority(&s.ranks, cudaStreamNonBlocking, lo) != cudaSuccess) return nullptr;
-        cudaEvent_t* ev[6] = {&s.fork, &s.pass_ready, &s.ranks_done, &s.chain_done, &s.gate_fork, &s.gate_join};
-        for (auto e : ev)
-            if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-        s.ready = true;
-    }
-    return &s;
+    std::lock_guard<std::mutex> lock(g_default_mutex);
+    if (!g_default_ctx[dev]) g_default_ctx[dev] = ctx_make();
+    return g_default_ctx[dev];
 }
 }  // namespace
+
+extern "C" {
+
+slimdp_status slimdp_round_ctx_create(slimdp_round_ctx** ctx) {
+    if (!ctx) return SLIMDP_ERR_INVALID_ARG;
+    *ctx = ctx_make();
+    return *ctx ? SLIMDP_OK : SLIMDP_ERR_CUDA;
+}
+
+slimdp_status slimdp_round_ctx_destroy(slimdp_round_ctx* ctx) {
+    if (!ctx) return SLIMDP_ERR_INVALID_ARG;
+    ctx_release(ctx);
+    return SLIMDP_OK;
+}
+
+slimdp_status slimdp_round_release_default_ctx(void) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SLIMDP_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_default_mutex);
+    if (g_default_ctx[dev]) {
+        ctx_release(g_default_ctx[dev]);
+        g_default_ctx[dev] = nullptr;
+    }
+    return SLIMDP_OK;
+}
+
+size_t slimdp_round_stage_bytes(uint64_t n, uint32_t K, uint64_t k_core) {
+    if (!n_ok(n) || !k_ok(K) || k_core > n) return 0;
+    return stage_bytes_for(n, K, k_core);
+}
 
 slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t K, uint64_t n, float c,
                            uint64_t k_core, uint64_t k_exp, uint64_t seed, uint32_t round, float eta, float* scores,
                            uint32_t* core_idx, void* core_aux, uint32_t* const* exp_idx, float* const* val,
                            float* const* pulled, void* select_ws, size_t select_ws_bytes, void* explore_ws,
-                           size_t explore_ws_bytes, void* stream) {
+                           size_t explore_ws_bytes, void* stage, size_t stage_bytes, slimdp_round_ctx* ctx,
+                           void* stream) {
     if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !w_global || !grads || !scores || !core_aux || !select_ws ||
         !explore_ws || !isfinite(c) || !isfinite(eta))
         return SLIMDP_ERR_INVALID_ARG;
     if (!aligned4(w_global) || !aligned4(scores) || !aligned16(core_aux) || !aligned16(select_ws) ||
         !aligned16(explore_ws))
         return SLIMDP_ERR_INVALID_ARG;
+    if (stage && (reinterpret_cast<uintptr_t>(stage) & 255u) != 0) return SLIMDP_ERR_INVALID_ARG;
     if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
     PtrArray<const float> g;
     PtrArray<uint32_t> exp_out;
@@ -391,12 +552,16 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
     }
     bool vec = aligned16(w_global) && aligned16(scores);
     for (uint32_t k = 0; k < K; ++k) vec = vec && aligned16(g.p[k]);
-    const bool fusable = score_select_fusable(n, k_core, vec);
+    const bool fusable = score_select_fusable(n, k_core, K, vec);
 
     cudaStream_t st = (cudaStream_t)stream;
-    std::lock_guard<std::mutex> lock(g_side_mutex);
-    SideStream* side = side_stream_locked();
+    slimdp_round_ctx* side = ctx ? ctx : default_ctx();
     if (!side) return SLIMDP_ERR_CUDA;
+    {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev != side->device) return SLIMDP_ERR_INVALID_ARG;
+    }
+    std::lock_guard<std::mutex> lock(side->lock);
     cudaStream_t ch = side->chain, rk = side->ranks;
 
     if (cudaEventRecord(side->fork, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
@@ -432,12 +597,12 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
         return r;
     };
     // chain: the core, scored and selected in one pass where sizes and alignment allow
+    bool staged = false;
     if (fusable) {
         rank_work.after = side->pass_ready;   // recorded by the call below just before its pass
         rank_work.lean = true;
         step(launch_score_select(w_global, g, K, c, n, scores, k_core, core_idx, core_aux, select_ws, mark0, mark1,
-                                 side->gate, side->gate_fork, side->gate_join, enqueue_ranks, &rank_work,
-                                 side->pass_ready, ch));
+                                 enqueue_ranks, &rank_work, side->pass_ready, stage, stage_bytes, &staged, ch));
         // (if the call failed before it reached the hook, ranks_done keeps an earlier record: nothing to wait for)
     } else {
         step(enqueue_ranks(&rank_work));
@@ -449,21 +614,28 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
     // chain: explorer indices from the sorted ranks and the core, then the exchange; where the
     // exchange's warp ranges line up with the core's directory it computes the indices itself
     cuda(cudaStreamWaitEvent(ch, side->ranks_done, 0));
+    const uint32_t* aux_bitmap = reinterpret_cast<const uint32_t*>(core_aux);
+    const uint32_t* aux_dir =
+        reinterpret_cast<const uint32_t*>(static_cast<const char*>(core_aux) + slimdp_core_aux_dir_offset(n));
+    ExchangeStage xs{};
+    if (staged) {
+        const SelectWs SL = select_ws_layout(select_ws, n);
+        const StageArea A = stage_layout(stage, n, K, k_core, (uint32_t)sm_count() * 8u);
+        xs = ExchangeStage{A.fill, A.chunks, (uint32_t)A.max_chunks, SL.hdr, (uint32_t)SL.cand_cap};
+    }
+    const ExchangeStage* xsp = staged ? &xs : nullptr;
     if (exchange_takes_ranks(n, k_exp)) {
         const ExploreWs EL = explore_ws_layout(explore_ws, n, k_exp, K);
         if (rc == SLIMDP_OK)
             step(launch_exchange(w_global, n, K, g, core_idx, k_core, exp_in, k_exp, eta, v, o, EL.rho, EL.rho_stride,
-                                 reinterpret_cast<const uint32_t*>(core_aux),
-                                 reinterpret_cast<const uint32_t*>(static_cast<const char*>(core_aux) +
-                                                                   slimdp_core_aux_dir_offset(n)),
-                                 &EL.hdr->status, ch));
+                                 aux_bitmap, aux_dir, &EL.hdr->status, xsp, ch));
     } else {
         if (rc == SLIMDP_OK)
             step(launch_explore_parts(core_aux, n, k_core, k_exp, seed, 0, K, round, exp_out, explore_ws, 2, false,
                                       ch));
         if (rc == SLIMDP_OK && k_core + k_exp > 0)
-            step(launch_exchange(w_global, n, K, g, core_idx, k_core, exp_in, k_exp, eta, v, o, nullptr, 0, nullptr,
-                                 nullptr, nullptr, ch));
+            step(launch_exchange(w_global, n, K, g, core_idx, k_core, exp_in, k_exp, eta, v, o, nullptr, 0,
+                                 aux_bitmap, aux_dir, nullptr, xsp, ch));
     }
     if (cudaEventRecord(side->chain_done, ch) != cudaSuccess || cudaStreamWaitEvent(st, side->chain_done, 0) != cudaSuccess)
         step(SLIMDP_ERR_CUDA);
@@ -488,6 +660,8 @@ struct Arena {
     size_t select_ws_bytes;
     void* explore_ws;
     size_t explore_ws_bytes;
+    void* stage;
+    size_t stage_bytes;
     uint32_t* exp_idx[SLIMDP_MAX_WORKERS];
     float* val[SLIMDP_MAX_WORKERS];
     float* pulled[SLIMDP_MAX_WORKERS];
@@ -514,6 +688,8 @@ Arena arena_layout(void* base, uint64_t n, uint32_t K, uint64_t k_core, uint64_t
     A.select_ws = take(A.select_ws_bytes);
     A.explore_ws_bytes = slimdp_explore_workspace_bytes(n, k_exp, K);
     A.explore_ws = take(A.explore_ws_bytes);
+    A.stage_bytes = slimdp_round_stage_bytes(n, K, k_core);
+    A.stage = A.stage_bytes ? take(A.stage_bytes) : nullptr;
     for (uint32_t k = 0; k < K; ++k) A.exp_idx[k] = reinterpret_cast<uint32_t*>(take(k_exp * 4));
     for (uint32_t k = 0; k < K; ++k) A.val[k] = reinterpret_cast<float*>(take(m * 4));
     for (uint32_t k = 0; k < K; ++k) A.pulled[k] = reinterpret_cast<float*>(take(m * 4));
@@ -558,7 +734,7 @@ slimdp_status slimdp_round_host(float* w_host, const float* const* grads_host, u
         SLIMDP_CUDA(cudaMemcpyAsync(A.delta[k], grads_host[k], n * 4, cudaMemcpyHostToDevice, st));
     SLIMDP_TRY(slimdp_round(A.w, A.delta, K, n, c, k_core, k_exp, seed, round, eta, A.scores, A.core_idx, A.core_aux,
                             A.exp_idx, A.val, A.pulled, A.select_ws, A.select_ws_bytes, A.explore_ws,
-                            A.explore_ws_bytes, stream));
+                            A.explore_ws_bytes, A.stage, A.stage_bytes, nullptr, stream));
     SLIMDP_CUDA(cudaMemcpyAsync(w_host, A.w, n * 4, cudaMemcpyDeviceToHost, st));
     if (k_core) SLIMDP_CUDA(cudaMemcpyAsync(core_idx_host, A.core_idx, k_core * 4, cudaMemcpyDeviceToHost, st));
     for (uint32_t k = 0; k < K; ++k) {

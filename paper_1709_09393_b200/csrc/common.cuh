@@ -14,9 +14,9 @@ constexpr uint32_t kDirStride = SLIMDP_DIR_STRIDE;      // parameters per direct
 constexpr uint32_t kDirPerBlock = kBlock / kDirStride;  // 16 directory entries per bitmap block
 constexpr uint32_t kWordsPerDir = kDirStride / 32;      // 2 bitmap words per directory entry
 static_assert(kWordsPerDir == 2, "select0 walks exactly two bitmap words per directory entry");
-constexpr uint32_t kScanTile = 1024;             // bitmap blocks per scan tile
 constexpr uint32_t kSampleBits = 18;             // the selection's bracket is estimated from 2^18 sampled keys
 constexpr uint64_t kBracketMinN = 1ull << 21;    // below this the selection reads the keys three more times instead
+constexpr uint32_t kStageChunk = 512;            // entries per chunk of the staging area (see layout.cuh)
 
 // K device pointers passed by value as a kernel argument (512 bytes).
 template <typename T>
@@ -37,13 +37,22 @@ struct WsHeader {
     uint32_t ticket[8];  // "last CTA done" counters, one per kernel that needs one
     uint32_t coarse_x[2];  // sample: coarse bins in which the two target ranks are crossed
     uint32_t next_block;   // fused scoring pass: the next 1024-parameter block to hand out
-    uint32_t reserved[45];
+    uint32_t barrier;      // finishing kernel: arrivals at its grid barrier so far (all epochs)
+    uint32_t abort;        // finishing kernel: a bounded wait ran out; every CTA leaves
+    uint32_t next_chunk;   // fused scoring pass: the next free chunk of the staging area
+    uint32_t stage_lost;   // fused scoring pass: the staging area ran out of chunks
+    uint32_t reserved[41];
 };
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 
+// True when the selection's pass over all keys proved that the threshold lies inside the sampled
+// bracket and every candidate was stored (k = k_core, cap = capacity of the candidate list).
+__host__ __device__ __forceinline__ bool bracket_held(uint32_t n_def, uint32_t n_cand, uint32_t k, uint32_t cap) {
+    return n_def < k && k - n_def <= n_cand && n_cand <= cap;
+}
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline uint64_t num_blocks(uint64_t n) { return (n + kBlock - 1) / kBlock; }
-inline uint64_t num_scan_tiles(uint64_t n) { return (num_blocks(n) + kScanTile - 1) / kScanTile; }
 
 // Number of SMs of the current device (cached per device id).
 int sm_count();
@@ -149,13 +158,5 @@ __device__ __forceinline__ float score_one(float c, float g, float w) {
 // canonical quiet NaN, as scores are.  Once NaN a parameter stays NaN, so one check after the last of a
 // chain of updates gives the same bits as a check after each.
 __device__ __forceinline__ float stored_model_value(float x) { return (x != x) ? __uint_as_float(0x7FC00000u) : x; }
-
-// ---- internal launchers (each enqueues on `st`, returns a slimdp_status) ---
-
-// Exclusive scan over bitmap blocks of 64-bit counters: cnt[y][nb] -> pref[y][nb],
-// totals[y] = sum.  y = 0 .. batch-1; rows are `stride` entries apart.
-slimdp_status launch_block_scan(const unsigned long long* cnt, unsigned long long* pref,
-                                unsigned long long* tile_sums, unsigned long long* totals, uint64_t nb,
-                                uint32_t batch, uint64_t stride, uint64_t tile_stride, cudaStream_t st);
 
 }  // namespace slimdp

@@ -7,13 +7,13 @@
 // parameter.  select0 is monotone, so sorting the ranks sorts the indices, and
 // the ranks are uniform on [0, M), so a bucket sort by the ranks' high bits
 // is balanced:
-//   1. setup: round keys (three Philox-4x32-10 blocks per worker);
-//   2. rank: thread j evaluates pi(j) (10-round alternating Feistel network
+//   1. rank: every CTA derives its worker's round keys (three Philox-4x32-10
+//      blocks); thread j evaluates pi(j) (10-round alternating Feistel network
 //      with cycle walking), stores it and counts it into its bucket (rank >> s);
-//   3. two-kernel exclusive scan of the bucket counts;
-//   4. scatter: every rank goes to its bucket's slice (order inside a bucket
+//      the last CTA of a worker to finish scans that worker's bucket counts;
+//   2. scatter: every rank goes to its bucket's slice (order inside a bucket
 //      is arbitrary here and is fixed by the next step);
-//   5. bucket: one CTA per (bucket, worker) marks its ranks in a 2^s-bit
+//   3. bucket: one CTA per (bucket, worker) marks its ranks in a 2^s-bit
 //      shared-memory bitmap, which sorts them; a block scan of the popcounts
 //      gives each rank its output position, and a select0 query (binary
 //      search of the per-64 non-core directory inside the bucket's range,
@@ -71,38 +71,44 @@ __device__ __forceinline__ uint32_t find_block(const uint32_t* __restrict__ dir,
     return lo;
 }
 
-// Round keys of every worker of the call.
-__global__ void explore_setup_kernel(WsHeader* hdr, uint32_t* __restrict__ rk, uint32_t seed_lo, uint32_t seed_hi,
-                                     uint32_t first_worker, uint32_t workers, uint32_t round) {
-    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
-    if (t == 0) hdr->status = SLIMDP_OK;
-    if (t < workers * 3) {
-        const uint32_t w = t / 3, b = t % 3;
-        uint32_t out[4];
-        philox4x32_10(seed_lo, seed_hi, b, first_worker + w, round, 0x534C494Du, out);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) rk[w * 12 + b * 4 + q] = out[q];
-    }
-}
+// What identifies a call's random stream, and where the rank step leaves its by-products.
+struct RankStream {
+    uint32_t seed_lo, seed_hi, first_worker, round;
+    WsHeader* hdr;
+    uint32_t* ticket;              // per worker, cleared before the launch
+    unsigned long long* pref;      // per worker: exclusive prefix sums of the bucket counts
+    unsigned long long* totals;    // per worker: their sum
+};
 
-// grid = (chunks, workers).  rho[w][j] = pi(j) for the CTA's chunk of j; cnt[w][rho >> s] += 1.
-// Lanes whose walk has ended take the next j of their warp's range at once, so a
-// long cycle walk in one lane does not idle the other 31.
+// grid = (chunks, workers), 1024 threads.  rho[w][j] = pi(j) for the CTA's chunk of j;
+// cnt[w][rho >> s] += 1.  Every CTA derives its worker's round keys itself (three Philox-4x32-10
+// blocks).  Lanes whose walk has ended take the next j of their warp's range at once, so a
+// long cycle walk in one lane does not idle the other 31.  The last CTA of a worker to finish
+// turns that worker's bucket counts into their exclusive prefix sums.
 template <bool SMEM_HIST>
 __global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, uint32_t chunk, uint32_t bits,
-                                                    uint32_t s, uint32_t buckets,
-                                                    const uint32_t* __restrict__ rk_all, uint32_t* __restrict__ rho,
-                                                    uint64_t rho_stride, unsigned long long* __restrict__ cnt,
-                                                    uint64_t cnt_stride, uint32_t* __restrict__ cta_hist) {
+                                                    uint32_t s, uint32_t buckets, RankStream rs,
+                                                    uint32_t* __restrict__ rho, uint64_t rho_stride,
+                                                    unsigned long long* __restrict__ cnt, uint64_t cnt_stride,
+                                                    uint32_t* __restrict__ cta_hist) {
     extern __shared__ uint32_t sh_hist[];
+    __shared__ uint32_t sh_rk[12];
+    __shared__ unsigned long long scan_smem[33];
+    __shared__ bool last_of_worker;
     const uint32_t worker = blockIdx.y, lane = lane_id();
-    if (SMEM_HIST) {
-        for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) sh_hist[b] = 0;
-        __syncthreads();
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) rs.hdr->status = SLIMDP_OK;   // no kernel before this one reports
+    if (threadIdx.x < 3) {
+        uint32_t out[4];
+        philox4x32_10(rs.seed_lo, rs.seed_hi, threadIdx.x, rs.first_worker + worker, rs.round, 0x534C494Du, out);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) sh_rk[threadIdx.x * 4 + q] = out[q];
     }
+    if (SMEM_HIST)
+        for (uint32_t b = threadIdx.x; b < buckets; b += blockDim.x) sh_hist[b] = 0;
+    __syncthreads();
     uint32_t rk[10];
 #pragma unroll
-    for (int r = 0; r < 10; ++r) rk[r] = rk_all[worker * 12 + r];
+    for (int r = 0; r < 10; ++r) rk[r] = sh_rk[r];
     // x = A * 2^c + B, A of a = floor(bits / 2) bits, B of c = bits - a bits
     const uint32_t a = bits >> 1, c = bits - a;
     const uint32_t maskA = (1u << a) - 1u, maskB = (1u << c) - 1u;
@@ -164,6 +170,27 @@ __global__ void __launch_bounds__(1024) rank_kernel(uint32_t M, uint32_t k_exp, 
             if (c) atomicAdd(&my_cnt[b], (unsigned long long)c);
         }
     }
+    // "last CTA done" per worker: the block barrier orders this CTA's atomics before thread 0's
+    // device-wide fence, the fence orders them before the ticket
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        last_of_worker = atomicAdd(&rs.ticket[worker], 1u) == gridDim.x - 1;
+        __threadfence();
+    }
+    __syncthreads();
+    if (!last_of_worker) return;
+    unsigned long long* my_pref = rs.pref + (uint64_t)worker * cnt_stride;
+    unsigned long long carry = 0;
+    for (uint32_t b0 = 0; b0 < buckets; b0 += 1024) {
+        const uint32_t b = b0 + threadIdx.x;
+        const unsigned long long v = (b < buckets) ? __ldcg(my_cnt + b) : 0ull;
+        unsigned long long total;
+        const unsigned long long ex = block_exclusive_scan64<32>(v, scan_smem, &total);
+        if (b < buckets) my_pref[b] = carry + ex;
+        carry += total;
+    }
+    if (threadIdx.x == 0) rs.totals[worker] = carry;
 }
 
 // grid = (chunks, workers).  Move every rank of the chunk into its bucket's slice of `sorted`.
@@ -517,13 +544,10 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
     const uint32_t s = explore_bucket_shift(M);
     const uint64_t buckets = (M + (1ull << s) - 1) >> s;
 
-    if (parts & 1) {
-        explore_setup_kernel<<<(3 * workers + 255) / 256, 256, 0, st>>>(L.hdr, L.round_keys, (uint32_t)seed,
-                                                                        (uint32_t)(seed >> 32), first_worker,
-                                                                        workers, round);
-        SLIMDP_LAUNCHED(1);
+    if (k_exp == 0) {   // nothing to draw; the status word is still this call's
+        if ((parts & 1) && cudaMemsetAsync(L.hdr, 0, sizeof(int32_t), st) != cudaSuccess) return SLIMDP_ERR_CUDA;
+        return SLIMDP_OK;
     }
-    if (k_exp == 0) return SLIMDP_OK;
     if (parts & 1) {
     if (cudaMemsetAsync(L.cnt, 0, L.zero_bytes, st) != cudaSuccess) return SLIMDP_ERR_CUDA;
 
@@ -549,22 +573,18 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
     if (!prefer_max_shared(rank_kernel<true>) || !prefer_max_shared(rank_kernel<false>) ||
         !prefer_max_shared(scatter_kernel<true, true>) || !prefer_max_shared(scatter_kernel<true, false>) ||
         !prefer_max_shared(scatter_kernel<false, false>) || !prefer_max_shared(bucket_sort_kernel<false>) ||
-        !prefer_max_shared(bucket_sort_kernel<true>) ||
-        !prefer_max_shared(explore_setup_kernel))
+        !prefer_max_shared(bucket_sort_kernel<true>))
         return SLIMDP_ERR_CUDA;
+    const RankStream rs{(uint32_t)seed, (uint32_t)(seed >> 32), first_worker, round, L.hdr, L.ticket, L.pref, L.totals};
     if (smem) {
         rank_kernel<true><<<grid, 1024, buckets * 4, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, bits, s,
-                                                           (uint32_t)buckets, L.round_keys, L.rho, L.rho_stride,
-                                                           L.cnt, L.cnt_stride, L.cta_hist);
+                                                           (uint32_t)buckets, rs, L.rho, L.rho_stride, L.cnt,
+                                                           L.cnt_stride, L.cta_hist);
     } else {
-        rank_kernel<false><<<grid, 1024, 0, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, bits, s, (uint32_t)buckets,
-                                                  L.round_keys, L.rho, L.rho_stride, L.cnt, L.cnt_stride,
-                                                  L.cta_hist);
+        rank_kernel<false><<<grid, 1024, 0, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, bits, s, (uint32_t)buckets, rs,
+                                                  L.rho, L.rho_stride, L.cnt, L.cnt_stride, L.cta_hist);
     }
     SLIMDP_LAUNCHED(1);
-    slimdp_status rc =
-        launch_block_scan(L.cnt, L.pref, L.tile_sums, L.totals, buckets, workers, L.cnt_stride, L.tile_stride, st);
-    if (rc != SLIMDP_OK) return rc;
     const size_t group_smem = (3 * buckets + chunk) * 4;
     if (smem && group_smem <= (lean ? kGroupSmemLean : kGroupSmemMax)) {
         if (group_smem > 48 * 1024 &&

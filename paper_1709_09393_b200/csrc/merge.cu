@@ -14,6 +14,7 @@
 // Inside one worker the indices are distinct, and no other warp touches the
 // range, so a parameter receives its updates in ascending k without atomics.
 #include "common.cuh"
+#include "layout.cuh"
 
 namespace slimdp {
 
@@ -372,6 +373,74 @@ __device__ __forceinline__ void exchange_explore_ranks_body(float* w, const Rank
     if (sink == 0x9E3779B9u && lane >= 32) w[0] = 0.0f;   // never true: keeps the early requests alive
 }
 
+// ---- core segment from the staging area ------------------------------------------------------
+//
+// In the one-call round the pass over all parameters has set aside, for every parameter that is
+// certainly in the core and for every candidate, its index and its K update values (chunks of
+// kStageChunk entries, see layout.cuh).  The core segment then streams those chunks instead of
+// gathering K + 1 scattered lines per core parameter: the entry's place in the core comes from
+// the core's bitmap and directory (a candidate that did not make it has its bit clear and is
+// skipped), the K values go out as the pushed values, the model value is read, updated in worker
+// order and written back, and the merged value goes to all K workers' pulls.  Entries of one
+// chunk are in ascending parameter order, so all of these accesses are runs.
+struct StagedSource {
+    const uint32_t* fill;      // null: nothing was staged, the core segment gathers
+    const uint32_t* chunks;
+    uint32_t max_chunks;
+    const WsHeader* sel;       // the selection's header: staging is valid only if its bracket held
+    uint32_t k, cap;
+    const uint32_t* bitmap;    // the core's bitmap and directory (core_aux)
+    const uint32_t* dir;
+    int32_t* status;
+};
+
+__device__ __forceinline__ bool staged_valid(const StagedSource& s) {
+    return s.fill != nullptr && s.sel->stage_lost == 0u && bracket_held(s.sel->n_def, s.sel->n_cand, s.k, s.cap);
+}
+
+__device__ __forceinline__ void exchange_core_staged_body(float* __restrict__ w, const StagedSource& src,
+                                                          uint64_t k_core, const PtrArray<float>& val,
+                                                          const PtrArray<float>& pulled, int K, float neg_eta,
+                                                          uint32_t chunk) {
+    const uint32_t f = __ldg(src.fill + chunk);
+    const uint32_t* __restrict__ base = src.chunks + (size_t)chunk * (size_t)(K + 1) * kStageChunk;
+    for (uint32_t e = threadIdx.x; e < f; e += blockDim.x) {
+        const uint32_t i = __ldcs(base + e);
+        const uint32_t d = i >> 6, bit = i & 63u;
+        const uint2 words = __ldg(reinterpret_cast<const uint2*>(src.bitmap) + d);
+        const uint32_t word = (bit < 32u) ? words.x : words.y;
+        if (!((word >> (bit & 31u)) & 1u)) continue;   // a candidate below the threshold
+        const uint32_t below = (bit < 32u) ? __popc(words.x & ((1u << bit) - 1u))
+                                           : __popc(words.x) + __popc(words.y & ((1u << (bit - 32u)) - 1u));
+        const uint64_t j = (uint64_t)d * 64u - __ldg(src.dir + d) + below;   // core parameters below i
+        if (j >= k_core) {
+            *src.status = SLIMDP_ERR_INTERNAL;
+            continue;
+        }
+        float x = w[i];
+        int k = 0;
+        for (; k + 8 <= K; k += 8) {
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(__ldcs(base + (size_t)(k + q + 1) * kStageChunk + e));
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                __stcs(val.p[k + q] + j, v[q]);
+                x = __fmaf_rn(neg_eta, v[q], x);
+            }
+        }
+        for (; k < K; ++k) {
+            const float v = __uint_as_float(__ldcs(base + (size_t)(k + 1) * kStageChunk + e));
+            __stcs(val.p[k] + j, v);
+            x = __fmaf_rn(neg_eta, v, x);
+        }
+        x = stored_model_value(x);
+        w[i] = x;
+#pragma unroll 8
+        for (int q = 0; q < K; ++q) __stcs(pulled.p[q] + j, x);
+    }
+}
+
 // One launch for both segments.  The core segment streams whole lines of the dense layers and is
 // bound by DRAM bandwidth; the explorer segments issue sparse accesses and are bound by their
 // latency and rate.  CTAs of both kinds are interleaved in the grid (core_ctas of every
@@ -382,13 +451,20 @@ __global__ void __launch_bounds__(256) exchange_kernel(float* w, const uint32_t*
                                                        PtrArray<const float> delta, PtrArray<float> val,
                                                        PtrArray<float> pulled, int K, float neg_eta,
                                                        uint32_t range_shift, uint64_t core_ctas, uint64_t total_ctas,
-                                                       RankSource from_ranks) {
+                                                       uint64_t gather_ctas, RankSource from_ranks,
+                                                       StagedSource staged) {
     __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
     const uint64_t b = blockIdx.x;
     const uint64_t core_before = b * core_ctas / total_ctas;            // core CTAs among blocks [0, b)
     const bool is_core = (b + 1) * core_ctas / total_ctas > core_before;
     if (is_core) {
-        exchange_core_body(w, core_idx, k_core, delta, val, pulled, K, neg_eta, core_before, core_ctas);
+        // core CTA number core_before: one staged chunk, or one slice of the gather
+        if (staged_valid(staged)) {
+            if (core_before < staged.max_chunks)
+                exchange_core_staged_body(w, staged, k_core, val, pulled, K, neg_eta, (uint32_t)core_before);
+        } else if (core_before < gather_ctas) {
+            exchange_core_body(w, core_idx, k_core, delta, val, pulled, K, neg_eta, core_before, gather_ctas);
+        }
     } else if (from_ranks.ranks != nullptr) {
         // the explorers are not there yet: `exp` is where this launch writes them
         exchange_explore_ranks_body(w, from_ranks, exp, k_exp, delta, val, pulled, k_core, K, neg_eta, range_shift,
@@ -441,19 +517,30 @@ bool exchange_takes_ranks(uint64_t n, uint64_t k_exp) {
 
 // ranks / rank_stride / core_aux_* / explore_status non-null: the explorers `exp` do not exist yet;
 // the launch computes them from every worker's sorted ranks and the core's bitmap and directory
-// (exchange_takes_ranks must hold) and writes them to `exp`.
+// (exchange_takes_ranks must hold) and writes them to `exp`.  stage non-null: the core segment may
+// stream the staging area that the selection's pass filled (core_bitmap / core_dir are needed then).
 slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<const float>& delta,
                               const uint32_t* core_idx, uint64_t k_core, const PtrArray<const uint32_t>& exp,
                               uint64_t k_exp, float eta, const PtrArray<float>& val, const PtrArray<float>& pulled,
                               const uint32_t* ranks, uint64_t rank_stride, const uint32_t* core_bitmap,
-                              const uint32_t* core_dir, int32_t* explore_status, cudaStream_t st) {
+                              const uint32_t* core_dir, int32_t* explore_status, const ExchangeStage* stage,
+                              cudaStream_t st) {
     static_assert(kMergeWarps * 32 == 256, "both kinds of CTA have 256 threads");
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
-    uint64_t core_ctas = 0, explore_ctas = 0;
+    uint64_t core_ctas = 0, explore_ctas = 0, gather_ctas = 0;
     uint32_t shift = 0;
+    StagedSource staged{};
     if (k_core > 0) {
-        core_ctas = (k_core + 255) / 256;   // one core parameter per thread: short CTAs interleave best
+        gather_ctas = (k_core + 255) / 256;   // one core parameter per thread: short CTAs interleave best
+        core_ctas = gather_ctas;
+        if (stage != nullptr && stage->fill != nullptr) {
+            // which of the two ways the core segment takes is known on the device only (did the
+            // selection's bracket hold?): the grid has room for either, the other's CTAs return at once
+            staged = StagedSource{stage->fill, stage->chunks, stage->max_chunks, stage->select_hdr, (uint32_t)k_core,
+                                  stage->cand_cap, core_bitmap, core_dir, &stage->select_hdr->status};
+            if (stage->max_chunks > core_ctas) core_ctas = stage->max_chunks;
+        }
     }
     if (k_exp > 0) {
         shift = explore_range_shift(n, k_exp);
@@ -469,7 +556,7 @@ slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<c
                          explore_status};
     }
     exchange_kernel<<<(unsigned)total, 256, 0, st>>>(w, core_idx, k_core, exp, (uint32_t)k_exp, delta, val, pulled,
-                                                     (int)K, -eta, shift, core_ctas, total, src);
+                                                     (int)K, -eta, shift, core_ctas, total, gather_ctas, src, staged);
     SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }

@@ -52,7 +52,7 @@ def test_size_queries(P):
         off = P.core_aux_dir_offset(n)
         assert off >= nb * 128 and off % 256 == 0
         assert P.core_aux_bytes(n) >= off + 4 * (16 * nb + 1)
-        assert P.select_workspace_bytes(n) >= 256 + 6 * 4096 * 4 + (1 << 18) * 4 + 2 * nb * 128 + 2 * nb * 8
+        assert P.select_workspace_bytes(n) >= 256 + 6 * 4096 * 4 + (1 << 18) * 4 + 2 * nb * 128 + ((nb + 63) // 64) * 8
         k_exp = n // 100
         assert P.explore_workspace_bytes(n, k_exp, 8) > P.explore_workspace_bytes(n, k_exp, 1) >= 256 + 8 * k_exp
         assert P.explore_workspace_bytes(n, n, 1) >= 8 * n

@@ -93,8 +93,10 @@ def test_large_flat_sweep_full_size():
         r_val = [torch.empty(m, dtype=torch.float32, device="cuda") for _ in range(K)]
         r_pulled = [torch.empty(m, dtype=torch.float32, device="cuda") for _ in range(K)]
         scratch = torch.empty(n, dtype=torch.float32, device="cuda")
+        stage_bytes = P.round_stage_bytes(n, K, k_core)
+        stage = torch.empty(stage_bytes, dtype=torch.uint8, device="cuda") if stage_bytes else None
         P.slimdp_round(r_w, d_gs, base.c, cfg.seed, pct, cfg.eta, scratch, r_core, r_aux, r_exp, r_val, r_pulled,
-                       sel_ws, exp_ws)
+                       sel_ws, exp_ws, stage)
         P.read_status(sel_ws)
         P.read_status(exp_ws)
         assert torch.equal(r_core, core_idx), f"one-call core at {pct} %"
@@ -103,6 +105,6 @@ def test_large_flat_sweep_full_size():
             assert torch.equal(r_exp[k], exp_idx[k]), f"one-call explorer {k} at {pct} %"
             assert torch.equal(r_val[k].view(torch.int32), val[k].view(torch.int32)), f"one-call packed {k} at {pct} %"
             assert torch.equal(r_pulled[k].view(torch.int32), pulled[k].view(torch.int32)), f"one-call pulled {k} at {pct} %"
-        del r_w, r_core, r_aux, r_exp, r_val, r_pulled, scratch
+        del r_w, r_core, r_aux, r_exp, r_val, r_pulled, scratch, stage
         del d_w, val, pulled, exp_idx, exp_ws, core_idx
         torch.cuda.empty_cache()

@@ -155,8 +155,10 @@ def test_maximum_vector_length():
     P.slimdp_exchange(w_a, deltas, a["core"], a["exp"], eta, a["val"], a["pulled"])
     P.read_status(sel_ws)
     P.read_status(exp_ws)
+    stage = torch.empty(P.round_stage_bytes(N, K, k_core), dtype=torch.uint8, device="cuda")
+    assert stage.numel() > 0
     P.slimdp_round(w, deltas, c, 78, 4, eta, scores, b["core"], b["aux"], b["exp"], b["val"], b["pulled"], sel_ws,
-                   exp_ws)
+                   exp_ws, stage)
     P.read_status(sel_ws)
     P.read_status(exp_ws)
     assert torch.equal(a["core"], b["core"])
@@ -165,7 +167,7 @@ def test_maximum_vector_length():
         assert torch.equal(a["exp"][k], b["exp"][k])
         assert torch.equal(a["val"][k].view(torch.int32), b["val"][k].view(torch.int32))
         assert torch.equal(a["pulled"][k].view(torch.int32), b["pulled"][k].view(torch.int32))
-    del a, w_a, scores, sel_ws, exp_ws
+    del a, w_a, scores, sel_ws, exp_ws, stage
     torch.cuda.empty_cache()
 
     # ... and the one-call round against the definitions, evaluated on the host without the library:

@@ -292,9 +292,9 @@ def test_merge_collisions_follow_worker_order(P):
 
 # --------------------------------------------------------------- whole round
 
-def gpu_round(P, w, gs, cfg_c, k_core, k_exp, seed, rnd, eta, fused=True, one_call=False):
+def gpu_round(P, w, gs, cfg_c, k_core, k_exp, seed, rnd, eta, fused=True, one_call=False, staging=True):
     n, K = w.size, len(gs)
-    buf = P.RoundBuffers(n, K, k_core, k_exp)
+    buf = P.RoundBuffers(n, K, k_core, k_exp, staging=staging)
     d_w, d_gs = dev(w), [dev(g) for g in gs]
     P.run_round(d_w, d_gs, cfg_c, seed, rnd, eta, buf, fused_exchange=fused, overlapped=one_call)
     P.read_status(buf.select_ws)
@@ -319,9 +319,9 @@ def assert_round_equal(P, d_w, buf, ref, n, scores=True):
 def _round_case(P, cfg, rnd=0):
     w, gs = all_inputs(cfg)
     ref = oracle.run_round(w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta)
-    # slimdp_exchange, the three separate calls, and the whole round as one call
-    for fused, one_call in ((True, False), (False, False), (True, True)):
-        d_w, buf = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta, fused, one_call)
+    # slimdp_exchange, the three separate calls, and the whole round as one call with and without its staging area
+    for fused, one_call, staging in ((True, False, False), (False, False, False), (True, True, True), (True, True, False)):
+        d_w, buf = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, rnd, cfg.eta, fused, one_call, staging)
         assert_round_equal(P, d_w, buf, ref, cfg.N, scores=not one_call)
         del d_w, buf
     return w, gs, ref
@@ -369,9 +369,10 @@ def test_round_degenerate_ratios(P, case):
 FUSED_N = (1 << 21) + 1061      # several thousand bitmap blocks, a ragged last block, n % 4 == 1
 
 
+@pytest.mark.parametrize("staging", [True, False])
 @pytest.mark.parametrize("case", ["ragged", "k_core_one", "everything_core", "all_scores_equal", "two_values",
-                                  "nan_and_inf"])
-def test_round_one_call_fused_cases(P, case):
+                                  "nan_and_inf", "half_core", "wide_bracket"])
+def test_round_one_call_fused_cases(P, case, staging):
     cfg = scaled_config(CONFIGS["vgg16"], FUSED_N)
     w, gs = all_inputs(cfg)
     w, gs = w.copy(), [g.copy() for g in gs]
@@ -390,6 +391,11 @@ def test_round_one_call_fused_cases(P, case):
             g[:] = 0.0
         k_core = n // 2 + 12_345
         k_exp = 1000
+    elif case == "half_core":             # the largest core that is still staged
+        k_core, k_exp = n // 2, n // 8
+    elif case == "wide_bracket":          # a few huge scores: the bracket spans many octaves (three counting rounds)
+        k_core, k_exp = 5, 1000
+        w[::50_021] *= np.float32(1e30)
     elif case == "nan_and_inf":
         w[7::1001] = np.nan
         w.view(np.uint32)[9::5003] = 0xFFC12345          # a NaN with a sign and a payload
@@ -398,7 +404,7 @@ def test_round_one_call_fused_cases(P, case):
         gs[2][5::3001] = -np.inf
         w[11::4001] = np.float32(-0.0)
     ref = oracle.run_round(w, gs, cfg.c, k_core, k_exp, cfg.seed, 2, cfg.eta)
-    d_w, buf = gpu_round(P, w, gs, cfg.c, k_core, k_exp, cfg.seed, 2, cfg.eta, one_call=True)
+    d_w, buf = gpu_round(P, w, gs, cfg.c, k_core, k_exp, cfg.seed, 2, cfg.eta, one_call=True, staging=staging)
     assert_round_equal(P, d_w, buf, ref, n, scores=False)
     if case == "all_scores_equal":        # and there the scratch does hold the scores
         assert np.array_equal(host_bits(buf.scores), bits(ref["scores"]))
@@ -558,3 +564,112 @@ def test_core_signature_parity(P, count):
     P.slimdp_core_signature(dev(keys), sig)
     assert int(sig.cpu().numpy().view(np.uint64)[0]) == oracle.core_signature(keys)
     assert P.wire_bytes(1000, 50) == 4 * 1000 + 8 * 50 + 8
+
+
+# ---------------------------------------------------------------- wire message (Section 3.5)
+
+def u64_dev(x: int) -> torch.Tensor:
+    """A one-element int64 CUDA tensor holding the 64-bit pattern x."""
+    return torch.from_numpy(np.array([x], np.uint64).view(np.int64)).cuda()
+
+
+def u64_host(t: torch.Tensor) -> int:
+    return int(t.cpu().numpy().view(np.uint64)[0])
+
+
+@pytest.mark.parametrize("k_core,k_exp", [(0, 0), (1, 0), (0, 1), (7, 5), (700, 333), (100_003, 40_001)])
+def test_wire_pack_and_unpack_match_the_oracle(P, k_core, k_exp):
+    rng = np.random.default_rng(100 + k_core)
+    n = 3 * (k_core + k_exp) + 10
+    idx = rng.permutation(n).astype(np.uint32)
+    core, exp = np.sort(idx[:k_core]), np.sort(idx[k_core:k_core + k_exp])
+    val = rng.standard_normal(k_core + k_exp).astype(np.float32)
+    if val.size:
+        val.view(np.uint32)[0] = 0x7FC12345          # the message moves bits
+    i32 = lambda a: torch.from_numpy(a.view(np.int32)).cuda()
+    d_core, d_exp, d_val = i32(core), i32(exp), dev(val)
+    d_sig = torch.zeros(1, dtype=torch.int64, device="cuda")
+    P.slimdp_core_signature(d_core, d_sig)
+    for with_keys in (False, True):
+        want = oracle.wire_pack(core, exp, val, 3, 17, with_keys)
+        msg = torch.zeros(P.wire_message_bytes(k_core, k_exp, with_keys), dtype=torch.uint8, device="cuda")
+        assert msg.numel() == want.size
+        P.slimdp_wire_pack(d_core, d_exp, d_val, d_sig, 3, 17, with_keys, msg)
+        assert np.array_equal(msg.cpu().numpy(), want), f"message bytes, with_keys={with_keys}"
+        # the receiver: cached keys current / stale
+        for stale in (False, True):
+            cached = u64_dev(oracle.core_signature(core) ^ (0x55 if stale else 0))
+            o_core = torch.full((k_core,), -1, dtype=torch.int32, device="cuda")
+            o_exp = torch.full((k_exp,), -1, dtype=torch.int32, device="cuda")
+            o_val = torch.full((k_core + k_exp,), 7.0, dtype=torch.float32, device="cuda")
+            o_sig = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+            status = torch.zeros(4, dtype=torch.int32, device="cuda")
+            P.slimdp_wire_unpack(msg, cached, o_core, o_exp, o_val, o_sig, status)
+            st = P.wire_read_status(status)
+            ref_st, ref_core, ref_exp, ref_val, ref_sig = oracle.wire_unpack(want, u64_host(cached), k_core, k_exp)
+            assert st == ref_st
+            if st == 0:
+                assert np.array_equal(host_u32(o_exp), ref_exp)
+                assert np.array_equal(host_bits(o_val), bits(ref_val))
+                assert u64_host(o_sig) == ref_sig
+                if with_keys:
+                    assert np.array_equal(host_u32(o_core), ref_core)
+                else:
+                    assert bool((o_core == -1).all())
+            else:       # keys wanted: nothing was written
+                assert st == P.WIRE_KEYS_WANTED and not with_keys and stale
+                assert bool((o_exp == -1).all()) and bool((o_val == 7.0).all()) and int(o_sig.item()) == -1
+
+
+def test_wire_malformed_messages_are_refused_on_the_device(P):
+    core, exp = np.array([1, 4, 6], np.uint32), np.array([2, 3], np.uint32)
+    val = np.arange(5, dtype=np.float32)
+    good = oracle.wire_pack(core, exp, val, 0, 0, True)
+    cached = u64_dev(oracle.core_signature(core))
+
+    def verdict(msg_bytes, k_core=3, k_exp=2):
+        msg = torch.from_numpy(msg_bytes.copy()).cuda()
+        o_core = torch.zeros(k_core, dtype=torch.int32, device="cuda")
+        o_exp = torch.zeros(k_exp, dtype=torch.int32, device="cuda")
+        o_val = torch.zeros(k_core + k_exp, dtype=torch.float32, device="cuda")
+        o_sig = torch.zeros(1, dtype=torch.int64, device="cuda")
+        status = torch.zeros(4, dtype=torch.int32, device="cuda")
+        P.slimdp_wire_unpack(msg, cached, o_core, o_exp, o_val, o_sig, status)
+        return P.wire_read_status(status)
+
+    assert verdict(good) == 0
+    for mutate in (lambda m: m.__setitem__(0, m[0] ^ 1), lambda m: m.__setitem__(32, m[32] ^ 1),
+                   lambda m: m.__setitem__(4, 2)):
+        bad = good.copy()
+        mutate(bad)
+        with pytest.raises(P.SlimDPError):
+            verdict(bad)
+    with pytest.raises(P.SlimDPError):
+        verdict(good[:-4])
+    with pytest.raises(P.SlimDPError):
+        verdict(good, k_core=2, k_exp=2)
+
+
+def test_wire_unpack_feeds_the_merge(P):
+    cfg = CONFIGS["tiny"]
+    w, gs = all_inputs(cfg)
+    ref = oracle.run_round(w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 0, cfg.eta)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int32)).cuda()
+    d_core = i32(ref["core_idx"])
+    d_sig = torch.zeros(1, dtype=torch.int64, device="cuda")
+    P.slimdp_core_signature(d_core, d_sig)
+    exps, vals = [], []
+    for k in range(cfg.K):      # every worker's push goes through a message and is taken apart again
+        msg = torch.empty(P.wire_message_bytes(cfg.k_core, cfg.k_exp, False), dtype=torch.uint8, device="cuda")
+        P.slimdp_wire_pack(d_core, i32(ref["exp_idx"][k]), dev(ref["val"][k]), d_sig, k, 0, False, msg)
+        o_core = torch.empty(cfg.k_core, dtype=torch.int32, device="cuda")
+        o_exp = torch.empty(cfg.k_exp, dtype=torch.int32, device="cuda")
+        o_val = torch.empty(cfg.m, dtype=torch.float32, device="cuda")
+        status = torch.zeros(4, dtype=torch.int32, device="cuda")
+        P.slimdp_wire_unpack(msg, d_sig, o_core, o_exp, o_val, d_sig.clone(), status)
+        assert P.wire_read_status(status) == 0
+        exps.append(o_exp)
+        vals.append(o_val)
+    d_w = dev(w)
+    P.slimdp_merge(d_w, d_core, exps, vals, cfg.eta)
+    assert np.array_equal(host_bits(d_w), bits(ref["w"]))
