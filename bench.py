@@ -227,7 +227,7 @@ def run_ours(args):
     w_host, g_host = all_inputs(cfg)
     w = torch.from_numpy(w_host).to(device)
     grads = [torch.from_numpy(g).to(device) for g in g_host]
-    buf = P.RoundBuffers(N, K, k_core, k_exp, device, staging=not args.no_staging)
+    buf = P.RoundBuffers(N, K, k_core, k_exp, device, staging=args.staging)
     bytes_model = model_bytes(N, K, k_core, k_exp)
 
     def barrier():
@@ -431,8 +431,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
-    ap.add_argument("--no-staging", action="store_true",
-                    help="run slimdp_round without its staging area (the exchange then gathers the core's values)")
+    ap.add_argument("--staging", action="store_true",
+                    help="give slimdp_round its optional staging area (the exchange then streams the core's values)")
     ap.add_argument("--timeline", default="",
                     help="also write the kernel timeline of three extra rounds (start, duration, stream) to this file")
     ap.add_argument("--scale", type=int, default=0,

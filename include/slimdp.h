@@ -123,6 +123,22 @@ slimdp_status slimdp_score(const float* w, const float* const* grads, uint32_t K
 slimdp_status slimdp_select_core(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx,
                                  void* core_aux, void* ws, size_t ws_bytes, void* stream);
 
+/* Per-layer selection: the ranking of Section 3.2 done segment by segment, the simplest of the
+ * "model-specific" significance measures that Section 5 leaves open.  The vector is cut into
+ * `segments` consecutive segments (layers), segment s = [seg_off[s], seg_off[s+1]); segment s
+ * contributes its seg_k[s] parameters of largest score, ties to the smaller index; the core is
+ * their union.  core_idx (ascending, sum of seg_k entries) and core_aux come out exactly as from
+ * slimdp_select_core, so every other call works on the result unchanged.
+ *   seg_off  HOST array [segments + 1], seg_off[0] = 0, non-decreasing, seg_off[segments] = n
+ *   seg_k    HOST array [segments], seg_k[s] <= length of segment s
+ *   (both are copied during the call and may be freed when it returns)
+ *   ws       [ws_bytes >= slimdp_select_segmented_workspace_bytes(n, segments)] scratch */
+#define SLIMDP_MAX_SEGMENTS 65536
+size_t slimdp_select_segmented_workspace_bytes(uint64_t n, uint32_t segments);
+slimdp_status slimdp_select_core_segmented(const float* scores, uint64_t n, const uint64_t* seg_off,
+                                           const uint64_t* seg_k, uint32_t segments, uint32_t* core_idx,
+                                           void* core_aux, void* ws, size_t ws_bytes, void* stream);
+
 /* -------------------------------------------------------------- explore ---
  * Exploration operator T_R^k (Section 3.1 item 2, Section 3.3 step 2): worker
  * `worker` draws, for communication `round`, k_exp distinct parameters
@@ -283,6 +299,32 @@ slimdp_status slimdp_worker_merge_batched(float* const* w_local, uint32_t K, uin
  * i.e. (2 alpha - beta) n words as in Section 3.5, against 4 n for Plump-DP. */
 slimdp_status slimdp_core_signature(const uint32_t* keys, uint64_t count, uint64_t* signature, void* stream);
 size_t slimdp_wire_bytes(uint64_t k_core, uint64_t k_exp);
+
+/* ------------------------------------------------ 8-bit pushed values ---
+ * Section 2.2 closes by noting that the method combines with quantisation of
+ * what is sent.  The paper defines no quantiser; this library fixes a
+ * deterministic one so that sender, receiver and a reference agree bit for bit.
+ * A worker's packed buffer (core values, then explorer values: k_core + k_exp
+ * entries) is cut into buckets of SLIMDP_Q8_BUCKET consecutive entries; a
+ * bucket's scale is its largest finite magnitude; a value v becomes the code
+ *     rint(v * (127 / scale)) clamped to [-127, 127]   (fp32 division, fp32 product, ties to even),
+ * 0 if the scale is 0 or v is a NaN, +-127 if v is an infinity; the receiver
+ * reads code * (scale / 127) (fp32 division, fp32 product).  A push then costs
+ * k_core + k_exp bytes of codes and one fp32 scale per bucket instead of
+ * 4 (k_core + k_exp) bytes of values.
+ * slimdp_pack_q8_batched: slimdp_pack_batched with the quantiser folded into its
+ *   stores (the fp32 packed buffer is never written).
+ *   codes   HOST array of K device pointers, each int8 [k_core + k_exp] (written)
+ *   scales  HOST array of K device pointers, each fp32 [ceil((k_core + k_exp) / SLIMDP_Q8_BUCKET)] (written)
+ * slimdp_merge_q8: slimdp_merge reading its values through the codes: bit-identical to
+ *   slimdp_merge on the decoded values. */
+#define SLIMDP_Q8_BUCKET 256
+slimdp_status slimdp_pack_q8_batched(const float* const* deltas, uint32_t K, uint64_t n, const uint32_t* core_idx,
+                                     uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
+                                     int8_t* const* codes, float* const* scales, void* stream);
+slimdp_status slimdp_merge_q8(float* w_global, uint64_t n, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+                              const uint32_t* const* exp_idx, uint64_t k_exp, const int8_t* const* codes,
+                              const float* const* scales, float eta, void* stream);
 
 /* ------------------------------------------ selection over a sharded model ---
  * The parameter-server setting of Section 2.1 with the global model cut into

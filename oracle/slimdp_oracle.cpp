@@ -375,7 +375,13 @@ void oracle_quantize_q8(const float* val, uint64_t m, uint32_t bucket, int8_t* c
         const float inv = (amax > 0.0f) ? 127.0f / amax : 0.0f;
         for (uint64_t j = b0; j < b1; ++j) {
             const float v = val[j];
-            float q = std::isnan(v) ? 0.0f : std::rint(v * inv);
+            float q;
+            if (std::isnan(v))
+                q = 0.0f;
+            else if (std::isinf(v))
+                q = (v > 0.0f) ? 127.0f : -127.0f;   // whatever the scale, 0 included
+            else
+                q = std::rint(v * inv);
             if (q > 127.0f) q = 127.0f;
             if (q < -127.0f) q = -127.0f;
             codes[j] = (int8_t)q;

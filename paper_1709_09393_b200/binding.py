@@ -51,6 +51,10 @@ EXPORTS = {
     "slimdp_worker_merge_batched": (ctypes.c_int32, [_pp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _vp]),
     "slimdp_core_signature": (ctypes.c_int32, [_vp, _u64, _vp, _vp]),
     "slimdp_wire_bytes": (_sz, [_u64, _u64]),
+    "slimdp_select_segmented_workspace_bytes": (_sz, [_u64, _u32]),
+    "slimdp_select_core_segmented": (ctypes.c_int32, [_vp, _u64, _vp, _vp, _u32, _vp, _vp, _vp, _sz, _vp]),
+    "slimdp_pack_q8_batched": (ctypes.c_int32, [_pp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _pp, _vp]),
+    "slimdp_merge_q8": (ctypes.c_int32, [_vp, _u64, _u32, _vp, _u64, _pp, _u64, _pp, _pp, _f32, _vp]),
     "slimdp_select_shard_begin": (ctypes.c_int32, [_u64, _vp, _vp]),
     "slimdp_select_hist": (ctypes.c_int32, [_vp, _u64, _u32, _vp, _vp, _vp]),
     "slimdp_select_resolve": (ctypes.c_int32, [_vp, _u32, _vp, _vp]),
@@ -404,6 +408,60 @@ def slimdp_core_signature(keys: torch.Tensor, signature: torch.Tensor, stream=No
 
 def wire_bytes(k_core: int, k_exp: int) -> int:
     return lib.slimdp_wire_bytes(k_core, k_exp)
+
+
+def select_segmented_workspace_bytes(n: int, segments: int) -> int:
+    return lib.slimdp_select_segmented_workspace_bytes(n, segments)
+
+
+def slimdp_select_core_segmented(scores: torch.Tensor, seg_off: Sequence[int], seg_k: Sequence[int],
+                                 core_idx: torch.Tensor, core_aux: torch.Tensor, ws: torch.Tensor, stream=None):
+    """Per-layer selection: segment s = [seg_off[s], seg_off[s+1]) contributes its seg_k[s] largest scores."""
+    _dev(scores, torch.float32, "scores")
+    _dev(core_idx, IDX, "core_idx")
+    S = len(seg_k)
+    if len(seg_off) != S + 1:
+        raise ValueError("seg_off must have one entry more than seg_k")
+    if core_idx.numel() != sum(int(k) for k in seg_k):
+        raise ValueError("core_idx: length differs from the sum of seg_k")
+    off = (ctypes.c_uint64 * (S + 1))(*[int(x) for x in seg_off])
+    ks = (ctypes.c_uint64 * S)(*[int(x) for x in seg_k])
+    _check("slimdp_select_core_segmented",
+           lib.slimdp_select_core_segmented(scores.data_ptr(), scores.numel(), off, ks, S, _ptr(core_idx),
+                                            core_aux.data_ptr(), ws.data_ptr(), ws.numel(), _stream(stream)))
+
+
+Q8_BUCKET = 256
+
+
+def slimdp_pack_q8_batched(deltas: Sequence[torch.Tensor], core_idx: torch.Tensor, exp_idx: Sequence[torch.Tensor],
+                           codes: Sequence[torch.Tensor], scales: Sequence[torch.Tensor], stream=None):
+    """Extraction with the 8-bit quantiser folded in: codes[k] int8[m], scales[k] float32[ceil(m / 256)]."""
+    K, n = len(deltas), deltas[0].numel()
+    m = core_idx.numel() + exp_idx[0].numel()
+    for d, e, c, s in zip(deltas, exp_idx, codes, scales):
+        _dev(d, torch.float32, "deltas")
+        _dev(e, IDX, "exp_idx")
+        if _dev(c, torch.int8, "codes").numel() != m or _dev(s, torch.float32, "scales").numel() != (m + 255) // 256:
+            raise ValueError("codes / scales: wrong length")
+    _check("slimdp_pack_q8_batched",
+           lib.slimdp_pack_q8_batched(_ptr_array(deltas), K, n, _ptr(core_idx), core_idx.numel(), _ptr_array(exp_idx),
+                                      exp_idx[0].numel(), _ptr_array(codes), _ptr_array(scales), _stream(stream)))
+
+
+def slimdp_merge_q8(w_global: torch.Tensor, core_idx: torch.Tensor, exp_idx: Sequence[torch.Tensor],
+                    codes: Sequence[torch.Tensor], scales: Sequence[torch.Tensor], eta: float, stream=None):
+    """Server update reading the pushed values through their 8-bit codes."""
+    _dev(w_global, torch.float32, "w_global")
+    K = len(codes)
+    for e, c, s in zip(exp_idx, codes, scales):
+        _dev(e, IDX, "exp_idx")
+        _dev(c, torch.int8, "codes")
+        _dev(s, torch.float32, "scales")
+    _check("slimdp_merge_q8",
+           lib.slimdp_merge_q8(w_global.data_ptr(), w_global.numel(), K, _ptr(core_idx), core_idx.numel(),
+                               _ptr_array(exp_idx), exp_idx[0].numel(), _ptr_array(codes), _ptr_array(scales), eta,
+                               _stream(stream)))
 
 
 def slimdp_select_shard_begin(k_total: int, state: torch.Tensor, stream=None):

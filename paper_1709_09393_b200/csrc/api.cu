@@ -58,6 +58,17 @@ slimdp_status launch_worker_merge(const PtrArray<float>& w_local, uint32_t worke
                                   uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp,
                                   const PtrArray<const float>& pulled, cudaStream_t st);
 
+size_t seg_select_ws_bytes(uint64_t n, uint32_t segments);
+slimdp_status launch_select_segmented(const float* scores, uint64_t n, const uint64_t* seg_off, const uint64_t* seg_k,
+                                      uint32_t segments, uint64_t k_total, uint32_t* core_idx, void* core_aux,
+                                      void* ws, cudaStream_t st);
+slimdp_status launch_pack_q8(const PtrArray<const float>& delta, uint32_t K, const uint32_t* core_idx,
+                             uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp,
+                             const PtrArray<int8_t>& codes, const PtrArray<float>& scales, cudaStream_t st);
+slimdp_status launch_merge_q8(float* w, uint64_t n, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+                              const PtrArray<const uint32_t>& exp, uint64_t k_exp,
+                              const PtrArray<const int8_t>& codes, const PtrArray<const float>& scales, float eta,
+                              cudaStream_t st);
 slimdp_status launch_select_given(const float* scores, uint64_t n, uint32_t T, uint32_t ties, uint64_t k_shard,
                                   uint32_t* core_idx, void* core_aux, void* ws, cudaStream_t st);
 slimdp_status launch_shard_state_init(void* state, uint64_t k, cudaStream_t st);
@@ -319,6 +330,68 @@ slimdp_status slimdp_core_signature(const uint32_t* keys, uint64_t count, uint64
 }
 
 size_t slimdp_wire_bytes(uint64_t k_core, uint64_t k_exp) { return (size_t)(4 * k_core + 8 * k_exp + 8); }
+
+// ---- per-segment selection --------------------------------------------------
+
+size_t slimdp_select_segmented_workspace_bytes(uint64_t n, uint32_t segments) {
+    if (!n_ok(n) || segments < 1 || segments > SLIMDP_MAX_SEGMENTS) return 0;
+    return seg_select_ws_bytes(n, segments);
+}
+
+slimdp_status slimdp_select_core_segmented(const float* scores, uint64_t n, const uint64_t* seg_off,
+                                           const uint64_t* seg_k, uint32_t segments, uint32_t* core_idx,
+                                           void* core_aux, void* ws, size_t ws_bytes, void* stream) {
+    if (!n_ok(n) || segments < 1 || segments > SLIMDP_MAX_SEGMENTS || !scores || !seg_off || !seg_k || !core_aux ||
+        !ws)
+        return SLIMDP_ERR_INVALID_ARG;
+    if (!aligned4(scores) || !aligned16(core_aux) || !aligned16(ws)) return SLIMDP_ERR_INVALID_ARG;
+    if (seg_off[0] != 0 || seg_off[segments] != n) return SLIMDP_ERR_INVALID_ARG;
+    uint64_t k_total = 0;
+    for (uint32_t s = 0; s < segments; ++s) {
+        if (seg_off[s + 1] < seg_off[s] || seg_k[s] > seg_off[s + 1] - seg_off[s]) return SLIMDP_ERR_INVALID_ARG;
+        k_total += seg_k[s];
+    }
+    if (k_total > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (ws_bytes < slimdp_select_segmented_workspace_bytes(n, segments)) return SLIMDP_ERR_WORKSPACE;
+    return launch_select_segmented(scores, n, seg_off, seg_k, segments, k_total, core_idx, core_aux, ws,
+                                   (cudaStream_t)stream);
+}
+
+// ---- 8-bit pushed values ---------------------------------------------------
+
+slimdp_status slimdp_pack_q8_batched(const float* const* deltas, uint32_t K, uint64_t n, const uint32_t* core_idx,
+                                     uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
+                                     int8_t* const* codes, float* const* scales, void* stream) {
+    if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !deltas) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned4(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    PtrArray<const float> d;
+    PtrArray<const uint32_t> exp;
+    PtrArray<int8_t> c;
+    PtrArray<float> sc;
+    const bool any = k_core + k_exp > 0;
+    if (!fill<const float>(d, deltas, K, true, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<int8_t>(c, codes, K, any, 1)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<float>(sc, scales, K, any, 4)) return SLIMDP_ERR_INVALID_ARG;
+    return launch_pack_q8(d, K, core_idx, k_core, exp, k_exp, c, sc, (cudaStream_t)stream);
+}
+
+slimdp_status slimdp_merge_q8(float* w_global, uint64_t n, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+                              const uint32_t* const* exp_idx, uint64_t k_exp, const int8_t* const* codes,
+                              const float* const* scales, float eta, void* stream) {
+    if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !w_global || !aligned4(w_global) || !isfinite(eta))
+        return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned4(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    PtrArray<const uint32_t> exp;
+    PtrArray<const int8_t> c;
+    PtrArray<const float> sc;
+    const bool any = k_core + k_exp > 0;
+    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const int8_t>(c, codes, K, any, 1)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const float>(sc, scales, K, any, 4)) return SLIMDP_ERR_INVALID_ARG;
+    if (!any) return SLIMDP_OK;
+    return launch_merge_q8(w_global, n, K, core_idx, k_core, exp, k_exp, c, sc, eta, (cudaStream_t)stream);
+}
 
 // ---- selection over a range-sharded model ---------------------------------
 

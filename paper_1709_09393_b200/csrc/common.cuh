@@ -16,6 +16,7 @@ constexpr uint32_t kWordsPerDir = kDirStride / 32;      // 2 bitmap words per di
 static_assert(kWordsPerDir == 2, "select0 walks exactly two bitmap words per directory entry");
 constexpr uint32_t kSampleBits = 18;             // the selection's bracket is estimated from 2^18 sampled keys
 constexpr uint64_t kBracketMinN = 1ull << 21;    // below this the selection reads the keys three more times instead
+constexpr uint32_t kQ8Bucket = SLIMDP_Q8_BUCKET;   // packed entries that share one scale of the 8-bit codes
 constexpr uint32_t kStageChunk = 512;            // entries per chunk of the staging area (see layout.cuh)
 
 // K device pointers passed by value as a kernel argument (512 bytes).

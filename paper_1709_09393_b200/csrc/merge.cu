@@ -22,9 +22,24 @@ namespace {
 
 constexpr int kMergeWarps = 8;
 
+// Where the pushed values come from: fp32 buffers as slimdp_pack writes them, or 8-bit codes with
+// one fp32 scale per bucket of kQ8Bucket packed entries (value = code * (scale / 127), fp32).
+struct F32Vals {
+    PtrArray<const float> p;
+    __device__ __forceinline__ float get(int k, uint64_t j) const { return __ldcs(p.p[k] + j); }
+};
+struct Q8Vals {
+    PtrArray<const int8_t> codes;
+    PtrArray<const float> scales;
+    __device__ __forceinline__ float get(int k, uint64_t j) const {
+        const float step = __fdiv_rn(__ldg(scales.p[k] + j / kQ8Bucket), 127.0f);
+        return __fmul_rn((float)__ldg(codes.p[k] + j), step);
+    }
+};
+
+template <typename Vals>
 __global__ void __launch_bounds__(256) merge_core_kernel(float* __restrict__ w, const uint32_t* __restrict__ core_idx,
-                                                         uint64_t k_core, PtrArray<const float> val, int K,
-                                                         float neg_eta) {
+                                                         uint64_t k_core, Vals val, int K, float neg_eta) {
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
     for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k_core; j += stride) {
         const uint32_t i = __ldg(core_idx + j);
@@ -33,11 +48,11 @@ __global__ void __launch_bounds__(256) merge_core_kernel(float* __restrict__ w, 
         for (; k + 8 <= K; k += 8) {
             float v[8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = __ldcs(val.p[k + q] + j);
+            for (int q = 0; q < 8; ++q) v[q] = val.get(k + q, j);
 #pragma unroll
             for (int q = 0; q < 8; ++q) x = __fmaf_rn(neg_eta, v[q], x);
         }
-        for (; k < K; ++k) x = __fmaf_rn(neg_eta, __ldcs(val.p[k] + j), x);
+        for (; k < K; ++k) x = __fmaf_rn(neg_eta, val.get(k, j), x);
         w[i] = stored_model_value(x);
     }
 }
@@ -123,10 +138,10 @@ __device__ __forceinline__ uint32_t touch_range(const float* w, const PtrArray<c
 // One CTA owns 8 consecutive ranges of 2^range_shift parameters, one per warp.  Every warp, on
 // its own, first requests all lines it is going to touch (L2 prefetch), then applies worker 0's
 // entries of its range, a warp barrier, worker 1's entries, ...
+template <typename Vals>
 __global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* w, PtrArray<const uint32_t> exp,
-                                                                         uint32_t k_exp, PtrArray<const float> val,
-                                                                         uint64_t k_core, int K, float neg_eta,
-                                                                         uint32_t range_shift) {
+                                                                         uint32_t k_exp, Vals val, uint64_t k_core,
+                                                                         int K, float neg_eta, uint32_t range_shift) {
     __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
     find_bounds(bound, exp, k_exp, K, range_shift, blockIdx.x);
     const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
@@ -134,11 +149,10 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* 
     const uint32_t sink = touch_range<false>(w, exp, none, bound, K, wid, lane);
     for (int k = 0; k < K; ++k) {
         const uint32_t* __restrict__ idx = exp.p[k];
-        const float* __restrict__ v = val.p[k] + k_core;
         const uint32_t b = bound[k][wid + 1];
         for (uint32_t e = bound[k][wid] + lane; e < b; e += 32) {
             const uint32_t i = __ldg(idx + e);
-            w[i] = stored_model_value(__fmaf_rn(neg_eta, __ldcs(v + e), ld_sparse(w + i)));
+            w[i] = stored_model_value(__fmaf_rn(neg_eta, val.get(k, k_core + e), ld_sparse(w + i)));
         }
         __syncwarp();   // worker k's updates are visible to the whole warp before worker k+1 starts
     }
@@ -484,27 +498,41 @@ uint32_t explore_range_shift(uint64_t n, uint64_t k_exp) {
 
 }  // namespace
 
-slimdp_status launch_merge(float* w, uint64_t n, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
-                           const PtrArray<const uint32_t>& exp, uint64_t k_exp, const PtrArray<const float>& val,
-                           float eta, cudaStream_t st) {
+template <typename Vals>
+static slimdp_status launch_merge_with(float* w, uint64_t n, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+                                       const PtrArray<const uint32_t>& exp, uint64_t k_exp, const Vals& val, float eta,
+                                       cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
     const float neg_eta = -eta;
     if (k_core > 0) {
         uint64_t grid = (k_core + 255) / 256;
         if (grid > (uint64_t)sms * 32) grid = (uint64_t)sms * 32;
-        merge_core_kernel<<<(unsigned)grid, 256, 0, st>>>(w, core_idx, k_core, val, (int)K, neg_eta);
+        merge_core_kernel<Vals><<<(unsigned)grid, 256, 0, st>>>(w, core_idx, k_core, val, (int)K, neg_eta);
         SLIMDP_LAUNCHED(1);
     }
     if (k_exp > 0) {
         const uint32_t shift = explore_range_shift(n, k_exp);
         const uint64_t per_cta = (uint64_t)kMergeWarps << shift;
         const uint64_t ctas = (n + per_cta - 1) / per_cta;
-        merge_explore_kernel<<<(unsigned)ctas, kMergeWarps * 32, 0, st>>>(w, exp, (uint32_t)k_exp, val, k_core,
-                                                                          (int)K, neg_eta, shift);
+        merge_explore_kernel<Vals><<<(unsigned)ctas, kMergeWarps * 32, 0, st>>>(w, exp, (uint32_t)k_exp, val, k_core,
+                                                                                (int)K, neg_eta, shift);
         SLIMDP_LAUNCHED(1);
     }
     return SLIMDP_OK;
+}
+
+slimdp_status launch_merge(float* w, uint64_t n, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+                           const PtrArray<const uint32_t>& exp, uint64_t k_exp, const PtrArray<const float>& val,
+                           float eta, cudaStream_t st) {
+    return launch_merge_with(w, n, K, core_idx, k_core, exp, k_exp, F32Vals{val}, eta, st);
+}
+
+slimdp_status launch_merge_q8(float* w, uint64_t n, uint32_t K, const uint32_t* core_idx, uint64_t k_core,
+                              const PtrArray<const uint32_t>& exp, uint64_t k_exp,
+                              const PtrArray<const int8_t>& codes, const PtrArray<const float>& scales, float eta,
+                              cudaStream_t st) {
+    return launch_merge_with(w, n, K, core_idx, k_core, exp, k_exp, Q8Vals{codes, scales}, eta, st);
 }
 
 // Whether the exchange can turn sorted ranks into explorer indices itself: a warp's range must be

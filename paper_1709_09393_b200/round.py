@@ -14,7 +14,7 @@ class RoundBuffers:
     """Device buffers one round needs for n parameters, K workers and the
     integer set sizes k_core, k_exp.  Allocated once, reused every round."""
 
-    def __init__(self, n: int, K: int, k_core: int, k_exp: int, device="cuda", staging: bool = True):
+    def __init__(self, n: int, K: int, k_core: int, k_exp: int, device="cuda", staging: bool = False):
         self.n, self.K, self.k_core, self.k_exp = n, K, k_core, k_exp
         m = k_core + k_exp
         dev = torch.device(device)
@@ -23,7 +23,8 @@ class RoundBuffers:
         self.core_aux = torch.empty(B.core_aux_bytes(n), dtype=torch.uint8, device=dev)
         self.select_ws = torch.empty(B.select_workspace_bytes(n), dtype=torch.uint8, device=dev)
         self.explore_ws = torch.empty(B.explore_workspace_bytes(n, k_exp, K), dtype=torch.uint8, device=dev)
-        # the one-call round's staging area (None where staging does not apply or is not wanted)
+        # the one-call round's optional staging area (off by default: on the measured workloads the pass
+        # loses more by filling it than the exchange gains by streaming it)
         stage_bytes = B.round_stage_bytes(n, K, k_core) if staging else 0
         self.stage = torch.empty(stage_bytes, dtype=torch.uint8, device=dev) if stage_bytes else None
         self.exp_idx: List[torch.Tensor] = [torch.empty(k_exp, dtype=B.IDX, device=dev) for _ in range(K)]

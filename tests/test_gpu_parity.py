@@ -292,7 +292,7 @@ def test_merge_collisions_follow_worker_order(P):
 
 # --------------------------------------------------------------- whole round
 
-def gpu_round(P, w, gs, cfg_c, k_core, k_exp, seed, rnd, eta, fused=True, one_call=False, staging=True):
+def gpu_round(P, w, gs, cfg_c, k_core, k_exp, seed, rnd, eta, fused=True, one_call=False, staging=False):
     n, K = w.size, len(gs)
     buf = P.RoundBuffers(n, K, k_core, k_exp, staging=staging)
     d_w, d_gs = dev(w), [dev(g) for g in gs]
@@ -673,3 +673,91 @@ def test_wire_unpack_feeds_the_merge(P):
     d_w = dev(w)
     P.slimdp_merge(d_w, d_core, exps, vals, cfg.eta)
     assert np.array_equal(host_bits(d_w), bits(ref["w"]))
+
+
+# ------------------------------------------------------------- 8-bit pushed values (Section 2.2, last remark)
+
+@pytest.mark.parametrize("n,k_core,k_exp,K", [(1000, 100, 37, 1), (100_003, 20_000, 5_001, 3), (5000, 0, 700, 2),
+                                               (5000, 256, 0, 2), (300_000, 65_536, 30_000, 8)])
+def test_q8_pack_and_merge_match_the_oracle(P, n, k_core, k_exp, K):
+    rng = np.random.default_rng(n + K)
+    idx = rng.permutation(n).astype(np.uint32)
+    core = np.sort(idx[:k_core])
+    exps = [np.sort(rng.permutation(np.setdiff1d(np.arange(n, dtype=np.uint32), core))[:k_exp]) for _ in range(K)]
+    w = rng.standard_normal(n).astype(np.float32)
+    ds = [(rng.standard_normal(n) * np.exp(rng.uniform(-6, 1, n))).astype(np.float32) for _ in range(K)]
+    ds[0][::97] = 0.0
+    if k_core:                                   # non-finite values, and a bucket with nothing but zeros
+        ds[0][core[:3]] = [np.nan, np.inf, -np.inf]
+        ds[-1][core[:min(256, k_core)]] = 0.0
+    m = k_core + k_exp
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int32)).cuda()
+    d_core, d_exps = i32(core), [i32(e) for e in exps]
+    codes = [torch.zeros(m, dtype=torch.int8, device="cuda") for _ in range(K)]
+    scales = [torch.zeros((m + 255) // 256, dtype=torch.float32, device="cuda") for _ in range(K)]
+    P.slimdp_pack_q8_batched([dev(d) for d in ds], d_core, d_exps, codes, scales)
+    deq = []
+    for k in range(K):
+        ref_codes, ref_scales = oracle.quantize_q8(oracle.pack(ds[k], core, exps[k]))
+        assert np.array_equal(codes[k].cpu().numpy(), ref_codes), f"codes of worker {k}"
+        assert np.array_equal(host_bits(scales[k]), bits(ref_scales)), f"scales of worker {k}"
+        deq.append(oracle.dequantize_q8(ref_codes, ref_scales))
+    d_w = dev(w)
+    P.slimdp_merge_q8(d_w, d_core, d_exps, codes, scales, 1.0 / K)
+    assert np.array_equal(host_bits(d_w), bits(oracle.merge(w, core, exps, deq, 1.0 / K)))
+
+
+# ------------------------------------------------------------- per-layer selection (Section 5)
+
+def _segmented_case(P, S, off, ks):
+    n = S.size
+    k = int(sum(ks))
+    core_idx = torch.empty(k, dtype=torch.int32, device="cuda")
+    aux = torch.empty(P.core_aux_bytes(n), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(P.select_segmented_workspace_bytes(n, len(ks)), dtype=torch.uint8, device="cuda")
+    P.slimdp_select_core_segmented(dev(S), off, ks, core_idx, aux, ws)
+    P.read_status(ws)
+    ref = oracle.select_core_segmented(S, off, ks)
+    assert np.array_equal(host_u32(core_idx), ref)
+    check_aux(P, aux, ref, n)
+
+
+@pytest.mark.parametrize("name", ["googlenet", "resnet50_ties", "vgg16"])
+def test_segmented_select_on_the_layer_tables(P, name):
+    # the layers of the shaped workloads (biases and batch-norm vectors are segments of their own);
+    # every layer keeps the workload's core ratio of its own parameters
+    cfg = CONFIGS[name] if name != "vgg16" else scaled_config(CONFIGS["vgg16"], 20_000_003)
+    w, gs = all_inputs(cfg)
+    S = oracle.score(w, gs, cfg.c)
+    off = [0]
+    for seg in cfg.segments:
+        off.append(off[-1] + seg.size)
+    ks = [(off[i + 1] - off[i]) * cfg.core_pct // 100 for i in range(len(off) - 1)]
+    _segmented_case(P, S, off, ks)
+
+
+@pytest.mark.parametrize("case", ["ties", "edges", "one_segment", "bits"])
+def test_segmented_select_adversarial(P, case):
+    rng = np.random.default_rng(77)
+    if case == "ties":            # few distinct scores: thresholds sit in tie groups that cross block and CTA boundaries
+        n = 700_001
+        S = (rng.integers(0, 8, n) / 8.0).astype(np.float32)
+        off = [0, 1, 33, 1024, 1025, 100_000, 100_000, 350_011, n]
+        ks = [1, 7, 500, 0, 33_333, 0, 125_000, 200_000]
+    elif case == "edges":         # nothing / everything of a segment, empty segments, segments of one parameter
+        n = 50_000
+        S = np.abs(rng.standard_normal(n)).astype(np.float32)
+        off = [0, 0, 10, 11, 2048, 2048, 30_000, n]
+        ks = [0, 10, 0, 2037, 0, 1, n - 30_000]
+    elif case == "one_segment":   # reduces to the selection over the whole vector
+        n = 300_007
+        S = np.abs(rng.standard_normal(n)).astype(np.float32)
+        off, ks = [0, n], [n // 7]
+    else:                          # arbitrary bit patterns
+        n = 200_003
+        S = rng.integers(0, 2 ** 32, n, dtype=np.uint64).astype(np.uint32).view(np.float32)
+        off = [0, 50_000, 50_064, n]
+        ks = [25_000, 64, 1]
+    _segmented_case(P, S, off, ks)
+    if case == "one_segment":
+        assert np.array_equal(oracle.select_core_segmented(S, off, ks), oracle.select_core(S, ks[0]))

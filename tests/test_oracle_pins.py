@@ -572,6 +572,8 @@ def test_q8_hand_example_and_special_values():
     codes, scales = oracle.quantize_q8(v, bucket=4)
     assert scales.tolist() == [0.0, 2.0, 3.0]
     assert codes.tolist() == [0, 0, 0, 0, 0, 127, -127, 127, -127]
+    codes, scales = oracle.quantize_q8(np.array([np.inf, 0.0, -np.inf, np.nan], np.float32), bucket=4)
+    assert scales.tolist() == [0.0] and codes.tolist() == [127, 0, -127, 0]      # no finite magnitude at all
 
 
 def test_q8_codes_are_one_rounding_of_the_scaled_value_and_the_error_is_half_a_step():
