@@ -50,20 +50,24 @@ def model_bytes(N: int, K: int, k_core: int, k_exp: int) -> dict:
     }
     b["round"] = sum(b.values())
     b["round_without_score"] = b["round"] - b["score"]
+    # what the one-call round must move: the scores are neither written (4N) nor read back by the selection (4N)
+    b["round_fused"] = b["round"] - 8 * N
     return b
 
 
-def fused_pass_kernel_name(K: int) -> str:
+def fused_pass_kernel_name(K: int, staging: bool):
     """Which kernel slimdp_round's pass over all parameters is for K workers (the library's own rule:
-    a ring of 2..8 stages of 8 x (K + 1) x 512 bytes within 112 KB, or two stages within 176 KB)."""
+    a ring of 2..8 stages of 8 x (K + 1) x 512 bytes within 112 KB, or two stages within 160 KB;
+    K = 4 and K = 8 have instantiations of their own).  None: the round does not fuse for this K."""
     stage = 8 * (K + 1) * 512
     stages = (112 * 1024) // stage
-    if stages < 2 and 2 * stage <= 176 * 1024:
+    if stages < 2 and 2 * stage <= 160 * 1024:
         stages = 2
     stages = min(stages, 8)
-    if stages >= 2 and stages * stage >= 64 * 1024:
-        return f"score_bracket_async_kernel<{stages}, 8>"
-    return f"score_bracket_kernel<{K if K in (4, 8) else 0}>"
+    if stages < 2 or stages * stage < 64 * 1024:
+        return None
+    kt = K if (K, stages) in ((8, 3), (4, 5)) else 0
+    return f"score_bracket_async_kernel<{stages}, {kt}, {'true' if staging else 'false'}>"
 
 
 def measured_peak():
@@ -160,7 +164,7 @@ def aggregate_value(params_per_rank: int, world: int, ms_per_step: float) -> flo
 def time_oracle(cfg, n_sample: int, steps: int, warmup: int):
     import oracle
     from workloads import all_inputs, scaled_config
-    sample = scaled_config(cfg, n_sample)
+    sample = scaled_config(cfg, n_sample) if n_sample < cfg.N else cfg
     w, gs = all_inputs(sample)
     times = []
     for s in range(warmup + steps):
@@ -171,6 +175,60 @@ def time_oracle(cfg, n_sample: int, steps: int, warmup: int):
         if s >= warmup:
             times.append(dt)
     return sample, times
+
+
+def oracle_round_threaded(w, gs, c, k_core, k_exp, seed, rnd, eta, threads: int):
+    """The oracle's round with its loops spread over host threads, the "multi-thread scanning" of
+    Section 3.5: scoring over index chunks, explorers / extraction / pull over workers.  The sort of
+    the selection and the worker-ordered merge stay serial.  Same results as oracle.run_round."""
+    import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
+    import oracle
+    n, K = w.size, len(gs)
+    cuts = [n * i // threads for i in range(threads + 1)]
+    S = np.empty(n, np.float32)
+
+    def score_chunk(i):
+        a, b = cuts[i], cuts[i + 1]
+        if b > a:
+            S[a:b] = oracle.score(w[a:b], [g[a:b] for g in gs], c)
+
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        list(pool.map(score_chunk, range(threads)))
+        core = oracle.select_core(S, k_core)
+        exp = list(pool.map(lambda k: oracle.sample_explore(core, n, k_exp, seed, k, rnd), range(K)))
+        val = list(pool.map(lambda k: oracle.pack(gs[k], core, exp[k]), range(K)))
+        merged = oracle.merge(w, core, exp, val, eta)
+        pulled = list(pool.map(lambda k: oracle.pull(merged, core, exp[k]), range(K)))
+    return {"scores": S, "core_idx": core, "exp_idx": exp, "val": val, "w": merged, "pulled": pulled}
+
+
+def time_oracle_threaded(cfg, n_sample: int, threads: int):
+    from workloads import all_inputs, scaled_config
+    sample = scaled_config(cfg, n_sample) if n_sample < cfg.N else cfg
+    w, gs = all_inputs(sample)
+    t0 = time.perf_counter()
+    oracle_round_threaded(w, gs, sample.c, sample.k_core, sample.k_exp, sample.seed, 0, sample.eta, threads)
+    return sample, time.perf_counter() - t0
+
+
+def dominant_traffic(kernel: str, n: int):
+    """DRAM bytes of one launch of `kernel` over n parameters, from the tracked summary of its ncu
+    capture (bytes per parameter on a small case; traffic grows in proportion to n).  None when the
+    summary is for another kernel: counters of a kernel that has changed since are not reported."""
+    path = os.path.join(ROOT, "profiles", "dominant_kernel_traffic.txt")
+    try:
+        with open(path) as f:
+            for line in f:
+                if line.startswith("#") or not line.strip():
+                    continue
+                name, per_param, date = [x.strip() for x in line.split("|")][:3]
+                if name == kernel:
+                    return {"bytes": int(float(per_param) * n), "bytes_per_parameter": float(per_param),
+                            "captured": date, "source": "profiles/dominant_kernel_traffic.txt"}
+    except Exception:
+        pass
+    return None
 
 
 def run_reference(args):
@@ -204,6 +262,101 @@ def run_reference(args):
 
 # ------------------------------------------------------------------ ours ---
 
+def timed_rounds(P, torch, cfg, w, grads, buf, steps: int, warmup: int, t0: int, flush=None, mark=True):
+    """`steps` one-call rounds after `warmup` untimed ones, device-timed.  Returns the time of the whole
+    timed region, every step's own time (between events recorded on the caller's stream after each
+    round), the pass's times (events the library records around its dominant kernel) and the next round
+    index.  flush: a buffer larger than L2 that is overwritten before every timed round; its time is
+    not counted (each round is then bracketed by its own pair of events)."""
+    def one_round(t):
+        P.slimdp_round(w, grads, cfg.c, cfg.seed, t, cfg.eta, buf.scores, buf.core_idx, buf.core_aux, buf.exp_idx,
+                       buf.val, buf.pulled, buf.select_ws, buf.explore_ws, buf.stage)
+    t = t0
+    for _ in range(warmup):
+        one_round(t)
+        t += 1
+    torch.cuda.synchronize()
+    P.read_status(buf.select_ws)
+    P.read_status(buf.explore_ws)
+    new_ev = lambda: torch.cuda.Event(enable_timing=True)
+    marks = [(new_ev(), new_ev()) for _ in range(steps)]
+    for a, b in marks:      # torch creates the CUDA event at the first record
+        a.record()
+        b.record()
+    begins = [new_ev() for _ in range(steps)]
+    ends = [new_ev() for _ in range(steps)]
+    ev_start, ev_end = new_ev(), new_ev()
+    torch.cuda.synchronize()
+    ev_start.record()
+    for s in range(steps):
+        if flush is not None:
+            flush.zero_()
+        begins[s].record()
+        if mark:
+            P.mark_dominant_kernel(marks[s][0], marks[s][1])
+        one_round(t)
+        ends[s].record()
+        t += 1
+    ev_end.record()
+    torch.cuda.synchronize()
+    P.read_status(buf.select_ws)
+    P.read_status(buf.explore_ws)
+    per_step = [begins[s].elapsed_time(ends[s]) for s in range(steps)]
+    pass_ms = [a.elapsed_time(b) for a, b in marks] if mark else []
+    return ev_start.elapsed_time(ev_end), per_step, pass_ms, t
+
+
+def parity_with_oracle(P, torch, cfg, w_host, g_host, staging: bool) -> bool:
+    """One one-call round on a fresh copy of the inputs against the CPU oracle, bit for bit."""
+    import numpy as np
+    import oracle
+    ref = oracle.run_round(w_host, g_host, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 0, cfg.eta)
+    d_w = torch.from_numpy(w_host).cuda()
+    d_g = [torch.from_numpy(g).cuda() for g in g_host]
+    buf = P.RoundBuffers(cfg.N, cfg.K, cfg.k_core, cfg.k_exp, staging=staging)
+    P.slimdp_round(d_w, d_g, cfg.c, cfg.seed, 0, cfg.eta, buf.scores, buf.core_idx, buf.core_aux, buf.exp_idx, buf.val,
+                   buf.pulled, buf.select_ws, buf.explore_ws, buf.stage)
+    P.read_status(buf.select_ws)
+    P.read_status(buf.explore_ws)
+    same = lambda t, a: np.array_equal(t.cpu().numpy().view(np.uint32), np.ascontiguousarray(a).view(np.uint32))
+    ok = same(buf.core_idx, ref["core_idx"]) and same(d_w, ref["w"])
+    for k in range(cfg.K):
+        ok = ok and same(buf.exp_idx[k], ref["exp_idx"][k]) and same(buf.val[k], ref["val"][k]) \
+            and same(buf.pulled[k], ref["pulled"][k])
+    return bool(ok)
+
+
+def config_report(P, torch, name: str, args, device, peak: float):
+    """Short report for one of the other configs: warm and L2-flushed round times, both roofline
+    fractions, and parity with the oracle re-checked on the spot."""
+    from workloads import CONFIGS, all_inputs
+    cfg = CONFIGS[name]
+    N, K = cfg.N, cfg.K
+    w_host, g_host = all_inputs(cfg)
+    parity = parity_with_oracle(P, torch, cfg, w_host, g_host, args.staging) if N <= (1 << 26) else None
+    w = torch.from_numpy(w_host).to(device)
+    grads = [torch.from_numpy(g).to(device) for g in g_host]
+    buf = P.RoundBuffers(N, K, cfg.k_core, cfg.k_exp, device, staging=args.staging)
+    steps = max(20, min(args.steps, 50))
+    _, warm, pass_ms, t = timed_rounds(P, torch, cfg, w, grads, buf, steps, 5, 0)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)
+    _, cold, _, t = timed_rounds(P, torch, cfg, w, grads, buf, steps, 3, t, flush=flush, mark=False)
+    bm = model_bytes(N, K, cfg.k_core, cfg.k_exp)
+    med = statistics.median(warm)
+    out = {"N": N, "K": K, "k_core": cfg.k_core, "k_exp": cfg.k_exp,
+           "us_per_round_median": round(med * 1e3, 1), "us_per_round_min": round(min(warm) * 1e3, 1),
+           "us_per_round_l2_flushed_median": round(statistics.median(cold) * 1e3, 1),
+           "us_per_round_l2_flushed_min": round(min(cold) * 1e3, 1),
+           "gparams_per_s": N / (med * 1e-3) / 1e9,
+           "frac_of_8TBs": bm["round"] / (med * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+           "frac_of_measured": bm["round"] / (med * 1e-3) / 1e9 / peak,
+           "pass_us_median": round(statistics.median(pass_ms) * 1e3, 1) if pass_ms else None,
+           "inputs_fit_l2": 4 * N * (K + 1) <= 126e6, "parity_with_oracle": parity}
+    del buf, w, grads, flush
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -234,49 +387,24 @@ def run_ours(args):
         if world > 1:
             torch.distributed.barrier()
 
-    def one_round(t):
-        # the whole round as ONE C-ABI call on device buffers (scoring folded into the selection's pass
-        # over all parameters, explorer ranks beside it, then explorer indices and the exchange)
-        P.slimdp_round(w, grads, cfg.c, cfg.seed, t, cfg.eta, buf.scores, buf.core_idx, buf.core_aux, buf.exp_idx,
-                       buf.val, buf.pulled, buf.select_ws, buf.explore_ws, buf.stage)
-
-    # warm-up: successive rounds t = 0, 1, ... on the evolving model, as in training
-    t = 0
-    for _ in range(args.warmup):
-        one_round(t)
-        t += 1
-    torch.cuda.synchronize()
-    P.read_status(buf.select_ws)
-    P.read_status(buf.explore_ws)
-
-    # ---- timed region: exactly `steps` rounds, device-timed -----------------
-    # ev[s]: recorded by the library around the round's pass over all parameters (its dominant kernel)
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for a, b in ev:     # torch creates the CUDA event at the first record
-        a.record()
-        b.record()
-    ev_start, ev_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # ---- timed region: exactly `steps` rounds (successive rounds t = 0, 1, ... on the evolving model, as
+    # in training), each the ONE C-ABI call slimdp_round; device-timed
     sampler = ClockSampler(torch.cuda.current_device())
     launches0 = P.launch_count()
     barrier()
-    torch.cuda.synchronize()
     sampler.start()
-    ev_start.record()
-    for s in range(args.steps):
-        P.mark_dominant_kernel(ev[s][0], ev[s][1])
-        one_round(t)
-        t += 1
-    ev_end.record()
-    torch.cuda.synchronize()
+    total_ms, per_step, pass_ms, t = timed_rounds(P, torch, cfg, w, grads, buf, args.steps, args.warmup, 0)
     clocks = sampler.stop()
     barrier()
     launches = P.launch_count() - launches0
-    P.read_status(buf.select_ws)
-    P.read_status(buf.explore_ws)
-    total_ms = max_over_ranks(ev_start.elapsed_time(ev_end), world, device)
+    total_ms = max_over_ranks(total_ms, world, device)
     ms_per_step = total_ms / args.steps
-    dominant_ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
+    dominant_ms = sum(pass_ms) / args.steps
     value = aggregate_value(N, world, ms_per_step)
+
+    def one_round(tt):
+        P.slimdp_round(w, grads, cfg.c, cfg.seed, tt, cfg.eta, buf.scores, buf.core_idx, buf.core_aux, buf.exp_idx,
+                       buf.val, buf.pulled, buf.select_ws, buf.explore_ws, buf.stage)
 
     # ---- optional: kernel timeline of three more rounds (CUPTI through torch.profiler) ----
     # Start, duration and stream of every kernel, relative to the first: shows which kernels of the
@@ -301,64 +429,83 @@ def run_ours(args):
                 f.write(f'{e["ts"] - events[0]["ts"]:10.1f} {e["dur"]:8.1f} s{e["args"].get("stream")} {name}\n')
 
     # ---- per-call breakdown (untimed for the headline; 5 more rounds) -------
-    # "exchange" is the fused pack + merge + pull the timed rounds use; the three separate calls
-    # are timed after it for comparison (they repeat the exchange's work on the next model state)
-    # after them the two steps either side of the path: the worker-side merge and the dense push
-    # (+ scoring) of a reselection boundary
+    # the steps as separate C-ABI calls on one stream ("exchange" is the fused pack + merge + pull; the
+    # three separate calls follow for comparison), then the steps either side of the path
     names = ["score", "select", "explore", "exchange", "pack_alone", "merge_alone", "pull_alone", "worker_merge",
              "dense_merge_score"]
     acc = {nm: [] for nm in names}
-    local = [w.clone() for _ in range(K)]
-    for _ in range(5):
-        marks = [torch.cuda.Event(enable_timing=True) for _ in range(10)]
-        marks[0].record()
-        P.slimdp_score(w, grads, cfg.c, buf.scores); marks[1].record()
-        P.slimdp_select_core(buf.scores, k_core, buf.core_idx, buf.core_aux, buf.select_ws); marks[2].record()
-        P.slimdp_sample_explore_batched(buf.core_aux, N, k_core, k_exp, cfg.seed, 0, t, buf.exp_idx, buf.explore_ws)
-        marks[3].record()
-        P.slimdp_exchange(w, grads, buf.core_idx, buf.exp_idx, cfg.eta, buf.val, buf.pulled); marks[4].record()
-        P.slimdp_pack_batched(grads, buf.core_idx, buf.exp_idx, buf.val); marks[5].record()
-        P.slimdp_merge(w, buf.core_idx, buf.exp_idx, buf.val, cfg.eta); marks[6].record()
-        P.slimdp_pull_batched(w, buf.core_idx, buf.exp_idx, buf.pulled); marks[7].record()
-        P.slimdp_worker_merge_batched(local, buf.core_idx, buf.exp_idx, buf.pulled); marks[8].record()
-        P.slimdp_dense_merge_score(w, grads, cfg.eta, cfg.c, buf.scores); marks[9].record()
-        torch.cuda.synchronize()
-        t += 1
-        for i, nm in enumerate(names):
-            acc[nm].append(marks[i].elapsed_time(marks[i + 1]) * 1e3)
-    # the steps as separate C-ABI calls, one after the other on one stream; the timed rounds above run
-    # them as the single slimdp_round call, whose time and dominant kernel come first
     breakdown_us = {"round_one_call": round(ms_per_step * 1e3, 1), "dominant_kernel": round(dominant_ms * 1e3, 1)}
-    breakdown_us.update({nm: round(statistics.median(v), 1) for nm, v in acc.items()})
-    del local
+    if not args.no_breakdown:
+        local = [w.clone() for _ in range(K)]
+        for _ in range(5):
+            marks = [torch.cuda.Event(enable_timing=True) for _ in range(10)]
+            marks[0].record()
+            P.slimdp_score(w, grads, cfg.c, buf.scores); marks[1].record()
+            P.slimdp_select_core(buf.scores, k_core, buf.core_idx, buf.core_aux, buf.select_ws); marks[2].record()
+            P.slimdp_sample_explore_batched(buf.core_aux, N, k_core, k_exp, cfg.seed, 0, t, buf.exp_idx, buf.explore_ws)
+            marks[3].record()
+            P.slimdp_exchange(w, grads, buf.core_idx, buf.exp_idx, cfg.eta, buf.val, buf.pulled); marks[4].record()
+            P.slimdp_pack_batched(grads, buf.core_idx, buf.exp_idx, buf.val); marks[5].record()
+            P.slimdp_merge(w, buf.core_idx, buf.exp_idx, buf.val, cfg.eta); marks[6].record()
+            P.slimdp_pull_batched(w, buf.core_idx, buf.exp_idx, buf.pulled); marks[7].record()
+            P.slimdp_worker_merge_batched(local, buf.core_idx, buf.exp_idx, buf.pulled); marks[8].record()
+            P.slimdp_dense_merge_score(w, grads, cfg.eta, cfg.c, buf.scores); marks[9].record()
+            torch.cuda.synchronize()
+            t += 1
+            for i, nm in enumerate(names):
+                acc[nm].append(marks[i].elapsed_time(marks[i + 1]) * 1e3)
+        breakdown_us.update({nm: round(statistics.median(v), 1) for nm, v in acc.items()})
+        del local
 
     peak, peak_src = measured_peak()
-    fused = N >= (1 << 21) and k_core > 0      # sizes from which slimdp_round scores inside the selection's pass
+    fused_kernel = fused_pass_kernel_name(K, buf.stage is not None)
+    fused = N >= (1 << 21) and k_core > 0 and fused_kernel is not None   # the round scores inside the selection's pass
     if fused:
         # per parameter: K + 1 fp32 values read, one bit in each of the two bitmaps written (the
         # candidates, about 1 % of the parameters at 8 B each, are not counted)
-        dominant = {"kernel": fused_pass_kernel_name(K),
-                    "bytes": 4 * N * (K + 1) + 2 * (N // 8), "traffic": TRAFFIC_DOMINANT_BYTES.get(cfg.name)}
+        dominant = {"kernel": fused_kernel, "bytes": 4 * N * (K + 1) + 2 * (N // 8)}
     else:
-        dominant = {"kernel": f"score_vec4_kernel<{K}>", "bytes": bytes_model["score"], "traffic": None}
+        dominant = {"kernel": f"score_vec4_kernel<{K}>", "bytes": bytes_model["score"]}
+    traffic = dominant_traffic(dominant["kernel"], N)
     achieved = dominant["bytes"] / (dominant_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dominant["kernel"], "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "traffic": dominant["traffic"],
-                "algorithmic_bytes_per_launch": dominant["bytes"], "avg_launch_ms": dominant_ms,
-                "peak_source": peak_src}
+                "unit": "GB/s", "frac": achieved / peak, "traffic": traffic["bytes"] if traffic else None,
+                "traffic_source": traffic, "algorithmic_bytes_per_launch": dominant["bytes"],
+                "avg_launch_ms": dominant_ms, "peak_source": peak_src}
     round_gbs = bytes_model["round"] / (ms_per_step * 1e-3) / 1e9
-    # the model's "round without score" against the round's time less the score step's share of the fused
-    # pass (that pass's time scaled by the score step's part of its bytes)
+    fused_gbs = bytes_model["round_fused"] / (ms_per_step * 1e-3) / 1e9
+    # "round without score": the model's bytes of select + explore + pack + merge + pull against the
+    # round's time less the score step's share of the fused pass (that pass's time scaled by the score
+    # step's part of its bytes: an attribution), and, beside it, against the round's time less the
+    # separately timed slimdp_score call (a measurement; that call also writes the scores)
     score_ms = dominant_ms * (4 * N * (K + 1) / dominant["bytes"]) if fused else dominant_ms
     rest_ms = ms_per_step - score_ms
     rest_gbs = bytes_model["round_without_score"] / (rest_ms * 1e-3) / 1e9
+    without = {"model_bytes": bytes_model["round_without_score"], "ms": rest_ms, "achieved_gbs": rest_gbs,
+               "frac_of_8TBs": rest_gbs / NOMINAL_HBM_GBS, "frac_of_measured": rest_gbs / peak,
+               "how": "round time less the score step's byte share of the fused pass"}
+    if "score" in breakdown_us and ms_per_step * 1e3 > breakdown_us["score"]:
+        alt_ms = ms_per_step - breakdown_us["score"] * 1e-3
+        alt_gbs = bytes_model["round_without_score"] / (alt_ms * 1e-3) / 1e9
+        without["less_separate_score_call"] = {"ms": alt_ms, "frac_of_8TBs": alt_gbs / NOMINAL_HBM_GBS,
+                                               "frac_of_measured": alt_gbs / peak}
+    if not args.no_breakdown:
+        sep_ms = (breakdown_us["select"] + breakdown_us["explore"] + breakdown_us["exchange"]) * 1e-3
+        sep_gbs = bytes_model["round_without_score"] / (sep_ms * 1e-3) / 1e9
+        without["as_separate_calls"] = {"ms": sep_ms, "frac_of_8TBs": sep_gbs / NOMINAL_HBM_GBS,
+                                        "frac_of_measured": sep_gbs / peak}
     round_roofline = {
         "model_bytes": bytes_model["round"], "achieved_gbs": round_gbs,
         "frac_of_8TBs": round_gbs / NOMINAL_HBM_GBS, "frac_of_measured": round_gbs / peak,
-        "without_score": {"model_bytes": bytes_model["round_without_score"], "ms": rest_ms, "achieved_gbs": rest_gbs,
-                          "frac_of_8TBs": rest_gbs / NOMINAL_HBM_GBS, "frac_of_measured": rest_gbs / peak},
+        "label": "unfused model bytes (scores written and read back) over the one-call round's time",
+        "moved_bytes": {"model_bytes": bytes_model["round_fused"], "achieved_gbs": fused_gbs,
+                        "frac_of_8TBs": fused_gbs / NOMINAL_HBM_GBS, "frac_of_measured": fused_gbs / peak,
+                        "label": "bytes the one-call round must move (no score write, no re-read)"},
+        "without_score": without,
     }
-
+    step_stats = {"median_ms": statistics.median(per_step), "min_ms": min(per_step), "max_ms": max(per_step),
+                  "note": "per step, between events recorded around each round; ms_per_step is the whole timed "
+                          "region over the step count"}
     # ---- end to end: host buffers through the C ABI, copies inside the timed region
     e2e = None
     if (rank == 0 or world > 1) and not args.no_e2e:
@@ -388,14 +535,31 @@ def run_ours(args):
         e2e = {"value": aggregate_value(N, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms, "steps": e2e_steps,
                "h2d_bytes_per_step": 4 * N * (K + 1),
                "d2h_bytes_per_step": 4 * N + 4 * k_core + K * (4 * k_exp + 4 * m)}
+        del arena, w_pin, g_pin
+        torch.cuda.empty_cache()
 
-    cpu_baseline = None
+    # ---- the other configs (rank 0, one GPU): warm and L2-flushed times, parity re-checked
+    per_config = None
+    if rank == 0 and world == 1 and args.per_config != "none" and not args.scale:
+        del w, grads
+        torch.cuda.empty_cache()
+        names_pc = ["tiny", "googlenet", "resnet50_ties", "vgg16"] + (["large"] if args.per_config == "all" else [])
+        per_config = {nm: config_report(P, torch, nm, args, device, peak) for nm in names_pc if nm != args.config}
+
+    cpu_baseline = cpu_baseline_mt = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        sample, times = time_oracle(cfg, CPU_BASELINE_SAMPLE, 1, 0)
+        n_cpu = cfg.N if args.cpu_baseline_full else min(cfg.N, CPU_BASELINE_SAMPLE)
+        sample, times = time_oracle(cfg, n_cpu, 1, 0)
+        what = (f"one oracle round on {'all' if sample.N == cfg.N else 'the leading'} {sample.N} parameters of the "
+                f"{cfg.name}-shaped workload (K={sample.K}, k_core={sample.k_core}, k_exp={sample.k_exp})")
         cpu_baseline = {"value": sample.N / times[0] / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-                        "seconds": times[0],
-                        "sample": f"one oracle round on the leading {sample.N} parameters of the {cfg.name}-shaped "
-                                  f"workload (K={sample.K}, k_core={sample.k_core}, k_exp={sample.k_exp})"}
+                        "seconds": times[0], "sample": what}
+        threads = os.cpu_count() or 1
+        sample, secs = time_oracle_threaded(cfg, n_cpu, threads)
+        cpu_baseline_mt = {"value": sample.N / secs / 1e9, "unit": UNIT, "cores": threads,
+                           "kind": "oracle, its loops spread over host threads (scoring over index chunks; "
+                                   "explorers, extraction and pull over workers; sort and merge serial)",
+                           "seconds": secs, "sample": what}
 
     if rank == 0:
         line = {
@@ -405,21 +569,17 @@ def run_ours(args):
             "config": {"workload": f"{cfg.name}-shaped: N={N} fp32 parameters, K={K} workers, k_core={k_core} "
                                    f"({cfg.core_pct}%), k_exp={k_exp} ({cfg.explore_pct}% of the non-core)",
                        "N": N, "K": K, "k_core": k_core, "k_exp": k_exp, "seed": cfg.seed,
+                       "staging_area": bool(args.staging),
                        "l2": "inputs larger than L2 (no flush needed)" if 4 * N * (K + 1) > 4 * 126e6
                        else "inputs fit L2 (warm)",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+            "clocks": clocks, "step_ms": step_stats, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
             "round_roofline": round_roofline, "breakdown_us": breakdown_us, "cpu_baseline": cpu_baseline,
+            "cpu_baseline_threaded": cpu_baseline_mt, "per_config": per_config,
         }
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()
-
-
-# DRAM bytes (read + write) of one launch of the fused pass, per workload: from an ncu capture of the
-# same kernel on the leading 40 M parameters of the workload (1447.6 MB = 36.19 B per parameter;
-# traffic grows in proportion to n), scaled to the full launch of 138 357 544 parameters.
-TRAFFIC_DOMINANT_BYTES: dict = {"vgg16": 5_007_158_000}
 
 
 def main():
@@ -431,6 +591,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-breakdown", action="store_true", help="skip the steps timed as separate calls")
+    ap.add_argument("--per-config", default="default", choices=["default", "all", "none"],
+                    help="short reports for the other configs: default = tiny, googlenet, resnet50_ties; "
+                         "all = also the 10^9-parameter vector; none")
+    ap.add_argument("--cpu-baseline-full", action="store_true",
+                    help="time the CPU oracle on the whole workload instead of its leading 2^25 parameters")
     ap.add_argument("--staging", action="store_true",
                     help="give slimdp_round its optional staging area (the exchange then streams the core's values)")
     ap.add_argument("--timeline", default="",

@@ -26,10 +26,12 @@
  *     other work on that stream.
  *   - Arguments are validated on the host before anything is enqueued.  A
  *     negative return value means nothing (more) was enqueued by that call.
- *   - Indices are 0-based uint32_t, so 1 <= n < 2^32.  fp32 buffers must be
- *     4-byte aligned; 16-byte alignment of all of them selects the vectorised
- *     kernels (any alignment is still computed correctly).  Index buffers and
- *     core_aux / workspaces must be 16-byte aligned.
+ *   - Indices are 0-based uint32_t, so 1 <= n < 2^32.  fp32 and index buffers
+ *     must be 4-byte aligned.  16-byte alignment of all fp32 tensors of a call
+ *     selects the vectorised kernels; slimdp_score also takes them when all
+ *     tensors are off a 16-byte boundary by the same amount (slices of one
+ *     allocation), after one to three leading parameters.  Any alignment is
+ *     computed correctly.  core_aux and workspaces must be 16-byte aligned.
  *   - Input and output buffers of one call must not overlap, except where a
  *     buffer is documented as updated in place.
  *   - Results are deterministic: the same inputs give the same bytes on every
@@ -86,8 +88,8 @@ size_t slimdp_select_workspace_bytes(uint64_t n);
  * draw k_exp parameters per worker (any k_core). */
 size_t slimdp_explore_workspace_bytes(uint64_t n, uint64_t k_exp, uint32_t num_workers);
 
-/* max(select, explore for K workers): one workspace that serves every call of a round. */
-size_t slimdp_workspace_bytes(uint64_t n, uint64_t k_exp, uint32_t K);
+/* max(select, explore for K workers): one workspace that serves every separate call of a round. */
+size_t slimdp_workspace_bytes(uint64_t n, uint32_t K, uint64_t k_core, uint64_t k_exp);
 
 /* ---------------------------------------------------------------- score ---
  * Eq. 1 (Section 3.2).  For every i < n, in fp32:
@@ -188,7 +190,8 @@ slimdp_status slimdp_sample_explore_batched(const void* core_aux, uint64_t n, ui
  *            call's device-side consistency status (SLIMDP_OK or SLIMDP_ERR_INTERNAL).
  * The first call on each device looks up the scratch array's device address
  * (cudaGetSymbolAddress, with that device current); make that first call
- * outside any stream capture.  All calls on a device share the one array and
+ * outside any stream capture.  The address is kept for the life of the device's
+ * primary context.  All calls on a device share the one array and
  * each call overwrites what the last one left (it clears what it needs at zero
  * itself), so two calls that may run at the same time on the GPU, e.g. on
  * different streams, race; order them. */

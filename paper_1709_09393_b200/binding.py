@@ -34,7 +34,7 @@ EXPORTS = {
     "slimdp_core_aux_dir_offset": (_sz, [_u64]),
     "slimdp_select_workspace_bytes": (_sz, [_u64]),
     "slimdp_explore_workspace_bytes": (_sz, [_u64, _u64, _u32]),
-    "slimdp_workspace_bytes": (_sz, [_u64, _u64, _u32]),
+    "slimdp_workspace_bytes": (_sz, [_u64, _u32, _u64, _u64]),
     "slimdp_score": (ctypes.c_int32, [_vp, _pp, _u32, _f32, _u64, _vp, _vp]),
     "slimdp_select_core": (ctypes.c_int32, [_vp, _u64, _u64, _vp, _vp, _vp, _sz, _vp]),
     "slimdp_sample_explore": (ctypes.c_int32, [_vp, _u64, _u64, _u64, _u64, _u32, _u32, _vp, _vp, _sz, _vp]),
@@ -137,8 +137,8 @@ def explore_workspace_bytes(n: int, k_exp: int, num_workers: int) -> int:
     return lib.slimdp_explore_workspace_bytes(n, k_exp, num_workers)
 
 
-def workspace_bytes(n: int, k_exp: int, K: int) -> int:
-    return lib.slimdp_workspace_bytes(n, k_exp, K)
+def workspace_bytes(n: int, K: int, k_core: int, k_exp: int) -> int:
+    return lib.slimdp_workspace_bytes(n, K, k_core, k_exp)
 
 
 def round_arena_bytes(n: int, K: int, k_core: int, k_exp: int) -> int:

@@ -158,7 +158,8 @@ size_t slimdp_explore_workspace_bytes(uint64_t n, uint64_t k_exp, uint32_t num_w
     return explore_ws_layout(nullptr, n, k_exp, num_workers).bytes;
 }
 
-size_t slimdp_workspace_bytes(uint64_t n, uint64_t k_exp, uint32_t K) {
+size_t slimdp_workspace_bytes(uint64_t n, uint32_t K, uint64_t k_core, uint64_t k_exp) {
+    if (!sets_ok(n, k_core, k_exp)) return 0;
     const size_t a = slimdp_select_workspace_bytes(n), b = slimdp_explore_workspace_bytes(n, k_exp, K);
     if (a == 0 || b == 0) return 0;
     return a > b ? a : b;
@@ -172,6 +173,21 @@ slimdp_status slimdp_score(const float* w, const float* const* grads, uint32_t K
     if (!fill<const float>(g, grads, K, true, 4)) return SLIMDP_ERR_INVALID_ARG;
     bool vec = aligned16(w) && aligned16(scores);
     for (uint32_t k = 0; k < K; ++k) vec = vec && aligned16(g.p[k]);
+    if (!vec) {
+        // all tensors off a 16-byte boundary by the same amount (slices of one allocation): the first
+        // one to three parameters go through the scalar kernel, the rest is aligned
+        const uintptr_t mis = reinterpret_cast<uintptr_t>(w) & 15u;
+        bool same = (reinterpret_cast<uintptr_t>(scores) & 15u) == mis;
+        for (uint32_t k = 0; k < K; ++k) same = same && (reinterpret_cast<uintptr_t>(g.p[k]) & 15u) == mis;
+        const uint64_t head = (16u - mis) / 4u;
+        if (same && n > head) {
+            slimdp_status rc = launch_score(w, g, K, c, head, scores, false, (cudaStream_t)stream);
+            if (rc != SLIMDP_OK) return rc;
+            PtrArray<const float> g2 = g;
+            for (uint32_t k = 0; k < K; ++k) g2.p[k] = g.p[k] + head;
+            return launch_score(w + head, g2, K, c, n - head, scores + head, true, (cudaStream_t)stream);
+        }
+    }
     return launch_score(w, g, K, c, n, scores, vec, (cudaStream_t)stream);
 }
 
@@ -179,7 +195,7 @@ slimdp_status slimdp_select_core(const float* scores, uint64_t n, uint64_t k_cor
                                  void* core_aux, void* ws, size_t ws_bytes, void* stream) {
     if (!n_ok(n) || k_core > n || !scores || !core_aux || !ws) return SLIMDP_ERR_INVALID_ARG;
     if (k_core > 0 && !core_idx) return SLIMDP_ERR_INVALID_ARG;
-    if (!aligned4(scores) || !aligned16(core_aux) || !aligned16(ws) || (core_idx && !aligned16(core_idx)))
+    if (!aligned4(scores) || !aligned16(core_aux) || !aligned16(ws) || (core_idx && !aligned4(core_idx)))
         return SLIMDP_ERR_INVALID_ARG;
     if (ws_bytes < slimdp_select_workspace_bytes(n)) return SLIMDP_ERR_WORKSPACE;
     return launch_select(scores, n, k_core, core_idx, core_aux, ws, (cudaStream_t)stream);
@@ -193,7 +209,7 @@ slimdp_status slimdp_sample_explore_batched(const void* core_aux, uint64_t n, ui
     if ((uint64_t)first_worker + num_workers > 0x100000000ull) return SLIMDP_ERR_INVALID_ARG;
     if (!aligned16(core_aux) || !aligned16(ws)) return SLIMDP_ERR_INVALID_ARG;
     PtrArray<uint32_t> out;
-    if (!fill<uint32_t>(out, exp_idx, num_workers, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<uint32_t>(out, exp_idx, num_workers, k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (ws_bytes < slimdp_explore_workspace_bytes(n, k_exp, num_workers)) return SLIMDP_ERR_WORKSPACE;
     return launch_explore(core_aux, n, k_core, k_exp, seed, first_worker, num_workers, round, out, ws,
                           (cudaStream_t)stream);
@@ -211,7 +227,7 @@ slimdp_status slimdp_sample_explore_static(const void* core_aux, uint64_t n, uin
                                            uint64_t seed, uint32_t worker, uint32_t round, uint32_t* exp_idx,
                                            int32_t* status, void* stream) {
     if (!sets_ok(n, k_core, k_exp) || !core_aux || !aligned16(core_aux)) return SLIMDP_ERR_INVALID_ARG;
-    if (k_exp > 0 && (!exp_idx || !aligned16(exp_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_exp > 0 && (!exp_idx || !aligned4(exp_idx))) return SLIMDP_ERR_INVALID_ARG;
     if (status && !aligned4(status)) return SLIMDP_ERR_INVALID_ARG;
     if (n > SLIMDP_STATIC_MAX_N || k_exp > SLIMDP_STATIC_MAX_K_EXP) return SLIMDP_ERR_UNSUPPORTED;
     return launch_explore_static(core_aux, n, k_core, k_exp, seed, worker, round, exp_idx, status,
@@ -222,7 +238,7 @@ static slimdp_status gather_common(const float* const* srcs, bool same_src, cons
                                    uint64_t n, const uint32_t* core_idx, uint64_t k_core,
                                    const uint32_t* const* exp_idx, uint64_t k_exp, float* const* out, void* stream) {
     if (!sets_ok(n, k_core, k_exp) || !k_ok(K)) return SLIMDP_ERR_INVALID_ARG;
-    if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned4(core_idx))) return SLIMDP_ERR_INVALID_ARG;
     PtrArray<const float> src;
     PtrArray<const uint32_t> exp;
     PtrArray<float> dst;
@@ -233,7 +249,7 @@ static slimdp_status gather_common(const float* const* srcs, bool same_src, cons
     } else if (!fill<const float>(src, srcs, K, true, 4)) {
         return SLIMDP_ERR_INVALID_ARG;
     }
-    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (!fill<float>(dst, out, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (k_core + k_exp == 0) return SLIMDP_OK;
     return launch_gather(src, same_src, K, core_idx, k_core, exp, k_exp, dst, (cudaStream_t)stream);
@@ -271,10 +287,10 @@ slimdp_status slimdp_merge(float* w_global, uint64_t n, uint32_t K, const uint32
                            void* stream) {
     if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !w_global || !aligned4(w_global) || !isfinite(eta))
         return SLIMDP_ERR_INVALID_ARG;
-    if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned4(core_idx))) return SLIMDP_ERR_INVALID_ARG;
     PtrArray<const uint32_t> exp;
     PtrArray<const float> v;
-    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (!fill<const float>(v, val, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (k_core + k_exp == 0) return SLIMDP_OK;
     return launch_merge(w_global, n, K, core_idx, k_core, exp, k_exp, v, eta, (cudaStream_t)stream);
@@ -285,12 +301,12 @@ slimdp_status slimdp_exchange(float* w_global, uint64_t n, uint32_t K, const flo
                               uint64_t k_exp, float eta, float* const* val, float* const* pulled, void* stream) {
     if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !w_global || !aligned4(w_global) || !isfinite(eta))
         return SLIMDP_ERR_INVALID_ARG;
-    if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned4(core_idx))) return SLIMDP_ERR_INVALID_ARG;
     PtrArray<const float> d;
     PtrArray<const uint32_t> exp;
     PtrArray<float> v, o;
     if (!fill<const float>(d, deltas, K, true, 4)) return SLIMDP_ERR_INVALID_ARG;
-    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (!fill<float>(v, val, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (!fill<float>(o, pulled, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (k_core + k_exp == 0) return SLIMDP_OK;
@@ -313,12 +329,12 @@ slimdp_status slimdp_worker_merge_batched(float* const* w_local, uint32_t K, uin
                                           uint64_t k_core, const uint32_t* const* exp_idx, uint64_t k_exp,
                                           const float* const* pulled, void* stream) {
     if (!sets_ok(n, k_core, k_exp) || !k_ok(K) || !w_local) return SLIMDP_ERR_INVALID_ARG;
-    if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned4(core_idx))) return SLIMDP_ERR_INVALID_ARG;
     PtrArray<float> w;
     PtrArray<const uint32_t> exp;
     PtrArray<const float> v;
     if (!fill<float>(w, w_local, K, true, 4)) return SLIMDP_ERR_INVALID_ARG;
-    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<const uint32_t>(exp, exp_idx, K, k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (!fill<const float>(v, pulled, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     return launch_worker_merge(w, K, core_idx, k_core, exp, k_exp, v, (cudaStream_t)stream);
 }
@@ -351,7 +367,7 @@ slimdp_status slimdp_select_core_segmented(const float* scores, uint64_t n, cons
         if (seg_off[s + 1] < seg_off[s] || seg_k[s] > seg_off[s + 1] - seg_off[s]) return SLIMDP_ERR_INVALID_ARG;
         k_total += seg_k[s];
     }
-    if (k_total > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_total > 0 && (!core_idx || !aligned4(core_idx))) return SLIMDP_ERR_INVALID_ARG;
     if (ws_bytes < slimdp_select_segmented_workspace_bytes(n, segments)) return SLIMDP_ERR_WORKSPACE;
     return launch_select_segmented(scores, n, seg_off, seg_k, segments, k_total, core_idx, core_aux, ws,
                                    (cudaStream_t)stream);
@@ -431,7 +447,7 @@ slimdp_status slimdp_select_emit(const float* scores, uint64_t n_shard, uint32_t
     if (!n_ok(n_shard) || k_shard > n_shard || tie_quota > k_shard || !scores || !core_aux || !ws)
         return SLIMDP_ERR_INVALID_ARG;
     if (k_shard > 0 && !core_idx) return SLIMDP_ERR_INVALID_ARG;
-    if (!aligned4(scores) || !aligned16(core_aux) || !aligned16(ws) || (core_idx && !aligned16(core_idx)))
+    if (!aligned4(scores) || !aligned16(core_aux) || !aligned16(ws) || (core_idx && !aligned4(core_idx)))
         return SLIMDP_ERR_INVALID_ARG;
     if (ws_bytes < slimdp_select_workspace_bytes(n_shard)) return SLIMDP_ERR_WORKSPACE;
     return launch_select_given(scores, n_shard, threshold_bits, (uint32_t)tie_quota, k_shard, core_idx, core_aux, ws,
@@ -605,13 +621,13 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
         !aligned16(explore_ws))
         return SLIMDP_ERR_INVALID_ARG;
     if (stage && (reinterpret_cast<uintptr_t>(stage) & 255u) != 0) return SLIMDP_ERR_INVALID_ARG;
-    if (k_core > 0 && (!core_idx || !aligned16(core_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (k_core > 0 && (!core_idx || !aligned4(core_idx))) return SLIMDP_ERR_INVALID_ARG;
     PtrArray<const float> g;
     PtrArray<uint32_t> exp_out;
     PtrArray<const uint32_t> exp_in;
     PtrArray<float> v, o;
     if (!fill<const float>(g, grads, K, true, 4)) return SLIMDP_ERR_INVALID_ARG;
-    if (!fill<uint32_t>(exp_out, exp_idx, K, k_exp > 0, 16)) return SLIMDP_ERR_INVALID_ARG;
+    if (!fill<uint32_t>(exp_out, exp_idx, K, k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (!fill<float>(v, val, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     if (!fill<float>(o, pulled, K, k_core + k_exp > 0, 4)) return SLIMDP_ERR_INVALID_ARG;
     memset(&exp_in, 0, sizeof(exp_in));

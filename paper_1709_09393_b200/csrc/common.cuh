@@ -42,7 +42,9 @@ struct WsHeader {
     uint32_t abort;        // finishing kernel: a bounded wait ran out; every CTA leaves
     uint32_t next_chunk;   // fused scoring pass: the next free chunk of the staging area
     uint32_t stage_lost;   // fused scoring pass: the staging area ran out of chunks
-    uint32_t reserved[41];
+    uint32_t threshold;    // what the finishing kernel hands the emitting kernel: the threshold key T ...
+    uint32_t tie_quota;    // ... and how many keys equal to T belong to the core
+    uint32_t reserved[39];
 };
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 

@@ -21,6 +21,7 @@
 //      the group holds no core parameter) turns it into the parameter index.
 // No global bitmap, no inter-CTA waiting; the result does not depend on the
 // order in which atomics land.
+#include <atomic>
 #include <type_traits>
 
 #include "common.cuh"
@@ -503,7 +504,7 @@ __global__ void __launch_bounds__(kSelThreads, 5) select0_kernel(const uint32_t*
         hdr->status = SLIMDP_ERR_INTERNAL;   // directory and bitmap disagree, or the ranks are not sorted
         return;
     }
-    if (e0 + kSelPer <= m) {
+    if (e0 + kSelPer <= m && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {   // 16-byte stores where the list allows
 #pragma unroll
         for (uint32_t q = 0; q < kSelPer; q += 4)
             *reinterpret_cast<uint4*>(dst + e0 + q) = make_uint4(idx[q], idx[q + 1], idx[q + 2], idx[q + 3]);
@@ -641,19 +642,22 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 slimdp_status launch_explore_static(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                     uint32_t worker, uint32_t round, uint32_t* exp_idx, int32_t* status_out,
                                     cudaStream_t st) {
-    static void* scratch_addr[64];   // per device; every thread that races here stores the same value
+    // per device; every thread that gets here first stores the same value.  The address holds for the
+    // life of the device's primary context.
+    static std::atomic<void*> scratch_addr[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SLIMDP_ERR_CUDA;
-    if (scratch_addr[dev] == nullptr) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return SLIMDP_ERR_CUDA;
-        scratch_addr[dev] = p;
+    void* scratch = scratch_addr[dev].load(std::memory_order_relaxed);
+    if (scratch == nullptr) {
+        if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || scratch == nullptr)
+            return SLIMDP_ERR_CUDA;
+        scratch_addr[dev].store(scratch, std::memory_order_relaxed);
     }
     if (explore_ws_layout(nullptr, n, k_exp, 1).bytes > kStaticScratchBytes) return SLIMDP_ERR_UNSUPPORTED;
     PtrArray<uint32_t> out;
     for (auto& q : out.p) q = nullptr;
     out.p[0] = exp_idx;
-    void* ws = scratch_addr[dev];
+    void* ws = scratch;
     // launch_explore clears the counters it needs at zero and resets the status word on every call
     slimdp_status rc = launch_explore(core_aux, n, k_core, k_exp, seed, worker, 1, round, out, ws, st);
     if (rc != SLIMDP_OK) return rc;

@@ -174,7 +174,6 @@ __global__ void __launch_bounds__(kFinishThreads, 2) seg_select_kernel(SegArgs a
     __shared__ uint32_t sh[4096];
     __shared__ unsigned long long scan_smem[33];
     __shared__ uint32_t res[3];
-    __shared__ unsigned long long red[kFinishThreads / 32];
     const uint32_t t = threadIdx.x, lane = lane_id(), wid = t >> 5;
     uint32_t epoch = 0;
     // segment states (k = 0: nothing, k = length: everything, else the rounds decide)
@@ -234,9 +233,6 @@ __global__ void __launch_bounds__(kFinishThreads, 2) seg_select_kernel(SegArgs a
         const uint32_t c = __reduce_add_sync(0xFFFFFFFFu, __popc(mine));
         if (lane == 0 && c) atomicAdd(&a.tile_sum[blk / kEmitTile], (unsigned long long)c);
     }
-    if (!grid_barrier(a.hdr, &epoch)) return;
-    emit_phase(a.G, nullptr, 0u, 0u, a.tile_sum, a.n, a.nb, a.k_total, a.hdr, a.core_idx, a.bitmap, a.dir, scan_smem,
-               red);
 }
 
 }  // namespace
@@ -332,7 +328,7 @@ slimdp_status launch_select_segmented(const float* scores, uint64_t n, const uin
                                     dim3(kFinishThreads), args, 0, st) != cudaSuccess)
         return SLIMDP_ERR_CUDA;
     SLIMDP_LAUNCHED(1);
-    return SLIMDP_OK;
+    return launch_emit(L.G, nullptr, L.tile_sum, n, (uint32_t)k_total, L.hdr, core_idx, a.bitmap, a.dir, st);
 }
 
 }  // namespace slimdp

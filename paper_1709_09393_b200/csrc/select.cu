@@ -808,7 +808,6 @@ __global__ void __launch_bounds__(kFinishThreads, 2) finish_kernel(FinishArgs a)
     __shared__ uint32_t sh[kDigitBins];   // a counting round's histogram
     __shared__ unsigned long long scan_smem[33];
     __shared__ uint32_t res[3];
-    __shared__ unsigned long long red[kFinishThreads / 32];
     WsHeader* hdr = a.hdr;
     const uint32_t t = threadIdx.x, lane = lane_id(), wid = t >> 5;
     const uint32_t lt_mask = (1u << lane) - 1u;
@@ -870,7 +869,6 @@ __global__ void __launch_bounds__(kFinishThreads, 2) finish_kernel(FinishArgs a)
                                                      ((unsigned long long)__popc(peers & ~gt) << 32));
             }
         }
-        if (!grid_barrier(hdr, &epoch)) return;
     } else {
         if (a.given) {
             T = a.T_given;
@@ -945,14 +943,16 @@ __global__ void __launch_bounds__(kFinishThreads, 2) finish_kernel(FinishArgs a)
                     atomicAdd(&a.tile_sum[blk / kEmitTile], (unsigned long long)cg | ((unsigned long long)ce << 32));
             }
         }
-        if (!grid_barrier(hdr, &epoch)) return;
     }
     if (failed) {
         if (t == 0) hdr->status = SLIMDP_ERR_INTERNAL;
         return;
     }
 
-    emit_phase(a.G, a.E, T, ties, a.tile_sum, a.n, a.nb, k, hdr, a.core_idx, a.bitmap, a.dir, scan_smem, red);
+    if (blockIdx.x == 0 && t == 0) {   // for the emitting kernel, and for whoever reads the header afterwards
+        hdr->threshold = T;
+        hdr->tie_quota = ties;
+    }
 }
 
 }  // namespace
@@ -1142,7 +1142,7 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
                                     dim3(kFinishThreads), args, 0, st) != cudaSuccess)
         return SLIMDP_ERR_CUDA;
     SLIMDP_LAUNCHED(1);
-    return SLIMDP_OK;
+    return launch_emit(L.G, L.E, L.tile_sum, n, k, L.hdr, core_idx, bitmap, dir, st);
 }
 
 slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx, void* core_aux,

@@ -110,25 +110,36 @@ __device__ __forceinline__ unsigned long long cta_sum64(unsigned long long v, un
     return s;
 }
 
-// Last phase of a selection, run by every CTA of a kernel of kFinishThreads threads after a grid
-// barrier: G holds the parameters above the threshold, E (may be null: none) those equal to it, of
-// which the first `ties` in index order belong to the core; tile_sum their counts per tile of
-// kEmitTile blocks.  Writes the core's bitmap, its non-core rank directory and its ascending index
-// list, and checks the totals against k.
-__device__ __forceinline__ void emit_phase(const uint32_t* G, const uint32_t* E, uint32_t T, uint32_t ties,
-                                           const unsigned long long* tile_sum, uint64_t n, uint64_t nb, uint32_t k,
-                                           WsHeader* hdr, uint32_t* core_idx, uint32_t* bitmap, uint32_t* dir,
-                                           unsigned long long* scan_smem, unsigned long long* red) {
+// Last step of a selection, a kernel of its own (one CTA of kFinishThreads threads per kEmitGroup
+// tiles): G holds the parameters above the threshold, E (may be null: none) those equal to it, of
+// which the first hdr->tie_quota in index order belong to the core; tile_sum their counts per tile
+// of kEmitTile blocks.  Writes the core's bitmap, its non-core rank directory and its ascending
+// index list, and checks the totals against k.
+constexpr uint32_t kEmitGroup = 4;
+constexpr uint32_t kEmitOwnLists = 2048;   // members in a warp's 128 words up to which every thread writes its own
+
+__global__ void __launch_bounds__(kFinishThreads, 3) emit_kernel(const uint32_t* __restrict__ G,
+                                                                 const uint32_t* __restrict__ E,
+                                                                 const unsigned long long* __restrict__ tile_sum,
+                                                                 uint64_t n, uint64_t nb, uint32_t k, WsHeader* hdr,
+                                                                 uint32_t* __restrict__ core_idx,
+                                                                 uint32_t* __restrict__ bitmap,
+                                                                 uint32_t* __restrict__ dir) {
+    __shared__ unsigned long long scan_smem[33];
+    __shared__ unsigned long long red[kFinishThreads / 32];
+    if (hdr->abort != 0u) return;   // the finishing kernel gave up (status says so)
+    const uint32_t ties = (E != nullptr) ? hdr->tie_quota : 0u;
     const uint32_t t = threadIdx.x, lane = lane_id();
     const uint32_t lt_mask = (1u << lane) - 1u;
     const uint64_t ntiles = (nb + kEmitTile - 1) / kEmitTile;
+    // this CTA's tiles: blockIdx.x, blockIdx.x + gridDim.x, ... (the core clusters in some layers:
+    // neighbouring tiles go to different CTAs, so that the heavy ones are worked on all over the GPU)
+    const uint64_t tile_first = blockIdx.x, tile_step = gridDim.x, tile_last = ntiles;
     if (blockIdx.x == 0) {
         unsigned long long all = 0;
-        for (uint64_t x = t; x < ntiles; x += kFinishThreads) all += __ldcg(tile_sum + x);
+        for (uint64_t x = t; x < ntiles; x += kFinishThreads) all += __ldg(tile_sum + x);
         all = cta_sum64<kFinishThreads>(all, red);
         if (t == 0) {
-            hdr->prefix = T;
-            hdr->ties = ties;
             // whole-vector check: (#greater) + min(#equal, r) must be k
             const uint32_t ng = (uint32_t)all, ne = (uint32_t)(all >> 32);
             if (ng + min(ne, ties) != k) hdr->status = SLIMDP_ERR_INTERNAL;
@@ -136,27 +147,26 @@ __device__ __forceinline__ void emit_phase(const uint32_t* G, const uint32_t* E,
         }
     }
 
-    // Bitmaps to core bitmap, directory and ascending index list.  One tile of kEmitTile blocks per
-    // step, four consecutive bitmap words per thread; tiles are dealt out to the CTAs in turn (the
-    // core clusters in some layers); a scan over the tile's words places every member.
+    // One tile of kEmitTile blocks per step, four consecutive bitmap words per thread; a scan over
+    // the tile's words places every member.
     unsigned long long before = 0;   // counts in the tiles below the current one
     uint64_t counted = 0;            // tiles whose counts `before` holds
     const uint32_t w0 = (t & 7u) * 4u;   // first of this thread's four words in its block
     auto load_words = [&](uint64_t tile, uint4* Gw, uint4* Ew) {
         const uint64_t blk = tile * kEmitTile + (t >> 3);
         *Gw = *Ew = make_uint4(0, 0, 0, 0);
-        if (tile < ntiles && blk < nb) {
-            *Gw = __ldcg(reinterpret_cast<const uint4*>(G + blk * kWordsPerBlock + w0));
-            if (E != nullptr) *Ew = __ldcg(reinterpret_cast<const uint4*>(E + blk * kWordsPerBlock + w0));
+        if (tile < tile_last && blk < nb) {
+            *Gw = __ldg(reinterpret_cast<const uint4*>(G + blk * kWordsPerBlock + w0));
+            if (E != nullptr) *Ew = __ldg(reinterpret_cast<const uint4*>(E + blk * kWordsPerBlock + w0));
         }
     };
     uint4 Gnext, Enext;   // the next tile's words are requested before this tile's are worked on
-    load_words(blockIdx.x, &Gnext, &Enext);
-    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    load_words(tile_first, &Gnext, &Enext);
+    for (uint64_t tile = tile_first; tile < tile_last; tile += tile_step) {
         const uint4 Gw = Gnext, Ew = Enext;
-        load_words(tile + gridDim.x, &Gnext, &Enext);
+        load_words(tile + tile_step, &Gnext, &Enext);
         unsigned long long v = 0;
-        for (uint64_t x = counted + t; x < tile; x += kFinishThreads) v += __ldcg(tile_sum + x);
+        for (uint64_t x = counted + t; x < tile; x += kFinishThreads) v += __ldg(tile_sum + x);
         before += cta_sum64<kFinishThreads>(v, red);
         counted = tile;
         const uint64_t blk = tile * kEmitTile + (t >> 3);
@@ -198,7 +208,7 @@ __device__ __forceinline__ void emit_phase(const uint32_t* G, const uint32_t* E,
         const uint32_t first0 = (uint32_t)(blk * kBlock) + w0 * 32u;
         const uint32_t warp_members = __reduce_add_sync(0xFFFFFFFFu, members);
         bool bad = false;
-        if (warp_members <= 128u) {
+        if (warp_members <= kEmitOwnLists) {
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 uint32_t pos = pos0[q];
@@ -232,6 +242,17 @@ __device__ __forceinline__ void emit_phase(const uint32_t* G, const uint32_t* E,
         before += total;
         counted = tile + 1;
     }
+}
+
+inline slimdp_status launch_emit(const uint32_t* G, const uint32_t* E, const unsigned long long* tile_sum, uint64_t n,
+                                 uint32_t k, WsHeader* hdr, uint32_t* core_idx, uint32_t* bitmap, uint32_t* dir,
+                                 cudaStream_t st) {
+    const uint64_t nb = num_blocks(n);
+    const uint64_t ntiles = (nb + kEmitTile - 1) / kEmitTile;
+    emit_kernel<<<(unsigned)((ntiles + kEmitGroup - 1) / kEmitGroup), kFinishThreads, 0, st>>>(
+        G, E, tile_sum, n, nb, k, hdr, core_idx, bitmap, dir);
+    SLIMDP_LAUNCHED(1);
+    return SLIMDP_OK;
 }
 
 }  // namespace

@@ -56,8 +56,8 @@ def test_size_queries(P):
         k_exp = n // 100
         assert P.explore_workspace_bytes(n, k_exp, 8) > P.explore_workspace_bytes(n, k_exp, 1) >= 256 + 8 * k_exp
         assert P.explore_workspace_bytes(n, n, 1) >= 8 * n
-        assert P.workspace_bytes(n, k_exp, 8) == max(P.select_workspace_bytes(n),
-                                                     P.explore_workspace_bytes(n, k_exp, 8))
+        assert P.workspace_bytes(n, 8, 0, k_exp) == max(P.select_workspace_bytes(n),
+                                                        P.explore_workspace_bytes(n, k_exp, 8))
     # out-of-range arguments size to zero
     assert P.core_aux_bytes(0) == 0 and P.core_aux_bytes(2 ** 32) == 0
     assert P.explore_workspace_bytes(1000, 10, 0) == 0 and P.explore_workspace_bytes(1000, 10, 65) == 0

@@ -107,6 +107,54 @@ def test_score_unaligned_views(P):
     assert np.array_equal(got[3:].view(np.uint32), bits(exp)) and np.all(got[:3] == 0)
 
 
+@pytest.mark.parametrize("shift", [1, 2, 3])
+def test_score_views_with_one_common_misalignment(P, shift):
+    # slices of larger allocations that all start `shift` floats past a 16-byte boundary: the vectorised
+    # kernel runs after the first 4 - shift parameters; the bytes around the outputs stay untouched
+    n, K = 100_003, 4
+    rng = np.random.default_rng(50 + shift)
+    w = rng.standard_normal(n + 8).astype(np.float32)
+    gs = [rng.standard_normal(n + 8).astype(np.float32) for _ in range(K)]
+    dw, dg = dev(w), [dev(g) for g in gs]
+    out = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+    P.slimdp_score(dw[shift:shift + n], [g[shift:shift + n] for g in dg], 0.75, out[shift:shift + n])
+    exp = oracle.score(w[shift:shift + n], [g[shift:shift + n] for g in gs], 0.75)
+    got = out.cpu().numpy()
+    assert np.array_equal(got[shift:shift + n].view(np.uint32), bits(exp))
+    assert np.all(got[:shift] == 0) and np.all(got[shift + n:] == 0)
+
+
+def test_index_buffers_need_only_four_byte_alignment(P):
+    # core_idx / exp_idx that start 4 bytes past a 16-byte boundary go through select, explore and the exchange
+    cfg = CONFIGS["tiny"]
+    w, gs = all_inputs(cfg)
+    ref = oracle.run_round(w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 3, cfg.eta)
+    n, K = cfg.N, cfg.K
+    d_w, d_gs = dev(w), [dev(g) for g in gs]
+    scores = torch.empty(n, dtype=torch.float32, device="cuda")
+    core_store = torch.empty(cfg.k_core + 1, dtype=torch.int32, device="cuda")
+    core_idx = core_store[1:]
+    exp_store = [torch.empty(cfg.k_exp + 3, dtype=torch.int32, device="cuda") for _ in range(K)]
+    exp_idx = [e[3:] for e in exp_store]
+    assert core_idx.data_ptr() % 16 == 4 and exp_idx[0].data_ptr() % 16 == 12
+    aux = torch.empty(P.core_aux_bytes(n), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(P.workspace_bytes(n, K, cfg.k_core, cfg.k_exp), dtype=torch.uint8, device="cuda")
+    val = [torch.empty(cfg.m, dtype=torch.float32, device="cuda") for _ in range(K)]
+    pulled = [torch.empty(cfg.m, dtype=torch.float32, device="cuda") for _ in range(K)]
+    P.slimdp_score(d_w, d_gs, cfg.c, scores)
+    P.slimdp_select_core(scores, cfg.k_core, core_idx, aux, ws)
+    P.read_status(ws)
+    P.slimdp_sample_explore_batched(aux, n, cfg.k_core, cfg.k_exp, cfg.seed, 0, 3, exp_idx, ws)
+    P.read_status(ws)
+    P.slimdp_exchange(d_w, d_gs, core_idx, exp_idx, cfg.eta, val, pulled)
+    assert np.array_equal(host_u32(core_idx), ref["core_idx"])
+    for k in range(K):
+        assert np.array_equal(host_u32(exp_idx[k]), ref["exp_idx"][k])
+        assert np.array_equal(host_bits(val[k]), bits(ref["val"][k]))
+        assert np.array_equal(host_bits(pulled[k]), bits(ref["pulled"][k]))
+    assert np.array_equal(host_bits(d_w), bits(ref["w"]))
+
+
 # -------------------------------------------------------------------- select
 
 def _score_patterns(n, rng):
@@ -761,3 +809,58 @@ def test_segmented_select_adversarial(P, case):
     _segmented_case(P, S, off, ks)
     if case == "one_segment":
         assert np.array_equal(oracle.select_core_segmented(S, off, ks), oracle.select_core(S, ks[0]))
+
+
+
+# ------------------------------------------------------------- round contexts
+
+def test_two_host_threads_run_rounds_on_one_device_at_once(P):
+    """Two host threads, each with its own stream, round context and buffers, enqueue rounds on one
+    device at the same time; both must leave the oracle's bytes.  A third pair of rounds shares the
+    library's default context from two threads (serialised by its lock)."""
+    import threading
+    cfg = scaled_config(CONFIGS["vgg16"], FUSED_N)
+    w, gs = all_inputs(cfg)
+    refs, w_ref = [], w
+    for t in range(3):                       # three successive rounds on the evolving model
+        r = oracle.run_round(w_ref, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, t, cfg.eta)
+        refs.append(r)
+        w_ref = r["w"]
+
+    def worker(own_ctx, errors, slot):
+        try:
+            torch.cuda.set_device(0)
+            stream = torch.cuda.Stream()
+            ctx = P.RoundContext() if own_ctx else None
+            with torch.cuda.stream(stream):
+                d_w, d_gs = dev(w), [dev(g) for g in gs]
+                buf = P.RoundBuffers(cfg.N, cfg.K, cfg.k_core, cfg.k_exp)
+                for t in range(3):
+                    P.slimdp_round(d_w, d_gs, cfg.c, cfg.seed, t, cfg.eta, buf.scores, buf.core_idx, buf.core_aux,
+                                   buf.exp_idx, buf.val, buf.pulled, buf.select_ws, buf.explore_ws, None, ctx, stream)
+                stream.synchronize()
+                P.read_status(buf.select_ws, stream)
+                P.read_status(buf.explore_ws, stream)
+                ok = np.array_equal(host_bits(d_w), bits(refs[2]["w"])) and \
+                    np.array_equal(host_u32(buf.core_idx), refs[2]["core_idx"])
+                for k in range(cfg.K):
+                    ok = ok and np.array_equal(host_u32(buf.exp_idx[k]), refs[2]["exp_idx"][k]) and \
+                        np.array_equal(host_bits(buf.pulled[k]), bits(refs[2]["pulled"][k]))
+                if not ok:
+                    errors.append(f"thread {slot}: results differ from the oracle")
+            if ctx is not None:
+                ctx.close()
+        except Exception as e:          # noqa: BLE001  (reported to the main thread)
+            errors.append(f"thread {slot}: {e!r}")
+
+    for own_ctx in (True, False):
+        errors = []
+        threads = [threading.Thread(target=worker, args=(own_ctx, errors, i)) for i in range(2)]
+        for th in threads:
+            th.start()
+        for th in threads:
+            th.join()
+        assert not errors, errors
+    P.release_default_round_ctx()            # and the default context can be given back and made again
+    d_w, buf = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 0, cfg.eta, one_call=True)
+    assert np.array_equal(host_bits(d_w), bits(refs[0]["w"]))
