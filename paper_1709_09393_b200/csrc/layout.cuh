@@ -15,6 +15,7 @@ struct SelectWs {
     uint32_t* G;                    // greater-than-threshold bitmap, nb * 32 words
     uint32_t* E;                    // equal-to-threshold bitmap, nb * 32 words
     unsigned long long* tile_sum;   // per tile of kEmitTile blocks: #greater | #equal << 32
+    unsigned long long* super_pref; // per group of 64 tiles: the counts in the tiles below the group
     uint32_t* cand_key;             // keys inside the bracket
     uint32_t* cand_idx;             // and their parameter indices
     uint64_t cand_cap;              // entries in each candidate array
@@ -22,7 +23,7 @@ struct SelectWs {
     size_t bytes;
 };
 
-constexpr uint32_t kEmitTile = 64;    // 1024-parameter blocks per step of the finishing kernel's last phase
+constexpr uint32_t kEmitTile = 8;     // 1024-parameter blocks per tile of the selection's last step (one CTA, a warp per block)
 
 inline SelectWs select_ws_layout(void* ws, uint64_t n) {
     const uint64_t nb = num_blocks(n);
@@ -40,6 +41,7 @@ inline SelectWs select_ws_layout(void* ws, uint64_t n) {
     L.fine_hist = reinterpret_cast<uint32_t*>(take(512 * sizeof(uint32_t)));
     L.tile_sum = reinterpret_cast<unsigned long long*>(take(((nb + kEmitTile - 1) / kEmitTile) * 8));
     L.zero_bytes = off;
+    L.super_pref = reinterpret_cast<unsigned long long*>(take((((nb + kEmitTile - 1) / kEmitTile + 63) / 64) * 8));
     L.coarse_incl = reinterpret_cast<uint32_t*>(take(256 * sizeof(uint32_t)));
     L.sample = reinterpret_cast<uint32_t*>(take((size_t)(1u << kSampleBits) * sizeof(uint32_t)));
     L.G = reinterpret_cast<uint32_t*>(take(nb * kWordsPerBlock * 4));

@@ -55,6 +55,7 @@ struct SegArgs {
     WsHeader* hdr;
     uint32_t* G;
     unsigned long long* tile_sum;
+    unsigned long long* super_pref;
     uint32_t* core_idx;
     uint32_t* bitmap;
     uint32_t* dir;
@@ -233,6 +234,9 @@ __global__ void __launch_bounds__(kFinishThreads, 2) seg_select_kernel(SegArgs a
         const uint32_t c = __reduce_add_sync(0xFFFFFFFFu, __popc(mine));
         if (lane == 0 && c) atomicAdd(&a.tile_sum[blk / kEmitTile], (unsigned long long)c);
     }
+    if (!grid_barrier(a.hdr, &epoch)) return;
+    if (blockIdx.x == 0)
+        tile_scan_phase<kFinishThreads>(a.tile_sum, a.super_pref, a.n, a.nb, a.k_total, 0u, a.hdr, a.dir, scan_smem);
 }
 
 }  // namespace
@@ -243,6 +247,7 @@ struct SegWs {
     WsHeader* hdr;
     uint32_t* flags;
     unsigned long long* tile_sum;
+    unsigned long long* super_pref;
     uint32_t* hist;
     size_t zero_bytes;   // header, flags, tile counts and histograms, contiguous
     unsigned long long* seg_off;
@@ -267,6 +272,7 @@ SegWs seg_ws_layout(void* ws, uint64_t n, uint32_t segments) {
     L.tile_sum = reinterpret_cast<unsigned long long*>(take(((nb + kEmitTile - 1) / kEmitTile) * 8));
     L.hist = reinterpret_cast<uint32_t*>(take((size_t)2 * segments * kSegHistWords * 4));
     L.zero_bytes = off;
+    L.super_pref = reinterpret_cast<unsigned long long*>(take(num_super_tiles(nb) * 8));
     L.seg_off = reinterpret_cast<unsigned long long*>(take(((size_t)segments + 1) * 8));
     L.seg_k = reinterpret_cast<unsigned long long*>(take((size_t)segments * 8));
     L.state = reinterpret_cast<SegState*>(take((size_t)segments * sizeof(SegState)));
@@ -320,6 +326,7 @@ slimdp_status launch_select_segmented(const float* scores, uint64_t n, const uin
     a.hdr = L.hdr;
     a.G = L.G;
     a.tile_sum = L.tile_sum;
+    a.super_pref = L.super_pref;
     a.core_idx = core_idx;
     a.bitmap = reinterpret_cast<uint32_t*>(core_aux);
     a.dir = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(core_aux) + slimdp_core_aux_dir_offset(n));
@@ -328,7 +335,7 @@ slimdp_status launch_select_segmented(const float* scores, uint64_t n, const uin
                                     dim3(kFinishThreads), args, 0, st) != cudaSuccess)
         return SLIMDP_ERR_CUDA;
     SLIMDP_LAUNCHED(1);
-    return launch_emit(L.G, nullptr, L.tile_sum, n, (uint32_t)k_total, L.hdr, core_idx, a.bitmap, a.dir, st);
+    return launch_emit(L.G, nullptr, L.tile_sum, L.super_pref, n, (uint32_t)k_total, L.hdr, core_idx, a.bitmap, a.dir, st);
 }
 
 }  // namespace slimdp

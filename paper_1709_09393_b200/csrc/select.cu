@@ -756,6 +756,7 @@ struct FinishArgs {
     uint32_t* G;
     uint32_t* E;
     unsigned long long* tile_sum;   // per tile of kEmitTile blocks: #greater | #equal << 32
+    unsigned long long* super_pref; // per group of tiles: the counts below the group (written here)
     uint32_t* core_idx;
     uint32_t* bitmap;
     uint32_t* dir;
@@ -949,10 +950,14 @@ __global__ void __launch_bounds__(kFinishThreads, 2) finish_kernel(FinishArgs a)
         return;
     }
 
-    if (blockIdx.x == 0 && t == 0) {   // for the emitting kernel, and for whoever reads the header afterwards
+    // the tile counts are complete once every CTA is here; one CTA turns them into the groups' prefixes
+    if (!grid_barrier(hdr, &epoch)) return;
+    if (blockIdx.x != 0) return;
+    if (t == 0) {   // for the emitting kernel, and for whoever reads the header afterwards
         hdr->threshold = T;
         hdr->tie_quota = ties;
     }
+    tile_scan_phase<kFinishThreads>(a.tile_sum, a.super_pref, a.n, a.nb, k, ties, hdr, a.dir, scan_smem);
 }
 
 }  // namespace
@@ -1134,6 +1139,7 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
     fa.G = L.G;
     fa.E = L.E;
     fa.tile_sum = L.tile_sum;
+    fa.super_pref = L.super_pref;
     fa.core_idx = core_idx;
     fa.bitmap = bitmap;
     fa.dir = dir;
@@ -1142,7 +1148,7 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
                                     dim3(kFinishThreads), args, 0, st) != cudaSuccess)
         return SLIMDP_ERR_CUDA;
     SLIMDP_LAUNCHED(1);
-    return launch_emit(L.G, L.E, L.tile_sum, n, k, L.hdr, core_idx, bitmap, dir, st);
+    return launch_emit(L.G, L.E, L.tile_sum, L.super_pref, n, k, L.hdr, core_idx, bitmap, dir, st);
 }
 
 slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx, void* core_aux,

@@ -9,7 +9,6 @@ namespace slimdp {
 namespace {
 
 constexpr int kFinishThreads = 512;   // two CTAs per SM: one's waits are the other's work
-static_assert(kFinishThreads / 8 == kEmitTile, "a tile is four bitmap words per thread of the finishing kernel");
 constexpr uint32_t kBarrierSpins = 1u << 24;   // x 64 ns of back-off: about a second
 
 
@@ -110,147 +109,155 @@ __device__ __forceinline__ unsigned long long cta_sum64(unsigned long long v, un
     return s;
 }
 
-// Last step of a selection, a kernel of its own (one CTA of kFinishThreads threads per kEmitGroup
-// tiles): G holds the parameters above the threshold, E (may be null: none) those equal to it, of
-// which the first hdr->tie_quota in index order belong to the core; tile_sum their counts per tile
-// of kEmitTile blocks.  Writes the core's bitmap, its non-core rank directory and its ascending
-// index list, and checks the totals against k.
-constexpr uint32_t kEmitGroup = 4;
-constexpr uint32_t kEmitOwnLists = 2048;   // members in a warp's 128 words up to which every thread writes its own
+// ---- last step of a selection: bitmaps to core bitmap, directory and ascending index list ----
+//
+// G holds the parameters above the threshold, E (may be null: none) those equal to it, of which the
+// first hdr->tie_quota in index order belong to the core; tile_sum holds their counts per tile of
+// kEmitTile blocks.  The finishing kernel ends with tile_scan_phase (one CTA, after a grid barrier):
+// the counts before every group of kSuperTile tiles.  emit_kernel then runs one small CTA per tile
+// (a warp per 1024-parameter block, no waiting between CTAs): the counts before the tile are the
+// group's plus those of the tiles before it in the group.
+constexpr uint32_t kSuperTile = 64;    // tiles per group
+constexpr int kEmitThreads = 32 * kEmitTile;
+static_assert(kEmitThreads >= (int)kSuperTile, "one thread per tile of a group");
 
-__global__ void __launch_bounds__(kFinishThreads, 3) emit_kernel(const uint32_t* __restrict__ G,
-                                                                 const uint32_t* __restrict__ E,
-                                                                 const unsigned long long* __restrict__ tile_sum,
-                                                                 uint64_t n, uint64_t nb, uint32_t k, WsHeader* hdr,
-                                                                 uint32_t* __restrict__ core_idx,
-                                                                 uint32_t* __restrict__ bitmap,
-                                                                 uint32_t* __restrict__ dir) {
-    __shared__ unsigned long long scan_smem[33];
-    __shared__ unsigned long long red[kFinishThreads / 32];
-    if (hdr->abort != 0u) return;   // the finishing kernel gave up (status says so)
-    const uint32_t ties = (E != nullptr) ? hdr->tie_quota : 0u;
-    const uint32_t t = threadIdx.x, lane = lane_id();
-    const uint32_t lt_mask = (1u << lane) - 1u;
+inline uint64_t num_tiles(uint64_t nb) { return (nb + kEmitTile - 1) / kEmitTile; }
+inline uint64_t num_super_tiles(uint64_t nb) { return (num_tiles(nb) + kSuperTile - 1) / kSuperTile; }
+
+// One CTA of THREADS threads: super_pref[s] = counts in the tiles below group s; checks the totals
+// against k ((#greater) + min(#equal, r) must be k) and writes the directory's last entry.
+template <int THREADS>
+__device__ __forceinline__ void tile_scan_phase(const unsigned long long* tile_sum, unsigned long long* super_pref,
+                                                uint64_t n, uint64_t nb, uint32_t k, uint32_t ties, WsHeader* hdr,
+                                                uint32_t* dir, unsigned long long* scan_smem) {
     const uint64_t ntiles = (nb + kEmitTile - 1) / kEmitTile;
-    // this CTA's tiles: blockIdx.x, blockIdx.x + gridDim.x, ... (the core clusters in some layers:
-    // neighbouring tiles go to different CTAs, so that the heavy ones are worked on all over the GPU)
-    const uint64_t tile_first = blockIdx.x, tile_step = gridDim.x, tile_last = ntiles;
-    if (blockIdx.x == 0) {
-        unsigned long long all = 0;
-        for (uint64_t x = t; x < ntiles; x += kFinishThreads) all += __ldg(tile_sum + x);
-        all = cta_sum64<kFinishThreads>(all, red);
-        if (t == 0) {
-            // whole-vector check: (#greater) + min(#equal, r) must be k
-            const uint32_t ng = (uint32_t)all, ne = (uint32_t)(all >> 32);
-            if (ng + min(ne, ties) != k) hdr->status = SLIMDP_ERR_INTERNAL;
-            dir[nb * kDirPerBlock] = (uint32_t)(n - k);
-        }
-    }
-
-    // One tile of kEmitTile blocks per step, four consecutive bitmap words per thread; a scan over
-    // the tile's words places every member.
-    unsigned long long before = 0;   // counts in the tiles below the current one
-    uint64_t counted = 0;            // tiles whose counts `before` holds
-    const uint32_t w0 = (t & 7u) * 4u;   // first of this thread's four words in its block
-    auto load_words = [&](uint64_t tile, uint4* Gw, uint4* Ew) {
-        const uint64_t blk = tile * kEmitTile + (t >> 3);
-        *Gw = *Ew = make_uint4(0, 0, 0, 0);
-        if (tile < tile_last && blk < nb) {
-            *Gw = __ldg(reinterpret_cast<const uint4*>(G + blk * kWordsPerBlock + w0));
-            if (E != nullptr) *Ew = __ldg(reinterpret_cast<const uint4*>(E + blk * kWordsPerBlock + w0));
-        }
-    };
-    uint4 Gnext, Enext;   // the next tile's words are requested before this tile's are worked on
-    load_words(tile_first, &Gnext, &Enext);
-    for (uint64_t tile = tile_first; tile < tile_last; tile += tile_step) {
-        const uint4 Gw = Gnext, Ew = Enext;
-        load_words(tile + tile_step, &Gnext, &Enext);
+    const uint64_t nsuper = (ntiles + kSuperTile - 1) / kSuperTile;
+    unsigned long long carry = 0;
+    for (uint64_t s0 = 0; s0 < nsuper; s0 += THREADS) {
+        const uint64_t s = s0 + threadIdx.x;
         unsigned long long v = 0;
-        for (uint64_t x = counted + t; x < tile; x += kFinishThreads) v += __ldg(tile_sum + x);
-        before += cta_sum64<kFinishThreads>(v, red);
-        counted = tile;
-        const uint64_t blk = tile * kEmitTile + (t >> 3);
-        const bool have = blk < nb;
-        const uint32_t gw[4] = {Gw.x, Gw.y, Gw.z, Gw.w}, ew[4] = {Ew.x, Ew.y, Ew.z, Ew.w};
-        unsigned long long sum = 0;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) sum += (unsigned long long)__popc(gw[q]) | ((unsigned long long)__popc(ew[q]) << 32);
+        if (s < nsuper) {
+            const uint64_t first = s * kSuperTile;
+            const uint64_t last = (first + kSuperTile < ntiles) ? first + kSuperTile : ntiles;
+            for (uint64_t x = first; x < last; ++x) v += __ldcg(tile_sum + x);
+        }
         unsigned long long total;
-        unsigned long long run = before + block_exclusive_scan64<kFinishThreads / 32>(sum, scan_smem, &total);
-        uint32_t sel[4], pos0[4], dirv[2] = {0, 0};
-        uint32_t members = 0;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t g_before = (uint32_t)run, e_before = (uint32_t)(run >> 32);
-            const uint32_t pe = __popc(ew[q]);
-            // equal keys: admit those whose rank among all equal keys (index order) is below r
-            const uint32_t admit = (ties > e_before) ? min(ties - e_before, pe) : 0u;
-            uint32_t Ea;
-            if (admit == pe)
-                Ea = ew[q];
-            else if (admit == 0)
-                Ea = 0;
-            else
-                Ea = ew[q] & ((1u << nth_set_bit(ew[q], admit)) - 1u);
-            sel[q] = gw[q] | Ea;
-            pos0[q] = g_before + min(e_before, ties);   // core parameters below this word
-            members += __popc(sel[q]);
-            const uint32_t first = (uint32_t)(blk * kBlock) + (w0 + q) * 32u;
-            if ((q & 1) == 0) dirv[q >> 1] = first - pos0[q];   // one directory entry per 64 parameters (2 words)
-            run += (unsigned long long)__popc(gw[q]) | ((unsigned long long)pe << 32);
-        }
-        if (have) {
-            *reinterpret_cast<uint4*>(bitmap + blk * kWordsPerBlock + w0) = make_uint4(sel[0], sel[1], sel[2], sel[3]);
-            *reinterpret_cast<uint2*>(dir + blk * kDirPerBlock + (w0 >> 1)) = make_uint2(dirv[0], dirv[1]);
-        }
-        // the index list.  Few members in the warp's 128 words: every thread writes its own; many:
-        // the warp writes one word's members at a time (coalesced)
-        const uint32_t first0 = (uint32_t)(blk * kBlock) + w0 * 32u;
-        const uint32_t warp_members = __reduce_add_sync(0xFFFFFFFFu, members);
-        bool bad = false;
-        if (warp_members <= kEmitOwnLists) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t pos = pos0[q];
-                for (uint32_t word = sel[q]; word; word &= word - 1) {
-                    if (pos < k)
-                        core_idx[pos] = first0 + q * 32u + (uint32_t)__ffs(word) - 1u;
-                    else
-                        bad = true;
-                    ++pos;
-                }
-            }
-        } else {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                for (uint32_t m = __ballot_sync(0xFFFFFFFFu, sel[q] != 0); m; m &= m - 1) {
-                    const int src = __ffs(m) - 1;
-                    const uint32_t word = __shfl_sync(0xFFFFFFFFu, sel[q], src);
-                    const uint32_t base = __shfl_sync(0xFFFFFFFFu, pos0[q], src);
-                    const uint32_t first = __shfl_sync(0xFFFFFFFFu, first0, src) + q * 32u;
-                    if ((word >> lane) & 1u) {
-                        const uint32_t pos = base + __popc(word & lt_mask);
-                        if (pos < k)
-                            core_idx[pos] = first + lane;
-                        else
-                            bad = true;
-                    }
-                }
-            }
-        }
-        if (bad) hdr->status = SLIMDP_ERR_INTERNAL;
-        before += total;
-        counted = tile + 1;
+        const unsigned long long ex = block_exclusive_scan64<THREADS / 32>(v, scan_smem, &total);
+        if (s < nsuper) super_pref[s] = carry + ex;
+        carry += total;
+    }
+    if (threadIdx.x == 0) {
+        const uint32_t ng = (uint32_t)carry, ne = (uint32_t)(carry >> 32);
+        if (ng + min(ne, ties) != k) hdr->status = SLIMDP_ERR_INTERNAL;
+        dir[nb * kDirPerBlock] = (uint32_t)(n - k);
     }
 }
 
-inline slimdp_status launch_emit(const uint32_t* G, const uint32_t* E, const unsigned long long* tile_sum, uint64_t n,
-                                 uint32_t k, WsHeader* hdr, uint32_t* core_idx, uint32_t* bitmap, uint32_t* dir,
-                                 cudaStream_t st) {
-    const uint64_t nb = num_blocks(n);
+__global__ void __launch_bounds__(kEmitThreads) emit_kernel(const uint32_t* __restrict__ G,
+                                                            const uint32_t* __restrict__ E,
+                                                            const unsigned long long* __restrict__ tile_sum,
+                                                            const unsigned long long* __restrict__ super_pref,
+                                                            uint64_t nb, uint32_t k, WsHeader* hdr,
+                                                            uint32_t* __restrict__ core_idx,
+                                                            uint32_t* __restrict__ bitmap,
+                                                            uint32_t* __restrict__ dir) {
+    __shared__ unsigned long long red[kEmitThreads / 32];
+    __shared__ unsigned long long warp_cnt[kEmitTile];
+    if (hdr->abort != 0u) return;   // the finishing kernel gave up (the status word says so)
+    const uint32_t ties = (E != nullptr) ? hdr->tie_quota : 0u;
+    const uint32_t t = threadIdx.x, lane = lane_id(), wid = t >> 5;
+    const uint32_t lt_mask = (1u << lane) - 1u;
     const uint64_t ntiles = (nb + kEmitTile - 1) / kEmitTile;
-    emit_kernel<<<(unsigned)((ntiles + kEmitGroup - 1) / kEmitGroup), kFinishThreads, 0, st>>>(
-        G, E, tile_sum, n, nb, k, hdr, core_idx, bitmap, dir);
+    // what an iteration needs from memory is requested one iteration ahead
+    uint32_t Gn = 0, En = 0;
+    unsigned long long vn = 0;
+    auto request = [&](uint64_t tile) {
+        Gn = En = 0u;
+        vn = 0ull;
+        if (tile >= ntiles) return;
+        const uint64_t blk = tile * kEmitTile + wid;
+        if (blk < nb) {   // this warp's block: one bitmap word per lane
+            Gn = __ldg(G + blk * kWordsPerBlock + lane);
+            if (E != nullptr) En = __ldg(E + blk * kWordsPerBlock + lane);
+        }
+        // counts before the tile: the group's, plus the tiles of the group below this one
+        const uint64_t super = tile / kSuperTile, in_super = tile % kSuperTile;
+        if (t < in_super) vn = __ldg(tile_sum + super * kSuperTile + t);
+        if (t == 0) vn += __ldg(super_pref + super);
+    };
+    request(blockIdx.x);
+    bool bad = false;
+    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const uint32_t Gw = Gn, Ew = En;
+        const unsigned long long v = vn;
+        request(tile + gridDim.x);
+        const uint64_t blk = tile * kEmitTile + wid;
+        const bool have = blk < nb;
+        const unsigned long long mine = (unsigned long long)__popc(Gw) | ((unsigned long long)__popc(Ew) << 32);
+        const unsigned long long in_warp = warp_inclusive_scan64(mine);
+        if (lane == 31) warp_cnt[wid] = in_warp;
+        unsigned long long run = cta_sum64<kEmitThreads>(v, red);   // (its barriers also publish warp_cnt)
+        for (uint32_t x = 0; x < wid; ++x) run += warp_cnt[x];
+        run += in_warp - mine;   // counts before this lane's word
+        const uint32_t g_before = (uint32_t)run, e_before = (uint32_t)(run >> 32);
+        const uint32_t pe = __popc(Ew);
+        // equal keys: admit those whose rank among all equal keys (index order) is below r
+        const uint32_t admit = (ties > e_before) ? min(ties - e_before, pe) : 0u;
+        uint32_t Ea;
+        if (admit == pe)
+            Ea = Ew;
+        else if (admit == 0)
+            Ea = 0;
+        else
+            Ea = Ew & ((1u << nth_set_bit(Ew, admit)) - 1u);
+        const uint32_t sel = Gw | Ea;
+        const uint32_t pos0 = g_before + min(e_before, ties);   // core parameters below this word
+        if (!have) continue;
+        const uint32_t first = (uint32_t)(blk * kBlock);
+        bitmap[blk * kWordsPerBlock + lane] = sel;
+        if ((lane & (kWordsPerDir - 1)) == 0)   // one directory entry per 64 parameters (2 words)
+            dir[blk * kDirPerBlock + lane / kWordsPerDir] = first + lane * 32u - pos0;
+        const uint32_t in_block = __reduce_add_sync(0xFFFFFFFFu, __popc(sel));
+        if (in_block == 0) continue;
+        if (in_block <= 256) {
+            // sparse block: every lane writes out its own word's members
+            uint32_t pos = pos0;
+            for (uint32_t word = sel; word; word &= word - 1, ++pos) {
+                if (pos < k)
+                    core_idx[pos] = first + lane * 32u + (uint32_t)__ffs(word) - 1u;
+                else
+                    bad = true;
+            }
+        } else {
+            // dense block: the warp writes one word's members at a time (coalesced)
+            for (uint32_t m = __ballot_sync(0xFFFFFFFFu, sel != 0); m; m &= m - 1) {
+                const int wd = __ffs(m) - 1;
+                const uint32_t word = __shfl_sync(0xFFFFFFFFu, sel, wd);
+                const uint32_t base = __shfl_sync(0xFFFFFFFFu, pos0, wd);
+                if ((word >> lane) & 1u) {
+                    const uint32_t pos = base + __popc(word & lt_mask);
+                    if (pos < k)
+                        core_idx[pos] = first + wd * 32u + lane;
+                    else
+                        bad = true;
+                }
+            }
+        }
+    }
+    if (bad) hdr->status = SLIMDP_ERR_INTERNAL;
+}
+
+inline slimdp_status launch_emit(const uint32_t* G, const uint32_t* E, const unsigned long long* tile_sum,
+                                 const unsigned long long* super_pref, uint64_t n, uint32_t k, WsHeader* hdr,
+                                 uint32_t* core_idx, uint32_t* bitmap, uint32_t* dir, cudaStream_t st) {
+    const uint64_t nb = num_blocks(n);
+    const int sms = sm_count();
+    if (sms <= 0) return SLIMDP_ERR_CUDA;
+    // CTAs that are all resident at once (8 per SM) walk the tiles in turn
+    uint64_t grid = num_tiles(nb);
+    if (grid > (uint64_t)sms * 8) grid = (uint64_t)sms * 8;
+    emit_kernel<<<(unsigned)grid, kEmitThreads, 0, st>>>(G, E, tile_sum, super_pref, nb, k, hdr, core_idx,
+                                                                   bitmap, dir);
     SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }
