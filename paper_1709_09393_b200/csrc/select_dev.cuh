@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(kEmitThreads) emit_kernel(const uint32_t* __re
                                                             uint32_t* __restrict__ bitmap,
                                                             uint32_t* __restrict__ dir) {
     __shared__ unsigned long long red[kEmitThreads / 32];
-    __shared__ unsigned long long warp_cnt[kEmitTile];
+    __shared__ unsigned long long warp_cnt[2][kEmitTile];   // by iteration parity: a warp may be one iteration ahead
     if (hdr->abort != 0u) return;   // the finishing kernel gave up (the status word says so)
     const uint32_t ties = (E != nullptr) ? hdr->tie_quota : 0u;
     const uint32_t t = threadIdx.x, lane = lane_id(), wid = t >> 5;
@@ -187,7 +187,8 @@ __global__ void __launch_bounds__(kEmitThreads) emit_kernel(const uint32_t* __re
     };
     request(blockIdx.x);
     bool bad = false;
-    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    uint32_t parity = 0;
+    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, parity ^= 1u) {
         const uint32_t Gw = Gn, Ew = En;
         const unsigned long long v = vn;
         request(tile + gridDim.x);
@@ -195,9 +196,9 @@ __global__ void __launch_bounds__(kEmitThreads) emit_kernel(const uint32_t* __re
         const bool have = blk < nb;
         const unsigned long long mine = (unsigned long long)__popc(Gw) | ((unsigned long long)__popc(Ew) << 32);
         const unsigned long long in_warp = warp_inclusive_scan64(mine);
-        if (lane == 31) warp_cnt[wid] = in_warp;
+        if (lane == 31) warp_cnt[parity][wid] = in_warp;
         unsigned long long run = cta_sum64<kEmitThreads>(v, red);   // (its barriers also publish warp_cnt)
-        for (uint32_t x = 0; x < wid; ++x) run += warp_cnt[x];
+        for (uint32_t x = 0; x < wid; ++x) run += warp_cnt[parity][x];
         run += in_warp - mine;   // counts before this lane's word
         const uint32_t g_before = (uint32_t)run, e_before = (uint32_t)(run >> 32);
         const uint32_t pe = __popc(Ew);

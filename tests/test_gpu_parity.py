@@ -864,3 +864,26 @@ def test_two_host_threads_run_rounds_on_one_device_at_once(P):
     P.release_default_round_ctx()            # and the default context can be given back and made again
     d_w, buf = gpu_round(P, w, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, 0, cfg.eta, one_call=True)
     assert np.array_equal(host_bits(d_w), bits(refs[0]["w"]))
+
+
+def test_rounds_back_to_back_on_a_vector_with_several_tiles_per_cta(P):
+    """Six one-call rounds enqueued without a synchronisation in between, on a vector long enough that the
+    persistent CTAs of the selection's last kernel walk several tiles each; the model after the last round and
+    that round's outputs must be the oracle's."""
+    cfg = scaled_config(CONFIGS["vgg16"], 24_000_007)
+    w, gs = all_inputs(cfg)
+    rounds = 6
+    w_ref = w
+    for t in range(rounds):
+        ref = oracle.run_round(w_ref, gs, cfg.c, cfg.k_core, cfg.k_exp, cfg.seed, t, cfg.eta)
+        w_ref = ref["w"]
+    d_w, d_gs = dev(w), [dev(g) for g in gs]
+    buf = P.RoundBuffers(cfg.N, cfg.K, cfg.k_core, cfg.k_exp)
+    for rep in range(3):                 # the whole sequence three times over: races show up as flakiness
+        d_w.copy_(torch.from_numpy(w))
+        for t in range(rounds):
+            P.slimdp_round(d_w, d_gs, cfg.c, cfg.seed, t, cfg.eta, buf.scores, buf.core_idx, buf.core_aux, buf.exp_idx,
+                           buf.val, buf.pulled, buf.select_ws, buf.explore_ws)
+        P.read_status(buf.select_ws)
+        P.read_status(buf.explore_ws)
+        assert_round_equal(P, d_w, buf, ref, cfg.N, scores=False)
