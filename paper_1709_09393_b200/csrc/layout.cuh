@@ -14,8 +14,8 @@ struct SelectWs {
     uint32_t* sample;               // 2^18 sampled keys
     uint32_t* G;                    // greater-than-threshold bitmap, nb * 32 words
     uint32_t* E;                    // equal-to-threshold bitmap, nb * 32 words
-    unsigned long long* tile_sum;   // per tile of kEmitTile blocks: #greater | #equal << 32
-    unsigned long long* super_pref; // per group of 64 tiles: the counts in the tiles below the group
+    unsigned long long* tile_sum;   // per 1024-parameter block: #greater | #equal << 32
+    unsigned long long* super_pref; // per group of 64 blocks: their counts, then the counts below the group
     uint32_t* cand_key;             // keys inside the bracket
     uint32_t* cand_idx;             // and their parameter indices
     uint64_t cand_cap;              // entries in each candidate array
@@ -23,7 +23,7 @@ struct SelectWs {
     size_t bytes;
 };
 
-constexpr uint32_t kEmitTile = 8;     // 1024-parameter blocks per tile of the selection's last step (one CTA, a warp per block)
+constexpr uint32_t kEmitTile = 1;     // 1024-parameter blocks per counter of the selection's members (see select_dev.cuh)
 
 inline SelectWs select_ws_layout(void* ws, uint64_t n) {
     const uint64_t nb = num_blocks(n);

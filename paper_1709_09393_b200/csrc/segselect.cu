@@ -235,8 +235,10 @@ __global__ void __launch_bounds__(kFinishThreads, 2) seg_select_kernel(SegArgs a
         if (lane == 0 && c) atomicAdd(&a.tile_sum[blk / kEmitTile], (unsigned long long)c);
     }
     if (!grid_barrier(a.hdr, &epoch)) return;
+    super_sum_phase<kFinishThreads>(a.tile_sum, a.super_pref, a.nb);
+    if (!grid_barrier(a.hdr, &epoch)) return;
     if (blockIdx.x == 0)
-        tile_scan_phase<kFinishThreads>(a.tile_sum, a.super_pref, a.n, a.nb, a.k_total, 0u, a.hdr, a.dir, scan_smem);
+        tile_scan_phase<kFinishThreads>(a.super_pref, a.n, a.nb, a.k_total, 0u, a.hdr, a.dir, scan_smem);
 }
 
 }  // namespace

@@ -950,14 +950,17 @@ __global__ void __launch_bounds__(kFinishThreads, 2) finish_kernel(FinishArgs a)
         return;
     }
 
-    // the tile counts are complete once every CTA is here; one CTA turns them into the groups' prefixes
+    // the block counts are complete once every CTA is here: sums per group of blocks by all CTAs, then
+    // one CTA turns them into the groups' prefixes
+    if (!grid_barrier(hdr, &epoch)) return;
+    super_sum_phase<kFinishThreads>(a.tile_sum, a.super_pref, a.nb);
     if (!grid_barrier(hdr, &epoch)) return;
     if (blockIdx.x != 0) return;
-    if (t == 0) {   // for the emitting kernel, and for whoever reads the header afterwards
+    if (t == 0) {   // for whoever places the core's members next, and for whoever reads the header afterwards
         hdr->threshold = T;
         hdr->tie_quota = ties;
     }
-    tile_scan_phase<kFinishThreads>(a.tile_sum, a.super_pref, a.n, a.nb, k, ties, hdr, a.dir, scan_smem);
+    tile_scan_phase<kFinishThreads>(a.super_pref, a.n, a.nb, k, ties, hdr, a.dir, scan_smem);
 }
 
 }  // namespace

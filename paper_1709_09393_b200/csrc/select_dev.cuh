@@ -112,38 +112,49 @@ __device__ __forceinline__ unsigned long long cta_sum64(unsigned long long v, un
 // ---- last step of a selection: bitmaps to core bitmap, directory and ascending index list ----
 //
 // G holds the parameters above the threshold, E (may be null: none) those equal to it, of which the
-// first hdr->tie_quota in index order belong to the core; tile_sum holds their counts per tile of
-// kEmitTile blocks.  The finishing kernel ends with tile_scan_phase (one CTA, after a grid barrier):
-// the counts before every group of kSuperTile tiles.  emit_kernel then runs one small CTA per tile
-// (a warp per 1024-parameter block, no waiting between CTAs): the counts before the tile are the
-// group's plus those of the tiles before it in the group.
-constexpr uint32_t kSuperTile = 64;    // tiles per group
-constexpr int kEmitThreads = 32 * kEmitTile;
-static_assert(kEmitThreads >= (int)kSuperTile, "one thread per tile of a group");
+// first hdr->tie_quota in index order belong to the core; cnt holds their counts per 1024-parameter
+// block (#greater | #equal << 32).  The finishing kernels end with super_sum_phase (every CTA: the
+// counts of each group of kSuperTile blocks) and, after a grid barrier, tile_scan_phase (one CTA:
+// the counts below every group).  From then on any warp finds, without waiting for any other, what
+// lies below a block (the group's prefix plus at most 63 block counts) and hence every member's
+// place in the core: block_selection.  emit_kernel uses it to write the core's bitmap, directory
+// and index list; the one-call round's exchange uses it directly and needs no emit.
+constexpr uint32_t kSuperTile = 64;    // blocks per group
+constexpr int kEmitWarps = 8;
 
-inline uint64_t num_tiles(uint64_t nb) { return (nb + kEmitTile - 1) / kEmitTile; }
-inline uint64_t num_super_tiles(uint64_t nb) { return (num_tiles(nb) + kSuperTile - 1) / kSuperTile; }
+inline uint64_t num_super_tiles(uint64_t nb) { return (nb + kSuperTile - 1) / kSuperTile; }
 
-// One CTA of THREADS threads: super_pref[s] = counts in the tiles below group s; checks the totals
-// against k ((#greater) + min(#equal, r) must be k) and writes the directory's last entry.
+// Every CTA of the grid: super[s] = sum of cnt over group s (a warp per group).
 template <int THREADS>
-__device__ __forceinline__ void tile_scan_phase(const unsigned long long* tile_sum, unsigned long long* super_pref,
-                                                uint64_t n, uint64_t nb, uint32_t k, uint32_t ties, WsHeader* hdr,
-                                                uint32_t* dir, unsigned long long* scan_smem) {
-    const uint64_t ntiles = (nb + kEmitTile - 1) / kEmitTile;
-    const uint64_t nsuper = (ntiles + kSuperTile - 1) / kSuperTile;
+__device__ __forceinline__ void super_sum_phase(const unsigned long long* cnt, unsigned long long* super,
+                                                uint64_t nb) {
+    const uint64_t nsuper = (nb + kSuperTile - 1) / kSuperTile;
+    const uint32_t lane = lane_id();
+    const uint64_t warps = (uint64_t)gridDim.x * (THREADS / 32);
+    for (uint64_t s = (uint64_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5); s < nsuper; s += warps) {
+        const uint64_t b0 = s * kSuperTile + lane, b1 = b0 + 32;
+        unsigned long long v = (b0 < nb ? __ldcg(cnt + b0) : 0ull) + (b1 < nb ? __ldcg(cnt + b1) : 0ull);
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+        if (lane == 0) super[s] = v;
+    }
+}
+
+// One CTA of THREADS threads, after a grid barrier: super[s] <- counts in the groups below s (in
+// place); checks the totals against k ((#greater) + min(#equal, r) must be k) and writes the
+// directory's last entry.
+template <int THREADS>
+__device__ __forceinline__ void tile_scan_phase(unsigned long long* super, uint64_t n, uint64_t nb, uint32_t k,
+                                                uint32_t ties, WsHeader* hdr, uint32_t* dir,
+                                                unsigned long long* scan_smem) {
+    const uint64_t nsuper = (nb + kSuperTile - 1) / kSuperTile;
     unsigned long long carry = 0;
     for (uint64_t s0 = 0; s0 < nsuper; s0 += THREADS) {
         const uint64_t s = s0 + threadIdx.x;
-        unsigned long long v = 0;
-        if (s < nsuper) {
-            const uint64_t first = s * kSuperTile;
-            const uint64_t last = (first + kSuperTile < ntiles) ? first + kSuperTile : ntiles;
-            for (uint64_t x = first; x < last; ++x) v += __ldcg(tile_sum + x);
-        }
+        const unsigned long long v = (s < nsuper) ? __ldcg(super + s) : 0ull;
         unsigned long long total;
         const unsigned long long ex = block_exclusive_scan64<THREADS / 32>(v, scan_smem, &total);
-        if (s < nsuper) super_pref[s] = carry + ex;
+        if (s < nsuper) super[s] = carry + ex;
         carry += total;
     }
     if (threadIdx.x == 0) {
@@ -153,73 +164,73 @@ __device__ __forceinline__ void tile_scan_phase(const unsigned long long* tile_s
     }
 }
 
-__global__ void __launch_bounds__(kEmitThreads) emit_kernel(const uint32_t* __restrict__ G,
-                                                            const uint32_t* __restrict__ E,
-                                                            const unsigned long long* __restrict__ tile_sum,
-                                                            const unsigned long long* __restrict__ super_pref,
-                                                            uint64_t nb, uint32_t k, WsHeader* hdr,
-                                                            uint32_t* __restrict__ core_idx,
-                                                            uint32_t* __restrict__ bitmap,
-                                                            uint32_t* __restrict__ dir) {
-    __shared__ unsigned long long red[kEmitThreads / 32];
-    __shared__ unsigned long long warp_cnt[2][kEmitTile];   // by iteration parity: a warp may be one iteration ahead
+// One warp, one 1024-parameter block (lane = bitmap word; blk < nb): the block's part of the core
+// (*sel) and the number of core parameters below this lane's word (*pos0).  Returns the number of
+// core parameters in the block.
+__device__ __forceinline__ uint32_t block_selection(const uint32_t* __restrict__ G, const uint32_t* __restrict__ E,
+                                                    const unsigned long long* __restrict__ cnt,
+                                                    const unsigned long long* __restrict__ super_pref, uint32_t ties,
+                                                    uint64_t blk, uint32_t* sel, uint32_t* pos0) {
+    const uint32_t lane = lane_id();
+    const uint32_t Gw = __ldg(G + blk * kWordsPerBlock + lane);
+    const uint32_t Ew = (E != nullptr) ? __ldg(E + blk * kWordsPerBlock + lane) : 0u;
+    // counts below the block: the group's prefix plus the blocks of the group below this one
+    const uint64_t super = blk / kSuperTile, first = super * kSuperTile;
+    unsigned long long v = 0;
+    if (first + lane < blk) v += __ldg(cnt + first + lane);
+    if (first + 32 + lane < blk) v += __ldg(cnt + first + 32 + lane);
+    if (lane == 0) v += __ldg(super_pref + super);
+    const unsigned long long mine = (unsigned long long)__popc(Gw) | ((unsigned long long)__popc(Ew) << 32);
+    unsigned long long in_warp = warp_inclusive_scan64(mine);
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+    const unsigned long long run = v + in_warp - mine;   // counts below this lane's word
+    const uint32_t g_before = (uint32_t)run, e_before = (uint32_t)(run >> 32);
+    const uint32_t pe = __popc(Ew);
+    // equal keys: admit those whose rank among all equal keys (index order) is below r
+    const uint32_t admit = (ties > e_before) ? min(ties - e_before, pe) : 0u;
+    uint32_t Ea;
+    if (admit == pe)
+        Ea = Ew;
+    else if (admit == 0)
+        Ea = 0;
+    else
+        Ea = Ew & ((1u << nth_set_bit(Ew, admit)) - 1u);
+    *sel = Gw | Ea;
+    *pos0 = g_before + min(e_before, ties);
+    return __reduce_add_sync(0xFFFFFFFFu, __popc(*sel));
+}
+
+// The block's words of the core bitmap and its 16 directory entries.
+__device__ __forceinline__ void write_block_aux(uint32_t* __restrict__ bitmap, uint32_t* __restrict__ dir, uint64_t blk,
+                                                uint32_t sel, uint32_t pos0) {
+    const uint32_t lane = lane_id();
+    bitmap[blk * kWordsPerBlock + lane] = sel;
+    if ((lane & (kWordsPerDir - 1)) == 0)   // one directory entry per 64 parameters (2 words)
+        dir[blk * kDirPerBlock + lane / kWordsPerDir] = (uint32_t)(blk * kBlock) + lane * 32u - pos0;
+}
+
+// A warp per block; warps walk the blocks in turn and wait for nobody.
+__global__ void __launch_bounds__(kEmitWarps * 32) emit_kernel(const uint32_t* __restrict__ G,
+                                                               const uint32_t* __restrict__ E,
+                                                               const unsigned long long* __restrict__ cnt,
+                                                               const unsigned long long* __restrict__ super_pref,
+                                                               uint64_t nb, uint32_t k, WsHeader* hdr,
+                                                               uint32_t* __restrict__ core_idx,
+                                                               uint32_t* __restrict__ bitmap,
+                                                               uint32_t* __restrict__ dir) {
     if (hdr->abort != 0u) return;   // the finishing kernel gave up (the status word says so)
     const uint32_t ties = (E != nullptr) ? hdr->tie_quota : 0u;
-    const uint32_t t = threadIdx.x, lane = lane_id(), wid = t >> 5;
+    const uint32_t lane = lane_id();
     const uint32_t lt_mask = (1u << lane) - 1u;
-    const uint64_t ntiles = (nb + kEmitTile - 1) / kEmitTile;
-    // what an iteration needs from memory is requested one iteration ahead
-    uint32_t Gn = 0, En = 0;
-    unsigned long long vn = 0;
-    auto request = [&](uint64_t tile) {
-        Gn = En = 0u;
-        vn = 0ull;
-        if (tile >= ntiles) return;
-        const uint64_t blk = tile * kEmitTile + wid;
-        if (blk < nb) {   // this warp's block: one bitmap word per lane
-            Gn = __ldg(G + blk * kWordsPerBlock + lane);
-            if (E != nullptr) En = __ldg(E + blk * kWordsPerBlock + lane);
-        }
-        // counts before the tile: the group's, plus the tiles of the group below this one
-        const uint64_t super = tile / kSuperTile, in_super = tile % kSuperTile;
-        if (t < in_super) vn = __ldg(tile_sum + super * kSuperTile + t);
-        if (t == 0) vn += __ldg(super_pref + super);
-    };
-    request(blockIdx.x);
+    const uint64_t warps = (uint64_t)gridDim.x * kEmitWarps;
     bool bad = false;
-    uint32_t parity = 0;
-    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, parity ^= 1u) {
-        const uint32_t Gw = Gn, Ew = En;
-        const unsigned long long v = vn;
-        request(tile + gridDim.x);
-        const uint64_t blk = tile * kEmitTile + wid;
-        const bool have = blk < nb;
-        const unsigned long long mine = (unsigned long long)__popc(Gw) | ((unsigned long long)__popc(Ew) << 32);
-        const unsigned long long in_warp = warp_inclusive_scan64(mine);
-        if (lane == 31) warp_cnt[parity][wid] = in_warp;
-        unsigned long long run = cta_sum64<kEmitThreads>(v, red);   // (its barriers also publish warp_cnt)
-        for (uint32_t x = 0; x < wid; ++x) run += warp_cnt[parity][x];
-        run += in_warp - mine;   // counts before this lane's word
-        const uint32_t g_before = (uint32_t)run, e_before = (uint32_t)(run >> 32);
-        const uint32_t pe = __popc(Ew);
-        // equal keys: admit those whose rank among all equal keys (index order) is below r
-        const uint32_t admit = (ties > e_before) ? min(ties - e_before, pe) : 0u;
-        uint32_t Ea;
-        if (admit == pe)
-            Ea = Ew;
-        else if (admit == 0)
-            Ea = 0;
-        else
-            Ea = Ew & ((1u << nth_set_bit(Ew, admit)) - 1u);
-        const uint32_t sel = Gw | Ea;
-        const uint32_t pos0 = g_before + min(e_before, ties);   // core parameters below this word
-        if (!have) continue;
-        const uint32_t first = (uint32_t)(blk * kBlock);
-        bitmap[blk * kWordsPerBlock + lane] = sel;
-        if ((lane & (kWordsPerDir - 1)) == 0)   // one directory entry per 64 parameters (2 words)
-            dir[blk * kDirPerBlock + lane / kWordsPerDir] = first + lane * 32u - pos0;
-        const uint32_t in_block = __reduce_add_sync(0xFFFFFFFFu, __popc(sel));
+    for (uint64_t blk = (uint64_t)blockIdx.x * kEmitWarps + (threadIdx.x >> 5); blk < nb; blk += warps) {
+        uint32_t sel, pos0;
+        const uint32_t in_block = block_selection(G, E, cnt, super_pref, ties, blk, &sel, &pos0);
+        write_block_aux(bitmap, dir, blk, sel, pos0);
         if (in_block == 0) continue;
+        const uint32_t first = (uint32_t)(blk * kBlock);
         if (in_block <= 256) {
             // sparse block: every lane writes out its own word's members
             uint32_t pos = pos0;
@@ -248,17 +259,15 @@ __global__ void __launch_bounds__(kEmitThreads) emit_kernel(const uint32_t* __re
     if (bad) hdr->status = SLIMDP_ERR_INTERNAL;
 }
 
-inline slimdp_status launch_emit(const uint32_t* G, const uint32_t* E, const unsigned long long* tile_sum,
+inline slimdp_status launch_emit(const uint32_t* G, const uint32_t* E, const unsigned long long* cnt,
                                  const unsigned long long* super_pref, uint64_t n, uint32_t k, WsHeader* hdr,
                                  uint32_t* core_idx, uint32_t* bitmap, uint32_t* dir, cudaStream_t st) {
     const uint64_t nb = num_blocks(n);
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
-    // CTAs that are all resident at once (8 per SM) walk the tiles in turn
-    uint64_t grid = num_tiles(nb);
+    uint64_t grid = (nb + kEmitWarps - 1) / kEmitWarps;
     if (grid > (uint64_t)sms * 8) grid = (uint64_t)sms * 8;
-    emit_kernel<<<(unsigned)grid, kEmitThreads, 0, st>>>(G, E, tile_sum, super_pref, nb, k, hdr, core_idx,
-                                                                   bitmap, dir);
+    emit_kernel<<<(unsigned)grid, kEmitWarps * 32, 0, st>>>(G, E, cnt, super_pref, nb, k, hdr, core_idx, bitmap, dir);
     SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }
