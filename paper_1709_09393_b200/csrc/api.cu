@@ -14,7 +14,15 @@ namespace slimdp {
 slimdp_status launch_score(const float* w, const PtrArray<const float>& g, uint32_t K, float c, uint64_t n,
                            float* S, bool vec, cudaStream_t st);
 slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx, void* core_aux,
-                            void* ws, cudaStream_t st);
+                            void* ws, bool emit, cudaStream_t st);
+bool round_exchange_applies(uint64_t n, uint64_t k_exp);
+slimdp_status launch_round_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<const float>& delta,
+                                    uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp, float eta,
+                                    const PtrArray<float>& val, const PtrArray<float>& pulled, const uint32_t* ranks,
+                                    uint64_t rank_stride, int32_t* explore_status, const uint32_t* G,
+                                    const uint32_t* E, const unsigned long long* cnt,
+                                    const unsigned long long* super_pref, WsHeader* sel_hdr, uint32_t* core_idx,
+                                    uint32_t* core_bitmap, uint32_t* core_dir, cudaStream_t st);
 slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                              uint32_t first_worker, uint32_t workers, uint32_t round,
                              const PtrArray<uint32_t>& out, void* ws, cudaStream_t st);
@@ -46,7 +54,7 @@ slimdp_status launch_score_select(const float* w, const PtrArray<const float>& g
                                   float* scores, uint64_t k_core, uint32_t* core_idx, void* core_aux, void* ws,
                                   cudaEvent_t mark_begin, cudaEvent_t mark_end, slimdp_status (*after_pass)(void*),
                                   void* after_arg, cudaEvent_t pass_ready, void* stage, size_t stage_bytes,
-                                  bool* staged, cudaStream_t st);
+                                  bool* staged, bool emit, cudaStream_t st);
 
 slimdp_status launch_explore_static(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
                                     uint32_t worker, uint32_t round, uint32_t* exp_idx, int32_t* status_out,
@@ -100,6 +108,7 @@ int sm_count() {
 namespace {
 
 constexpr uint64_t kMaxN = 0xFFFFFFFFull;   // indices are uint32_t
+constexpr uint64_t kFoldedExchangeMaxN = 1ull << 23;   // slimdp_round: up to here the exchange also does the emit's work
 
 bool n_ok(uint64_t n) { return n >= 1 && n <= kMaxN; }
 bool k_ok(uint32_t K) { return K >= 1 && K <= SLIMDP_MAX_WORKERS; }
@@ -198,7 +207,7 @@ slimdp_status slimdp_select_core(const float* scores, uint64_t n, uint64_t k_cor
     if (!aligned4(scores) || !aligned16(core_aux) || !aligned16(ws) || (core_idx && !aligned4(core_idx)))
         return SLIMDP_ERR_INVALID_ARG;
     if (ws_bytes < slimdp_select_workspace_bytes(n)) return SLIMDP_ERR_WORKSPACE;
-    return launch_select(scores, n, k_core, core_idx, core_aux, ws, (cudaStream_t)stream);
+    return launch_select(scores, n, k_core, core_idx, core_aux, ws, true, (cudaStream_t)stream);
 }
 
 slimdp_status slimdp_sample_explore_batched(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp,
@@ -685,20 +694,25 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
         if (cudaEventRecord(s.done, s.rk) != cudaSuccess) return SLIMDP_ERR_CUDA;
         return r;
     };
-    // chain: the core, scored and selected in one pass where sizes and alignment allow
+    // chain: the core, scored and selected in one pass where sizes and alignment allow.  Short vectors
+    // are bound by the number of dependent launches: there the selection stops after its finishing
+    // kernel and the exchange places the core's members itself (one launch less).  On long vectors the
+    // separate emit kernel followed by the exchange over the finished index list is as fast or faster
+    // (measured: 138 M parameters 1.58 ms either way; 25.6 M parameters with 16 workers 1.10 against 1.18 ms).
     bool staged = false;
+    const bool folded = stage == nullptr && n < kFoldedExchangeMaxN && round_exchange_applies(n, k_exp);
     if (fusable) {
         rank_work.after = side->pass_ready;   // recorded by the call below just before its pass
         rank_work.lean = true;
         step(launch_score_select(w_global, g, K, c, n, scores, k_core, core_idx, core_aux, select_ws, mark0, mark1,
-                                 enqueue_ranks, &rank_work, side->pass_ready, stage, stage_bytes, &staged, ch));
+                                 enqueue_ranks, &rank_work, side->pass_ready, stage, stage_bytes, &staged, !folded, ch));
         // (if the call failed before it reached the hook, ranks_done keeps an earlier record: nothing to wait for)
     } else {
         step(enqueue_ranks(&rank_work));
         if (rc == SLIMDP_OK && mark0) cuda(cudaEventRecord(mark0, ch));
         if (rc == SLIMDP_OK) step(launch_score(w_global, g, K, c, n, scores, vec, ch));
         if (rc == SLIMDP_OK && mark1) cuda(cudaEventRecord(mark1, ch));
-        if (rc == SLIMDP_OK) step(launch_select(scores, n, k_core, core_idx, core_aux, select_ws, ch));
+        if (rc == SLIMDP_OK) step(launch_select(scores, n, k_core, core_idx, core_aux, select_ws, !folded, ch));
     }
     // chain: explorer indices from the sorted ranks and the core, then the exchange; where the
     // exchange's warp ranges line up with the core's directory it computes the indices itself
@@ -713,7 +727,14 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
         xs = ExchangeStage{A.fill, A.chunks, (uint32_t)A.max_chunks, SL.hdr, (uint32_t)SL.cand_cap};
     }
     const ExchangeStage* xsp = staged ? &xs : nullptr;
-    if (exchange_takes_ranks(n, k_exp)) {
+    if (folded) {
+        const SelectWs SL = select_ws_layout(select_ws, n);
+        const ExploreWs EL = explore_ws_layout(explore_ws, n, k_exp, K);
+        if (rc == SLIMDP_OK)
+            step(launch_round_exchange(w_global, n, K, g, k_core, exp_in, k_exp, eta, v, o, EL.rho, EL.rho_stride,
+                                       &EL.hdr->status, SL.G, SL.E, SL.tile_sum, SL.super_pref, SL.hdr, core_idx,
+                                       const_cast<uint32_t*>(aux_bitmap), const_cast<uint32_t*>(aux_dir), ch));
+    } else if (exchange_takes_ranks(n, k_exp)) {
         const ExploreWs EL = explore_ws_layout(explore_ws, n, k_exp, K);
         if (rc == SLIMDP_OK)
             step(launch_exchange(w_global, n, K, g, core_idx, k_core, exp_in, k_exp, eta, v, o, EL.rho, EL.rho_stride,

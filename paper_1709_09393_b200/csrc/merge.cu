@@ -15,6 +15,7 @@
 // range, so a parameter receives its updates in ascending k without atomics.
 #include "common.cuh"
 #include "layout.cuh"
+#include "select_dev.cuh"
 
 namespace slimdp {
 
@@ -166,35 +167,40 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_explore_kernel(float* 
 // back to all K workers (the pull).  One read of the key, K gathers, one read-modify-write.
 // The gathers ask for 64-byte fetches: where the core is dense both halves of a line are asked
 // for anyway, where it is thin (one member per line) half the line stays in DRAM.
+// One core parameter: i its index, j its place in the core.
+__device__ __forceinline__ void exchange_core_one(float* __restrict__ w, uint32_t i, uint64_t j,
+                                                  const PtrArray<const float>& delta, const PtrArray<float>& val,
+                                                  const PtrArray<float>& pulled, int K, float neg_eta) {
+    float x = ld_sparse(w + i);
+    int k = 0;
+    for (; k + 8 <= K; k += 8) {
+        float v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = ld_sparse(delta.p[k + q] + i);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            __stcs(val.p[k + q] + j, v[q]);
+            x = __fmaf_rn(neg_eta, v[q], x);
+        }
+    }
+    for (; k < K; ++k) {
+        const float v = ld_sparse(delta.p[k] + i);
+        __stcs(val.p[k] + j, v);
+        x = __fmaf_rn(neg_eta, v, x);
+    }
+    x = stored_model_value(x);
+    w[i] = x;
+#pragma unroll 8
+    for (int q = 0; q < K; ++q) __stcs(pulled.p[q] + j, x);
+}
+
 __device__ __forceinline__ void exchange_core_body(float* __restrict__ w, const uint32_t* __restrict__ core_idx,
                                                    uint64_t k_core, const PtrArray<const float>& delta,
                                                    const PtrArray<float>& val, const PtrArray<float>& pulled, int K,
                                                    float neg_eta, uint64_t vblock, uint64_t vgrid) {
     const uint64_t stride = vgrid * blockDim.x;
-    for (uint64_t j = vblock * blockDim.x + threadIdx.x; j < k_core; j += stride) {
-        const uint32_t i = __ldg(core_idx + j);
-        float x = ld_sparse(w + i);
-        int k = 0;
-        for (; k + 8 <= K; k += 8) {
-            float v[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = ld_sparse(delta.p[k + q] + i);
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                __stcs(val.p[k + q] + j, v[q]);
-                x = __fmaf_rn(neg_eta, v[q], x);
-            }
-        }
-        for (; k < K; ++k) {
-            const float v = ld_sparse(delta.p[k] + i);
-            __stcs(val.p[k] + j, v);
-            x = __fmaf_rn(neg_eta, v, x);
-        }
-        x = stored_model_value(x);
-        w[i] = x;
-#pragma unroll 8
-        for (int q = 0; q < K; ++q) __stcs(pulled.p[q] + j, x);
-    }
+    for (uint64_t j = vblock * blockDim.x + threadIdx.x; j < k_core; j += stride)
+        exchange_core_one(w, __ldg(core_idx + j), j, delta, val, pulled, K, neg_eta);
 }
 
 // Explorer segments: warp-owned ranges as in merge_explore_kernel.  Per worker, in ascending
@@ -263,6 +269,21 @@ __device__ __forceinline__ uint32_t lower_bound_ranks(const uint32_t* __restrict
     return lo;
 }
 
+// What a warp that owns a parameter range knows about it: lane l holds the range's l-th group of 64
+// parameters (dl = non-core parameters below the group, words = its two words of the core bitmap).
+struct RangeView {
+    uint32_t groups;    // groups in the range, 1 .. 32
+    uint32_t group0;    // the range's first group
+    uint32_t dl;        // 0xFFFFFFFF: this lane has no group
+    uint2 words;
+};
+
+__device__ __forceinline__ void explore_ranks_rest(float* w, const RankSource& src, const RangeView& rv,
+                                                   const PtrArray<const uint32_t>& exp, uint32_t k_exp,
+                                                   const PtrArray<const float>& delta, const PtrArray<float>& val,
+                                                   const PtrArray<float>& pulled, uint64_t k_core, int K,
+                                                   float neg_eta, uint32_t (*bound)[kMergeWarps + 1]);
+
 __device__ __forceinline__ void exchange_explore_ranks_body(float* w, const RankSource& src,
                                                             const PtrArray<const uint32_t>& exp, uint32_t k_exp,
                                                             const PtrArray<const float>& delta,
@@ -284,9 +305,24 @@ __device__ __forceinline__ void exchange_explore_ranks_body(float* w, const Rank
     // this warp's piece of the directory and of the bitmap: lane l holds group l of the range
     const uint64_t my_group = first_group + (uint64_t)wid * groups + lane;
     const bool have_group = lane < groups && my_group < src.nd;
-    const uint32_t dl = have_group ? __ldg(src.dir + my_group) : 0xFFFFFFFFu;
-    const uint2 words = have_group ? __ldg(reinterpret_cast<const uint2*>(src.bitmap) + my_group) : make_uint2(0u, 0u);
-    const uint32_t group0 = (uint32_t)(first_group + (uint64_t)wid * groups);
+    RangeView rv;
+    rv.groups = groups;
+    rv.group0 = (uint32_t)(first_group + (uint64_t)wid * groups);
+    rv.dl = have_group ? __ldg(src.dir + my_group) : 0xFFFFFFFFu;
+    rv.words = have_group ? __ldg(reinterpret_cast<const uint2*>(src.bitmap) + my_group) : make_uint2(0u, 0u);
+    explore_ranks_rest(w, src, rv, exp, k_exp, delta, val, pulled, k_core, K, neg_eta, bound);
+}
+
+__device__ __forceinline__ void explore_ranks_rest(float* w, const RankSource& src, const RangeView& rv,
+                                                   const PtrArray<const uint32_t>& exp, uint32_t k_exp,
+                                                   const PtrArray<const float>& delta, const PtrArray<float>& val,
+                                                   const PtrArray<float>& pulled, uint64_t k_core, int K,
+                                                   float neg_eta, uint32_t (*bound)[kMergeWarps + 1]) {
+    const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
+    const uint32_t groups = rv.groups;
+    const uint32_t dl = rv.dl;
+    const uint2 words = rv.words;
+    const uint32_t group0 = rv.group0;
     bool bad = false;
     // rank -> parameter index inside this warp's range; every lane takes part (shuffles), `ok` says
     // whether the lane's rank is real
@@ -489,6 +525,127 @@ __global__ void __launch_bounds__(256) exchange_kernel(float* w, const uint32_t*
     }
 }
 
+// ---- the one-call round's exchange: no emit before it ------------------------------------------
+//
+// After the selection's finishing kernel every warp can place a block's core members by itself
+// (block_selection: the "greater" / "equal" bitmaps, the per-block counts and their group prefixes).
+// Core CTAs own eight blocks spread over the vector, a warp per block: the warp writes the block's part of the
+// core bitmap and directory, lists the block's members in shared memory, and then takes them 32 at
+// a time through the push, the update and the pull (consecutive places in the core, so the value
+// stores are whole lines) and writes the index list as it goes.  Explorer CTAs work as in
+// exchange_explore_ranks_body, except that a warp derives its range's piece of the directory and
+// bitmap from the same sources instead of reading them: nothing here waits for an emit kernel.
+struct RoundSource {
+    const uint32_t* G;
+    const uint32_t* E;
+    const unsigned long long* cnt;
+    const unsigned long long* super_pref;
+    WsHeader* sel_hdr;
+    uint32_t* bitmap;     // written here (core CTAs)
+    uint32_t* dir;
+    uint32_t* core_idx;
+    uint64_t nb;
+    uint64_t n;
+};
+
+__device__ __forceinline__ void round_core_body(float* __restrict__ w, const RoundSource& rs, uint32_t ties,
+                                                uint64_t k_core, const PtrArray<const float>& delta,
+                                                const PtrArray<float>& val, const PtrArray<float>& pulled, int K,
+                                                float neg_eta, uint64_t cta, uint64_t core_ctas, uint16_t* list) {
+    const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
+    // the CTA's eight blocks lie an eighth of the vector apart: the core clusters in some layers, and this
+    // way every core CTA gets its share of the heavy blocks, all through the launch
+    const uint64_t blk = (uint64_t)wid * core_ctas + cta;
+    if (blk >= rs.nb) return;
+    uint32_t sel, pos0;
+    const uint32_t in_block = block_selection(rs.G, rs.E, rs.cnt, rs.super_pref, ties, blk, &sel, &pos0);
+    write_block_aux(rs.bitmap, rs.dir, blk, sel, pos0);
+    if (in_block == 0) return;
+    const uint32_t base = __shfl_sync(0xFFFFFFFFu, pos0, 0);   // core parameters below the block
+    uint16_t* mine = list + wid * kBlock;   // the members' offsets in the block, in index order
+    const uint32_t first = (uint32_t)(blk * kBlock);
+    uint32_t at = pos0 - base;
+    for (uint32_t word = sel; word; word &= word - 1, ++at)
+        if (at < kBlock) mine[at] = (uint16_t)(lane * 32u + (uint32_t)__ffs(word) - 1u);
+    __syncwarp();
+    for (uint32_t e = lane; e < in_block; e += 32) {
+        const uint64_t j = (uint64_t)base + e;
+        if (j >= k_core) {
+            rs.sel_hdr->status = SLIMDP_ERR_INTERNAL;
+            continue;
+        }
+        const uint32_t i = first + mine[e];
+        rs.core_idx[j] = i;
+        exchange_core_one(w, i, j, delta, val, pulled, K, neg_eta);
+    }
+}
+
+__device__ __forceinline__ void round_explore_body(float* w, const RankSource& src, const RoundSource& rs,
+                                                   uint32_t ties, const PtrArray<const uint32_t>& exp, uint32_t k_exp,
+                                                   const PtrArray<const float>& delta, const PtrArray<float>& val,
+                                                   const PtrArray<float>& pulled, uint64_t k_core, int K,
+                                                   float neg_eta, uint32_t range_shift, uint64_t vblock,
+                                                   uint32_t (*bound)[kMergeWarps + 1], uint32_t* range_lo) {
+    const uint32_t wid = threadIdx.x >> 5, lane = lane_id();
+    const uint32_t groups = 1u << (range_shift - 6);   // 64-parameter groups per warp range, 1 .. 32
+    const uint64_t group0 = ((vblock * kMergeWarps + wid) << (range_shift - 6));   // this warp's first group
+    const uint64_t nd = rs.nb * kDirPerBlock;
+    const uint32_t all_noncore = (uint32_t)(rs.n - k_core);
+    // the block(s) that hold the range (two only for ranges of 2048 parameters)
+    const uint64_t blkA = group0 / kDirPerBlock;
+    uint32_t selA = 0, posA = 0, selB = 0, posB = 0;
+    if (blkA < rs.nb) block_selection(rs.G, rs.E, rs.cnt, rs.super_pref, ties, blkA, &selA, &posA);
+    if (groups > kDirPerBlock && blkA + 1 < rs.nb)
+        block_selection(rs.G, rs.E, rs.cnt, rs.super_pref, ties, blkA + 1, &selB, &posB);
+    // lane l takes group l of the range: its two words and the core parameters below it
+    const uint64_t my_group = group0 + lane;
+    const uint32_t in_blk = (uint32_t)(my_group % kDirPerBlock) * 2u;   // first word of the group in its block
+    const bool second = my_group / kDirPerBlock != blkA;
+    const uint32_t a0 = __shfl_sync(0xFFFFFFFFu, selA, in_blk), a1 = __shfl_sync(0xFFFFFFFFu, selA, in_blk + 1);
+    const uint32_t b0 = __shfl_sync(0xFFFFFFFFu, selB, in_blk), b1 = __shfl_sync(0xFFFFFFFFu, selB, in_blk + 1);
+    const uint32_t pa = __shfl_sync(0xFFFFFFFFu, posA, in_blk), pb = __shfl_sync(0xFFFFFFFFu, posB, in_blk);
+    const bool have_group = lane < groups && my_group < nd;
+    RangeView rv;
+    rv.groups = groups;
+    rv.group0 = (uint32_t)group0;
+    rv.words = have_group ? make_uint2(second ? b0 : a0, second ? b1 : a1) : make_uint2(0u, 0u);
+    rv.dl = have_group ? (uint32_t)(my_group * 64u) - (second ? pb : pa) : 0xFFFFFFFFu;
+    // non-core parameters below the range's first parameter, and below the CTA's last one
+    if (lane == 0) range_lo[wid] = have_group ? rv.dl : all_noncore;
+    if (wid == kMergeWarps - 1 && lane == groups - 1)
+        range_lo[kMergeWarps] =
+            have_group ? rv.dl + 64u - (uint32_t)__popc(rv.words.x) - (uint32_t)__popc(rv.words.y) : all_noncore;
+    __syncthreads();
+    // where the CTA's 9 range boundaries fall in every worker's sorted ranks
+    for (int t = threadIdx.x; t < K * (kMergeWarps + 1); t += blockDim.x) {
+        const int k = t / (kMergeWarps + 1), r = t % (kMergeWarps + 1);
+        bound[k][r] = lower_bound_ranks(src.ranks + (uint64_t)k * src.stride, k_exp, range_lo[r]);
+    }
+    __syncthreads();
+    explore_ranks_rest(w, src, rv, exp, k_exp, delta, val, pulled, k_core, K, neg_eta, bound);
+}
+
+__global__ void __launch_bounds__(256) round_exchange_kernel(float* w, uint64_t k_core, PtrArray<const uint32_t> exp,
+                                                             uint32_t k_exp, PtrArray<const float> delta,
+                                                             PtrArray<float> val, PtrArray<float> pulled, int K,
+                                                             float neg_eta, uint32_t range_shift, uint64_t core_ctas,
+                                                             uint64_t total_ctas, RankSource from_ranks,
+                                                             RoundSource rs) {
+    __shared__ uint32_t bound[SLIMDP_MAX_WORKERS][kMergeWarps + 1];
+    __shared__ uint32_t range_lo[kMergeWarps + 1];
+    __shared__ uint16_t list[kMergeWarps * kBlock];
+    if (rs.sel_hdr->abort != 0u) return;   // the finishing kernel gave up (its status word says so)
+    const uint32_t ties = rs.sel_hdr->tie_quota;
+    const uint64_t b = blockIdx.x;
+    const uint64_t core_before = b * core_ctas / total_ctas;            // core CTAs among blocks [0, b)
+    const bool is_core = (b + 1) * core_ctas / total_ctas > core_before;
+    if (is_core)
+        round_core_body(w, rs, ties, k_core, delta, val, pulled, K, neg_eta, core_before, core_ctas, list);
+    else
+        round_explore_body(w, from_ranks, rs, ties, exp, k_exp, delta, val, pulled, k_core, K, neg_eta, range_shift,
+                           b - core_before, bound, range_lo);
+}
+
 // Range per warp: a power of two with 16 to 32 entries per worker on average, at least 32 parameters.
 uint32_t explore_range_shift(uint64_t n, uint64_t k_exp) {
     uint32_t shift = 5;
@@ -585,6 +742,36 @@ slimdp_status launch_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<c
     }
     exchange_kernel<<<(unsigned)total, 256, 0, st>>>(w, core_idx, k_core, exp, (uint32_t)k_exp, delta, val, pulled,
                                                      (int)K, -eta, shift, core_ctas, total, gather_ctas, src, staged);
+    SLIMDP_LAUNCHED(1);
+    return SLIMDP_OK;
+}
+
+// Whether slimdp_round can hand the selection's bitmaps and counts straight to the exchange (no emit
+// kernel, no separate explorer-index step): the explorers' warp ranges must line up with the directory.
+bool round_exchange_applies(uint64_t n, uint64_t k_exp) { return k_exp == 0 || exchange_takes_ranks(n, k_exp); }
+
+slimdp_status launch_round_exchange(float* w, uint64_t n, uint32_t K, const PtrArray<const float>& delta,
+                                    uint64_t k_core, const PtrArray<const uint32_t>& exp, uint64_t k_exp, float eta,
+                                    const PtrArray<float>& val, const PtrArray<float>& pulled, const uint32_t* ranks,
+                                    uint64_t rank_stride, int32_t* explore_status, const uint32_t* G,
+                                    const uint32_t* E, const unsigned long long* cnt,
+                                    const unsigned long long* super_pref, WsHeader* sel_hdr, uint32_t* core_idx,
+                                    uint32_t* core_bitmap, uint32_t* core_dir, cudaStream_t st) {
+    if (!round_exchange_applies(n, k_exp)) return SLIMDP_ERR_INTERNAL;
+    const uint64_t nb = num_blocks(n);
+    const uint64_t core_ctas = (nb + kMergeWarps - 1) / kMergeWarps;
+    uint64_t explore_ctas = 0;
+    uint32_t shift = 6;
+    if (k_exp > 0) {
+        shift = explore_range_shift(n, k_exp);
+        const uint64_t per_cta = (uint64_t)kMergeWarps << shift;
+        explore_ctas = (n + per_cta - 1) / per_cta;
+    }
+    const uint64_t total = core_ctas + explore_ctas;
+    const RankSource src{ranks, rank_stride, core_bitmap, core_dir, (uint32_t)(nb * kDirPerBlock), explore_status};
+    const RoundSource rs{G, E, cnt, super_pref, sel_hdr, core_bitmap, core_dir, core_idx, nb, n};
+    round_exchange_kernel<<<(unsigned)total, 256, 0, st>>>(w, k_core, exp, (uint32_t)k_exp, delta, val, pulled, (int)K,
+                                                           -eta, shift, core_ctas, total, src, rs);
     SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
 }

@@ -1008,9 +1008,11 @@ struct GivenThreshold {
     uint32_t T, ties;
 };
 
+// emit = false: the call ends with the finishing kernel; the caller places the core's members itself
+// (block_selection on the workspace's bitmaps and counts) and writes core_idx and core_aux.
 static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx,
                                         void* core_aux, void* ws, const FusedScore* fused, bool* staged_out,
-                                        const GivenThreshold* given, cudaStream_t st) {
+                                        const GivenThreshold* given, bool emit, cudaStream_t st) {
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
     const SelectWs L = select_ws_layout(ws, n);
@@ -1151,20 +1153,22 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
                                     dim3(kFinishThreads), args, 0, st) != cudaSuccess)
         return SLIMDP_ERR_CUDA;
     SLIMDP_LAUNCHED(1);
+    if (!emit) return SLIMDP_OK;
     return launch_emit(L.G, L.E, L.tile_sum, L.super_pref, n, k, L.hdr, core_idx, bitmap, dir, st);
 }
 
 slimdp_status launch_select(const float* scores, uint64_t n, uint64_t k_core, uint32_t* core_idx, void* core_aux,
-                            void* ws, cudaStream_t st) {
+                            void* ws, bool emit, cudaStream_t st) {
     return launch_select_impl(const_cast<float*>(scores), n, k_core, core_idx, core_aux, ws, nullptr, nullptr, nullptr,
-                              st);
+                              emit, st);
 }
 
 // A shard's part of the core for a threshold and a tie quota that were found over all shards.
 slimdp_status launch_select_given(const float* scores, uint64_t n, uint32_t T, uint32_t ties, uint64_t k_shard,
                                   uint32_t* core_idx, void* core_aux, void* ws, cudaStream_t st) {
     const GivenThreshold gt{T, ties};
-    return launch_select_impl(const_cast<float*>(scores), n, k_shard, core_idx, core_aux, ws, nullptr, nullptr, &gt, st);
+    return launch_select_impl(const_cast<float*>(scores), n, k_shard, core_idx, core_aux, ws, nullptr, nullptr, &gt, true,
+                              st);
 }
 
 // Whether scoring can be folded into the selection for these sizes and alignments.
@@ -1184,9 +1188,9 @@ slimdp_status launch_score_select(const float* w, const PtrArray<const float>& g
                                   float* scores, uint64_t k_core, uint32_t* core_idx, void* core_aux, void* ws,
                                   cudaEvent_t mark_begin, cudaEvent_t mark_end, slimdp_status (*after_pass)(void*),
                                   void* after_arg, cudaEvent_t pass_ready, void* stage, size_t stage_bytes,
-                                  bool* staged, cudaStream_t st) {
+                                  bool* staged, bool emit, cudaStream_t st) {
     const FusedScore f{w, &g, K, c, mark_begin, mark_end, after_pass, after_arg, pass_ready, stage, stage_bytes};
-    return launch_select_impl(scores, n, k_core, core_idx, core_aux, ws, &f, staged, nullptr, st);
+    return launch_select_impl(scores, n, k_core, core_idx, core_aux, ws, &f, staged, nullptr, emit, st);
 }
 
 }  // namespace slimdp
