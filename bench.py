@@ -373,6 +373,8 @@ def run_ours(args):
     from workloads import CONFIGS, all_inputs
 
     cfg = CONFIGS[args.config]
+    if args.core_pct:
+        cfg = cfg.with_core_pct(args.core_pct)   # another point of the core-ratio sweep
     if args.scale:
         from workloads import scaled_config
         cfg = scaled_config(cfg, args.scale)     # leading parameters only: a small case for profiling
@@ -601,6 +603,7 @@ def main():
                     help="give slimdp_round its optional staging area (the exchange then streams the core's values)")
     ap.add_argument("--timeline", default="",
                     help="also write the kernel timeline of three extra rounds (start, duration, stream) to this file")
+    ap.add_argument("--core-pct", type=int, default=0, help="core ratio in percent (default: the config's own)")
     ap.add_argument("--scale", type=int, default=0,
                     help="run on the leading SCALE parameters of the config (small case for profiler captures)")
     args = ap.parse_args()

@@ -16,19 +16,21 @@
 //      inside the bracket are copied, with their indices, to a candidate list
 //      and counted by the top 12 bits of their offset in the bracket; the
 //      pass's last CTA finds the 12-bit bin that holds T;
-//   3. the finishing kernel (one cooperative launch, one CTA per SM, phases
+//   3. the finishing kernel (one cooperative launch, two CTAs per SM, phases
 //      separated by a grid barrier): if the counts prove the bracket right
 //      (n_def < k <= n_def + n_cand, list not overflowed) it resolves the
 //      remaining low bits of T from the candidates alone (at most two more
 //      counting rounds) and adds the candidates >= T to the "greater" /
-//      "equal" bitmaps; otherwise (one score value repeated millions of times,
-//      a defeated sample, small inputs) it takes the full path: three
-//      most-significant-digit-first counting rounds over all keys
-//      (12 + 10 + 10 bits) and one classifying round that writes both bitmaps.
-//      Either way it ends with a scan over all bitmap words that admits the
-//      first r equal keys in index order and writes the core bitmap, the
-//      non-core rank directory and the ascending index list (ordered
-//      compaction, no atomic cursors).
+//      "equal" bitmaps and to the per-block counts; otherwise (one score value
+//      repeated millions of times, a defeated sample, small inputs) it takes the
+//      full path: three most-significant-digit-first counting rounds over all
+//      keys (12 + 10 + 10 bits) and one classifying round that writes both
+//      bitmaps and the counts.  Either way it ends by turning the per-block
+//      counts into prefixes per group of 64 blocks;
+//   4. the emit kernel (select_dev.cuh; a warp per 1024-parameter block, no
+//      waiting between warps): admits the first r equal keys in index order
+//      and writes the core bitmap, the non-core rank directory and the
+//      ascending index list (ordered compaction, no atomic cursors).
 // Every wait of the grid barrier is bounded: if it runs out the kernel records
 // SLIMDP_ERR_INTERNAL in the workspace header and every CTA returns.
 #include <atomic>
