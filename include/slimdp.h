@@ -358,7 +358,26 @@ slimdp_status slimdp_merge_q8(float* w_global, uint64_t n, uint32_t K, const uin
  *           uint64 remaining rank (after round 2: r)
  *   hist    DEVICE uint64[4096] (rounds 1 and 2 use the first 1024), added to
  *   counts  DEVICE uint64[2], added to
- *   scores  the shard's scores [n_shard] (n_shard may be 0 in hist / count) */
+ *   scores  the shard's scores [n_shard] (n_shard may be 0 in hist / count)
+ * With the core in place, pack, merge and pull run per shard on shard-local indices as they are.
+ * slimdp_sample_explore_shard: one shard's share of a worker's explorer (Section 3.3 step 2 on the
+ *   sharded model).  The explorer is drawn over the non-core parameters of ALL shards, numbered in index
+ *   order: every shard evaluates the same noncore_total-rank permutation prefix (the generator of
+ *   slimdp_sample_explore with M = noncore_total) and keeps the ranks of its own non-core parameters,
+ *   [noncore_below, noncore_below + n_shard - k_core_shard), as shard-local indices.  The shards'
+ *   lists, each shifted by its shard's offset and concatenated, are bit for bit the explorer that
+ *   slimdp_sample_explore draws on the whole vector.  noncore_below and noncore_total come from the
+ *   all-gather of the shards' core sizes.
+ *   core_aux   the shard's, as written by slimdp_select_emit
+ *   exp_idx    [cap] (written: *count entries, ascending); count: DEVICE uint32 (written)
+ *   If the shard's share exceeds cap nothing is written, *count = 0 and the workspace's status word
+ *   is set (slimdp_read_status).  noncore_total < 2^32.
+ *   ws         [ws_bytes >= slimdp_explore_shard_workspace_bytes(n_shard, noncore_total, k_exp)] */
+size_t slimdp_explore_shard_workspace_bytes(uint64_t n_shard, uint64_t noncore_total, uint64_t k_exp);
+slimdp_status slimdp_sample_explore_shard(const void* core_aux, uint64_t n_shard, uint64_t k_core_shard,
+                                          uint64_t noncore_total, uint64_t noncore_below, uint64_t k_exp,
+                                          uint64_t seed, uint32_t worker, uint32_t round, uint32_t* exp_idx,
+                                          uint64_t cap, uint32_t* count, void* ws, size_t ws_bytes, void* stream);
 slimdp_status slimdp_select_shard_begin(uint64_t k_total, void* state, void* stream);
 slimdp_status slimdp_select_hist(const float* scores, uint64_t n_shard, uint32_t round, const void* state,
                                  uint64_t* hist, void* stream);

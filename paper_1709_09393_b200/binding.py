@@ -55,6 +55,9 @@ EXPORTS = {
     "slimdp_select_core_segmented": (ctypes.c_int32, [_vp, _u64, _vp, _vp, _u32, _vp, _vp, _vp, _sz, _vp]),
     "slimdp_pack_q8_batched": (ctypes.c_int32, [_pp, _u32, _u64, _vp, _u64, _pp, _u64, _pp, _pp, _vp]),
     "slimdp_merge_q8": (ctypes.c_int32, [_vp, _u64, _u32, _vp, _u64, _pp, _u64, _pp, _pp, _f32, _vp]),
+    "slimdp_explore_shard_workspace_bytes": (_sz, [_u64, _u64, _u64]),
+    "slimdp_sample_explore_shard": (ctypes.c_int32, [_vp, _u64, _u64, _u64, _u64, _u64, _u64, _u32, _u32, _vp, _u64, _vp,
+                                                     _vp, _sz, _vp]),
     "slimdp_select_shard_begin": (ctypes.c_int32, [_u64, _vp, _vp]),
     "slimdp_select_hist": (ctypes.c_int32, [_vp, _u64, _u32, _vp, _vp, _vp]),
     "slimdp_select_resolve": (ctypes.c_int32, [_vp, _u32, _vp, _vp]),
@@ -462,6 +465,22 @@ def slimdp_merge_q8(w_global: torch.Tensor, core_idx: torch.Tensor, exp_idx: Seq
            lib.slimdp_merge_q8(w_global.data_ptr(), w_global.numel(), K, _ptr(core_idx), core_idx.numel(),
                                _ptr_array(exp_idx), exp_idx[0].numel(), _ptr_array(codes), _ptr_array(scales), eta,
                                _stream(stream)))
+
+
+def explore_shard_workspace_bytes(n_shard: int, noncore_total: int, k_exp: int) -> int:
+    return lib.slimdp_explore_shard_workspace_bytes(n_shard, noncore_total, k_exp)
+
+
+def slimdp_sample_explore_shard(core_aux: torch.Tensor, n_shard: int, k_core_shard: int, noncore_total: int,
+                                noncore_below: int, k_exp: int, seed: int, worker: int, rnd: int,
+                                exp_idx: torch.Tensor, count: torch.Tensor, ws: torch.Tensor, stream=None):
+    """One shard's share of a worker's explorer: count[0] shard-local indices into exp_idx (its length is the cap)."""
+    _dev(exp_idx, IDX, "exp_idx")
+    _dev(count, torch.int32, "count")
+    _check("slimdp_sample_explore_shard",
+           lib.slimdp_sample_explore_shard(core_aux.data_ptr(), n_shard, k_core_shard, noncore_total, noncore_below,
+                                           k_exp, seed, worker, rnd, _ptr(exp_idx), exp_idx.numel(), count.data_ptr(),
+                                           ws.data_ptr(), ws.numel(), _stream(stream)))
 
 
 def slimdp_select_shard_begin(k_total: int, state: torch.Tensor, stream=None):

@@ -79,6 +79,11 @@ slimdp_status launch_merge_q8(float* w, uint64_t n, uint32_t K, const uint32_t* 
                               cudaStream_t st);
 slimdp_status launch_select_given(const float* scores, uint64_t n, uint32_t T, uint32_t ties, uint64_t k_shard,
                                   uint32_t* core_idx, void* core_aux, void* ws, cudaStream_t st);
+slimdp_status launch_explore_shard(const void* core_aux, uint64_t n_shard, uint64_t k_core_shard,
+                                   uint64_t noncore_total, uint64_t noncore_below, uint64_t k_exp, uint64_t seed,
+                                   uint32_t worker, uint32_t round, uint32_t* exp_idx, uint64_t cap, uint32_t* count,
+                                   void* ws, cudaStream_t st);
+size_t explore_shard_ws_bytes(uint64_t n_shard, uint64_t noncore_total, uint64_t k_exp);
 slimdp_status launch_shard_state_init(void* state, uint64_t k, cudaStream_t st);
 slimdp_status launch_shard_hist(const float* scores, uint64_t n, uint32_t round, const void* state, uint64_t* hist,
                                 cudaStream_t st);
@@ -419,6 +424,26 @@ slimdp_status slimdp_merge_q8(float* w_global, uint64_t n, uint32_t K, const uin
 }
 
 // ---- selection over a range-sharded model ---------------------------------
+
+size_t slimdp_explore_shard_workspace_bytes(uint64_t n_shard, uint64_t noncore_total, uint64_t k_exp) {
+    if (!n_ok(n_shard) || noncore_total > kMaxN || k_exp > noncore_total) return 0;
+    return explore_shard_ws_bytes(n_shard, noncore_total, k_exp);
+}
+
+slimdp_status slimdp_sample_explore_shard(const void* core_aux, uint64_t n_shard, uint64_t k_core_shard,
+                                          uint64_t noncore_total, uint64_t noncore_below, uint64_t k_exp,
+                                          uint64_t seed, uint32_t worker, uint32_t round, uint32_t* exp_idx,
+                                          uint64_t cap, uint32_t* count, void* ws, size_t ws_bytes, void* stream) {
+    if (!n_ok(n_shard) || k_core_shard > n_shard || noncore_total > kMaxN || k_exp > noncore_total || !core_aux ||
+        !count || !ws)
+        return SLIMDP_ERR_INVALID_ARG;
+    if (noncore_below + (n_shard - k_core_shard) > noncore_total) return SLIMDP_ERR_INVALID_ARG;
+    if (!aligned16(core_aux) || !aligned16(ws) || !aligned4(count)) return SLIMDP_ERR_INVALID_ARG;
+    if (cap > 0 && (!exp_idx || !aligned4(exp_idx))) return SLIMDP_ERR_INVALID_ARG;
+    if (ws_bytes < slimdp_explore_shard_workspace_bytes(n_shard, noncore_total, k_exp)) return SLIMDP_ERR_WORKSPACE;
+    return launch_explore_shard(core_aux, n_shard, k_core_shard, noncore_total, noncore_below, k_exp, seed, worker,
+                                round, exp_idx, cap, count, ws, (cudaStream_t)stream);
+}
 
 slimdp_status slimdp_select_shard_begin(uint64_t k_total, void* state, void* stream) {
     if (!state || (reinterpret_cast<uintptr_t>(state) & 7u) != 0) return SLIMDP_ERR_INVALID_ARG;

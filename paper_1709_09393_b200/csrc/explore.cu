@@ -385,23 +385,31 @@ __global__ void __launch_bounds__(kSelThreads, 5) select0_kernel(const uint32_t*
                                                                  uint32_t cells, uint32_t k_exp,
                                                                  const uint32_t* __restrict__ ranks,
                                                                  uint64_t rho_stride, PtrArray<uint32_t> out,
-                                                                 WsHeader* hdr) {
+                                                                 WsHeader* hdr, const uint32_t* __restrict__ window,
+                                                                 uint32_t rank0) {
     __shared__ uint32_t dir_sh[kDirCache + 1];
     __shared__ uint32_t grp_bounds[2];
     const uint32_t worker = blockIdx.y, t = threadIdx.x;
+    // window (a shard's piece of the sorted ranks): positions [window[0], window[1]) of the row, whose ranks
+    // count from rank0; without it the whole row
+    uint32_t first = 0, count = k_exp;
+    if (window != nullptr) {
+        first = window[0];
+        count = window[1] - first;
+    }
     const uint32_t tile0 = blockIdx.x * kSelTile;
-    if (tile0 >= k_exp) return;
-    const uint32_t m = (k_exp - tile0 < kSelTile) ? k_exp - tile0 : kSelTile;
-    const uint32_t* src = ranks + (uint64_t)worker * rho_stride + tile0;
+    if (tile0 >= count) return;
+    const uint32_t m = (count - tile0 < kSelTile) ? count - tile0 : kSelTile;
+    const uint32_t* src = ranks + (uint64_t)worker * rho_stride + first + tile0;
     uint32_t* dst = out.p[worker] + tile0;
     if (t < 2) {   // the group of the first cell the tile touches, and of the cell after its last
-        const uint32_t cell = (__ldg(src + (t ? m - 1u : 0u)) >> kCellShift) + t;
+        const uint32_t cell = ((__ldg(src + (t ? m - 1u : 0u)) - rank0) >> kCellShift) + t;
         grp_bounds[t] = __ldg(cell_group + (cell < cells ? cell : cells));
     }
     // this thread's ranks (the row is 256-byte aligned and tile0, kSelPer are multiples of 4)
     const uint32_t e0 = t * kSelPer;
     uint32_t rank[kSelPer];
-    if (e0 + kSelPer <= m) {
+    if (window == nullptr && e0 + kSelPer <= m) {
 #pragma unroll
         for (uint32_t q = 0; q < kSelPer; q += 4) {
             const uint4 v = __ldg(reinterpret_cast<const uint4*>(src + e0 + q));
@@ -412,7 +420,7 @@ __global__ void __launch_bounds__(kSelThreads, 5) select0_kernel(const uint32_t*
         }
     } else {
 #pragma unroll
-        for (uint32_t q = 0; q < kSelPer; ++q) rank[q] = (e0 + q < m) ? __ldg(src + e0 + q) : 0u;
+        for (uint32_t q = 0; q < kSelPer; ++q) rank[q] = (e0 + q < m) ? __ldg(src + e0 + q) - rank0 : 0u;
     }
     __syncthreads();
     const uint32_t grp_lo = grp_bounds[0], grp_hi = grp_bounds[1];
@@ -619,9 +627,96 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
     if (tgrid > (uint64_t)sms * 8) tgrid = (uint64_t)sms * 8;
     cell_table_kernel<<<(unsigned)tgrid, 256, 0, st>>>(dir, (uint32_t)nd, cells, L.cell_group);
     select0_kernel<<<dim3((unsigned)((k_exp + kSelTile - 1) / kSelTile), workers), kSelThreads, 0, st>>>(
-        bitmap, dir, (uint32_t)nd, L.cell_group, cells, (uint32_t)k_exp, L.rho, L.rho_stride, out, L.hdr);
+        bitmap, dir, (uint32_t)nd, L.cell_group, cells, (uint32_t)k_exp, L.rho, L.rho_stride, out, L.hdr, nullptr, 0u);
     SLIMDP_LAUNCHED(2);
     return SLIMDP_OK;
+}
+
+namespace {
+
+// window[0], window[1]: where the ranks in [rank_lo, rank_hi) sit in the sorted row; *count = how many they
+// are, or 0 with the status word set if they do not fit `cap`.
+__global__ void rank_window_kernel(const uint32_t* __restrict__ ranks, uint32_t k_exp, uint32_t rank_lo,
+                                   unsigned long long rank_hi, unsigned long long cap, uint32_t* window,
+                                   uint32_t* count, WsHeader* hdr) {
+    uint32_t lo = 0, hi = k_exp;
+    while (lo < hi) {   // first position with rank >= rank_lo
+        const uint32_t mid = lo + ((hi - lo) >> 1);
+        if (ranks[mid] < rank_lo)
+            lo = mid + 1;
+        else
+            hi = mid;
+    }
+    const uint32_t a = lo;
+    hi = k_exp;
+    while (lo < hi) {   // first position with rank >= rank_hi
+        const uint32_t mid = lo + ((hi - lo) >> 1);
+        if ((unsigned long long)ranks[mid] < rank_hi)
+            lo = mid + 1;
+        else
+            hi = mid;
+    }
+    uint32_t b = lo;
+    if ((unsigned long long)(b - a) > cap) {
+        hdr->status = SLIMDP_ERR_INTERNAL;   // the caller's list is too short for this shard's share
+        b = a;
+    }
+    window[0] = a;
+    window[1] = b;
+    *count = b - a;
+}
+
+}  // namespace
+
+// One shard's share of a worker's explorer (see slimdp_sample_explore_shard).  The ranks are drawn and
+// sorted over ALL shards' non-core parameters (every shard computes the same row); the shard keeps the
+// ranks of its own non-core parameters, [noncore_below, noncore_below + n_shard - k_core_shard), and turns
+// them into shard-local indices with its own bitmap and directory.
+slimdp_status launch_explore_shard(const void* core_aux, uint64_t n_shard, uint64_t k_core_shard,
+                                   uint64_t noncore_total, uint64_t noncore_below, uint64_t k_exp, uint64_t seed,
+                                   uint32_t worker, uint32_t round, uint32_t* exp_idx, uint64_t cap, uint32_t* count,
+                                   void* ws, cudaStream_t st) {
+    const int sms = sm_count();
+    if (sms <= 0) return SLIMDP_ERR_CUDA;
+    const uint64_t n_layout = noncore_total > n_shard ? noncore_total : n_shard;
+    const ExploreWs L = explore_ws_layout(ws, n_layout, k_exp, 1);
+    uint32_t* window = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + L.bytes);   // 2 words after the layout
+    PtrArray<uint32_t> out;
+    for (auto& q : out.p) q = nullptr;
+    out.p[0] = exp_idx;
+    if (k_exp == 0) {
+        if (cudaMemsetAsync(L.hdr, 0, sizeof(int32_t), st) != cudaSuccess ||
+            cudaMemsetAsync(count, 0, sizeof(uint32_t), st) != cudaSuccess)
+            return SLIMDP_ERR_CUDA;
+        return SLIMDP_OK;
+    }
+    // the sorted ranks of the whole model's explorer: a vector of n_layout parameters with noncore_total of them outside the core
+    slimdp_status rc = launch_explore_parts(core_aux, n_layout, n_layout - noncore_total, k_exp, seed, worker, 1, round,
+                                            out, ws, 1, false, st);
+    if (rc != SLIMDP_OK) return rc;
+    const uint64_t m_shard = n_shard - k_core_shard;
+    rank_window_kernel<<<1, 1, 0, st>>>(L.rho, (uint32_t)k_exp, (uint32_t)noncore_below, noncore_below + m_shard, cap,
+                                        window, count, L.hdr);
+    const uint64_t nd = num_blocks(n_shard) * kDirPerBlock;
+    const uint32_t* bitmap = reinterpret_cast<const uint32_t*>(core_aux);
+    const uint32_t* dir =
+        reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(core_aux) + slimdp_core_aux_dir_offset(n_shard));
+    const uint32_t cells = (uint32_t)((m_shard + (1u << kCellShift) - 1) >> kCellShift);
+    uint64_t tgrid = (nd + 255) / 256;
+    if (tgrid > (uint64_t)sms * 8) tgrid = (uint64_t)sms * 8;
+    cell_table_kernel<<<(unsigned)tgrid, 256, 0, st>>>(dir, (uint32_t)nd, cells, L.cell_group);
+    // the grid covers the most ranks the shard can get; CTAs beyond its share return at once
+    const uint64_t most = (k_exp < m_shard ? k_exp : m_shard);
+    select0_kernel<<<dim3((unsigned)((most + kSelTile - 1) / kSelTile + 1), 1), kSelThreads, 0, st>>>(
+        bitmap, dir, (uint32_t)nd, L.cell_group, cells, (uint32_t)k_exp, L.rho, L.rho_stride, out, L.hdr, window,
+        (uint32_t)noncore_below);
+    SLIMDP_LAUNCHED(3);
+    return SLIMDP_OK;
+}
+
+size_t explore_shard_ws_bytes(uint64_t n_shard, uint64_t noncore_total, uint64_t k_exp) {
+    const uint64_t n_layout = noncore_total > n_shard ? noncore_total : n_shard;
+    return explore_ws_layout(nullptr, n_layout, k_exp, 1).bytes + 256;
 }
 
 slimdp_status launch_explore(const void* core_aux, uint64_t n, uint64_t k_core, uint64_t k_exp, uint64_t seed,
