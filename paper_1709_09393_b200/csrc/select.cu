@@ -834,10 +834,21 @@ __global__ void __launch_bounds__(kFinishThreads, 2) finish_kernel(FinishArgs a)
             uint32_t* hist = a.hist + (4 + round) * kBins0;
             for (uint32_t b = t; b < kDigitBins; b += kFinishThreads) sh[b] = 0;
             __syncthreads();
-            for (uint32_t c = gid; c < n_cand; c += gstride) {
-                const uint32_t rel = __ldcg(a.cand_key + c) - bot_key;
+            // (the list is long on long flat vectors: four keys per load, two loads in flight per thread)
+            auto count = [&](uint32_t key) {
+                const uint32_t rel = key - bot_key;
                 if ((rel >> low) == (prefix >> low)) atomicAdd(&sh[(rel >> shift) & ((1u << d) - 1u)], 1u);
+            };
+            const uint32_t n4 = n_cand / 4;
+            const uint4* key4 = reinterpret_cast<const uint4*>(a.cand_key);
+            for (uint32_t c = gid; c < n4; c += 2 * gstride) {
+                const uint4 v0 = __ldcg(key4 + c);
+                const bool two = c + gstride < n4;
+                const uint4 v1 = two ? __ldcg(key4 + c + gstride) : make_uint4(0u, 0u, 0u, 0u);
+                count(v0.x), count(v0.y), count(v0.z), count(v0.w);
+                if (two) count(v1.x), count(v1.y), count(v1.z), count(v1.w);
             }
+            if (gid < n_cand - 4 * n4) count(__ldcg(a.cand_key + 4 * n4 + gid));
             __syncthreads();
             for (uint32_t b = t; b < (1u << d); b += kFinishThreads)
                 if (sh[b]) atomicAdd(&hist[b], sh[b]);
@@ -858,18 +869,31 @@ __global__ void __launch_bounds__(kFinishThreads, 2) finish_kernel(FinishArgs a)
             // candidates at or above T into the bitmaps and the tile counts
             // (neighbours in the list come from neighbouring parameters: a warp adds to a tile's
             // counter once, not once per candidate)
-            for (uint32_t c0 = gid - lane; c0 < n_cand; c0 += gstride) {
-                const uint32_t c = c0 + lane;
-                const uint32_t key = (c < n_cand) ? __ldcg(a.cand_key + c) : 0u;
-                const bool take = c < n_cand && key >= T;
-                const uint32_t i = take ? __ldcg(a.cand_idx + c) : 0xFFFFFFFFu;
-                if (take) atomicOr(((key > T) ? a.G : a.E) + (i >> 5), 1u << (i & 31u));
-                const uint32_t tile = take ? i / (kBlock * kEmitTile) : 0xFFFFFFFFu;
-                const uint32_t peers = __match_any_sync(0xFFFFFFFFu, tile);
-                const uint32_t gt = __ballot_sync(0xFFFFFFFFu, take && key > T);
-                if (take && (peers & lt_mask) == 0)   // the first lane of each group adds for the group
-                    atomicAdd(&a.tile_sum[tile], (unsigned long long)__popc(peers & gt) |
-                                                     ((unsigned long long)__popc(peers & ~gt) << 32));
+            // (four stretches of the list per warp and turn, their loads in flight together)
+            for (uint64_t c0 = gid - lane; c0 < n_cand; c0 += 4ull * gstride) {
+                uint32_t key[4], idx[4];
+                bool take[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint64_t c = c0 + (uint64_t)j * gstride + lane;
+                    key[j] = (c < n_cand) ? __ldcg(a.cand_key + c) : 0u;
+                    take[j] = c < n_cand && key[j] >= T;
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    idx[j] = take[j] ? __ldcg(a.cand_idx + c0 + (uint64_t)j * gstride + lane) : 0xFFFFFFFFu;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (c0 + (uint64_t)j * gstride >= n_cand) break;   // warp-uniform
+                    const uint32_t i = idx[j];
+                    if (take[j]) atomicOr(((key[j] > T) ? a.G : a.E) + (i >> 5), 1u << (i & 31u));
+                    const uint32_t tile = take[j] ? i / (kBlock * kEmitTile) : 0xFFFFFFFFu;
+                    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, tile);
+                    const uint32_t gt = __ballot_sync(0xFFFFFFFFu, take[j] && key[j] > T);
+                    if (take[j] && (peers & lt_mask) == 0)   // the first lane of each group adds for the group
+                        atomicAdd(&a.tile_sum[tile], (unsigned long long)__popc(peers & gt) |
+                                                         ((unsigned long long)__popc(peers & ~gt) << 32));
+                }
             }
         }
     } else {

@@ -148,14 +148,28 @@ __device__ __forceinline__ void tile_scan_phase(unsigned long long* super, uint6
                                                 uint32_t ties, WsHeader* hdr, uint32_t* dir,
                                                 unsigned long long* scan_smem) {
     const uint64_t nsuper = (nb + kSuperTile - 1) / kSuperTile;
-    unsigned long long carry = 0;
-    for (uint64_t s0 = 0; s0 < nsuper; s0 += THREADS) {
-        const uint64_t s = s0 + threadIdx.x;
-        const unsigned long long v = (s < nsuper) ? __ldcg(super + s) : 0ull;
-        unsigned long long total;
-        const unsigned long long ex = block_exclusive_scan64<THREADS / 32>(v, scan_smem, &total);
-        if (s < nsuper) super[s] = carry + ex;
-        carry += total;
+    // every warp owns a stretch of consecutive groups: its sum (independent loads), one scan over the
+    // warps' sums, then the stretch again 32 groups at a time, the next 32 asked for ahead
+    constexpr uint32_t W = THREADS / 32;
+    const uint32_t lane = lane_id(), wid = threadIdx.x >> 5;
+    const uint64_t per = ((nsuper + W - 1) / W + 31) / 32 * 32;   // groups per warp, a multiple of 32
+    const uint64_t s_lo = min(nsuper, (uint64_t)wid * per), s_hi = min(nsuper, s_lo + per);
+    unsigned long long sum = 0;
+#pragma unroll 4
+    for (uint64_t s = s_lo + lane; s < s_hi; s += 32) sum += __ldcg(super + s);
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
+    unsigned long long carry;
+    unsigned long long run = block_exclusive_scan64<W>(lane == 0 ? sum : 0ull, scan_smem, &carry);
+    run = __shfl_sync(0xFFFFFFFFu, run, 0);   // counts below the warp's stretch
+    unsigned long long v = (s_lo + lane < s_hi) ? __ldcg(super + s_lo + lane) : 0ull;
+    for (uint64_t s0 = s_lo; s0 < s_hi; s0 += 32) {
+        const uint64_t s = s0 + lane;
+        const unsigned long long nxt = (s + 32 < s_hi) ? __ldcg(super + s + 32) : 0ull;
+        const unsigned long long inc = warp_inclusive_scan64(v);
+        if (s < s_hi) super[s] = run + inc - v;
+        run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+        v = nxt;
     }
     if (threadIdx.x == 0) {
         const uint32_t ng = (uint32_t)carry, ne = (uint32_t)(carry >> 32);
@@ -164,29 +178,50 @@ __device__ __forceinline__ void tile_scan_phase(unsigned long long* super, uint6
     }
 }
 
-// One warp, one 1024-parameter block (lane = bitmap word; blk < nb): the block's part of the core
-// (*sel) and the number of core parameters below this lane's word (*pos0).  Returns the number of
-// core parameters in the block.
-__device__ __forceinline__ uint32_t block_selection(const uint32_t* __restrict__ G, const uint32_t* __restrict__ E,
+// What a warp reads for one 1024-parameter block (lane = bitmap word; blk < nb): the lane's words of
+// the two bitmaps and its share of the counts below the block (the group's prefix plus the blocks
+// of the group below this one).  Asking and placing are separate so that a warp that walks several
+// blocks can ask for the next one before it works on the current one.
+struct BlockLoads {
+    uint32_t Gw, Ew;
+    uint32_t below_g, below_e;   // this lane's share of the group's blocks below the block
+    unsigned long long pref;     // counts below the group (every lane holds it)
+};
+
+__device__ __forceinline__ BlockLoads block_request(const uint32_t* __restrict__ G, const uint32_t* __restrict__ E,
                                                     const unsigned long long* __restrict__ cnt,
-                                                    const unsigned long long* __restrict__ super_pref, uint32_t ties,
-                                                    uint64_t blk, uint32_t* sel, uint32_t* pos0) {
+                                                    const unsigned long long* __restrict__ super_pref, uint64_t blk) {
     const uint32_t lane = lane_id();
-    const uint32_t Gw = __ldg(G + blk * kWordsPerBlock + lane);
-    const uint32_t Ew = (E != nullptr) ? __ldg(E + blk * kWordsPerBlock + lane) : 0u;
-    // counts below the block: the group's prefix plus the blocks of the group below this one
+    BlockLoads L;
+    L.Gw = __ldg(G + blk * kWordsPerBlock + lane);
+    L.Ew = (E != nullptr) ? __ldg(E + blk * kWordsPerBlock + lane) : 0u;
     const uint64_t super = blk / kSuperTile, first = super * kSuperTile;
-    unsigned long long v = 0;
-    if (first + lane < blk) v += __ldg(cnt + first + lane);
-    if (first + 32 + lane < blk) v += __ldg(cnt + first + 32 + lane);
-    if (lane == 0) v += __ldg(super_pref + super);
-    const unsigned long long mine = (unsigned long long)__popc(Gw) | ((unsigned long long)__popc(Ew) << 32);
-    unsigned long long in_warp = warp_inclusive_scan64(mine);
+    const unsigned long long c0 = (first + lane < blk) ? __ldg(cnt + first + lane) : 0ull;
+    const unsigned long long c1 = (first + 32 + lane < blk) ? __ldg(cnt + first + 32 + lane) : 0ull;
+    L.pref = __ldg(super_pref + super);
+    L.below_g = (uint32_t)c0 + (uint32_t)c1;   // a block counts at most 1024 of either kind
+    L.below_e = (uint32_t)(c0 >> 32) + (uint32_t)(c1 >> 32);
+    return L;
+}
+
+// The block's part of the core (*sel) and the number of core parameters below this lane's word
+// (*pos0).  Returns the number of core parameters in the block.
+__device__ __forceinline__ uint32_t block_place(const BlockLoads& L, uint32_t ties, uint32_t* sel, uint32_t* pos0) {
+    const uint32_t lane = lane_id();
+    const uint32_t Gw = L.Gw, Ew = L.Ew;
+    const uint32_t pg = __popc(Gw), pe = __popc(Ew);
+    // counts in the words below this lane's, both kinds in one word (at most 1024 each)
+    uint32_t incl = pg | (pe << 16);
 #pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
-    const unsigned long long run = v + in_warp - mine;   // counts below this lane's word
-    const uint32_t g_before = (uint32_t)run, e_before = (uint32_t)(run >> 32);
-    const uint32_t pe = __popc(Ew);
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= (uint32_t)d) incl += up;
+    }
+    // counts below this lane's word in the whole vector (the core is at most 2^32 - 1 long)
+    const uint32_t g_before =
+        (uint32_t)L.pref + __reduce_add_sync(0xFFFFFFFFu, L.below_g) + (incl & 0xFFFFu) - pg;
+    const uint32_t e_before =
+        (uint32_t)(L.pref >> 32) + __reduce_add_sync(0xFFFFFFFFu, L.below_e) + (incl >> 16) - pe;
     // equal keys: admit those whose rank among all equal keys (index order) is below r
     const uint32_t admit = (ties > e_before) ? min(ties - e_before, pe) : 0u;
     uint32_t Ea;
@@ -201,6 +236,14 @@ __device__ __forceinline__ uint32_t block_selection(const uint32_t* __restrict__
     return __reduce_add_sync(0xFFFFFFFFu, __popc(*sel));
 }
 
+__device__ __forceinline__ uint32_t block_selection(const uint32_t* __restrict__ G, const uint32_t* __restrict__ E,
+                                                    const unsigned long long* __restrict__ cnt,
+                                                    const unsigned long long* __restrict__ super_pref, uint32_t ties,
+                                                    uint64_t blk, uint32_t* sel, uint32_t* pos0) {
+    const BlockLoads L = block_request(G, E, cnt, super_pref, blk);
+    return block_place(L, ties, sel, pos0);
+}
+
 // The block's words of the core bitmap and its 16 directory entries.
 __device__ __forceinline__ void write_block_aux(uint32_t* __restrict__ bitmap, uint32_t* __restrict__ dir, uint64_t blk,
                                                 uint32_t sel, uint32_t pos0) {
@@ -210,7 +253,13 @@ __device__ __forceinline__ void write_block_aux(uint32_t* __restrict__ bitmap, u
         dir[blk * kDirPerBlock + lane / kWordsPerDir] = (uint32_t)(blk * kBlock) + lane * 32u - pos0;
 }
 
-// A warp per block; warps walk the blocks in turn and wait for nobody.
+// A warp per block; warps walk the blocks in turn and wait for nobody.  A block with few members
+// has every lane write out its own word's members; otherwise the lanes list their members' offsets
+// in the warp's piece of shared memory, in index order, and the warp writes the list out 32
+// consecutive places at a time (whole lines), which costs a tenth of the instructions and store
+// requests of word-by-word compaction on a dense block.
+constexpr uint32_t kEmitDirectMax = 160;   // members per block up to which the lanes write directly
+
 __global__ void __launch_bounds__(kEmitWarps * 32) emit_kernel(const uint32_t* __restrict__ G,
                                                                const uint32_t* __restrict__ E,
                                                                const unsigned long long* __restrict__ cnt,
@@ -219,20 +268,25 @@ __global__ void __launch_bounds__(kEmitWarps * 32) emit_kernel(const uint32_t* _
                                                                uint32_t* __restrict__ core_idx,
                                                                uint32_t* __restrict__ bitmap,
                                                                uint32_t* __restrict__ dir) {
+    __shared__ uint16_t list[kEmitWarps][kBlock];
     if (hdr->abort != 0u) return;   // the finishing kernel gave up (the status word says so)
     const uint32_t ties = (E != nullptr) ? hdr->tie_quota : 0u;
-    const uint32_t lane = lane_id();
-    const uint32_t lt_mask = (1u << lane) - 1u;
+    const uint32_t lane = lane_id(), wid = threadIdx.x >> 5;
     const uint64_t warps = (uint64_t)gridDim.x * kEmitWarps;
     bool bad = false;
-    for (uint64_t blk = (uint64_t)blockIdx.x * kEmitWarps + (threadIdx.x >> 5); blk < nb; blk += warps) {
+    uint64_t blk = (uint64_t)blockIdx.x * kEmitWarps + wid;
+    if (blk >= nb) return;
+    BlockLoads cur = block_request(G, E, cnt, super_pref, blk);
+    for (; blk < nb; blk += warps) {
+        BlockLoads nxt = cur;
+        if (blk + warps < nb) nxt = block_request(G, E, cnt, super_pref, blk + warps);
         uint32_t sel, pos0;
-        const uint32_t in_block = block_selection(G, E, cnt, super_pref, ties, blk, &sel, &pos0);
+        const uint32_t in_block = block_place(cur, ties, &sel, &pos0);
+        cur = nxt;
         write_block_aux(bitmap, dir, blk, sel, pos0);
         if (in_block == 0) continue;
         const uint32_t first = (uint32_t)(blk * kBlock);
-        if (in_block <= 256) {
-            // sparse block: every lane writes out its own word's members
+        if (in_block <= kEmitDirectMax) {
             uint32_t pos = pos0;
             for (uint32_t word = sel; word; word &= word - 1, ++pos) {
                 if (pos < k)
@@ -241,19 +295,19 @@ __global__ void __launch_bounds__(kEmitWarps * 32) emit_kernel(const uint32_t* _
                     bad = true;
             }
         } else {
-            // dense block: the warp writes one word's members at a time (coalesced)
-            for (uint32_t m = __ballot_sync(0xFFFFFFFFu, sel != 0); m; m &= m - 1) {
-                const int wd = __ffs(m) - 1;
-                const uint32_t word = __shfl_sync(0xFFFFFFFFu, sel, wd);
-                const uint32_t base = __shfl_sync(0xFFFFFFFFu, pos0, wd);
-                if ((word >> lane) & 1u) {
-                    const uint32_t pos = base + __popc(word & lt_mask);
-                    if (pos < k)
-                        core_idx[pos] = first + wd * 32u + lane;
-                    else
-                        bad = true;
-                }
+            const uint32_t base = __shfl_sync(0xFFFFFFFFu, pos0, 0);   // core parameters below the block
+            uint16_t* mine = list[wid];
+            uint32_t at = pos0 - base;
+            for (uint32_t word = sel; word; word &= word - 1, ++at)
+                if (at < kBlock) mine[at] = (uint16_t)(lane * 32u + (uint32_t)__ffs(word) - 1u);
+            __syncwarp();
+            for (uint32_t e = lane; e < in_block; e += 32) {
+                if (base + e < k)
+                    core_idx[base + e] = first + mine[e];
+                else
+                    bad = true;
             }
+            __syncwarp();   // the list is free again
         }
     }
     if (bad) hdr->status = SLIMDP_ERR_INTERNAL;
@@ -265,8 +319,13 @@ inline slimdp_status launch_emit(const uint32_t* G, const uint32_t* E, const uns
     const uint64_t nb = num_blocks(n);
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
+    // one wave: as many CTAs as are resident at once (a second, thinner wave would cost as much again)
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, emit_kernel, kEmitWarps * 32, 0) != cudaSuccess ||
+        per_sm < 1)
+        return SLIMDP_ERR_CUDA;
     uint64_t grid = (nb + kEmitWarps - 1) / kEmitWarps;
-    if (grid > (uint64_t)sms * 8) grid = (uint64_t)sms * 8;
+    if (grid > (uint64_t)sms * per_sm) grid = (uint64_t)sms * per_sm;
     emit_kernel<<<(unsigned)grid, kEmitWarps * 32, 0, st>>>(G, E, cnt, super_pref, nb, k, hdr, core_idx, bitmap, dir);
     SLIMDP_LAUNCHED(1);
     return SLIMDP_OK;
