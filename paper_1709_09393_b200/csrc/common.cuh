@@ -33,8 +33,8 @@ struct WsHeader {
     uint32_t ties;       // r: how many keys equal to T are admitted (smallest indices first)
     uint32_t n_def;      // bracket pass: keys in bins >= b_top (certainly in the core)
     uint32_t n_cand;     // bracket pass: keys inside the bracket (candidates)
-    uint32_t b_top;      // first 16-bit bin certainly above T (65536: none)
-    uint32_t b_bot;      // lowest 16-bit bin that may hold T
+    uint32_t b_top;      // first 18-bit bin (key >> 14) certainly above T (2^18: none)
+    uint32_t b_bot;      // lowest 18-bit bin that may hold T
     uint32_t ticket[8];  // "last CTA done" counters, one per kernel that needs one
     uint32_t coarse_x[2];  // sample: coarse bins in which the two target ranks are crossed
     uint32_t next_block;   // fused scoring pass: the next 1024-parameter block to hand out

@@ -9,7 +9,7 @@ struct SelectWs {
     WsHeader* hdr;
     uint32_t* hist;                 // 6 x 4096 bins: three passes over all keys, three over the candidates
     uint32_t* coarse_hist;          // 256 bins (top 8 key bits of the sampled keys)
-    uint32_t* fine_hist;            // 2 x 256 bins (top 16 key bits inside the two crossing coarse bins)
+    uint32_t* fine_hist;            // 2 x 1024 bins (top 18 key bits inside the two crossing coarse bins)
     uint32_t* coarse_incl;          // 256: samples in coarse bins >= c
     uint32_t* sample;               // 2^18 sampled keys
     uint32_t* G;                    // greater-than-threshold bitmap, nb * 32 words
@@ -38,7 +38,7 @@ inline SelectWs select_ws_layout(void* ws, uint64_t n) {
     L.hdr = reinterpret_cast<WsHeader*>(take(sizeof(WsHeader)));
     L.hist = reinterpret_cast<uint32_t*>(take(6 * 4096 * sizeof(uint32_t)));
     L.coarse_hist = reinterpret_cast<uint32_t*>(take(256 * sizeof(uint32_t)));
-    L.fine_hist = reinterpret_cast<uint32_t*>(take(512 * sizeof(uint32_t)));
+    L.fine_hist = reinterpret_cast<uint32_t*>(take(2 * 1024 * sizeof(uint32_t)));
     L.tile_sum = reinterpret_cast<unsigned long long*>(take(((nb + kEmitTile - 1) / kEmitTile) * 8));
     L.zero_bytes = off;
     L.super_pref = reinterpret_cast<unsigned long long*>(take((((nb + kEmitTile - 1) / kEmitTile + 63) / 64) * 8));

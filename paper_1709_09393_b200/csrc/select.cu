@@ -8,8 +8,8 @@
 // Large inputs (n >= 2^21) take the bracketed path, which reads the keys once:
 //   1. sample (two small kernels): 2^18 keys (sixteen at each of 2^14 evenly
 //      spaced places) are counted by their top 8 bits, then, around the two
-//      target ranks, by their top 16 bits; the last CTA of each kernel turns
-//      the counts into a bracket of 16-bit bins [b_bot, b_top) that holds T
+//      target ranks, by their top 18 bits; the last CTA of each kernel turns
+//      the counts into a bracket of 18-bit bins [b_bot, b_top) that holds T
 //      with overwhelming probability;
 //   2. bracket pass (one read of all keys): keys in bins >= b_top are
 //      certainly in the core and go straight into the "greater" bitmap; keys
@@ -52,12 +52,20 @@ __device__ __forceinline__ bool bracket_ok(const WsHeader* hdr, uint32_t k, uint
     return bracket_held(hdr->n_def, hdr->n_cand, k, cap);
 }
 
-// Candidates' keys lie in [b_bot << 16, b_top << 16).  Their offsets from the bottom of the bracket
-// need `width` bits; the first counting round takes the top kDigitBits of them and leaves this many.
+// The bracket's resolution: bins of 2^kBinShift consecutive keys (the keys' top 18 bits), found in two
+// steps (8 bits, then kFineBits more inside the two coarse bins that matter).
+constexpr uint32_t kFineBits = 10;
+constexpr uint32_t kFineBins = 1u << kFineBits;
+constexpr uint32_t kBinShift = 24 - kFineBits;
+constexpr uint32_t kNoBin = 1u << (32 - kBinShift);   // b_top when no bin is certainly above T
+
+// Candidates' keys lie in [b_bot << kBinShift, b_top << kBinShift).  Their offsets from the bottom of
+// the bracket need `width` bits; the first counting round takes the top kDigitBits of them and leaves
+// this many.
 __host__ __device__ __forceinline__ uint32_t cand_low_bits(uint32_t b_top, uint32_t b_bot) {
     if (b_top <= b_bot) return 0;
-    const unsigned long long span = (unsigned long long)(b_top - b_bot) << 16;   // <= 2^32
-    uint32_t width = 16;
+    const unsigned long long span = (unsigned long long)(b_top - b_bot) << kBinShift;   // <= 2^32
+    uint32_t width = kBinShift;
     while ((1ull << width) < span) ++width;
     return width > kDigitBits ? width - kDigitBits : 0;
 }
@@ -175,27 +183,31 @@ __global__ void __launch_bounds__(1024) sample_coarse_kernel(const uint32_t* __r
     }
 }
 
-// Sample kernel B: the members of the two crossing coarse bins are counted by their top 16 bits
-// (2 x 256 fine bins); the last CTA resolves each crossing to a 16-bit bin:
-// b_top = lowest bin b with (samples in bins >= b) <= lo_target, 65536 if there is none;
+// Sample kernel B: the members of the two crossing coarse bins are counted by the kFineBits key bits
+// that follow (2 x kFineBins fine bins); the last CTA resolves each crossing to an 18-bit bin:
+// b_top = lowest bin b with (samples in bins >= b) <= lo_target, kNoBin if there is none;
 // b_bot = highest bin b with (samples in bins >= b) >= hi_target, 0 if there is none.
 __global__ void __launch_bounds__(1024) sample_fine_kernel(const uint32_t* __restrict__ sample, uint64_t n,
                                                            uint32_t k, WsHeader* hdr,
                                                            uint32_t* __restrict__ fine_hist,
                                                            const uint32_t* __restrict__ coarse_incl) {
     __shared__ unsigned long long smem[33];
-    __shared__ uint32_t sh_fine[2][256];
+    __shared__ uint32_t sh_fine[2][kFineBins];
     __shared__ uint32_t s_val[2];
+    constexpr uint32_t kPer = kFineBins / 1024;   // fine bins per thread of the last CTA
     const uint32_t t = threadIdx.x;
     const uint32_t cx0 = hdr->coarse_x[0], cx1 = hdr->coarse_x[1];
-    if (t < 512) sh_fine[t >> 8][t & 255u] = 0;
+    for (uint32_t b = t; b < 2 * kFineBins; b += 1024) sh_fine[b / kFineBins][b % kFineBins] = 0;
     __syncthreads();
     const uint32_t key = sample[blockIdx.x * 1024 + t];
-    const uint32_t cb = key >> 24, fb = (key >> 16) & 255u;
+    const uint32_t cb = key >> 24, fb = (key >> kBinShift) & (kFineBins - 1u);
     if (cb == cx0) atomicAdd(&sh_fine[0][fb], 1u);
     if (cb == cx1) atomicAdd(&sh_fine[1][fb], 1u);
     __syncthreads();
-    if (t < 512 && sh_fine[t >> 8][t & 255u]) atomicAdd(&fine_hist[t], sh_fine[t >> 8][t & 255u]);
+    for (uint32_t b = t; b < 2 * kFineBins; b += 1024) {
+        const uint32_t c = sh_fine[b / kFineBins][b % kFineBins];
+        if (c) atomicAdd(&fine_hist[b], c);
+    }
     if (!last_cta_done(&hdr->ticket[7])) return;
     long long lo_target, hi_target;
     bracket_targets(k, n, &lo_target, &hi_target);
@@ -203,26 +215,34 @@ __global__ void __launch_bounds__(1024) sample_fine_kernel(const uint32_t* __res
         const long long target = which ? hi_target : lo_target;
         const uint32_t cx = which ? cx1 : cx0;
         if (cx == 0xFFFFFFFFu) {
-            // no crossing: which = 0: target < 0 (nothing is certain: 65536) or every bin qualifies (0);
+            // no crossing: which = 0: target < 0 (nothing is certain: kNoBin) or every bin qualifies (0);
             //              which = 1: target above the sample size: every bin may hold T (0)
-            if (t == 0) s_val[which] = which ? 0u : ((target < 0) ? 65536u : 0u);
+            if (t == 0) s_val[which] = which ? 0u : ((target < 0) ? kNoBin : 0u);
             __syncthreads();
             continue;
         }
         const long long above_cx = (cx == 255) ? 0 : (long long)coarse_incl[cx + 1];
-        // fine bins of coarse bin cx from the top down: thread t < 256 owns fine bin cx * 256 + 255 - t
+        // fine bins of coarse bin cx from the top down: thread t owns fine bins
+        // kFineBins - 1 - kPer t, ..., kFineBins - kPer (t + 1)
+        uint32_t f[kPer];
+        unsigned long long mine = 0;
+#pragma unroll
+        for (uint32_t q = 0; q < kPer; ++q) {
+            f[q] = __ldcg(fine_hist + which * kFineBins + (kFineBins - 1u - (kPer * t + q)));
+            mine += f[q];
+        }
         unsigned long long total;
-        const unsigned long long f = (t < 256) ? __ldcg(fine_hist + which * 256 + 255 - t) : 0ull;
-        const long long f_above = (long long)block_exclusive_scan64<32>(f, smem, &total);
-        if (t == 0) s_val[which] = which ? 0u : (cx + 1) * 256u;   // default when no fine bin of cx qualifies
+        long long run = above_cx + (long long)block_exclusive_scan64<32>(mine, smem, &total);
+        if (t == 0) s_val[which] = which ? 0u : (cx + 1) * kFineBins;   // default when no fine bin of cx qualifies
         __syncthreads();
-        if (t < 256) {
-            const uint32_t b = cx * 256 + 255 - t;
-            const long long incl = above_cx + f_above + (long long)f;
+#pragma unroll
+        for (uint32_t q = 0; q < kPer; ++q) {
+            const uint32_t b = cx * kFineBins + (kFineBins - 1u - (kPer * t + q));
+            run += (long long)f[q];   // samples in bins >= b
             if (which == 0) {
-                if (incl <= target) atomicMin(&s_val[0], b);
+                if (run <= target) atomicMin(&s_val[0], b);
             } else {
-                if (incl >= target) atomicMax(&s_val[1], b);
+                if (run >= target) atomicMax(&s_val[1], b);
             }
         }
         __syncthreads();
@@ -276,9 +296,9 @@ __device__ __forceinline__ void pass_begin(PassWarp& pw, const PassOut& out, uin
     pw.my_idx = cand_smem + (kPassWarps + wid) * kCandStage;
     pw.sh_hist = sh_hist;
     // keys >= top_key are certainly in the core; keys in [bot_key, top_key) are candidates
-    pw.has_top = b_top < 65536u;
-    pw.top_key = pw.has_top ? (b_top << 16) : 0xFFFFFFFFu;
-    pw.bot_key = b_bot << 16;
+    pw.has_top = b_top < kNoBin;
+    pw.top_key = pw.has_top ? (b_top << kBinShift) : 0xFFFFFFFFu;
+    pw.bot_key = b_bot << kBinShift;
     pw.low_bits = cand_low_bits(b_top, b_bot);
     pw.staged = 0;
     pw.def_acc = 0;
@@ -823,7 +843,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2) finish_kernel(FinishArgs a)
     if (cand_mode) {
         // tile_sum holds what the pass counted (certainly-core members only so far)
         const uint32_t b_top = hdr->b_top, b_bot = hdr->b_bot;
-        const uint32_t bot_key = b_bot << 16;
+        const uint32_t bot_key = b_bot << kBinShift;
         const uint32_t n_cand = hdr->n_cand;
         uint32_t low = cand_low_bits(b_top, b_bot);
         uint32_t prefix = hdr->prefix, rem = hdr->k_rem;   // first digit: found by the pass's last CTA

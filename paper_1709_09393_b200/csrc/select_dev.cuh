@@ -253,12 +253,42 @@ __device__ __forceinline__ void write_block_aux(uint32_t* __restrict__ bitmap, u
         dir[blk * kDirPerBlock + lane / kWordsPerDir] = (uint32_t)(blk * kBlock) + lane * 32u - pos0;
 }
 
-// A warp per block; warps walk the blocks in turn and wait for nobody.  A block with few members
-// has every lane write out its own word's members; otherwise the lanes list their members' offsets
-// in the warp's piece of shared memory, in index order, and the warp writes the list out 32
-// consecutive places at a time (whole lines), which costs a tenth of the instructions and store
-// requests of word-by-word compaction on a dense block.
-constexpr uint32_t kEmitDirectMax = 160;   // members per block up to which the lanes write directly
+// emit_kernel: half a warp per block, so that one instruction serves two blocks (the kernel is
+// bound by the instructions it issues, not by memory).  Lane h of a half holds the block's words 2h
+// and 2h + 1, which is one directory group.  Warps walk pairs of blocks in turn, wait for nobody and
+// ask for the next pair before they work on the current one.  A block with few members has every
+// lane write out its own words' members; otherwise the lanes list their members' offsets in the
+// half's piece of shared memory, in index order, and the half writes the list out 16 consecutive
+// places at a time.
+constexpr uint32_t kEmitDirectMax = 64;   // members per block up to which the lanes write directly
+
+struct HalfLoads {
+    uint2 G2, E2;
+    uint32_t below;            // this lane's share of the group's blocks below the block: #greater | #equal << 16
+    unsigned long long pref;   // counts below the group
+};
+
+__device__ __forceinline__ HalfLoads half_request(const uint32_t* __restrict__ G, const uint32_t* __restrict__ E,
+                                                  const unsigned long long* __restrict__ cnt,
+                                                  const unsigned long long* __restrict__ super_pref, uint64_t blk,
+                                                  uint64_t nb, uint32_t hl) {
+    HalfLoads L;
+    L.G2 = make_uint2(0u, 0u);
+    L.E2 = make_uint2(0u, 0u);
+    L.below = 0;
+    L.pref = 0;
+    if (blk >= nb) return L;
+    L.G2 = __ldg(reinterpret_cast<const uint2*>(G) + blk * (kWordsPerBlock / 2) + hl);
+    if (E != nullptr) L.E2 = __ldg(reinterpret_cast<const uint2*>(E) + blk * (kWordsPerBlock / 2) + hl);
+    const uint64_t super = blk / kSuperTile, first = super * kSuperTile;
+    unsigned long long c = 0;   // at most 4 blocks of at most 1024 of either kind: no carry between the halves
+#pragma unroll
+    for (uint32_t q = 0; q < kSuperTile / 16; ++q)
+        if (first + 16 * q + hl < blk) c += __ldg(cnt + first + 16 * q + hl);
+    L.below = (uint32_t)c | ((uint32_t)(c >> 32) << 16);
+    L.pref = __ldg(super_pref + super);
+    return L;
+}
 
 __global__ void __launch_bounds__(kEmitWarps * 32) emit_kernel(const uint32_t* __restrict__ G,
                                                                const uint32_t* __restrict__ E,
@@ -268,46 +298,97 @@ __global__ void __launch_bounds__(kEmitWarps * 32) emit_kernel(const uint32_t* _
                                                                uint32_t* __restrict__ core_idx,
                                                                uint32_t* __restrict__ bitmap,
                                                                uint32_t* __restrict__ dir) {
-    __shared__ uint16_t list[kEmitWarps][kBlock];
+    static_assert((kSuperTile - 1) * kBlock < 65536u, "the counts of a group's blocks below a block fit 16 bits each");
+    __shared__ uint16_t list[kEmitWarps][2][kBlock];
     if (hdr->abort != 0u) return;   // the finishing kernel gave up (the status word says so)
     const uint32_t ties = (E != nullptr) ? hdr->tie_quota : 0u;
     const uint32_t lane = lane_id(), wid = threadIdx.x >> 5;
+    const uint32_t half = lane >> 4, hl = lane & 15u;
+    const uint64_t pairs = (nb + 1) / 2;
     const uint64_t warps = (uint64_t)gridDim.x * kEmitWarps;
     bool bad = false;
-    uint64_t blk = (uint64_t)blockIdx.x * kEmitWarps + wid;
-    if (blk >= nb) return;
-    BlockLoads cur = block_request(G, E, cnt, super_pref, blk);
-    for (; blk < nb; blk += warps) {
-        BlockLoads nxt = cur;
-        if (blk + warps < nb) nxt = block_request(G, E, cnt, super_pref, blk + warps);
-        uint32_t sel, pos0;
-        const uint32_t in_block = block_place(cur, ties, &sel, &pos0);
+    uint64_t pair = (uint64_t)blockIdx.x * kEmitWarps + wid;
+    if (pair >= pairs) return;
+    HalfLoads cur = half_request(G, E, cnt, super_pref, 2 * pair + half, nb, hl);
+    for (; pair < pairs; pair += warps) {
+        const uint64_t blk = 2 * pair + half;
+        const bool live = blk < nb;
+        HalfLoads nxt = cur;
+        if (pair + warps < pairs) nxt = half_request(G, E, cnt, super_pref, 2 * (pair + warps) + half, nb, hl);
+        const uint2 G2 = cur.G2, E2 = cur.E2;
+        const uint32_t pg = __popc(G2.x) + __popc(G2.y), pe = __popc(E2.x) + __popc(E2.y);
+        // counts in the half's lanes below this one, and in the group's blocks below the block
+        uint32_t incl = pg | (pe << 16), below = cur.below;
+#pragma unroll
+        for (int d = 1; d < 16; d <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d, 16);
+            if (hl >= (uint32_t)d) incl += up;
+        }
+#pragma unroll
+        for (int d = 8; d >= 1; d >>= 1) below += __shfl_xor_sync(0xFFFFFFFFu, below, d, 16);
+        const uint32_t g_before = (uint32_t)cur.pref + (below & 0xFFFFu) + (incl & 0xFFFFu) - pg;
+        const uint32_t e_before = (uint32_t)(cur.pref >> 32) + (below >> 16) + (incl >> 16) - pe;
         cur = nxt;
-        write_block_aux(bitmap, dir, blk, sel, pos0);
-        if (in_block == 0) continue;
+        // equal keys: admit those whose rank among all equal keys (index order) is below r
+        const uint32_t admit = (ties > e_before) ? min(ties - e_before, pe) : 0u;
+        uint2 sel = G2;
+        if (admit == pe) {
+            sel.x |= E2.x;
+            sel.y |= E2.y;
+        } else if (admit != 0) {
+            const uint32_t c0 = __popc(E2.x);
+            if (admit < c0) {
+                sel.x |= E2.x & ((1u << nth_set_bit(E2.x, admit)) - 1u);
+            } else {
+                sel.x |= E2.x;
+                if (admit > c0) sel.y |= E2.y & ((1u << nth_set_bit(E2.y, admit - c0)) - 1u);
+            }
+        }
+        const uint32_t pos0 = g_before + min(e_before, ties);   // core parameters below this lane's words
+        uint32_t in_block = __popc(sel.x) + __popc(sel.y);
+#pragma unroll
+        for (int d = 8; d >= 1; d >>= 1) in_block += __shfl_xor_sync(0xFFFFFFFFu, in_block, d, 16);
+        const uint32_t base = __shfl_sync(0xFFFFFFFFu, pos0, 0, 16);   // core parameters below the block
         const uint32_t first = (uint32_t)(blk * kBlock);
-        if (in_block <= kEmitDirectMax) {
+        if (live) {
+            reinterpret_cast<uint2*>(bitmap)[blk * (kWordsPerBlock / 2) + hl] = sel;
+            dir[blk * kDirPerBlock + hl] = first + hl * 64u - pos0;
+        }
+        const bool staged = live && in_block > kEmitDirectMax;
+        if (live && !staged) {
             uint32_t pos = pos0;
-            for (uint32_t word = sel; word; word &= word - 1, ++pos) {
+            for (uint32_t word = sel.x; word; word &= word - 1, ++pos) {
                 if (pos < k)
-                    core_idx[pos] = first + lane * 32u + (uint32_t)__ffs(word) - 1u;
+                    core_idx[pos] = first + hl * 64u + (uint32_t)__ffs(word) - 1u;
                 else
                     bad = true;
             }
-        } else {
-            const uint32_t base = __shfl_sync(0xFFFFFFFFu, pos0, 0);   // core parameters below the block
-            uint16_t* mine = list[wid];
-            uint32_t at = pos0 - base;
-            for (uint32_t word = sel; word; word &= word - 1, ++at)
-                if (at < kBlock) mine[at] = (uint16_t)(lane * 32u + (uint32_t)__ffs(word) - 1u);
+            for (uint32_t word = sel.y; word; word &= word - 1, ++pos) {
+                if (pos < k)
+                    core_idx[pos] = first + hl * 64u + 32u + (uint32_t)__ffs(word) - 1u;
+                else
+                    bad = true;
+            }
+        }
+        if (__any_sync(0xFFFFFFFFu, staged)) {
+            uint16_t* mine = list[wid][half];
+            if (staged) {
+                uint32_t at = pos0 - base;
+                for (uint32_t word = sel.x; word; word &= word - 1, ++at)
+                    if (at < kBlock) mine[at] = (uint16_t)(hl * 64u + (uint32_t)__ffs(word) - 1u);
+                for (uint32_t word = sel.y; word; word &= word - 1, ++at)
+                    if (at < kBlock) mine[at] = (uint16_t)(hl * 64u + 32u + (uint32_t)__ffs(word) - 1u);
+            }
             __syncwarp();
-            for (uint32_t e = lane; e < in_block; e += 32) {
-                if (base + e < k)
-                    core_idx[base + e] = first + mine[e];
-                else
-                    bad = true;
+            if (staged) {
+                for (uint32_t e = hl; e < in_block; e += 16) {
+                    if (base + e < k)
+                        core_idx[base + e] = first + mine[e];
+                    else
+                        bad = true;
+                }
             }
-            __syncwarp();   // the list is free again
+            __syncwarp();   // the lists are free again
         }
     }
     if (bad) hdr->status = SLIMDP_ERR_INTERNAL;
@@ -324,7 +405,7 @@ inline slimdp_status launch_emit(const uint32_t* G, const uint32_t* E, const uns
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, emit_kernel, kEmitWarps * 32, 0) != cudaSuccess ||
         per_sm < 1)
         return SLIMDP_ERR_CUDA;
-    uint64_t grid = (nb + kEmitWarps - 1) / kEmitWarps;
+    uint64_t grid = ((nb + 1) / 2 + kEmitWarps - 1) / kEmitWarps;   // a warp per pair of blocks
     if (grid > (uint64_t)sms * per_sm) grid = (uint64_t)sms * per_sm;
     emit_kernel<<<(unsigned)grid, kEmitWarps * 32, 0, st>>>(G, E, cnt, super_pref, nb, k, hdr, core_idx, bitmap, dir);
     SLIMDP_LAUNCHED(1);
