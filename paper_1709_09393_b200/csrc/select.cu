@@ -27,7 +27,7 @@
 //      keys (12 + 10 + 10 bits) and one classifying round that writes both
 //      bitmaps and the counts.  Either way it ends by turning the per-block
 //      counts into prefixes per group of 64 blocks;
-//   4. the emit kernel (select_dev.cuh; a warp per 1024-parameter block, no
+//   4. the emit kernel (select_dev.cuh; half a warp per 1024-parameter block, no
 //      waiting between warps): admits the first r equal keys in index order
 //      and writes the core bitmap, the non-core rank directory and the
 //      ascending index list (ordered compaction, no atomic cursors).
