@@ -113,7 +113,7 @@ int sm_count() {
 namespace {
 
 constexpr uint64_t kMaxN = 0xFFFFFFFFull;   // indices are uint32_t
-constexpr uint64_t kFoldedExchangeMaxN = 1ull << 23;   // slimdp_round: up to here the exchange also does the emit's work
+constexpr uint64_t kFoldedExchangeMaxN = 1ull << 22;   // slimdp_round: up to here the exchange also does the emit's work
 
 bool n_ok(uint64_t n) { return n >= 1 && n <= kMaxN; }
 bool k_ok(uint32_t K) { return K >= 1 && K <= SLIMDP_MAX_WORKERS; }
@@ -723,7 +723,8 @@ slimdp_status slimdp_round(float* w_global, const float* const* grads, uint32_t 
     // are bound by the number of dependent launches: there the selection stops after its finishing
     // kernel and the exchange places the core's members itself (one launch less).  On long vectors the
     // separate emit kernel followed by the exchange over the finished index list is as fast or faster
-    // (measured: 138 M parameters 1.58 ms either way; 25.6 M parameters with 16 workers 1.10 against 1.18 ms).
+    // (measured: 138 M parameters 1.58 ms either way; 25.6 M parameters with 16 workers 1.10 against 1.18 ms;
+    // 7 M parameters with 8 workers 201 against 206 us).
     bool staged = false;
     const bool folded = stage == nullptr && n < kFoldedExchangeMaxN && round_exchange_applies(n, k_exp);
     if (fusable) {

@@ -1,6 +1,7 @@
 // Shared declarations of the Slim-DP CUDA library (sm_100a).
 #pragma once
 
+#include <atomic>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -73,6 +74,22 @@ inline bool prefer_max_shared(Kernel kernel) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                 (int)cudaSharedmemCarveoutMaxShared) == cudaSuccess;
 }
+
+// Marks, per device (bit d = device d, devices above 63 are never marked), that a setting the device
+// keeps has been made: kernel attributes are set on a kernel's first launch on a device, not on every call.
+struct DeviceOnce {
+    std::atomic<unsigned long long> done{0};
+    bool needed() const {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+        return ((done.load(std::memory_order_relaxed) >> dev) & 1ull) == 0;
+    }
+    void mark() {
+        int dev = -1;
+        if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64)
+            done.fetch_or(1ull << dev, std::memory_order_relaxed);
+    }
+};
 
 // After a group of `count` kernel launches: fail on a launch error, else count them.
 #define SLIMDP_LAUNCHED(count)                                          \

@@ -579,11 +579,17 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
     const dim3 grid((unsigned)chunks, workers);
     const bool smem = buckets <= kMaxSmemBuckets;
     // part 1 may run beside another kernel's CTAs on the same SMs: one shared-memory split for all
-    if (!prefer_max_shared(rank_kernel<true>) || !prefer_max_shared(rank_kernel<false>) ||
-        !prefer_max_shared(scatter_kernel<true, true>) || !prefer_max_shared(scatter_kernel<true, false>) ||
-        !prefer_max_shared(scatter_kernel<false, false>) || !prefer_max_shared(bucket_sort_kernel<false>) ||
-        !prefer_max_shared(bucket_sort_kernel<true>))
-        return SLIMDP_ERR_CUDA;
+    static DeviceOnce attributes;
+    if (attributes.needed()) {
+        if (!prefer_max_shared(rank_kernel<true>) || !prefer_max_shared(rank_kernel<false>) ||
+            !prefer_max_shared(scatter_kernel<true, true>) || !prefer_max_shared(scatter_kernel<true, false>) ||
+            !prefer_max_shared(scatter_kernel<false, false>) || !prefer_max_shared(bucket_sort_kernel<false>) ||
+            !prefer_max_shared(bucket_sort_kernel<true>) ||
+            cudaFuncSetAttribute(scatter_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kGroupSmemMax) != cudaSuccess)
+            return SLIMDP_ERR_CUDA;
+        attributes.mark();
+    }
     const RankStream rs{(uint32_t)seed, (uint32_t)(seed >> 32), first_worker, round, L.hdr, L.ticket, L.pref, L.totals};
     if (smem) {
         rank_kernel<true><<<grid, 1024, buckets * 4, st>>>((uint32_t)M, (uint32_t)k_exp, chunk, bits, s,
@@ -596,10 +602,6 @@ slimdp_status launch_explore_parts(const void* core_aux, uint64_t n, uint64_t k_
     SLIMDP_LAUNCHED(1);
     const size_t group_smem = (3 * buckets + chunk) * 4;
     if (smem && group_smem <= (lean ? kGroupSmemLean : kGroupSmemMax)) {
-        if (group_smem > 48 * 1024 &&
-            cudaFuncSetAttribute(scatter_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)group_smem) != cudaSuccess)
-            return SLIMDP_ERR_CUDA;
         scatter_kernel<true, true><<<grid, 1024, group_smem, st>>>((uint32_t)k_exp, chunk, s, (uint32_t)buckets,
                                                                    L.rho, L.rho_stride, L.pref, L.cnt_stride,
                                                                    L.cursor, L.cta_hist, L.sorted);

@@ -1113,9 +1113,19 @@ static slimdp_status launch_select_impl(float* scores, uint64_t n, uint64_t k_co
 #define SLIMDP_ASYNC_LAUNCH(SS, KK, ST)                                                                             \
     {                                                                                                               \
         auto kern = score_bracket_async_kernel<SS, KK, ST>;                                                             \
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||    \
-            !prefer_max_shared(kern))                                                                               \
-            return SLIMDP_ERR_CUDA;                                                                                 \
+        static DeviceOnce attributes;                                                                               \
+        if (attributes.needed()) {                                                                                  \
+            int dev = 0, optin = 0;                                                                                 \
+            cudaFuncAttributes fa;                                                                                  \
+            if (cudaGetDevice(&dev) != cudaSuccess ||                                                               \
+                cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||      \
+                cudaFuncGetAttributes(&fa, kern) != cudaSuccess ||                                                  \
+                cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,                             \
+                                     optin - (int)fa.sharedSizeBytes) != cudaSuccess ||                             \
+                !prefer_max_shared(kern))                                                                           \
+                return SLIMDP_ERR_CUDA;                                                                             \
+            attributes.mark();                                                                                      \
+        }                                                                                                           \
         kern<<<(unsigned)agrid, kPassWarps * 32, smem, st>>>(fused->w, *fused->g, (int)fused->K, fused->c, n, nb,   \
                                                              out, so);                                              \
     }

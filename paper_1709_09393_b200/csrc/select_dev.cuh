@@ -401,10 +401,16 @@ inline slimdp_status launch_emit(const uint32_t* G, const uint32_t* E, const uns
     const int sms = sm_count();
     if (sms <= 0) return SLIMDP_ERR_CUDA;
     // one wave: as many CTAs as are resident at once (a second, thinner wave would cost as much again)
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, emit_kernel, kEmitWarps * 32, 0) != cudaSuccess ||
-        per_sm < 1)
-        return SLIMDP_ERR_CUDA;
+    static std::atomic<int> per_sm_cached[64];   // per device; 0 = not asked yet
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SLIMDP_ERR_CUDA;
+    int per_sm = (dev >= 0 && dev < 64) ? per_sm_cached[dev].load(std::memory_order_relaxed) : 0;
+    if (per_sm == 0) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, emit_kernel, kEmitWarps * 32, 0) != cudaSuccess ||
+            per_sm < 1)
+            return SLIMDP_ERR_CUDA;
+        if (dev >= 0 && dev < 64) per_sm_cached[dev].store(per_sm, std::memory_order_relaxed);
+    }
     uint64_t grid = ((nb + 1) / 2 + kEmitWarps - 1) / kEmitWarps;   // a warp per pair of blocks
     if (grid > (uint64_t)sms * per_sm) grid = (uint64_t)sms * per_sm;
     emit_kernel<<<(unsigned)grid, kEmitWarps * 32, 0, st>>>(G, E, cnt, super_pref, nb, k, hdr, core_idx, bitmap, dir);
