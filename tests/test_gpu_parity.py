@@ -196,6 +196,26 @@ def test_select_large_tie_group_spanning_many_blocks(P):
     check_aux(P, aux, exp, n)
 
 
+def test_select_tie_cut_at_every_offset_of_a_directory_group(P):
+    # the emit step admits the first r equal keys in index order: r ends inside the first word of a
+    # 64-parameter group, exactly between its two words, inside the second, and at a group's end,
+    # in a sparse block (members written directly) and in a dense one (listed through shared memory);
+    # 5 blocks: the last pair of blocks has one block only
+    n = 5000
+    rng = np.random.default_rng(5)
+    sparse = np.zeros(n, np.float32)
+    sparse[rng.choice(n, 400, replace=False)] = 0.5          # 400 equal keys above zeros
+    dense = np.full(n, 0.5, np.float32)                      # every key equal
+    tie_idx = np.flatnonzero(sparse)
+    for S, ks in ((dense, range(2040, 2120)), (sparse, range(150, 230)), (dense, (n - 65, n - 64, n - 33, n - 32, n - 1, n))):
+        for k in ks:
+            core_idx, aux = gpu_select(P, S, k)
+            exp = oracle.select_core(S, k)
+            assert np.array_equal(host_u32(core_idx), exp), k
+            check_aux(P, aux, exp, n)
+    assert np.array_equal(oracle.select_core(sparse, 400), tie_idx.astype(np.uint32))
+
+
 @pytest.mark.parametrize("case", ["random", "all_equal", "sampler_fooled", "two_values", "narrow_band"])
 def test_select_bracketed_path_and_its_fallback(P, case):
     # n >= 2^21 takes the sampled-bracket path; inputs that defeat the sample or
