@@ -496,7 +496,7 @@ __device__ __forceinline__ void exchange_core_staged_body(float* __restrict__ w,
 // latency and rate.  CTAs of both kinds are interleaved in the grid (core_ctas of every
 // total_ctas, evenly spread), so both kinds are resident together and fill each other's gaps.
 // The two segments touch disjoint parameters and disjoint parts of val / pulled.
-__global__ void __launch_bounds__(256) exchange_kernel(float* w, const uint32_t* __restrict__ core_idx,
+__global__ void __launch_bounds__(256, 8) exchange_kernel(float* w, const uint32_t* __restrict__ core_idx,
                                                        uint64_t k_core, PtrArray<const uint32_t> exp, uint32_t k_exp,
                                                        PtrArray<const float> delta, PtrArray<float> val,
                                                        PtrArray<float> pulled, int K, float neg_eta,
