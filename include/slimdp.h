@@ -344,6 +344,7 @@ slimdp_status slimdp_merge_q8(float* w_global, uint64_t n, uint32_t K, const uin
  *     slimdp_select_resolve(hist, round, state)      the digit that holds the wanted rank; the same on every shard
  *   now state holds the threshold T (the k_total-th largest key of the whole model) and r, the
  *   number of keys equal to T that belong to the core
+ *   (k_total = 0, the empty core: T = 0xFFFFFFFF and r = 0, so that no key is above T and none is admitted)
  *   clear counts; slimdp_select_count(shard, state, counts)   counts[0] += keys > T, counts[1] += keys == T
  *   all-gather the counts: shard g admits quota_g = min(equal_g, max(0, r - sum of equal_h, h < g))
  *   of its equal keys (ties go to the smaller global index, and shards are index ranges), and its

@@ -70,7 +70,13 @@ __global__ void __launch_bounds__(1024) shard_resolve_kernel(const unsigned long
     }
     unsigned long long total;
     unsigned long long above = block_exclusive_scan64<32>(sum, smem, &total);
-    if (total < want || want == 0) {
+    if (want == 0) {
+        // an empty core (only ever at the first round: a resolved digit leaves a rank of at least 1):
+        // no key lies above the largest bit pattern, and no key equal to it is admitted
+        if (t == 0) state->prefix = 0xFFFFFFFFu;
+        return;
+    }
+    if (total < want) {
         if (t == 0) state->status = SLIMDP_ERR_INTERNAL;
         return;
     }

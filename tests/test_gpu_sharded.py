@@ -35,7 +35,7 @@ def test_sharded_selection_matches_the_oracle(P, case, shards):
     S = _scores(case, n, rng)
     bounds = P.shard_bounds(n, shards)
     parts = [torch.from_numpy(S[b:e].copy()).cuda() for b, e in bounds]
-    for k in (1, n // 20, n // 2 + 7):
+    for k in (0, 1, n // 20, n // 2 + 7, n):
         ref = oracle.select_core(S, k).astype(np.int64)
         out = P.select_core_sharded(parts, k, P.CudaBackend())
         got = np.concatenate([o[0].cpu().numpy().view(np.uint32).astype(np.int64) + b for o, (b, e) in zip(out, bounds)])
